@@ -1,0 +1,346 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA path: they make sure that a plausible
+mistake in the oracle (a dropped term, a wrong sign or index, a transposed
+operand) fails somewhere before the oracle is used to judge the kernels.
+"""
+import ctypes
+import itertools
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle as O
+from conftest import golden_rows
+
+
+# ---------------------------------------------------------------- levels
+def test_level_set_closed_form():
+    """Sec. 3.1: L = (0, 2^-s, ..., 1/2, 1); Fig. 1 uses s = 3."""
+    for row in golden_rows("levels.txt"):
+        s, want = int(row[0]), [Fraction(x) for x in row[1:]]
+        assert O.num_levels(O.LEVELS_EXP, s) == len(want) == s + 2
+        got = [Fraction(O.level_value(O.LEVELS_EXP, s, j)) for j in range(s + 2)]
+        assert got == want
+    for s in range(1, 15):
+        lv = [O.level_value(O.LEVELS_EXP, s, j) for j in range(s + 2)]
+        assert lv[0] == 0.0 and lv[-1] == 1.0 and lv[1] == 2.0 ** -s
+        assert all(lv[j + 1] == 2 * lv[j] for j in range(1, s + 1))
+
+
+def test_uniform_level_set():
+    for s in (1, 2, 4, 8):
+        n = O.num_levels(O.LEVELS_UNIFORM, s)
+        assert n == 2 ** s + 1
+        assert [O.level_value(O.LEVELS_UNIFORM, s, k) for k in range(n)] == [k / 2 ** s for k in range(n)]
+
+
+def test_fixed_width():
+    # sign bit + ceil(log2(number of levels))
+    assert [O.fixed_width(O.LEVELS_EXP, s) for s in (1, 2, 3, 4, 6, 7)] == [3, 3, 4, 4, 4, 5]
+    assert [O.fixed_width(O.LEVELS_UNIFORM, s) for s in (1, 2, 4, 8)] == [3, 4, 6, 10]
+
+
+# ---------------------------------------------------------------- ERC
+def _erc_len(n):
+    return 1 if n == 1 else n.bit_length() + _erc_len(n.bit_length() - 1)
+
+
+def test_erc_codewords_by_hand():
+    """Algorithm 2 executed by hand (tests/golden/erc_codewords.txt)."""
+    for n, word in golden_rows("erc_codewords.txt"):
+        assert O.erc_encode(int(n)) == word
+        assert O.erc_decode(word) == (int(n), len(word))
+
+
+def test_erc_lengths_and_round_trip():
+    # |ERC(N)| = floor(log2 N)+1 + |ERC(floor(log2 N))|, |ERC(1)| = 1  (App. A, property 1)
+    ns = list(range(1, 1 << 13)) + [2 ** k + j for k in range(13, 40) for j in (-1, 0, 1)]
+    for n in ns:
+        w = O.erc_encode(n)
+        assert len(w) == _erc_len(n)
+        assert O.erc_decode(w) == (n, len(w))
+        assert w[-1] == "0" and (n == 1 or w[0] == "1")
+    assert [_erc_len(n) for n in (32, 64, 128, 256, 65536)] == [12, 13, 14, 16, 28]
+
+
+def test_erc_prefix_free_concatenation():
+    # decoding without knowing an upper bound on N (App. A, property 3)
+    rng = np.random.default_rng(5)
+    vals = [int(v) for v in rng.integers(1, 5000, 400)] + [1, 1, 2, 1, 3]
+    s = "".join(O.erc_encode(v) for v in vals)
+    pos, out = 0, []
+    while pos < len(s):
+        v, pos = O.erc_decode(s, pos)
+        out.append(v)
+    assert out == vals
+    # a truncated string is reported, not misread
+    assert O.erc_decode(O.erc_encode(100)[:-3])[0] == 0
+
+
+def test_erc_is_prefix_code_small():
+    words = [O.erc_encode(n) for n in range(1, 600)]
+    assert len(set(words)) == len(words)
+    wl = sorted(words)
+    for a, b in zip(wl, wl[1:]):
+        assert not b.startswith(a)
+
+
+# ---------------------------------------------------------------- Philox
+def _curand_host(seed, n_words, offset=0):
+    try:
+        lib = ctypes.CDLL("libcurand.so.10")
+    except OSError:
+        try:
+            lib = ctypes.CDLL("/usr/local/cuda/lib64/libcurand.so.10")
+        except OSError:
+            pytest.skip("libcurand not available")
+    gen = ctypes.c_void_p()
+    if lib.curandCreateGeneratorHost(ctypes.byref(gen), 161) != 0:  # CURAND_RNG_PSEUDO_PHILOX4_32_10
+        pytest.skip("cuRAND host generator not available")
+    assert lib.curandSetPseudoRandomGeneratorSeed(gen, ctypes.c_ulonglong(seed)) == 0
+    assert lib.curandSetGeneratorOffset(gen, ctypes.c_ulonglong(offset)) == 0
+    out = np.zeros(n_words, np.uint32)
+    assert lib.curandGenerate(gen, out.ctypes.data_as(ctypes.c_void_p), ctypes.c_size_t(n_words)) == 0
+    lib.curandDestroyGenerator(gen)
+    return out
+
+
+def test_philox_against_curand_host_generator():
+    """An independent Philox4x32-10: cuRAND's host generator emits, as words 4n..4n+3 of its
+    sequence, the Philox output for the counter (m_lo, m_hi, n mod 2^16, 0), m = n div 2^16,
+    under key = seed (65536 interleaved subsequences)."""
+    def block(n, key):
+        m = n >> 16
+        return O.philox4x32_10([m & 0xFFFFFFFF, m >> 32, n & 0xFFFF, 0], key)
+
+    for seed in (0, 1, 0x0123456789ABCDEF, 0xFFFFFFFFFFFFFFFF):
+        key = [seed & 0xFFFFFFFF, seed >> 32]
+        ref = _curand_host(seed, 4 * 300)
+        assert np.array_equal(ref, np.concatenate([block(n, key) for n in range(300)]))
+        for first in (1, 7, 65534, 123456, (1 << 48) + 5, (0x2BCD << 48) + 0xFFFFFFFFFFFE):
+            ref = _curand_host(seed, 4 * 8, offset=4 * first)
+            assert np.array_equal(ref, np.concatenate([block(first + n, key) for n in range(8)])), (seed, first)
+
+
+def test_draw_mapping_and_uniformity():
+    seed, offset = 0xDEADBEEF12345678, 0x1_0000_0007
+    for i in (0, 1, 2, 3, 4, 5, 1023, (1 << 34) + 6):
+        q = i >> 2
+        blk = O.philox4x32_10([q & 0xFFFFFFFF, q >> 32, offset & 0xFFFFFFFF, offset >> 32],
+                              [seed & 0xFFFFFFFF, seed >> 32])
+        assert O.draw_word(seed, offset, i) == int(blk[i & 3])
+        assert O.draw_uniform(seed, offset, i) == (int(blk[i & 3]) >> 8) / 2.0 ** 24
+    # every counter and key word matters
+    base = O.philox4x32_10([1, 2, 3, 4], [5, 6])
+    for w in range(4):
+        c = [1, 2, 3, 4]; c[w] ^= 1
+        assert not np.array_equal(base, O.philox4x32_10(c, [5, 6]))
+    assert not np.array_equal(base, O.philox4x32_10([1, 2, 3, 4], [4, 6]))
+    assert not np.array_equal(base, O.philox4x32_10([1, 2, 3, 4], [5, 7]))
+    # u in [0,1), mean 1/2, variance 1/12, flat histogram
+    u = np.array([O.draw_uniform(7, 0, i) for i in range(200000)])
+    assert 0.0 <= u.min() and u.max() < 1.0
+    assert abs(u.mean() - 0.5) < 4 * math.sqrt(1 / 12 / u.size)
+    assert abs(u.var() - 1 / 12) < 2e-3
+    hist = np.histogram(u, bins=64, range=(0, 1))[0]
+    chi2 = ((hist - u.size / 64) ** 2 / (u.size / 64)).sum()
+    assert chi2 < 63 + 5 * math.sqrt(2 * 63)
+
+
+# ---------------------------------------------------------------- norm
+def test_norms():
+    rng = np.random.default_rng(1)
+    g = (rng.standard_normal(5000) * 10.0 ** rng.uniform(-6, 2, 5000)).astype(np.float32)
+    n = O.bucket_norms(g, 1024)
+    assert n.size == 5
+    for b in range(5):
+        seg = g[b * 1024:(b + 1) * 1024].astype(np.float64)
+        assert n[b] == np.float32(math.sqrt(float((seg * seg).sum()))) or \
+            abs(float(n[b]) - math.sqrt(float((seg * seg).sum()))) <= 1.2e-7 * float(n[b])
+    ninf = O.bucket_norms(g, 1024, O.NORM_LINF)
+    assert [float(x) for x in ninf] == [float(np.abs(g[b * 1024:(b + 1) * 1024]).max()) for b in range(5)]
+    assert O.norm(np.array([3.0, -4.0], np.float32)) == 5.0
+    assert O.norm(np.zeros(7, np.float32)) == 0.0
+
+
+# ---------------------------------------------------------------- Definition 1
+def _exact_split(v, nrm, s):
+    """lower level index and exact probability from the real-number definition:
+    r = |v|/||v||, l_j <= r <= l_{j+1}, p = (r - l_j)/(l_{j+1} - l_j)."""
+    r = Fraction(abs(float(v))) / Fraction(float(nrm))
+    lv = [Fraction(0)] + [Fraction(1, 2 ** (s + 1 - j)) for j in range(1, s + 2)]
+    j = max(k for k in range(s + 1) if lv[k] <= r)
+    return j, (r - lv[j]) / (lv[j + 1] - lv[j])
+
+
+def test_rounding_probability_matches_definition():
+    """App. B: p_1 = 2^s r on [0, 2^-s], p_2 = 2^(s-j) r - 1 on [2^(j-s), 2^(j+1-s)]."""
+    rng = np.random.default_rng(2)
+    for s in (1, 3, 4, 7):
+        for _ in range(300):
+            nrm = np.float32(10.0 ** rng.uniform(-3, 3))
+            v = np.float32(nrm * rng.uniform(0, 1) ** 3 * rng.choice([-1, 1]))
+            low, p = O.round_probability(v, nrm, s)
+            j, pe = _exact_split(v, nrm, s)
+            # fp32: one rounding in 2^s/norm and one in the product; the affine map is exact
+            assert abs(Fraction(float(p)) + low - (pe + j)) <= Fraction(3, 2 ** 24) * max(1, 2 ** j)
+            assert 0 <= p <= 1
+    # exact cases: r on a level and midway between levels
+    assert O.round_probability(0.25, 1.0, 3) in ((2, 0.0), (1, 1.0))
+    assert O.round_probability(0.1875, 1.0, 3) == (1, 0.5)     # midway between 1/8 and 1/4 (Fig. 1)
+    assert O.round_probability(-0.0625, 1.0, 3) == (0, 0.5)
+    assert O.round_probability(0.75, 1.0, 3) == (3, 0.5)
+    assert O.round_probability(1.0, 1.0, 3) == (3, 1.0)
+    assert O.round_probability(0.0, 1.0, 3) == (0, 0.0)
+
+
+def test_rounding_frequency_over_all_draws():
+    """Enumerate every 24-bit draw: #(u < p) = ceil(p 2^24); equal to p 2^24 when r >= 2^-s."""
+    u = (np.arange(1 << 24, dtype=np.float64) / 2.0 ** 24).astype(np.float32)
+    for s, v, nrm in ((3, 0.3, 1.0), (4, 0.01, 1.0), (3, 0.7, 2.0), (2, 1e-5, 0.003)):
+        v32, n32 = np.float32(v), np.float32(nrm)
+        low, p = O.round_probability(v32, n32, s)
+        sign, sym = O.quantize_with_draws(np.full(u.size, v32, np.float32), n32, s, O.LEVELS_EXP, u)
+        ups = int((sym == low + 1).sum())
+        assert int((sym == low).sum()) + ups == u.size
+        assert ups == math.ceil(Fraction(float(p)) * 2 ** 24)
+        if low >= 1:
+            assert Fraction(ups, 2 ** 24) == Fraction(float(p))
+        assert not sign.any()
+
+
+def test_unbiased_by_full_enumeration():
+    """Theorem 1, first claim: E[Q_s(v)] = v.  Enumerate all 2^d outcomes of a tiny vector."""
+    rng = np.random.default_rng(3)
+    for s, d in ((3, 8), (2, 10), (4, 6)):
+        v = (rng.standard_normal(d) * 10.0 ** rng.uniform(-2, 0, d)).astype(np.float32)
+        nrm = O.norm(v)
+        split = [O.round_probability(x, nrm, s) for x in v]
+        mean = [Fraction(0)] * d
+        total = Fraction(0)
+        for ups in itertools.product((0, 1), repeat=d):
+            u = np.array([0.0 if b else 0.99999994 for b in ups], np.float32)
+            pr = Fraction(1)
+            for b, (_, p) in zip(ups, split):
+                pr *= Fraction(float(p)) if b else 1 - Fraction(float(p))
+            if pr == 0:
+                continue
+            sign, sym = O.quantize_with_draws(v, nrm, s, O.LEVELS_EXP, u)
+            for i in range(d):
+                assert sym[i] == split[i][0] + (1 if (ups[i] and split[i][1] > 0) else 0)
+                q = O.dequantize(nrm, s, O.LEVELS_EXP, sign[i], sym[i])
+                mean[i] += pr * Fraction(float(q))
+            total += pr
+        assert total == 1
+        for i in range(d):
+            assert abs(float(mean[i]) - float(v[i])) <= 4e-7 * float(nrm)
+
+
+def test_unbiased_and_variance_monte_carlo():
+    """E[Q] = v and Lemma 7's closed form, on one N(0,1) bucket of 1024 with s = 3."""
+    v = np.random.default_rng(4).standard_normal(1024).astype(np.float32)
+    s, reps = 3, 4000
+    nrm = O.norm(v)
+    acc = np.zeros(1024)
+    err2 = np.zeros(reps)
+    for t in range(reps):
+        q = O.quantize_dequantize(v, 1024, s, O.NORM_L2, O.LEVELS_EXP, seed=1000 + t, offset=0).astype(np.float64)
+        acc += q
+        err2[t] = ((q - v) ** 2).sum()
+    var_cf = O.variance_closed_form(v, nrm, s)
+    # mean of err2 against the closed form, 4 standard errors
+    assert abs(err2.mean() - var_cf) < 4 * err2.std() / math.sqrt(reps)
+    # ||mean Q - v||^2 has expectation var_cf / reps
+    bias2 = ((acc / reps - v) ** 2).sum()
+    assert bias2 < 1.5 * var_cf / reps
+    assert bias2 > 0.5 * var_cf / reps          # and it is not suspiciously deterministic
+    # different offsets give different draws
+    a = O.quantize_dequantize(v, 1024, s, 0, 0, seed=1, offset=0)
+    b = O.quantize_dequantize(v, 1024, s, 0, 0, seed=1, offset=1)
+    assert not np.array_equal(a, b)
+
+
+def test_variance_closed_form_worked_examples():
+    """Lemma 7 on the all-equal vectors of Theorem 4 and Theorem 12."""
+    for d, s, frac in golden_rows("worked_examples.txt"):
+        d, s = int(d), int(s)
+        v = np.full(d, 0.37, np.float32)
+        nrm = O.norm(v)
+        got = O.variance_closed_form(v, nrm, s) / float(nrm) ** 2
+        assert abs(got - float(Fraction(frac))) < 2e-6 * max(1.0, float(Fraction(frac)))
+
+
+def _eps_q(d, s):
+    """Theorem 1's bound with the switch placed where its derivation puts it
+    (delta = sqrt(d)/2^s >= 2); never below the printed bound's first branch."""
+    delta = math.sqrt(d) / 2 ** s
+    return 1 / 8 + delta * delta / 4 if delta < 2 else delta - 7 / 8
+
+
+def test_variance_bound_theorem_1():
+    rng = np.random.default_rng(6)
+    for d, s in ((1024, 3), (8192, 4), (8192, 2), (512, 4), (64, 3)):
+        for kind in range(4):
+            if kind == 0:
+                v = rng.standard_normal(d)
+            elif kind == 1:
+                v = rng.standard_t(3, d)
+            elif kind == 2:
+                v = np.full(d, 1.0)
+            else:
+                v = rng.laplace(0, 1, d) * (rng.random(d) < 0.1)
+                v[0] = 1.0
+            v = v.astype(np.float32)
+            nrm = O.norm(v)
+            assert O.variance_closed_form(v, nrm, s) <= _eps_q(d, s) * float(nrm) ** 2 * (1 + 1e-6)
+    assert [round(_eps_q(b, s), 3) for b, s in ((1024, 3), (8192, 4), (8192, 3), (8192, 2), (65536, 4))] == \
+        [3.125, 4.782, 10.439, 21.752, 15.125]
+
+
+def test_sparsity_lemma_10():
+    """#{r_i > 2^-s} <= 2^(2s), and E||Q||_0 <= 2^(2s) + 2^s sqrt(d)."""
+    rng = np.random.default_rng(8)
+    for d, s in ((1024, 3), (8192, 4), (8192, 2)):
+        v = rng.standard_t(3, d).astype(np.float32)
+        nrm = float(O.norm(v))
+        r = np.abs(v.astype(np.float64)) / nrm
+        assert (r > 2.0 ** -s).sum() <= 2 ** (2 * s)
+        e_nnz = (r >= 2.0 ** -s).sum() + (2.0 ** s * r[r < 2.0 ** -s]).sum()
+        assert e_nnz <= 2 ** (2 * s) + 2 ** s * math.sqrt(d)
+        cnt = [np.count_nonzero(O.quantize(v, d, s, 0, 0, seed=t, offset=0)[1]) for t in range(200)]
+        assert abs(np.mean(cnt) - e_nnz) < 5 * math.sqrt(e_nnz / 200)
+
+
+def test_uniform_quantizer_definition():
+    """QSGD-style levels k/2^s: p = 2^s r - floor(2^s r); QSGD's variance bound min(d/s'^2, sqrt(d)/s')."""
+    assert O.round_probability(0.40625, 1.0, 4, O.LEVELS_UNIFORM) == (6, 0.5)
+    assert O.round_probability(1.0, 1.0, 4, O.LEVELS_UNIFORM) == (15, 1.0)
+    assert O.round_probability(0.01, 1.0, 4, O.LEVELS_UNIFORM)[0] == 0
+    v = np.random.default_rng(9).standard_normal(8192).astype(np.float32)
+    nrm = O.norm(v)
+    var = O.variance_closed_form(v, nrm, 4, O.LEVELS_UNIFORM) / float(nrm) ** 2
+    assert var <= min(8192 / 16 ** 2, math.sqrt(8192) / 16)
+    # L-infinity normalisation: r <= 1 exactly, the largest coordinate maps to the top level
+    ninf = O.norm(v, O.NORM_LINF)
+    sign, sym = O.quantize_bucket(v, ninf, 4, O.LEVELS_UNIFORM, 1, 0, 0)
+    assert sym.max() == 16 and sym[np.argmax(np.abs(v))] == 16
+    q = np.array([O.dequantize(ninf, 4, O.LEVELS_UNIFORM, a, b) for a, b in zip(sign, sym)])
+    assert np.abs(q - v).max() <= float(ninf) / 16 * (1 + 1e-6)
+
+
+def test_degenerate_buckets():
+    z = np.zeros(300, np.float32)
+    sign, sym, norms = O.quantize(z, 128, 3, 0, 0, 1, 0)
+    assert not sym.any() and not sign.any() and not norms.any()
+    v = np.ones(256, np.float32); v[7] = np.nan
+    assert not O.quantize(v, 256, 3, 0, 0, 1, 0)[1].any()
+    v[7] = np.inf
+    assert not O.quantize(v, 256, 3, 0, 0, 1, 0)[1].any()
+    v = np.full(256, 1e-42, np.float32)            # 2^s / norm overflows
+    assert not O.quantize(v, 256, 4, 0, 0, 1, 0)[1].any()
+    v = np.array([-0.0, 0.0, 1.0, -1.0], np.float32)
+    sign, sym, _ = O.quantize(v, 4, 3, 0, 0, 1, 0)
+    assert list(sym[:2]) == [0, 0] and list(sign[:2]) == [0, 0] and sign[3] == 1 and sign[2] == 0
