@@ -1,0 +1,139 @@
+/*
+ * nuq.h -- C ABI of the B200 (sm_100a) NUQSGD codec.
+ *
+ * The library implements the communication hot path of NUQSGD (arXiv
+ * 1908.06077): per-bucket norm, nonuniform stochastic quantization
+ * (Definition 1 with the level set (0, 2^-s, ..., 1/2, 1) of Sec. 3.1),
+ * ENCODE / DECODE with Elias recursive coding (App. A, Algorithm 2) and the
+ * aggregation sum of Algorithm 1, for K simulated workers on one GPU.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA global-memory addresses on the current device;
+ *     "host" pointers are ordinary process memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *   - Calls only enqueue work and return; argument errors are returned at once,
+ *     errors found by the kernels (malformed container, scan time-out) are
+ *     latched in a per-stream status word read by nuq_last_status().
+ *   - d = vector length, bucket = elements per norm bucket (Sec. 5, "bucket
+ *     size"), s = number of internal levels (Sec. 3.1).
+ *
+ * Limits: 1 <= d < 2^40; bucket a multiple of 256 with 256 <= bucket <= 8192,
+ * or bucket in {16384, 32768, 65536}; 1 <= s <= 14 (exponential levels) or
+ * 1 <= s <= 8 (uniform levels); 1 <= K <= 64.
+ *
+ * Container written by nuq_encode (all u32 words little endian; bit p of a bit
+ * string sits in word p>>5 at bit 31-(p&31)):
+ *   words 0..15   header: magic 'NUQ1', version, d (2 words), bucket, s,
+ *                 flags (norm | levels<<8 | mode<<16), 256, nblk (2),
+ *                 container_bits (2), code_bits (2), nnz (2)
+ *   ERC mode      (nblk+1) u64 bit offsets of the coding blocks, relative to
+ *                 the payload that follows the table.  A coding block is up to
+ *                 8192 consecutive elements of one bucket: norm (fp32 bits) |
+ *                 one u16 token-bit count per 256-element sub-block (padded to
+ *                 a word) | the sub-blocks' token strings back to back | zero
+ *                 padding to a word.  A token is ERC(gap) sign ERC(level
+ *                 index); the gap is counted from the start of the sub-block.
+ *   fixed mode    per bucket: norm word | fields of w bits (sign, level index)
+ *                 MSB first | zero padding to a word; no table.
+ */
+#ifndef NUQ_H_
+#define NUQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int nuq_status;
+#define NUQ_OK 0
+#define NUQ_ERR_INVALID_ARG (-1) /* null / misaligned pointer, size or parameter out of range      */
+#define NUQ_ERR_CAPACITY (-2)    /* reserved: output capacity too small                            */
+#define NUQ_ERR_BAD_STREAM (-3)  /* a container failed validation inside nuq_decode_accumulate     */
+#define NUQ_ERR_CUDA (-4)        /* a CUDA runtime call failed (allocation, launch)                */
+#define NUQ_ERR_TIMEOUT (-5)     /* the encoder's cross-tile scan gave up waiting (bounded spin)   */
+
+/* norm_kind argument of nuq_encode: bit fields */
+#define NUQ_NORM_L2 0u            /* bits 0-7: Euclidean norm (Sec. 2), the paper's choice        */
+#define NUQ_NORM_LINF 1u          /*           max-abs norm (QSGDinf comparison, Sec. 1)          */
+#define NUQ_LEVELS_EXP (0u << 8)  /* bits 8-15: levels (0, 2^-s, ..., 1/2, 1)  (Sec. 3.1)         */
+#define NUQ_LEVELS_UNIFORM (1u << 8) /*         levels k / 2^s, k = 0..2^s    (QSGD comparison)   */
+#define NUQ_MODE_ERC (0u << 16)   /* bits 16-23: Elias-recursive token stream (App. A)            */
+#define NUQ_MODE_FIXED (1u << 16) /*             fixed-width fields ("4-bit" variant of Sec. 5)   */
+#define NUQ_TEST_NORMS (1u << 24) /* take bucket norms from nuq_set_test_norms (parity testing)   */
+
+typedef struct nuq_info {
+    uint64_t d;
+    uint32_t bucket;
+    uint32_t s;
+    uint32_t flags;          /* norm | levels<<8 | mode<<16 */
+    uint32_t sub_block;      /* 256 */
+    uint64_t nblk;           /* coding blocks (ERC) or buckets (fixed) */
+    uint64_t container_bits; /* what a sender would transmit */
+    uint64_t code_bits;      /* token bits only (ERC) or d*w (fixed) */
+    uint64_t nnz;            /* coordinates quantized to a nonzero level */
+} nuq_info;
+
+/*
+ * c <- ENCODE(g)   (Algorithm 1, encode line; App. A; Definition 1).
+ *
+ * Splits g into buckets of `bucket` elements (the last may be short), takes
+ * each bucket's norm, quantizes every coordinate stochastically to the level
+ * set and writes the container described above.  Coordinate i (0-based within
+ * this call) draws u = (w >> 8) * 2^-24 from word (i & 3) of
+ * Philox4x32-10(key = seed, counter = (i >> 2, offset)) and moves to the upper
+ * level iff u < p(r_i), so equal (seed, offset) reproduce the stream exactly.
+ *
+ *   g         device, d floats, 16-byte aligned; read only
+ *   out       device, 16-byte aligned, at least nuq_encode_bound() bytes; need
+ *             not be zeroed; fully owned by the caller
+ *   out_bits  device u64 (may be NULL): receives container_bits
+ *   returns   NUQ_ERR_INVALID_ARG for bad arguments, NUQ_ERR_CUDA if the
+ *             per-stream workspace cannot be allocated or a launch fails.
+ * The call may allocate (and then synchronise the device) when the per-stream
+ * workspace has to grow; otherwise it is asynchronous.
+ */
+nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
+                      uint64_t offset, void* out, uint64_t* out_bits, void* stream);
+
+/*
+ * acc <- sum_k DECODE(c_k)   (Algorithm 1, decode and aggregation lines,
+ * without the alpha/K factor; App. A decoding).
+ *
+ *   streams  HOST array of K device pointers to containers written by
+ *            nuq_encode with the same (d, bucket, s); each buffer must hold
+ *            the container_bits its header declares.  The array is copied at
+ *            call time.
+ *   acc      device, d floats, 16-byte aligned; OVERWRITTEN with
+ *            ((0 + q_0[i]) + q_1[i]) + ... in fp32, k ascending.
+ * Each container's header, offsets, lengths and tokens are validated on the
+ * device; a violation latches NUQ_ERR_BAD_STREAM (the affected coordinates of
+ * acc are then unspecified, nothing outside acc[0..d) is written).
+ */
+nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
+                                 float* acc, void* stream);
+
+/* Bytes that `out` of nuq_encode must hold for these arguments (0 if they are invalid). */
+uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind);
+
+/* Parity-test hook: device array of ceil(d/bucket) bucket norms that nuq_encode uses in
+ * place of its own reduction when NUQ_TEST_NORMS is set; NULL clears it.  The pointer is
+ * kept, not copied.                                                                        */
+nuq_status nuq_set_test_norms(const float* norms);
+
+/* Synchronises `stream` and returns, then clears, the status latched by the kernels that
+ * ran on it since the last call (NUQ_OK, NUQ_ERR_BAD_STREAM, NUQ_ERR_TIMEOUT).            */
+nuq_status nuq_last_status(void* stream);
+
+/* Copies the header of a container (device) into *host_out; synchronises `stream`.        */
+nuq_status nuq_stream_info(const void* out, nuq_info* host_out, void* stream);
+
+/* Frees every per-stream workspace of the library. */
+void nuq_shutdown(void);
+
+const char* nuq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NUQ_H_ */

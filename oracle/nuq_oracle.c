@@ -454,6 +454,7 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
     if (check_args(d, bucket, s, flags & 0xff, levelset, mode) != ORC_OK) return ORC_ERR_STREAM;
     uint64_t nb = (d + bucket - 1) / bucket;
     uint64_t nblk = (uint64_t)words[8] | ((uint64_t)words[9] << 32);
+    uint64_t container_bits = (uint64_t)words[10] | ((uint64_t)words[11] << 32);
     uint32_t nlev = nuq_oracle_num_levels(levelset, s);
     uint32_t w = nuq_oracle_fixed_width(levelset, s);
     memset(sign, 0, (size_t)d);
@@ -461,6 +462,10 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
 
     if (mode == MODE_FIXED) {
         if (nblk != nb) return ORC_ERR_STREAM;
+        uint64_t last = d - (nb - 1) * (uint64_t)bucket;
+        if (container_bits != 32u * (ORC_HEADER_WORDS + (nb - 1) * (1 + ((uint64_t)bucket * w + 31) / 32) +
+                                     1 + (last * w + 31) / 32))
+            return ORC_ERR_STREAM;
         const uint32_t* payload = words + ORC_HEADER_WORDS;
         for (uint64_t b = 0; b < nb; ++b) {
             uint64_t lo = b * (uint64_t)bucket, n = lo + bucket < d ? bucket : d - lo;
@@ -482,6 +487,7 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
     if (nblk != count_blocks(d, bucket)) return ORC_ERR_STREAM;
     const uint64_t* table = (const uint64_t*)(words + ORC_HEADER_WORDS);
     const uint32_t* payload = words + ORC_HEADER_WORDS + 2 * (nblk + 1);
+    if (container_bits != 32u * (ORC_HEADER_WORDS + 2 * (nblk + 1)) + table[nblk]) return ORC_ERR_STREAM;
     uint64_t blk = 0;
     for (uint64_t b = 0; b < nb; ++b) {
         uint64_t lo = b * (uint64_t)bucket, n = lo + bucket < d ? bucket : d - lo;

@@ -1,0 +1,280 @@
+// C ABI of the library (see include/nuq.h): argument validation, geometry,
+// per-stream workspace, kernel launches.  No torch types, no CPU fallback: every
+// step of the path runs in the kernels of nuq_encode.cu / nuq_decode.cu.
+#include <map>
+#include <mutex>
+#include <set>
+#include <utility>
+
+#include "../../include/nuq.h"
+#include "nuq_common.cuh"
+#include "nuq_launch.h"
+
+namespace nuq {
+namespace {
+
+struct WsEntry {
+    Workspace* ptr = nullptr;
+    size_t bytes = 0;
+};
+
+std::mutex g_mu;
+std::map<std::pair<int, cudaStream_t>, WsEntry> g_ws;
+std::map<int, int> g_sms;                 // device -> SM count
+std::set<int> g_lut_ready;                // devices whose constant LUT is uploaded
+const float* g_test_norms = nullptr;
+uint32_t g_erc_len[256];
+bool g_erc_len_ready = false;
+
+uint32_t erc_len(uint32_t n) {            // |ERC(n)|, 1 <= n <= 256
+    if (!g_erc_len_ready) {
+        uint32_t lut[256];
+        build_erc_lut(lut);
+        for (int i = 0; i < 256; ++i) g_erc_len[i] = lut[i] >> 16;
+        g_erc_len_ready = true;
+    }
+    return g_erc_len[n - 1];
+}
+
+bool bucket_ok(uint32_t bucket) {
+    if (bucket >= kSB && bucket <= kBLK) return bucket % kSB == 0;
+    return bucket == 16384u || bucket == 32768u || bucket == 65536u;
+}
+
+bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geometry* G) {
+    const uint32_t norm_kind = flags & 0xffu, levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
+    if (d == 0 || d >= (1ull << 40) || !bucket_ok(bucket) || s < 1) return false;
+    if (norm_kind > 1 || levelset > 1 || mode > 1) return false;
+    if (s > (levelset == kLevelsExp ? 14u : 8u)) return false;
+    if (flags & ~(0x00ffffffu | NUQ_TEST_NORMS)) return false;
+    G->d = d;
+    G->bucket = bucket;
+    G->s = s;
+    G->norm_kind = norm_kind;
+    G->levelset = levelset;
+    G->mode = mode;
+    G->nb = (d + bucket - 1) / bucket;
+    G->nlev = levelset == kLevelsExp ? s + 2u : (1u << s) + 1u;
+    uint32_t b = 0;
+    while ((1u << b) < G->nlev) ++b;
+    G->width = b + 1u;
+    G->rec_words = 1u + (uint32_t)(((uint64_t)bucket * G->width + 31) / 32);
+    const uint64_t last = d - (G->nb - 1) * bucket;
+    if (bucket <= kBLK) {
+        G->blocks_per_tile = kBLK / bucket;
+        G->tile_elems = G->blocks_per_tile * bucket;
+        G->sb_per_block = bucket / kSB;
+        G->blk_per_bucket = 1;
+        G->nblk = G->nb;
+        G->ntiles = (G->nb + G->blocks_per_tile - 1) / G->blocks_per_tile;
+    } else {
+        G->blocks_per_tile = 1;
+        G->tile_elems = kBLK;
+        G->sb_per_block = 32;
+        G->blk_per_bucket = bucket / kBLK;
+        G->nblk = (G->nb - 1) * G->blk_per_bucket + (last + kBLK - 1) / kBLK;
+        G->ntiles = G->nblk;
+    }
+    return true;
+}
+
+uint32_t max_level_code_bits(const Geometry& G) {
+    uint32_t best = 0;
+    for (uint32_t sym = 1; sym < G.nlev; ++sym) best = erc_len(sym) > best ? erc_len(sym) : best;
+    return best;
+}
+
+// words of shared-memory staging one tile can need
+uint32_t stage_words_for(const Geometry& G) {
+    if (G.mode == kModeFixed) return G.bucket <= kBLK ? G.blocks_per_tile * G.rec_words : kBLK * G.width / 32u;
+    uint32_t head = 1u + (G.sb_per_block + 1u) / 2u + 1u;          // norm, lengths, padding
+    return G.blocks_per_tile * head + (kBLK * (2u + max_level_code_bits(G)) + 31u) / 32u;
+}
+
+uint64_t bound_bytes(const Geometry& G) {
+    if (G.mode == kModeFixed) return 4ull * (kHeaderWords + G.nb * G.rec_words);
+    uint64_t head = 1u + (G.sb_per_block + 1u) / 2u + 1u;
+    uint64_t token_words = (G.d * (2ull + max_level_code_bits(G)) + 31) / 32;
+    return 4ull * (kHeaderWords + 2 * (G.nblk + 1) + G.nblk * head + token_words);
+}
+
+int device_sms(int dev) {
+    auto it = g_sms.find(dev);
+    if (it != g_sms.end()) return it->second;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    g_sms[dev] = sms;
+    return sms;
+}
+
+// Workspace of (current device, stream), grown to `bytes`.  Growing synchronises the stream.
+nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int* dev_out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    *dev_out = dev;
+    WsEntry& e = g_ws[std::make_pair(dev, stream)];
+    if (e.bytes < bytes) {
+        int carried = 0;
+        if (e.ptr) {
+            if (cudaStreamSynchronize(stream) != cudaSuccess) return NUQ_ERR_CUDA;
+            if (cudaMemcpy(&carried, &e.ptr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
+            cudaFree(e.ptr);
+            e.ptr = nullptr;
+            e.bytes = 0;
+        }
+        size_t want = bytes + bytes / 2;
+        void* p = nullptr;
+        if (cudaMalloc(&p, want) != cudaSuccess) { cudaGetLastError(); return NUQ_ERR_CUDA; }
+        if (cudaMemset(p, 0, want) != cudaSuccess) return NUQ_ERR_CUDA;
+        e.ptr = static_cast<Workspace*>(p);
+        e.bytes = want;
+        if (carried && cudaMemcpy(&e.ptr->status, &carried, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
+            return NUQ_ERR_CUDA;
+    }
+    *out = e.ptr;
+    return NUQ_OK;
+}
+
+}  // namespace
+}  // namespace nuq
+
+using namespace nuq;
+
+extern "C" {
+
+uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    Geometry G;
+    if (!make_geometry(d, bucket, s, norm_kind, &G)) return 0;
+    return (bound_bytes(G) + 15) & ~15ull;
+}
+
+nuq_status nuq_set_test_norms(const float* norms) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    g_test_norms = norms;
+    return NUQ_OK;
+}
+
+nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
+                      uint64_t offset, void* out, uint64_t* out_bits, void* stream_) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    EncodeParams P;
+    Geometry& G = P.geo;
+    if (!g || !out || !make_geometry(d, bucket, s, norm_kind, &G)) return NUQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u) ||
+        (reinterpret_cast<uintptr_t>(out_bits) & 7u))
+        return NUQ_ERR_INVALID_ARG;
+    const bool test_norms = (norm_kind & NUQ_TEST_NORMS) != 0;
+    if (test_norms && !g_test_norms) return NUQ_ERR_INVALID_ARG;
+
+    const bool wide = bucket > kBLK;
+    const size_t state_bytes = sizeof(Workspace) + 8 * G.ntiles;
+    const size_t ws_bytes = state_bytes + (wide ? 4 * G.nb : 0);
+    Workspace* ws = nullptr;
+    int dev = 0;
+    nuq_status st = get_workspace(stream, ws_bytes, &ws, &dev);
+    if (st != NUQ_OK) return st;
+    if (!g_lut_ready.count(dev)) {
+        if (upload_erc_lut() != cudaSuccess) return NUQ_ERR_CUDA;
+        g_lut_ready.insert(dev);
+    }
+    if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, state_bytes - kWorkspaceClearFrom, stream) !=
+        cudaSuccess)
+        return NUQ_ERR_CUDA;
+
+    P.g = g;
+    P.norms_in = nullptr;
+    if (test_norms) {
+        P.norms_in = g_test_norms;
+    } else if (wide) {
+        float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + state_bytes);
+        if (launch_bucket_norms(g, d, bucket, G.norm_kind, norms, G.nb, stream) != cudaSuccess) return NUQ_ERR_CUDA;
+        P.norms_in = norms;
+    }
+    P.out = static_cast<uint32_t*>(out);
+    P.out_bits = out_bits;
+    P.ws = ws;
+    P.seed = seed;
+    P.offset = offset;
+    P.stage_words = stage_words_for(G);
+    if (launch_encode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    return NUQ_OK;
+}
+
+nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
+                                 float* acc, void* stream_) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    DecodeParams P;
+    if (!streams || !acc || K < 1 || K > kMaxK) return NUQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(acc) & 15u) return NUQ_ERR_INVALID_ARG;
+    // the level set and mode come from each container's header; geometry only needs (d, bucket, s)
+    if (!make_geometry(d, bucket, s, 0, &P.geo)) return NUQ_ERR_INVALID_ARG;
+    for (uint32_t k = 0; k < K; ++k) {
+        if (!streams[k] || (reinterpret_cast<uintptr_t>(streams[k]) & 15u)) return NUQ_ERR_INVALID_ARG;
+        P.streams[k] = static_cast<const uint32_t*>(streams[k]);
+    }
+    for (uint32_t k = K; k < kMaxK; ++k) P.streams[k] = nullptr;
+    P.K = K;
+    P.acc = acc;
+    Workspace* ws = nullptr;
+    int dev = 0;
+    nuq_status st = get_workspace(stream, sizeof(Workspace), &ws, &dev);
+    if (st != NUQ_OK) return st;
+    P.ws = ws;
+    if (launch_decode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    return NUQ_OK;
+}
+
+nuq_status nuq_last_status(void* stream_) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    auto it = g_ws.find(std::make_pair(dev, stream));
+    if (it == g_ws.end() || !it->second.ptr) return NUQ_OK;
+    int status = 0;
+    if (cudaMemcpy(&status, &it->second.ptr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (status != 0 && cudaMemset(&it->second.ptr->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
+    return status;
+}
+
+nuq_status nuq_stream_info(const void* out, nuq_info* host_out, void* stream_) {
+    if (!out || !host_out) return NUQ_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    uint32_t h[kHeaderWords];
+    if (cudaMemcpyAsync(h, out, sizeof(h), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (h[0] != kMagic || h[1] != kVersion) return NUQ_ERR_BAD_STREAM;
+    auto u64 = [&](int i) { return (uint64_t)h[i] | ((uint64_t)h[i + 1] << 32); };
+    host_out->d = u64(2);
+    host_out->bucket = h[4];
+    host_out->s = h[5];
+    host_out->flags = h[6];
+    host_out->sub_block = h[7];
+    host_out->nblk = u64(8);
+    host_out->container_bits = u64(10);
+    host_out->code_bits = u64(12);
+    host_out->nnz = u64(14);
+    return NUQ_OK;
+}
+
+void nuq_shutdown(void) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    int cur = 0;
+    cudaGetDevice(&cur);
+    for (auto& kv : g_ws) {
+        if (kv.second.ptr) {
+            cudaSetDevice(kv.first.first);
+            cudaFree(kv.second.ptr);
+        }
+    }
+    g_ws.clear();
+    cudaSetDevice(cur);
+}
+
+const char* nuq_version(void) { return "nuq-b200 0.1 (sm_100a)"; }
+
+}  // extern "C"

@@ -1,0 +1,88 @@
+// Shared definitions of the CUDA side: container constants, kernel parameter
+// blocks, small device helpers.  Nothing here is used by the CPU oracle.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace nuq {
+
+constexpr uint32_t kMagic = 0x3151554Eu;  // 'N','U','Q','1'
+constexpr uint32_t kVersion = 1u;
+constexpr uint32_t kSB = 256;             // elements per coding sub-block (one warp pass, 8 per lane)
+constexpr uint32_t kBLK = 32 * kSB;       // elements per coding block / per tile
+constexpr uint32_t kHeaderWords = 16;
+constexpr uint32_t kMaxK = 64;
+
+constexpr int kEncThreads = 256;          // 8 warps, 4 sub-blocks each
+constexpr int kEncWarps = kEncThreads / 32;
+constexpr int kSbPerWarp = 32 / kEncWarps;
+
+enum : uint32_t { kNormL2 = 0, kNormLinf = 1 };
+enum : uint32_t { kLevelsExp = 0, kLevelsUniform = 1 };
+enum : uint32_t { kModeErc = 0, kModeFixed = 1 };
+
+// status latched by kernels (most negative wins)
+enum : int { kOk = 0, kErrBadStream = -3, kErrTimeout = -5 };
+
+// look-back tile states, kept in the two top bits of a 64-bit word
+constexpr uint64_t kTileAggregate = 1ull << 62;
+constexpr uint64_t kTilePrefix = 2ull << 62;
+constexpr uint64_t kTilePoison = 3ull << 62;
+constexpr uint64_t kTileValueMask = (1ull << 62) - 1;
+
+// per-stream scratch owned by the library
+struct Workspace {
+    int status;             // latched kernel status; survives calls until nuq_last_status reads it
+    int pad;
+    // everything below is cleared at the start of every encode call
+    uint64_t ticket;        // next tile to hand out
+    uint64_t done;          // tiles finished
+    uint64_t code_bits;     // token bits of the whole call
+    uint64_t nnz;           // nonzero symbols of the whole call
+    uint64_t total_words;   // payload words of the whole call
+    uint64_t reserved[2];
+    // followed by: uint64_t tile_state[ntiles], then float norms[nb] for wide buckets
+};
+constexpr size_t kWorkspaceClearFrom = 8;
+
+struct Geometry {
+    uint64_t d;
+    uint64_t nb;             // buckets
+    uint64_t nblk;           // coding blocks (ERC) == table entries - 1
+    uint64_t ntiles;         // CTAs' work items (<= 8192 elements each)
+    uint32_t bucket;
+    uint32_t s;
+    uint32_t norm_kind, levelset, mode;
+    uint32_t tile_elems;     // elements a full tile covers
+    uint32_t blocks_per_tile;// buckets per tile when bucket <= 8192, else 1
+    uint32_t sb_per_block;   // sub-blocks of a full coding block
+    uint32_t blk_per_bucket; // coding blocks of a full bucket (1 when bucket <= 8192)
+    uint32_t nlev;           // number of levels including zero
+    uint32_t width;          // fixed-mode bits per element
+    uint32_t rec_words;      // fixed mode: words per full bucket record
+};
+
+struct EncodeParams {
+    Geometry geo;
+    const float* g;
+    const float* norms_in;   // bucket norms to use, or nullptr
+    uint32_t* out;
+    uint64_t* out_bits;
+    Workspace* ws;
+    uint64_t seed, offset;
+    uint32_t stage_words;    // capacity of the shared-memory staging buffer
+};
+
+struct DecodeParams {
+    Geometry geo;
+    const uint32_t* streams[kMaxK];
+    uint32_t K;
+    float* acc;
+    Workspace* ws;
+};
+
+__device__ __forceinline__ void latch_status(Workspace* ws, int code) { atomicMin(&ws->status, code); }
+
+__device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
+
+}  // namespace nuq

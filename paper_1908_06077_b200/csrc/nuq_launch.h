@@ -1,0 +1,17 @@
+// Host-side entry points of the kernel translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "nuq_common.cuh"
+
+namespace nuq {
+
+void build_erc_lut(uint32_t* lut256);                 // ERC(N), N = 1..256: code | len << 16
+cudaError_t upload_erc_lut();                         // into the current device's constant memory
+cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uint32_t norm_kind, float* norms,
+                                uint64_t nb, cudaStream_t stream);
+cudaError_t launch_encode(const EncodeParams& P, int sms, cudaStream_t stream);
+cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream);
+
+}  // namespace nuq

@@ -1,0 +1,133 @@
+"""Thin ctypes binding of libnuq.so: argument marshalling only.
+
+Every function has the name and the argument order of its C counterpart in
+include/nuq.h; tensors are passed as raw device pointers and the current torch
+CUDA stream is used unless one is given.  There is no CPU path: importing this
+module fails if the CUDA library cannot be built or loaded.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+NUQ_OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BAD_STREAM, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+NORM_L2, NORM_LINF = 0, 1
+LEVELS_EXP, LEVELS_UNIFORM = 0 << 8, 1 << 8
+MODE_ERC, MODE_FIXED = 0 << 16, 1 << 16
+TEST_NORMS = 1 << 24
+HEADER_WORDS = 16
+
+
+class NuqError(RuntimeError):
+    def __init__(self, where, code):
+        super().__init__(f"{where} failed with status {code}")
+        self.code = code
+
+
+class _Info(C.Structure):
+    _fields_ = [("d", C.c_uint64), ("bucket", C.c_uint32), ("s", C.c_uint32), ("flags", C.c_uint32),
+                ("sub_block", C.c_uint32), ("nblk", C.c_uint64), ("container_bits", C.c_uint64),
+                ("code_bits", C.c_uint64), ("nnz", C.c_uint64)]
+
+
+def _load():
+    path = _build.LIB
+    if not os.path.exists(path):
+        _build.build()
+    lib = C.CDLL(path)
+    lib.nuq_encode.restype = C.c_int
+    lib.nuq_encode.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
+                               C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.nuq_decode_accumulate.restype = C.c_int
+    lib.nuq_decode_accumulate.argtypes = [C.POINTER(C.c_void_p), C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32,
+                                          C.c_void_p, C.c_void_p]
+    lib.nuq_encode_bound.restype = C.c_uint64
+    lib.nuq_encode_bound.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
+    lib.nuq_set_test_norms.restype = C.c_int
+    lib.nuq_set_test_norms.argtypes = [C.c_void_p]
+    lib.nuq_last_status.restype = C.c_int
+    lib.nuq_last_status.argtypes = [C.c_void_p]
+    lib.nuq_stream_info.restype = C.c_int
+    lib.nuq_stream_info.argtypes = [C.c_void_p, C.POINTER(_Info), C.c_void_p]
+    lib.nuq_shutdown.restype = None
+    lib.nuq_shutdown.argtypes = []
+    lib.nuq_version.restype = C.c_char_p
+    lib.nuq_version.argtypes = []
+    return lib
+
+
+_lib = _load()
+LIBRARY_PATH = _build.LIB
+
+
+def _stream(stream):
+    if stream is None:
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, torch.cuda.Stream):
+        return C.c_void_p(stream.cuda_stream)
+    return C.c_void_p(int(stream))
+
+
+def version() -> str:
+    return _lib.nuq_version().decode()
+
+
+def encode_bound(d, bucket, s, norm_kind=0) -> int:
+    return int(_lib.nuq_encode_bound(d, bucket, s, norm_kind))
+
+
+def set_test_norms(norms: torch.Tensor | None):
+    """norms: CUDA float32 tensor of ceil(d/bucket) bucket norms (kept by reference), or None."""
+    rc = _lib.nuq_set_test_norms(C.c_void_p(norms.data_ptr()) if norms is not None else None)
+    if rc != NUQ_OK:
+        raise NuqError("nuq_set_test_norms", rc)
+
+
+def encode(g: torch.Tensor, bucket, s, norm_kind=0, seed=0, offset=0, out=None, out_bits=None, stream=None):
+    """c <- ENCODE(g).  Returns (out, out_bits): the container as an int32 CUDA tensor of
+    nuq_encode_bound bytes and a one-element int64 CUDA tensor that receives container_bits."""
+    assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()
+    d = g.numel()
+    if out is None:
+        nbytes = encode_bound(d, bucket, s, norm_kind)
+        if nbytes == 0:
+            raise NuqError("nuq_encode_bound", ERR_INVALID_ARG)
+        out = torch.empty(nbytes // 4, dtype=torch.int32, device=g.device)
+    if out_bits is None:
+        out_bits = torch.empty(1, dtype=torch.int64, device=g.device)
+    rc = _lib.nuq_encode(C.c_void_p(g.data_ptr()), d, bucket, s, norm_kind, seed, offset, C.c_void_p(out.data_ptr()),
+                         C.c_void_p(out_bits.data_ptr()), _stream(stream))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_encode", rc)
+    return out, out_bits
+
+
+def decode_accumulate(streams, d, bucket, s, acc=None, stream=None):
+    """acc <- sum_k DECODE(streams[k]); acc is overwritten."""
+    if acc is None:
+        acc = torch.empty(d, dtype=torch.float32, device=streams[0].device)
+    ptrs = (C.c_void_p * len(streams))(*[C.c_void_p(t.data_ptr()) for t in streams])
+    rc = _lib.nuq_decode_accumulate(ptrs, len(streams), d, bucket, s, C.c_void_p(acc.data_ptr()), _stream(stream))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_decode_accumulate", rc)
+    return acc
+
+
+def last_status(stream=None) -> int:
+    return int(_lib.nuq_last_status(_stream(stream)))
+
+
+def stream_info(out: torch.Tensor, stream=None) -> dict:
+    info = _Info()
+    rc = _lib.nuq_stream_info(C.c_void_p(out.data_ptr()), C.byref(info), _stream(stream))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_stream_info", rc)
+    return {k: int(getattr(info, k)) for k, _ in _Info._fields_}
+
+
+def shutdown():
+    _lib.nuq_shutdown()

@@ -1,0 +1,177 @@
+"""Element-by-element parity of the CUDA path (through the C ABI) with the CPU
+oracle on seeded inputs: sizes span several tiles and ragged tails."""
+import numpy as np
+import pytest
+
+import oracle as O
+from gpu_util import compare_symbols, gpu_decode, gpu_encode, require_cuda
+
+pytestmark = pytest.mark.gpu
+
+L2, LINF = O.NORM_L2, O.NORM_LINF
+EXP, UNI = O.LEVELS_EXP, O.LEVELS_UNIFORM
+
+# (d, bucket, s, norm, levels)
+CASES = [
+    (65536, 1024, 3, L2, EXP),
+    (100037, 8192, 4, L2, EXP),
+    (20000, 512, 4, L2, EXP),
+    (3 * 8192 + 5, 256, 2, L2, EXP),
+    (70000, 768, 3, L2, EXP),
+    (200000, 65536, 4, L2, EXP),
+    (150001, 16384, 4, L2, EXP),
+    (40000, 8192, 14, L2, EXP),
+    (40000, 2048, 1, L2, EXP),
+    (50000, 8192, 4, L2, UNI),
+    (50000, 8192, 4, LINF, UNI),
+    (30000, 4096, 8, L2, UNI),
+    (90000, 32768, 3, LINF, EXP),
+    (1, 512, 4, L2, EXP),
+    (255, 256, 3, L2, EXP),
+    (256, 256, 3, L2, EXP),
+    (257, 256, 3, L2, EXP),
+    (8193, 8192, 4, L2, EXP),
+]
+
+
+def _input(d, seed):
+    rng = np.random.default_rng(seed)
+    g = rng.standard_normal(d) * 10.0 ** rng.uniform(-4, 0, d)
+    g[rng.random(d) < 0.02] = 0.0
+    return g.astype(np.float32)
+
+
+@pytest.mark.parametrize("d,bucket,s,nk,ls", CASES)
+@pytest.mark.parametrize("mode", [O.MODE_ERC, O.MODE_FIXED])
+def test_bitstream_exact_with_oracle_norms(d, bucket, s, nk, ls, mode):
+    """Fed the oracle's bucket norms, the GPU container equals the oracle's bit for bit."""
+    flags = O.make_flags(nk, ls, mode)
+    g = _input(d, d + s)
+    norms = O.bucket_norms(g, bucket, nk)
+    want, want_bits = O.encode(g, bucket, s, flags, seed=11, offset=3, norms=norms)
+    got, got_bits = gpu_encode(g, bucket, s, flags, seed=11, offset=3, norms=norms)
+    assert got_bits == want_bits
+    assert np.array_equal(got[:16], want[:16]), "header"
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("d,bucket,s,nk,ls", CASES)
+def test_free_running_encode_matches_oracle(d, bucket, s, nk, ls):
+    """The GPU's own norms agree to 1e-6; signs and levels are equal except within 1e-6 of a threshold."""
+    flags = O.make_flags(nk, ls, O.MODE_ERC)
+    g = _input(d, 7 * d + s)
+    got, _ = gpu_encode(g, bucket, s, flags, seed=5, offset=0)
+    compare_symbols(g, bucket, s, flags, 5, 0, got)
+    got_fixed, _ = gpu_encode(g, bucket, s, O.make_flags(nk, ls, O.MODE_FIXED), seed=5, offset=0)
+    compare_symbols(g, bucket, s, flags, 5, 0, got_fixed)
+
+
+@pytest.mark.parametrize("d,bucket,s,nk,ls", CASES)
+@pytest.mark.parametrize("K", [1, 3])
+def test_decode_accumulate_matches_oracle(d, bucket, s, nk, ls, K):
+    """GPU decode of oracle-written containers equals the oracle's ordered sum bit for bit."""
+    streams = []
+    for k in range(K):
+        mode = O.MODE_FIXED if (k == 1) else O.MODE_ERC          # mixed modes in one call
+        g = _input(d, 1000 * k + d)
+        streams.append(O.encode(g, bucket, s, O.make_flags(nk, ls, mode), seed=k + 1, offset=0)[0])
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_c1_end_to_end():
+    """Config C1: encode on the GPU, decode on the GPU, against the oracle end to end."""
+    from paper_1908_06077_b200 import inputs
+    g = inputs.c1_input()
+    got, bits = gpu_encode(g, 1024, 3, 0, seed=0, offset=0)
+    nbad, nrel = compare_symbols(g, 1024, 3, 0, 0, 0, got)
+    want, _ = O.encode(g, 1024, 3, 0, 0, 0)
+    if nbad == 0 and nrel == 0.0:
+        assert np.array_equal(got, want)
+    acc = gpu_decode([got], g.size, 1024, 3)
+    rc, ref = O.decode_accumulate([want], g.size, 1024, 3)
+    err = np.linalg.norm(acc.astype(np.float64) - ref) / np.linalg.norm(ref)
+    assert err <= 1e-5
+
+
+def test_encode_is_deterministic_and_ignores_stale_output():
+    g = _input(300000, 1)
+    a, _ = gpu_encode(g, 8192, 4, 0, 9, 2)
+    b, _ = gpu_encode(g, 8192, 4, 0, 9, 2, prefill=0x7FFFFFFF)
+    c, _ = gpu_encode(g, 8192, 4, 0, 9, 3)
+    assert np.array_equal(a, b)
+    assert not np.array_equal(a, c)
+
+
+def test_stream_info_and_status():
+    torch, nuq = require_cuda()
+    g = torch.from_numpy(_input(50000, 2)).cuda()
+    out, bits = nuq.encode(g, 1024, 3, 0, 1, 0)
+    info = nuq.stream_info(out)
+    assert info["d"] == 50000 and info["bucket"] == 1024 and info["s"] == 3 and info["sub_block"] == 256
+    assert info["container_bits"] == int(bits.item()) and info["nblk"] == 49
+    assert nuq.last_status() == 0
+
+
+def test_invalid_arguments_are_refused():
+    torch, nuq = require_cuda()
+    g = torch.zeros(4096, device="cuda")
+    for bucket, s, flags in ((100, 3, 0), (0, 3, 0), (1024, 0, 0), (1024, 15, 0), (1024, 9, nuq.LEVELS_UNIFORM),
+                             (1024, 3, 2), (1024, 3, 1 << 25), (131072, 3, 0), (1024, 3, nuq.TEST_NORMS)):
+        assert nuq.encode_bound(4096, bucket, s, flags & ~nuq.TEST_NORMS) == 0 or flags & nuq.TEST_NORMS
+        with pytest.raises(nuq.NuqError) as e:
+            nuq.encode(g, bucket, s, flags, out=torch.empty(65536, dtype=torch.int32, device="cuda"))
+        assert e.value.code == nuq.ERR_INVALID_ARG
+    out, _ = nuq.encode(g, 1024, 3)
+    with pytest.raises(nuq.NuqError):
+        nuq.decode_accumulate([out] * 65, 4096, 1024, 3)
+    with pytest.raises(nuq.NuqError):
+        nuq.decode_accumulate([out], 4096, 1000, 3)
+    with pytest.raises(nuq.NuqError):                      # misaligned input
+        nuq.encode(torch.zeros(4097, device="cuda")[1:], 1024, 3)
+    assert nuq.last_status() == 0
+
+
+def test_malformed_containers_are_reported_not_trusted():
+    """Corrupt headers, offsets, lengths and tokens: the decoder latches BAD_STREAM and stays in bounds."""
+    d, bucket, s = 40000, 1024, 3
+    g = _input(d, 3)
+    good, _ = O.encode(g, bucket, s, 0, 1, 0)
+    nblk = 40
+    payload0 = 16 + 2 * (nblk + 1)
+    gpu_decode([good], d, bucket, s)
+    edits = [
+        (0, 0), (1, 9), (2, d - 1), (4, 2048), (5, 4), (7, 128), (8, nblk - 1), (10, 31),
+        (16 + 2 * 3, 5),                       # block 3 offset not a multiple of 32
+        (16 + 2 * 3, 0xFFFFFF00),              # block 3 offset beyond the payload
+        (payload0 + 1, 0xFFFFFFFF),            # sub-block lengths of block 0 beyond the block
+        (payload0 + 4, 0xFFFFFFFF),            # token soup
+    ]
+    for word, value in edits:
+        bad = good.copy()
+        bad[word] = value
+        assert O.decode_symbols(bad, d, bucket, s)[0] == -3, (word, value)
+        gpu_decode([bad], d, bucket, s, expect_status=-3)
+        gpu_decode([good, bad, good], d, bucket, s, expect_status=-3)
+    fx, _ = O.encode(g, bucket, s, O.make_flags(mode=O.MODE_FIXED), 1, 0)
+    bad = fx.copy(); bad[20] = 0xFFFFFFFF      # level index 7 does not exist for s = 3
+    gpu_decode([bad], d, bucket, s, expect_status=-3)
+    assert np.array_equal(gpu_decode([good], d, bucket, s), O.decode_accumulate([good], d, bucket, s)[1])
+
+
+def test_degenerate_buckets():
+    d, bucket = 5 * 1024, 1024
+    g = _input(d, 4)
+    g[0:1024] = 0.0                            # all-zero bucket
+    g[1024 + 5] = np.nan                       # NaN poisons bucket 1
+    g[2048 + 9] = np.inf                       # infinite norm
+    g[3072:4096] = 1e-42                       # 2^s / norm overflows
+    for flags in (0, O.make_flags(mode=O.MODE_FIXED), O.make_flags(L2, UNI), O.make_flags(LINF, UNI)):
+        want, _ = O.encode(g, bucket, 4, flags, 1, 0)
+        got, _ = gpu_encode(g, bucket, 4, flags, 1, 0)
+        assert np.array_equal(got, want)
+        acc = gpu_decode([got], d, bucket, 4)
+        assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([want], d, bucket, 4)[1].view(np.uint32))
+        assert not acc[:4096].any()
