@@ -110,6 +110,9 @@ uint32_t nuq_oracle_fixed_width(uint32_t levelset, uint32_t s) {
     return b + 1u;
 }
 
+static uint32_t float_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+static float bits_float(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
+
 /* ------------------------------------------------------------------ */
 /* Bucket norm (Euclidean norm of Sec. 2; max-abs for the QSGDinf case).*/
 /* ------------------------------------------------------------------ */
@@ -118,13 +121,14 @@ float nuq_oracle_norm(const float* v, uint64_t n, uint32_t norm_kind) {
         float m = 0.0f;
         for (uint64_t i = 0; i < n; ++i) {
             float a = fabsf(v[i]);
-            if (a != a) return a;   /* NaN poisons the bucket */
+            if (a != a) return bits_float(0x7FC00000u);   /* NaN poisons the bucket */
             if (a > m) m = a;
         }
         return m;
     }
     double acc = 0.0;
     for (uint64_t i = 0; i < n; ++i) acc += (double)v[i] * (double)v[i];
+    if (acc != acc) return bits_float(0x7FC00000u);       /* one NaN pattern, whatever the payloads were */
     return (float)sqrt(acc);
 }
 
@@ -311,8 +315,6 @@ static void put_bit(uint32_t* words, uint64_t p, uint32_t b) {
 static uint32_t get_bit(const uint32_t* words, uint64_t p) {
     return (words[p >> 5] >> (31u - (uint32_t)(p & 31u))) & 1u;
 }
-static uint32_t float_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
-static float bits_float(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
 
 static uint64_t count_blocks(uint64_t d, uint32_t bucket) {
     uint64_t nb = (d + bucket - 1) / bucket;

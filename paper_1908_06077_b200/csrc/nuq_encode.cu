@@ -269,6 +269,7 @@ __global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(const __grid_con
                 for (uint32_t sb = sb0; sb < sb1; ++sb) m = max(m, s_sb_maxbits[sb]);
                 norm = __uint_as_float(m);
             }
+            if (norm != norm) norm = __uint_as_float(0x7fc00000u);     // one NaN pattern in the stream
             float inv = 0.0f;
             if (norm > 0.0f && norm < __uint_as_float(0x7f800000u)) {
                 inv = __fdiv_rn(top, norm);                 // one IEEE division per bucket
@@ -547,7 +548,8 @@ __global__ void __launch_bounds__(256) bucket_norm_kernel(const float* __restric
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < 8; ++w) { acc += s_acc[w]; m = max(m, s_max[w]); }
-        norms[b] = norm_kind == kNormL2 ? (float)sqrt(acc) : __uint_as_float(m);
+        float norm = norm_kind == kNormL2 ? (float)sqrt(acc) : __uint_as_float(m);
+        norms[b] = norm != norm ? __uint_as_float(0x7fc00000u) : norm;
     }
 }
 
