@@ -32,5 +32,5 @@ def test_argument_only_calls_need_no_gpu():
     assert lib.nuq_encode_bound(65536, 1024, 3, 0) > 65536 // 8
     assert lib.nuq_encode_bound(65536, 1000, 3, 0) == 0          # bucket not a multiple of 256
     assert lib.nuq_encode_bound(65536, 1024, 0, 0) == 0
-    # fixed mode: header + per bucket one norm word and B*w/32 field words
-    assert lib.nuq_encode_bound(8192, 8192, 4, 1 << 16) == 4 * (16 + 1 + 8192 * 4 // 32)
+    # fixed mode: header + per bucket one norm word and B*w/32 field words, rounded up to 16 bytes
+    assert lib.nuq_encode_bound(8192, 8192, 4, 1 << 16) == (4 * (16 + 1 + 8192 * 4 // 32) + 15) // 16 * 16
