@@ -48,7 +48,7 @@ extern "C" {
 typedef int nuq_status;
 #define NUQ_OK 0
 #define NUQ_ERR_INVALID_ARG (-1) /* null / misaligned pointer, size or parameter out of range      */
-#define NUQ_ERR_CAPACITY (-2)    /* reserved: output capacity too small                            */
+#define NUQ_ERR_CAPACITY (-2)    /* a fixed capacity is too small (nuq_encode_static: scratch)     */
 #define NUQ_ERR_BAD_STREAM (-3)  /* a container failed validation inside nuq_decode_accumulate     */
 #define NUQ_ERR_CUDA (-4)        /* a CUDA runtime call failed (allocation, launch)                */
 #define NUQ_ERR_TIMEOUT (-5)     /* the encoder's cross-tile scan gave up waiting (bounded spin)   */
@@ -112,6 +112,43 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
  */
 nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
                                  float* acc, void* stream);
+
+/*
+ * nuq_encode for callers that must not allocate device memory.  (The paper has
+ * no counterpart; this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is forbidden or would stall --
+ * inside a framework that has handed all of the GPU's memory to its own caching
+ * allocator, in a latency-critical loop where the implicit device
+ * synchronisation of an allocation is not acceptable, or in a process whose
+ * memory budget is fixed at start-up.  nuq_encode keeps its cross-tile scan
+ * state in a workspace that it allocates (and regrows) on demand; this variant
+ * keeps the same state in a fixed array of NUQ_STATIC_SCRATCH_BYTES that is part
+ * of the library's device image, so it never calls cudaMalloc, cudaFree or any
+ * allocating routine.  Every GPU that loads the library holds that array until
+ * the process exits.
+ *
+ * Arguments, container, random draws and results are exactly those of
+ * nuq_encode.  Differences:
+ *   - Size limit: the scan state needs 64 + 8 * ceil(d / tile) bytes (a tile is
+ *     8192 elements, or floor(8192 / bucket) buckets), plus 4 bytes per bucket
+ *     when bucket > 8192.  If that exceeds NUQ_STATIC_SCRATCH_BYTES the call
+ *     returns NUQ_ERR_CAPACITY and enqueues nothing (d up to about 5.3e8 with
+ *     bucket = 8192).
+ *   - The first call on each device looks up the array's device address (the
+ *     device must be current, as for every call here) and uploads a 1 KB code
+ *     table.  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array, which still holds what the
+ *     previous call left; each call clears the part it uses, in stream order,
+ *     before its kernel runs.  Two calls whose kernels can overlap on the GPU
+ *     (different streams, no dependency between them) race on it and produce
+ *     garbage: serialise them.
+ *   - Kernel-detected errors (NUQ_ERR_TIMEOUT) are latched in the array and are
+ *     reported, and cleared, by nuq_last_status on any stream of that device.
+ */
+#define NUQ_STATIC_SCRATCH_BYTES (512u * 1024u)
+nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind,
+                             uint64_t seed, uint64_t offset, void* out, uint64_t* out_bits, void* stream);
 
 /* Bytes that `out` of nuq_encode must hold for these arguments (0 if they are invalid). */
 uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind);

@@ -13,6 +13,12 @@
 namespace nuq {
 namespace {
 
+// Scratch of nuq_encode_static: lives in the library's device image, so every
+// GPU that loads the library holds these bytes until the process exits.  In host
+// code this name is only a handle for cudaGetSymbolAddress, never an address.
+constexpr size_t kStaticScratchBytes = NUQ_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
 struct WsEntry {
     Workspace* ptr = nullptr;
     size_t bytes = 0;
@@ -23,6 +29,7 @@ std::map<std::pair<int, cudaStream_t>, WsEntry> g_ws;
 std::map<int, int> g_sms;                 // device -> SM count
 std::set<int> g_lut_ready;                // devices whose constant LUT is uploaded
 const float* g_test_norms = nullptr;
+std::map<int, Workspace*> g_static_ws;   // device -> address of g_static_scratch on that device
 uint32_t g_erc_len[256];
 bool g_erc_len_ready = false;
 
@@ -140,6 +147,51 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
 
 using namespace nuq;
 
+// Shared tail of the two encode entry points: clears the call's scan state in `ws` and
+// enqueues the kernels.  `ws` must hold state_bytes (+ 4 * nb for buckets wider than a tile).
+static nuq_status enqueue_encode(EncodeParams& P, const float* g, uint32_t norm_kind, uint64_t seed, uint64_t offset,
+                                 void* out, uint64_t* out_bits, Workspace* ws, size_t state_bytes, int dev,
+                                 cudaStream_t stream) {
+    Geometry& G = P.geo;
+    const bool test_norms = (norm_kind & NUQ_TEST_NORMS) != 0;
+    const bool wide = G.bucket > kBLK;
+    if (!g_lut_ready.count(dev)) {
+        if (upload_erc_lut() != cudaSuccess) return NUQ_ERR_CUDA;
+        g_lut_ready.insert(dev);
+    }
+    if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, state_bytes - kWorkspaceClearFrom, stream) !=
+        cudaSuccess)
+        return NUQ_ERR_CUDA;
+
+    P.g = g;
+    P.norms_in = nullptr;
+    if (test_norms) {
+        P.norms_in = g_test_norms;
+    } else if (wide) {
+        float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + state_bytes);
+        if (launch_bucket_norms(g, G.d, G.bucket, G.norm_kind, norms, G.nb, stream) != cudaSuccess) return NUQ_ERR_CUDA;
+        P.norms_in = norms;
+    }
+    P.out = static_cast<uint32_t*>(out);
+    P.out_bits = out_bits;
+    P.ws = ws;
+    P.seed = seed;
+    P.offset = offset;
+    P.stage_words = stage_words_for(G);
+    if (launch_encode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    return NUQ_OK;
+}
+
+static bool encode_args_ok(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, void* out,
+                           uint64_t* out_bits, Geometry* G) {
+    if (!g || !out || !make_geometry(d, bucket, s, norm_kind, G)) return false;
+    if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u) ||
+        (reinterpret_cast<uintptr_t>(out_bits) & 7u))
+        return false;
+    if ((norm_kind & NUQ_TEST_NORMS) && !g_test_norms) return false;
+    return true;
+}
+
 extern "C" {
 
 uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind) {
@@ -161,45 +213,39 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     EncodeParams P;
     Geometry& G = P.geo;
-    if (!g || !out || !make_geometry(d, bucket, s, norm_kind, &G)) return NUQ_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u) ||
-        (reinterpret_cast<uintptr_t>(out_bits) & 7u))
-        return NUQ_ERR_INVALID_ARG;
-    const bool test_norms = (norm_kind & NUQ_TEST_NORMS) != 0;
-    if (test_norms && !g_test_norms) return NUQ_ERR_INVALID_ARG;
-
-    const bool wide = bucket > kBLK;
+    if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
     const size_t state_bytes = sizeof(Workspace) + 8 * G.ntiles;
-    const size_t ws_bytes = state_bytes + (wide ? 4 * G.nb : 0);
+    const size_t ws_bytes = state_bytes + (bucket > kBLK ? 4 * G.nb : 0);
     Workspace* ws = nullptr;
     int dev = 0;
     nuq_status st = get_workspace(stream, ws_bytes, &ws, &dev);
     if (st != NUQ_OK) return st;
-    if (!g_lut_ready.count(dev)) {
-        if (upload_erc_lut() != cudaSuccess) return NUQ_ERR_CUDA;
-        g_lut_ready.insert(dev);
-    }
-    if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, state_bytes - kWorkspaceClearFrom, stream) !=
-        cudaSuccess)
-        return NUQ_ERR_CUDA;
+    return enqueue_encode(P, g, norm_kind, seed, offset, out, out_bits, ws, state_bytes, dev, stream);
+}
 
-    P.g = g;
-    P.norms_in = nullptr;
-    if (test_norms) {
-        P.norms_in = g_test_norms;
-    } else if (wide) {
-        float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + state_bytes);
-        if (launch_bucket_norms(g, d, bucket, G.norm_kind, norms, G.nb, stream) != cudaSuccess) return NUQ_ERR_CUDA;
-        P.norms_in = norms;
+nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind,
+                             uint64_t seed, uint64_t offset, void* out, uint64_t* out_bits, void* stream_) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    EncodeParams P;
+    Geometry& G = P.geo;
+    if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
+    const size_t state_bytes = sizeof(Workspace) + 8 * G.ntiles;
+    const size_t ws_bytes = state_bytes + (bucket > kBLK ? 4 * G.nb : 0);
+    if (ws_bytes > kStaticScratchBytes) return NUQ_ERR_CAPACITY;       // vector too long for the fixed scratch
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    auto it = g_static_ws.find(dev);
+    if (it == g_static_ws.end()) {
+        // first call on this device: ask the runtime where this device keeps the array
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return NUQ_ERR_CUDA;
+        }
+        it = g_static_ws.emplace(dev, static_cast<Workspace*>(p)).first;
     }
-    P.out = static_cast<uint32_t*>(out);
-    P.out_bits = out_bits;
-    P.ws = ws;
-    P.seed = seed;
-    P.offset = offset;
-    P.stage_words = stage_words_for(G);
-    if (launch_encode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
-    return NUQ_OK;
+    return enqueue_encode(P, g, norm_kind, seed, offset, out, out_bits, it->second, state_bytes, dev, stream);
 }
 
 nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
@@ -233,11 +279,19 @@ nuq_status nuq_last_status(void* stream_) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return NUQ_ERR_CUDA;
-    auto it = g_ws.find(std::make_pair(dev, stream));
-    if (it == g_ws.end() || !it->second.ptr) return NUQ_OK;
     int status = 0;
-    if (cudaMemcpy(&status, &it->second.ptr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
-    if (status != 0 && cudaMemset(&it->second.ptr->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
+    auto it = g_ws.find(std::make_pair(dev, stream));
+    if (it != g_ws.end() && it->second.ptr) {
+        if (cudaMemcpy(&status, &it->second.ptr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
+        if (status != 0 && cudaMemset(&it->second.ptr->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
+    }
+    auto st = g_static_ws.find(dev);               // kernels of nuq_encode_static latch into the static scratch
+    if (st != g_static_ws.end()) {
+        int s2 = 0;
+        if (cudaMemcpy(&s2, &st->second->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
+        if (s2 != 0 && cudaMemset(&st->second->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
+        if (s2 < status) status = s2;
+    }
     return status;
 }
 

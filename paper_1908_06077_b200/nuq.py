@@ -20,6 +20,7 @@ LEVELS_EXP, LEVELS_UNIFORM = 0 << 8, 1 << 8
 MODE_ERC, MODE_FIXED = 0 << 16, 1 << 16
 TEST_NORMS = 1 << 24
 HEADER_WORDS = 16
+STATIC_SCRATCH_BYTES = 512 * 1024
 
 
 class NuqError(RuntimeError):
@@ -42,6 +43,8 @@ def _load():
     lib.nuq_encode.restype = C.c_int
     lib.nuq_encode.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, C.c_uint64,
                                C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.nuq_encode_static.restype = C.c_int
+    lib.nuq_encode_static.argtypes = lib.nuq_encode.argtypes
     lib.nuq_decode_accumulate.restype = C.c_int
     lib.nuq_decode_accumulate.argtypes = [C.POINTER(C.c_void_p), C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32,
                                           C.c_void_p, C.c_void_p]
@@ -103,6 +106,20 @@ def encode(g: torch.Tensor, bucket, s, norm_kind=0, seed=0, offset=0, out=None, 
                          C.c_void_p(out_bits.data_ptr()), _stream(stream))
     if rc != NUQ_OK:
         raise NuqError("nuq_encode", rc)
+    return out, out_bits
+
+
+def encode_static(g: torch.Tensor, bucket, s, norm_kind=0, seed=0, offset=0, *, out, out_bits, stream=None):
+    """nuq_encode_static: the encoder for callers that may not allocate device memory.  Its
+    scan state lives in a fixed array inside the library instead of a cudaMalloc'ed workspace,
+    so `out` (encode_bound bytes) and `out_bits` (one int64) must be passed in and nothing is
+    allocated here either.  Raises NuqError(ERR_CAPACITY) when d is too long for that array.
+    Calls that could overlap on the GPU must be serialised by the caller."""
+    assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()
+    rc = _lib.nuq_encode_static(C.c_void_p(g.data_ptr()), g.numel(), bucket, s, norm_kind, seed, offset,
+                                C.c_void_p(out.data_ptr()), C.c_void_p(out_bits.data_ptr()), _stream(stream))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_encode_static", rc)
     return out, out_bits
 
 
