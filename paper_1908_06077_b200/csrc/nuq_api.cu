@@ -147,38 +147,65 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
 
 using namespace nuq;
 
+// What one encode call needs from its workspace and from shared memory.
+struct EncodePlan {
+    size_t state_bytes;      // control block + one look-back word per tile
+    size_t norms_bytes;      // bucket norms for buckets wider than a tile
+    size_t slot_bytes;       // one warp's tile image (ERC mode), 0 in the fixed-width mode
+    uint32_t want_grid;      // CTAs that give every SM its full share
+};
+
+static EncodePlan plan_encode(EncodeParams& P, int sms) {
+    const Geometry& G = P.geo;
+    EncodePlan pl;
+    pl.state_bytes = sizeof(Workspace) + 8 * G.ntiles;
+    pl.norms_bytes = G.bucket > kBLK ? 4 * G.nb : 0;
+    P.slot_words = G.mode == kModeErc ? (stage_words_for(G) + 3u) & ~3u : 0u;
+    pl.slot_bytes = 4u * (size_t)P.slot_words;
+    const uint32_t bits_per_elem = G.mode == kModeErc ? 2u + max_level_code_bits(G) : G.width;
+    P.window_words = (kEncChunk * bits_per_elem + 31u) / 32u + 4u;
+    const uint32_t group_words = G.levelset == kLevelsExp ? 2u : 3u;
+    P.warp_smem_words = P.window_words + (G.mode == kModeErc ? kEncChunk + (kEncChunk / 4u) * group_words : 0u);
+    P.warp_smem_words = (P.warp_smem_words + 3u) & ~3u;
+    const uint64_t need = (G.ntiles + kEncWarps - 1) / kEncWarps;
+    const uint64_t cap = (uint64_t)encode_max_blocks(sms);
+    pl.want_grid = (uint32_t)(need < cap ? need : cap);
+    return pl;
+}
+
+static size_t slots_offset(const EncodePlan& pl) { return (pl.state_bytes + pl.norms_bytes + 15) & ~(size_t)15; }
+
 // Shared tail of the two encode entry points: clears the call's scan state in `ws` and
-// enqueues the kernels.  `ws` must hold state_bytes (+ 4 * nb for buckets wider than a tile).
-static nuq_status enqueue_encode(EncodeParams& P, const float* g, uint32_t norm_kind, uint64_t seed, uint64_t offset,
-                                 void* out, uint64_t* out_bits, Workspace* ws, size_t state_bytes, int dev,
-                                 cudaStream_t stream) {
+// enqueues the kernels.  `ws` must hold slots_offset(pl) + P.grid * kEncWarps * pl.slot_bytes.
+static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const float* g, uint32_t norm_kind,
+                                 uint64_t seed, uint64_t offset, void* out, uint64_t* out_bits, Workspace* ws,
+                                 int dev, cudaStream_t stream) {
     Geometry& G = P.geo;
     const bool test_norms = (norm_kind & NUQ_TEST_NORMS) != 0;
-    const bool wide = G.bucket > kBLK;
     if (!g_lut_ready.count(dev)) {
         if (upload_erc_lut() != cudaSuccess) return NUQ_ERR_CUDA;
         g_lut_ready.insert(dev);
     }
-    if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, state_bytes - kWorkspaceClearFrom, stream) !=
-        cudaSuccess)
+    if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, pl.state_bytes - kWorkspaceClearFrom,
+                        stream) != cudaSuccess)
         return NUQ_ERR_CUDA;
 
     P.g = g;
     P.norms_in = nullptr;
     if (test_norms) {
         P.norms_in = g_test_norms;
-    } else if (wide) {
-        float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + state_bytes);
+    } else if (pl.norms_bytes) {
+        float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + pl.state_bytes);
         if (launch_bucket_norms(g, G.d, G.bucket, G.norm_kind, norms, G.nb, stream) != cudaSuccess) return NUQ_ERR_CUDA;
         P.norms_in = norms;
     }
     P.out = static_cast<uint32_t*>(out);
     P.out_bits = out_bits;
     P.ws = ws;
+    P.slots = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + slots_offset(pl));
     P.seed = seed;
     P.offset = offset;
-    P.stage_words = stage_words_for(G);
-    if (launch_encode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (launch_encode(P, stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;
 }
 
@@ -214,13 +241,14 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     EncodeParams P;
     Geometry& G = P.geo;
     if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
-    const size_t state_bytes = sizeof(Workspace) + 8 * G.ntiles;
-    const size_t ws_bytes = state_bytes + (bucket > kBLK ? 4 * G.nb : 0);
-    Workspace* ws = nullptr;
     int dev = 0;
-    nuq_status st = get_workspace(stream, ws_bytes, &ws, &dev);
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    const EncodePlan pl = plan_encode(P, device_sms(dev));
+    P.grid = pl.want_grid;
+    Workspace* ws = nullptr;
+    nuq_status st = get_workspace(stream, slots_offset(pl) + (size_t)P.grid * kEncWarps * pl.slot_bytes, &ws, &dev);
     if (st != NUQ_OK) return st;
-    return enqueue_encode(P, g, norm_kind, seed, offset, out, out_bits, ws, state_bytes, dev, stream);
+    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, dev, stream);
 }
 
 nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind,
@@ -230,11 +258,18 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
     EncodeParams P;
     Geometry& G = P.geo;
     if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
-    const size_t state_bytes = sizeof(Workspace) + 8 * G.ntiles;
-    const size_t ws_bytes = state_bytes + (bucket > kBLK ? 4 * G.nb : 0);
-    if (ws_bytes > kStaticScratchBytes) return NUQ_ERR_CAPACITY;       // vector too long for the fixed scratch
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    const EncodePlan pl = plan_encode(P, device_sms(dev));
+    // the fixed array must hold the scan state and the tile images of at least one CTA's warps;
+    // fewer CTAs than the device could run are launched when it cannot hold more
+    const size_t fixed_part = slots_offset(pl), per_cta = (size_t)kEncWarps * pl.slot_bytes;
+    if (fixed_part + per_cta > kStaticScratchBytes) return NUQ_ERR_CAPACITY;
+    P.grid = pl.want_grid;
+    if (per_cta) {
+        const size_t fit = (kStaticScratchBytes - fixed_part) / per_cta;
+        if (fit < P.grid) P.grid = (uint32_t)fit;
+    }
     auto it = g_static_ws.find(dev);
     if (it == g_static_ws.end()) {
         // first call on this device: ask the runtime where this device keeps the array
@@ -245,7 +280,7 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
         }
         it = g_static_ws.emplace(dev, static_cast<Workspace*>(p)).first;
     }
-    return enqueue_encode(P, g, norm_kind, seed, offset, out, out_bits, it->second, state_bytes, dev, stream);
+    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, it->second, dev, stream);
 }
 
 nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,

@@ -13,9 +13,10 @@ constexpr uint32_t kBLK = 32 * kSB;       // elements per coding block / per til
 constexpr uint32_t kHeaderWords = 16;
 constexpr uint32_t kMaxK = 64;
 
-constexpr int kEncThreads = 256;          // 8 warps, 4 sub-blocks each
+constexpr int kEncThreads = 256;          // 8 independent warps, each takes whole tiles
 constexpr int kEncWarps = kEncThreads / 32;
-constexpr int kSbPerWarp = 32 / kEncWarps;
+constexpr int kEncMinBlocks = 4;          // resident CTAs per SM the encoder is compiled for
+constexpr uint32_t kEncChunk = 512;       // elements a warp quantizes per step
 
 enum : uint32_t { kNormL2 = 0, kNormLinf = 1 };
 enum : uint32_t { kLevelsExp = 0, kLevelsUniform = 1 };
@@ -41,7 +42,8 @@ struct Workspace {
     uint64_t nnz;           // nonzero symbols of the whole call
     uint64_t total_words;   // payload words of the whole call
     uint64_t reserved[2];
-    // followed by: uint64_t tile_state[ntiles], then float norms[nb] for wide buckets
+    // followed by: uint64_t tile_state[ntiles], float norms[nb] for wide buckets, then (16-byte
+    // aligned) one scratch slot per encoder warp that holds the image of the tile it is working on
 };
 constexpr size_t kWorkspaceClearFrom = 8;
 
@@ -70,7 +72,11 @@ struct EncodeParams {
     uint64_t* out_bits;
     Workspace* ws;
     uint64_t seed, offset;
-    uint32_t stage_words;    // capacity of the shared-memory staging buffer
+    uint32_t* slots;         // ERC mode: grid * kEncWarps scratch slots of slot_words words
+    uint32_t slot_words;     // capacity of one slot = largest possible tile image
+    uint32_t window_words;   // shared-memory bit window of one warp
+    uint32_t warp_smem_words;// shared memory of one warp (window, token list, group list)
+    uint32_t grid;           // CTAs to launch
 };
 
 struct DecodeParams {

@@ -1,11 +1,29 @@
 // ENCODE of NUQSGD (App. A) for one gradient vector: bucket norm, stochastic
-// quantization (Definition 1) and Elias-recursive token packing in ONE pass over
-// the input.  A CTA owns a tile of up to 8192 consecutive elements (32 coding
-// sub-blocks of 256); every lane keeps its 4 x 8 consecutive elements in
-// registers between the norm reduction and the quantizer, so the gradient is
-// read from HBM exactly once.  Tiles are chained by a decoupled look-back scan
-// over their payload sizes, which gives each tile its place in the packed
-// stream without a second kernel.
+// quantization (Definition 1) and Elias-recursive token packing in one kernel.
+//
+// ONE WARP owns a tile of up to 8192 consecutive elements (whole buckets, or one
+// 8192-element coding block of a wider bucket) and there is no block-level
+// barrier anywhere: warps of a CTA only share two read-only code tables.  For
+// each bucket of its tile a warp
+//   1. reads the bucket once and reduces its norm (fp64 sums of exact squares);
+//   2. walks the bucket again in chunks of 512 elements (the second read is
+//      served by L2/L1): a lane handles 4 consecutive elements per 128-element
+//      row with one 128-bit load and one Philox block;
+//   3. keeps only the groups of 4 elements that hold a nonzero symbol (ballot /
+//      popc compaction into a shared-memory list), expands those groups to one
+//      entry per nonzero symbol (second compaction), and generates the tokens
+//      from that dense list, 32 tokens per step, OR-ing them into a small
+//      shared-memory bit window behind a running bit cursor;
+//   4. flushes the completed words of the window to the warp's scratch slot in
+//      global memory, which ends up holding the exact image of the tile
+//      (norm word, sub-block lengths, token strings, per bucket).
+// The tile's size is then chained to its predecessors by a decoupled look-back
+// scan, and the image is copied from the slot (still in L2) to its place in the
+// packed stream.  In the fixed-width mode the place is known in advance and the
+// window is flushed straight into the stream.
+//
+// The kernel is bound by instruction issue, not by HBM; the quantizer is branch
+// free and all per-symbol work runs on dense lists.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 
@@ -55,38 +73,47 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 }
 
 // ---------------------------------------------------------------------------
-// Definition 1 for one coordinate.  y = |v| * (2^s / norm), clamped to 2^s.
-// The draw is u = m * 2^-24 with m the top 24 bits of `word`; the coordinate moves
-// to the upper level iff u < p.  Both sides of that comparison are scaled by 2^24
-// (exact), and for y >= 1 the 23 mantissa bits of y ARE p * 2^23, so the test
-// becomes an integer comparison.
+// Definition 1 for one coordinate.  y = |v| * (2^s / norm), clamped to 2^s; the
+// draw is u = m * 2^-24 with m the top 24 bits of `word`; the coordinate moves to
+// the upper level iff u < p.
+//
+// Exponential levels, y >= 1 (r in [2^(e-s), 2^(e+1-s)], e = floor(log2 y)):
+//   p = y 2^-e - 1 = mant / 2^23, and u < p  <=>  (word >> 9) < mant.  Adding
+//   0x7FFFFF - (word >> 9) to the bit pattern of y carries into the exponent field
+//   exactly in that case, so (bits + 0x7FFFFF - (word >> 9)) >> 23 - 126 is the level
+//   index e + 1 + [u < p].  For y < 1 the same expression is at most 1, and it is 1
+//   only if u < y as well, so the maximum with [u < y] is the index in every case.
+// y < 1 (r in [0, 2^-s]): p = y, and u < y  <=>  float(m) - y 2^24 < 0 (both terms
+//   exact, the sign of a rounded difference is the sign of the exact one).
 // ---------------------------------------------------------------------------
-template <uint32_t LEVELSET>
-__device__ __forceinline__ uint32_t quantize_one(float v, float inv, float top, uint32_t s, uint32_t word) {
-    float y = fminf(__fmul_rn(fabsf(v), inv), top);
-    uint32_t m24 = word >> 8;
-    if (LEVELSET == kLevelsExp) {
-        if (y < 1.0f) {                                    // r in [0, 2^-s]:  p_1 = 2^s r
-            return (__uint2float_rn(m24) < y * 16777216.0f) ? 1u : 0u;
-        }
-        uint32_t yb = __float_as_uint(y);
-        uint32_t e = (yb >> 23) - 127u;                    // r in [2^(e-s), 2^(e+1-s)]:  p_2 = 2^(s-e) r - 1
-        if (e >= s) return s + 1u;                         // y == 2^s: p = 1
-        return e + 1u + (((m24 >> 1) < (yb & 0x7FFFFFu)) ? 1u : 0u);
-    } else {                                               // levels k / 2^s:  p = y - floor(y)
-        float fl = fminf(floorf(y), top - 1.0f);
-        float p = y - fl;
-        return (uint32_t)fl + ((__uint2float_rn(m24) < p * 16777216.0f) ? 1u : 0u);
-    }
+__device__ __forceinline__ uint32_t quantize_exp(float v, float inv, float top, uint32_t word) {
+    const float y = fminf(__fmul_rn(fabsf(v), inv), top);
+    const int hi = (int)(__float_as_uint(y) + (0x007FFFFFu - 0x3F000000u) - (word >> 9)) >> 23;
+    const float diff = __fsub_rn(__uint2float_rn(word >> 8), __fmul_rn(y, 16777216.0f));
+    const int up = (int)(__float_as_uint(diff) >> 31);
+    return (uint32_t)max(hi, up);
 }
 
-// OR `nbits` (<= 33) right-aligned bits of `value` into the MSB-first bit string `stage` at `bitpos`.
-__device__ __forceinline__ void stage_or(uint32_t* stage, uint32_t bitpos, uint64_t value, uint32_t nbits) {
-    uint32_t w = bitpos >> 5, sh = bitpos & 31u;
-    uint64_t placed = (value << (64u - nbits)) >> sh;      // nbits + sh <= 64
-    uint32_t hi = (uint32_t)(placed >> 32), lo = (uint32_t)placed;
-    atomicOr(stage + w, hi);
-    if (lo) atomicOr(stage + w + 1, lo);
+// Uniform levels k / 2^s:  p = y - floor(y).
+__device__ __forceinline__ uint32_t quantize_uniform(float v, float inv, float top, uint32_t word) {
+    const float y = fminf(__fmul_rn(fabsf(v), inv), top);
+    const float fl = fminf(floorf(y), top - 1.0f);
+    const float p = y - fl;
+    return (uint32_t)fl + ((__uint2float_rn(word >> 8) < p * 16777216.0f) ? 1u : 0u);
+}
+
+// OR `nbits` (1..64) right-aligned bits of `value` into the MSB-first bit string `dst` at
+// `bitpos`.  Up to three words are touched; dst[bitpos/32 + 2] must exist.
+__device__ __forceinline__ void or_bits(uint32_t* dst, uint32_t bitpos, uint64_t value, uint32_t nbits) {
+    const uint64_t a = value << (64u - nbits);
+    const uint32_t hi = (uint32_t)(a >> 32), lo = (uint32_t)a;
+    const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
+    const uint32_t w0 = hi >> sh;
+    const uint32_t w1 = __funnelshift_r(lo, hi, sh);
+    const uint32_t w2 = __funnelshift_r(0u, lo, sh);
+    if (w0) atomicOr(dst + w, w0);
+    if (w1) atomicOr(dst + w + 1, w1);
+    if (w2) atomicOr(dst + w + 2, w2);
 }
 
 __device__ __forceinline__ uint64_t ld_volatile_u64(const uint64_t* p) {
@@ -141,346 +168,431 @@ __device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile,
     return exclusive;
 }
 
-// symbols of the 8 consecutive elements one lane owns in one sub-block
-struct LaneSyms {
-    uint32_t masks;   // bits 0-7 nonzero mask, bits 8-15 sign mask
-    uint32_t lo, hi;  // (sym-1) of elements 0-3 / 4-7, one byte each
+constexpr uint32_t kChunk = 512;                 // elements quantized per step of a warp (2 sub-blocks, 4 rows)
+constexpr uint32_t kChunkRows = kChunk / 128;
+
+// Symbols travel as small fields: level index in the low bits, sign above it.
+template <uint32_t LEVELSET>
+struct Sym {
+    static constexpr uint32_t kBits = LEVELSET == kLevelsExp ? 7u : 15u;     // index <= 15 resp. <= 256
+    static constexpr uint32_t kMask = (1u << kBits) - 1u;
 };
 
-__device__ __forceinline__ uint32_t sym_of(const LaneSyms& q, uint32_t e) {
-    return (((e < 4 ? q.lo : q.hi) >> (8u * (e & 3u))) & 0xffu) + 1u;
+// OR `nbits` (1..32) right-aligned bits of `value` into the MSB-first bit string `dst` at `bitpos`.
+__device__ __forceinline__ void or_bits32(uint32_t* dst, uint32_t bitpos, uint32_t value, uint32_t nbits) {
+    const uint32_t a = value << (32u - nbits);
+    const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
+    const uint32_t w0 = a >> sh;
+    const uint32_t w1 = __funnelshift_r(0u, a, sh);
+    if (w0) atomicOr(dst + w, w0);
+    if (w1) atomicOr(dst + w + 1, w1);
 }
 
-template <uint32_t LEVELSET, uint32_t MODE>
-__global__ void __launch_bounds__(kEncThreads, 2) encode_kernel(const __grid_constant__ EncodeParams P) {
-    extern __shared__ __align__(16) uint32_t stage[];      // staged payload of the tile
-    __shared__ uint32_t s_lut[256];
-    __shared__ double s_sb_partial[32];
-    __shared__ uint32_t s_sb_maxbits[32];
-    __shared__ float s_blk_norm[32];
-    __shared__ float s_blk_inv[32];                        // 2^s / norm, or 0 for a bucket that is not quantized
-    __shared__ uint32_t s_sb_bits[32];
-    __shared__ uint32_t s_sb_bitoff[32];
-    __shared__ uint32_t s_blk_wordoff[33];
-    __shared__ unsigned long long s_tile, s_tile_off;
-    __shared__ uint32_t s_tile_words, s_abort, s_nnz;
+// Shared memory of one warp.
+struct WarpMem {
+    uint32_t* window;     // bit window behind the cursor
+    uint32_t* tokens;     // kChunk entries: position | field << 10
+    uint32_t* groups;     // kChunk / 4 entries of 2 (exponential) or 3 (uniform) words
+};
 
+template <uint32_t LEVELSET, uint32_t MODE>
+__global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(const __grid_constant__ EncodeParams P) {
+    extern __shared__ __align__(16) uint32_t smem[];
+    __shared__ uint32_t s_lut[256];                        // ERC(N), N = 1..256: code | len << 16
+    __shared__ uint32_t s_lut_signed[256];                 // exponential levels: sign bit + ERC(index) by field
+
+    using S = Sym<LEVELSET>;
+    constexpr uint32_t kGroupWords = LEVELSET == kLevelsExp ? 2u : 3u;
     const Geometry& G = P.geo;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t gwarp = blockIdx.x * kEncWarps + warp;
+    uint32_t* wmem = smem + warp * P.warp_smem_words;
+    WarpMem M;
+    M.window = wmem;
+    M.tokens = wmem + P.window_words;
+    M.groups = M.tokens + kChunk;
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
+    uint32_t* slot = P.slots + (uint64_t)gwarp * P.slot_words;
     uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
     uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
     const float top = __uint_as_float((127u + G.s) << 23);
     const uint32_t k0 = (uint32_t)P.seed, k1 = (uint32_t)(P.seed >> 32);
     const uint32_t c2 = (uint32_t)P.offset, c3 = (uint32_t)(P.offset >> 32);
+    const uint32_t lt_mask = (1u << lane) - 1u;
 
-    s_lut[tid] = c_erc_lut[tid];
-    for (uint32_t i = tid; i < P.stage_words; i += kEncThreads) stage[i] = 0;
+    {
+        const uint32_t e = c_erc_lut[tid];
+        s_lut[tid] = e;
+        // field = sign << 7 | index: the sign bit followed by ERC(index)
+        const uint32_t idx = tid & 0x7Fu;
+        uint32_t v = 0;
+        if (idx >= 1) {
+            const uint32_t l = c_erc_lut[idx - 1u], len = l >> 16;
+            v = ((tid >> 7) << len) | (l & 0xffffu) | ((len + 1u) << 16);
+        }
+        s_lut_signed[tid] = v;
+    }
+    for (uint32_t i = lane; i < P.window_words; i += 32) M.window[i] = 0;
+    __syncthreads();
 
     for (;;) {
-        __syncthreads();
-        if (tid == 0) {
-            s_tile = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
-            s_abort = 0;
-            s_nnz = 0;
-        }
-        __syncthreads();
-        const uint64_t tile = s_tile;
+        uint64_t tile = 0;
+        if (lane == 0) tile = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        tile = __shfl_sync(0xffffffffu, tile, 0);
         if (tile >= G.ntiles) break;
 
         // ---- tile geometry ------------------------------------------------------
         uint64_t elem0, first_block;
-        uint32_t tile_len, nblk_tile, spb, blk_elems;
+        uint32_t tile_len, nblk_tile, blk_elems;
         uint64_t bucket_idx = 0;
         uint32_t bib = 0;                                   // block within a wide bucket
         if (G.bucket <= kBLK) {
             first_block = tile * G.blocks_per_tile;
             elem0 = first_block * G.bucket;
-            uint64_t left = G.d - elem0;
+            const uint64_t left = G.d - elem0;
             tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
             blk_elems = G.bucket;
             nblk_tile = (tile_len + G.bucket - 1) / G.bucket;
-            spb = G.sb_per_block;
         } else {
             bucket_idx = tile / G.blk_per_bucket;
             bib = (uint32_t)(tile % G.blk_per_bucket);
             first_block = tile;
-            uint64_t b0 = bucket_idx * G.bucket;
-            uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
+            const uint64_t b0 = bucket_idx * G.bucket;
+            const uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
             elem0 = b0 + (uint64_t)bib * kBLK;
-            uint64_t left = blen - (uint64_t)bib * kBLK;
+            const uint64_t left = blen - (uint64_t)bib * kBLK;
             tile_len = left < kBLK ? (uint32_t)left : kBLK;
             blk_elems = kBLK;
             nblk_tile = 1;
-            spb = 32;
         }
-        const uint32_t nsb_tile = (tile_len + kSB - 1) / kSB;
+        const float* gt = P.g + elem0;
 
-        // ---- load: 4 sub-blocks per warp, 8 consecutive elements per lane --------
-        float x[kSbPerWarp][8];
-#pragma unroll
-        for (int j = 0; j < kSbPerWarp; ++j) {
-            uint32_t base = (warp * kSbPerWarp + j) * kSB + lane * 8u;
-            if (base + 8u <= tile_len) {
-                const float4* src = reinterpret_cast<const float4*>(P.g + elem0 + base);
-                float4 a = __ldg(src), b = __ldg(src + 1);
-                x[j][0] = a.x; x[j][1] = a.y; x[j][2] = a.z; x[j][3] = a.w;
-                x[j][4] = b.x; x[j][5] = b.y; x[j][6] = b.z; x[j][7] = b.w;
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) x[j][e] = base + e < tile_len ? __ldg(P.g + elem0 + base + e) : 0.0f;
-            }
-        }
+        uint32_t W = 0;                                     // ERC: words of the tile image so far
+        uint32_t my_blk_wordoff = 0;                        // ERC: lane bi keeps the word offset of block bi
+        uint32_t tile_code_bits = 0, tile_nnz = 0;
+        uint64_t fixed_off = 0;                             // fixed mode: word offset of the tile's first record
+        if (MODE == kModeFixed)
+            fixed_off = G.bucket <= kBLK ? first_block * G.rec_words
+                                         : bucket_idx * G.rec_words + 1u + (uint64_t)bib * (kBLK * G.width / 32u);
 
-        // ---- bucket norms ----------------------------------------------------------
-        if (P.norms_in == nullptr) {
-#pragma unroll
-            for (int j = 0; j < kSbPerWarp; ++j) {
-                if (G.norm_kind == kNormL2) {
-                    double acc = 0.0;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) acc = fma((double)x[j][e], (double)x[j][e], acc);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-                    if (lane == 0) s_sb_partial[warp * kSbPerWarp + j] = acc;
-                } else {                                    // max |x| on the bit patterns: NaN sorts above inf
-                    uint32_t m = 0;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) m = max(m, __float_as_uint(fabsf(x[j][e])));
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-                    if (lane == 0) s_sb_maxbits[warp * kSbPerWarp + j] = m;
-                }
-            }
-            __syncthreads();
-        }
-        if (tid < nblk_tile) {
+        for (uint32_t bi = 0; bi < nblk_tile; ++bi) {
+            const uint32_t blk_first = bi * blk_elems;
+            const uint32_t bl = min(blk_elems, tile_len - blk_first);
+            const uint32_t nsb = (bl + kSB - 1) / kSB;
+            const uint32_t head_words = 1u + (nsb + 1u) / 2u;
+            const float* gb = gt + blk_first;
+
+            // ---- bucket norm: fp64 sum of exact squares (or max |x|), one rounding to fp32 ----
             float norm;
             if (P.norms_in != nullptr) {
-                norm = P.norms_in[G.bucket <= kBLK ? first_block + tid : bucket_idx];
-            } else if (G.norm_kind == kNormL2) {
-                double acc = 0.0;
-                uint32_t sb0 = tid * spb, sb1 = min(sb0 + spb, nsb_tile);
-                for (uint32_t sb = sb0; sb < sb1; ++sb) acc += s_sb_partial[sb];
-                norm = (float)sqrt(acc);
+                norm = P.norms_in[G.bucket <= kBLK ? first_block + bi : bucket_idx];
             } else {
-                uint32_t m = 0;
-                uint32_t sb0 = tid * spb, sb1 = min(sb0 + spb, nsb_tile);
-                for (uint32_t sb = sb0; sb < sb1; ++sb) m = max(m, s_sb_maxbits[sb]);
-                norm = __uint_as_float(m);
-            }
-            if (norm != norm) norm = __uint_as_float(0x7fc00000u);     // one NaN pattern in the stream
-            float inv = 0.0f;
-            if (norm > 0.0f && norm < __uint_as_float(0x7f800000u)) {
-                inv = __fdiv_rn(top, norm);                 // one IEEE division per bucket
-                if (!(inv < __uint_as_float(0x7f800000u))) inv = 0.0f;
-            }
-            s_blk_norm[tid] = norm;
-            s_blk_inv[tid] = inv;
-        }
-        __syncthreads();
-
-        // ---- quantize (Definition 1) ------------------------------------------------
-        LaneSyms q[kSbPerWarp];
-        uint32_t lane_off[kSbPerWarp];
-        uint32_t my_nnz = 0;
-#pragma unroll
-        for (int j = 0; j < kSbPerWarp; ++j) {
-            const uint32_t sb = warp * kSbPerWarp + j;
-            q[j].masks = 0; q[j].lo = 0; q[j].hi = 0;
-            lane_off[j] = 0;
-            if (sb >= nsb_tile) continue;
-            const float inv = s_blk_inv[sb / spb];
-            if (inv != 0.0f) {
-                uint64_t ctr = (elem0 + (uint64_t)sb * kSB + lane * 8u) >> 2;
-                uint4 r0 = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, k0, k1);
-                ++ctr;
-                uint4 r1 = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, k0, k1);
-                const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    uint32_t sym = quantize_one<LEVELSET>(x[j][e], inv, top, G.s, rw[e]);
-                    if (sym) {
-                        uint32_t neg = __float_as_uint(x[j][e]) >> 31;
-                        q[j].masks |= (1u << e) | (neg << (8 + e));
-                        if (e < 4) q[j].lo |= (sym - 1u) << (8 * e);
-                        else q[j].hi |= (sym - 1u) << (8 * (e - 4));
+                double acc = 0.0;
+                uint32_t mx = 0;
+#pragma unroll 4
+                for (uint32_t base = lane * 4u; base < bl; base += 128u) {
+                    float4 x;
+                    if (base + 4u <= bl) {
+                        x = __ldg(reinterpret_cast<const float4*>(gb + base));
+                    } else {
+                        x.x = __ldg(gb + base);
+                        x.y = base + 1u < bl ? __ldg(gb + base + 1u) : 0.0f;
+                        x.z = base + 2u < bl ? __ldg(gb + base + 2u) : 0.0f;
+                        x.w = 0.0f;
+                    }
+                    if (G.norm_kind == kNormL2) {
+                        acc = fma((double)x.x, (double)x.x, acc);
+                        acc = fma((double)x.y, (double)x.y, acc);
+                        acc = fma((double)x.z, (double)x.z, acc);
+                        acc = fma((double)x.w, (double)x.w, acc);
+                    } else {                                // max |x| on the bit patterns: NaN sorts above inf
+                        mx = max(max(mx, __float_as_uint(fabsf(x.x))), __float_as_uint(fabsf(x.y)));
+                        mx = max(max(mx, __float_as_uint(fabsf(x.z))), __float_as_uint(fabsf(x.w)));
                     }
                 }
+                if (G.norm_kind == kNormL2) {
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                    norm = (float)sqrt(acc);
+                } else {
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    norm = __uint_as_float(mx);
+                }
             }
-            my_nnz += __popc(q[j].masks & 0xffu);
+            if (norm != norm) norm = __uint_as_float(0x7fc00000u);     // one NaN pattern in the stream
+            float inv = 0.0f;                                           // 0: the bucket is not quantized
+            if (norm > 0.0f && norm < __uint_as_float(0x7f800000u)) {
+                inv = __fdiv_rn(top, norm);                             // one IEEE division per bucket
+                if (!(inv < __uint_as_float(0x7f800000u))) inv = 0.0f;
+            }
 
+            // ---- where this block's bits go -----------------------------------------------
+            uint32_t* dst;                                  // words of the block's bit string are flushed here
             if (MODE == kModeErc) {
-                // token lengths: gap to the previous nonzero of the sub-block (1-based positions)
-                uint32_t nz = q[j].masks & 0xffu;
-                uint32_t last_pos = nz ? lane * 8u + (31u - __clz(nz)) + 1u : 0u;
-                uint32_t any = __ballot_sync(0xffffffffu, nz != 0);
-                uint32_t lower = any & ((1u << lane) - 1u);
-                uint32_t prev = __shfl_sync(0xffffffffu, last_pos, lower ? 31 - __clz(lower) : 0);
-                if (!lower) prev = 0;
-                uint32_t bits = 0;
-                while (nz) {
-                    uint32_t e = __ffs(nz) - 1u;
-                    nz &= nz - 1u;
-                    uint32_t pos = lane * 8u + e + 1u;
-                    bits += (s_lut[pos - prev - 1u] >> 16) + 1u + (s_lut[sym_of(q[j], e) - 1u] >> 16);
-                    prev = pos;
-                }
-                uint32_t incl = bits;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= (uint32_t)o) incl += t;
-                }
-                lane_off[j] = incl - bits;
-                if (lane == 31) s_sb_bits[sb] = incl;
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) my_nnz += __shfl_xor_sync(0xffffffffu, my_nnz, o);
-        if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
-        __syncthreads();
-
-        // ---- layout of the tile's records -------------------------------------------
-        uint64_t tile_off = 0;
-        uint32_t tile_words = 0;
-        if (MODE == kModeErc) {
-            if (warp == 0) {
-                const uint32_t sb = lane;
-                uint32_t v = sb < nsb_tile ? s_sb_bits[sb] : 0u;
-                uint32_t incl = v;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= (uint32_t)o) incl += t;
-                }
-                const uint32_t excl = incl - v;
-                const uint32_t bi = sb / spb, sb0 = bi * spb;
-                const uint32_t sb_last = min(sb0 + spb, nsb_tile) - 1u;     // meaningful when sb < nsb_tile
-                const uint32_t excl0 = __shfl_sync(0xffffffffu, excl, sb0 & 31u);
-                const uint32_t incl_last = __shfl_sync(0xffffffffu, incl, sb_last & 31u);
-                const uint32_t nsb_blk = sb_last - sb0 + 1u;
-                const uint32_t head_words = 1u + (nsb_blk + 1u) / 2u;
-                const bool leader = sb < nsb_tile && sb == sb0;
-                uint32_t blk_words = leader ? head_words + (incl_last - excl0 + 31u) / 32u : 0u;
-                uint32_t wincl = blk_words;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    uint32_t t = __shfl_up_sync(0xffffffffu, wincl, o);
-                    if (lane >= (uint32_t)o) wincl += t;
-                }
-                const uint32_t wexcl = wincl - blk_words;
-                if (leader) s_blk_wordoff[bi] = wexcl;
-                const uint32_t blk_off = __shfl_sync(0xffffffffu, wexcl, sb0 & 31u);
-                if (sb < nsb_tile) s_sb_bitoff[sb] = 32u * (blk_off + head_words) + (excl - excl0);
-                tile_words = __shfl_sync(0xffffffffu, wincl, 31);
-                uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
-                if (lane == 0) {
-                    s_tile_words = tile_words;
-                    s_blk_wordoff[nblk_tile] = tile_words;
-                    atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)code_bits);
-                }
-            }
-            __syncthreads();
-            tile_words = s_tile_words;
-            if (warp == 0) {                                // chain the tiles while the others emit tokens
-                bool failed;
-                uint64_t off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
-                if (lane == 0) {
-                    s_tile_off = off;
-                    if (failed) s_abort = 1;
-                }
-            }
-        } else {
-            if (G.bucket <= kBLK) {
-                tile_off = first_block * G.rec_words;
-                tile_words = (nblk_tile - 1u) * G.rec_words + 1u +
-                             ((tile_len - (nblk_tile - 1u) * G.bucket) * G.width + 31u) / 32u;
+                if (lane == bi) my_blk_wordoff = W;
+                dst = slot + W + head_words;
+            } else if (G.bucket <= kBLK) {
+                dst = payload + fixed_off + (uint64_t)bi * G.rec_words + 1u;
             } else {
-                tile_off = bucket_idx * G.rec_words + 1u + (uint64_t)bib * (kBLK * G.width / 32u);
-                tile_words = (tile_len * G.width + 31u) / 32u;
+                dst = payload + fixed_off;
+            }
+            uint32_t bits = 0;                              // bits of the block's string so far
+            uint32_t flushed = 0;                           // whole words already written to dst
+            uint32_t my_len = 0;                            // ERC: lane q keeps the token bits of sub-block q
+
+            for (uint32_t cb = 0; cb < bl; cb += kChunk) {
+                const uint32_t win0 = 32u * flushed;        // bit of the block string at window bit 0
+                uint32_t ngroups = 0, ntok = 0;
+
+                // ---- quantize (Definition 1), 128 elements per step ---------------------------
+                if (inv != 0.0f) {
+#pragma unroll 1
+                    for (uint32_t r = 0; r < kChunkRows; ++r) {
+                        const uint32_t base = cb + r * 128u + lane * 4u;        // element within the block
+                        if (cb + r * 128u >= bl) break;
+                        float4 x;
+                        if (base + 4u <= bl) {
+                            x = __ldg(reinterpret_cast<const float4*>(gb + base));
+                        } else {
+                            x.x = base + 0u < bl ? __ldg(gb + base + 0u) : 0.0f;
+                            x.y = base + 1u < bl ? __ldg(gb + base + 1u) : 0.0f;
+                            x.z = base + 2u < bl ? __ldg(gb + base + 2u) : 0.0f;
+                            x.w = 0.0f;
+                        }
+                        const uint64_t ctr = (elem0 + blk_first + base) >> 2;
+                        const uint4 rnd = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, k0, k1);
+                        uint32_t q0, q1, q2, q3;
+                        if (LEVELSET == kLevelsExp) {
+                            q0 = quantize_exp(x.x, inv, top, rnd.x);
+                            q1 = quantize_exp(x.y, inv, top, rnd.y);
+                            q2 = quantize_exp(x.z, inv, top, rnd.z);
+                            q3 = quantize_exp(x.w, inv, top, rnd.w);
+                        } else {
+                            q0 = quantize_uniform(x.x, inv, top, rnd.x);
+                            q1 = quantize_uniform(x.y, inv, top, rnd.y);
+                            q2 = quantize_uniform(x.z, inv, top, rnd.z);
+                            q3 = quantize_uniform(x.w, inv, top, rnd.w);
+                        }
+                        const uint32_t b0 = __float_as_uint(x.x), b1 = __float_as_uint(x.y);
+                        const uint32_t b2 = __float_as_uint(x.z), b3 = __float_as_uint(x.w);
+                        // fields (index | sign << kBits) of the 4 elements, packed; a zero symbol has no sign
+                        uint32_t f01, f23;                   // exponential: f01 holds all four bytes
+                        bool any;
+                        if (LEVELSET == kLevelsExp) {
+                            const uint32_t syms = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
+                            const uint32_t tops =
+                                __byte_perm(__byte_perm(b0, b1, 0x0073), __byte_perm(b2, b3, 0x0073), 0x5410);
+                            const uint32_t nzb = (syms + 0x7F7F7F7Fu) & 0x80808080u;   // bit 7 of a byte: symbol != 0
+                            f01 = syms | (tops & nzb);
+                            f23 = 0;
+                            any = syms != 0;
+                        } else {
+                            f01 = (q0 | (q0 ? (b0 >> 16) & 0x8000u : 0u)) | ((q1 | (q1 ? (b1 >> 16) & 0x8000u : 0u)) << 16);
+                            f23 = (q2 | (q2 ? (b2 >> 16) & 0x8000u : 0u)) | ((q3 | (q3 ? (b3 >> 16) & 0x8000u : 0u)) << 16);
+                            any = (f01 | f23) != 0;
+                        }
+                        if (MODE == kModeErc) {
+                            // keep the groups that hold a nonzero symbol
+                            const uint32_t vote = __ballot_sync(0xffffffffu, any);
+                            if (any) {
+                                uint32_t* ge = M.groups + (ngroups + __popc(vote & lt_mask)) * kGroupWords;
+                                ge[0] = f01;
+                                if (LEVELSET == kLevelsExp) {
+                                    ge[1] = r * 32u + lane;
+                                } else {
+                                    ge[1] = f23;
+                                    ge[2] = r * 32u + lane;
+                                }
+                            }
+                            ngroups += __popc(vote);
+                        } else if (any) {
+                            // fixed-width fields, MSB first, straight into the window
+                            const uint32_t wbits = G.width;
+                            uint32_t f[4];
+                            if (LEVELSET == kLevelsExp) {
+                                f[0] = f01 & 0xFFu; f[1] = (f01 >> 8) & 0xFFu; f[2] = (f01 >> 16) & 0xFFu; f[3] = f01 >> 24;
+                            } else {
+                                f[0] = f01 & 0xFFFFu; f[1] = f01 >> 16; f[2] = f23 & 0xFFFFu; f[3] = f23 >> 16;
+                            }
+                            uint64_t str = 0;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                str = (str << wbits) | ((f[c] & S::kMask) | ((f[c] >> S::kBits) << (wbits - 1u)));
+                                tile_nnz += (f[c] & S::kMask) != 0;
+                            }
+                            or_bits(M.window, base * wbits - win0, str, 4u * wbits);
+                        }
+                    }
+                }
+
+                if (MODE == kModeErc) {
+                    __syncwarp();
+                    // ---- expand the kept groups to one entry per nonzero symbol ---------------------
+                    for (uint32_t g0 = 0; g0 < ngroups; g0 += 32) {
+                        const bool valid = g0 + lane < ngroups;
+                        uint32_t f01 = 0, f23 = 0, gpos = 0;
+                        if (valid) {
+                            const uint32_t* ge = M.groups + (g0 + lane) * kGroupWords;
+                            f01 = ge[0];
+                            if (LEVELSET == kLevelsExp) { gpos = ge[1]; } else { f23 = ge[1]; gpos = ge[2]; }
+                        }
+                        uint32_t f[4];
+                        if (LEVELSET == kLevelsExp) {
+                            f[0] = f01 & 0xFFu; f[1] = (f01 >> 8) & 0xFFu; f[2] = (f01 >> 16) & 0xFFu; f[3] = f01 >> 24;
+                        } else {
+                            f[0] = f01 & 0xFFFFu; f[1] = f01 >> 16; f[2] = f23 & 0xFFFFu; f[3] = f23 >> 16;
+                        }
+                        const uint32_t cnt = (f[0] != 0) + (f[1] != 0) + (f[2] != 0) + (f[3] != 0);
+                        uint32_t incl = cnt;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= (uint32_t)o) incl += t;
+                        }
+                        uint32_t at = ntok + incl - cnt;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            if (f[c]) M.tokens[at++] = (gpos * 4u + (uint32_t)c) | (f[c] << 10);
+                        }
+                        ntok += __shfl_sync(0xffffffffu, incl, 31);
+                    }
+                    __syncwarp();
+
+                    // ---- tokens ERC(gap) sign ERC(index), 32 per step, behind the bit cursor ----------
+                    int carry_pos = -1;                     // position (within the chunk) of the last nonzero so far
+                    uint32_t my_start = 0xFFFFFFFFu;        // lane q < 2: where sub-block q's string starts
+                    for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
+                        const bool valid = t0 + lane < ntok;
+                        const uint32_t e = valid ? M.tokens[t0 + lane] : 0u;
+                        const int pos = (int)(e & 1023u);
+                        const uint32_t field = e >> 10;
+                        int prev = __shfl_up_sync(0xffffffffu, pos, 1);
+                        if (lane == 0) prev = carry_pos;
+                        const bool first_of_sb = (prev >> 8) != (pos >> 8);      // also when there is no predecessor
+                        if (first_of_sb) prev = (pos & ~255) - 1;                  // the run restarts: t_0 = 0
+                        uint32_t tlen = 0, tokA = 0, lenA = 0, tokB = 0, lenB = 0;
+                        if (valid) {
+                            const uint32_t gl = s_lut[pos - prev - 1];
+                            if (LEVELSET == kLevelsExp) {
+                                const uint32_t ll = s_lut_signed[field];
+                                lenB = ll >> 16;
+                                tokA = ((gl & 0xffffu) << lenB) | (ll & 0xffffu);                  // <= 16 + 8 bits
+                                lenA = (gl >> 16) + lenB;
+                                tlen = lenA;
+                            } else {
+                                const uint32_t ll = s_lut[(field & S::kMask) - 1u];
+                                tokA = gl & 0xffffu;
+                                lenA = gl >> 16;
+                                lenB = (ll >> 16) + 1u;                                           // sign + ERC(index) <= 17
+                                tokB = ((field >> S::kBits) << (lenB - 1u)) | (ll & 0xffffu);
+                                tlen = lenA + lenB;
+                            }
+                        }
+                        uint32_t incl = tlen;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= (uint32_t)o) incl += t;
+                        }
+                        const uint32_t off = bits + incl - tlen;    // bit of the block string where my token starts
+                        // the first token of a sub-block marks where that sub-block's string starts
+                        uint32_t starts = __ballot_sync(0xffffffffu, valid && first_of_sb);
+                        while (starts) {
+                            const int src = __ffs(starts) - 1;
+                            starts &= starts - 1;
+                            const uint32_t q = (uint32_t)__shfl_sync(0xffffffffu, pos, src) >> 8;
+                            const uint32_t o = __shfl_sync(0xffffffffu, off, src);
+                            if (lane == q) my_start = o;
+                        }
+                        if (valid) {
+                            if (LEVELSET == kLevelsExp) {
+                                or_bits32(M.window, off - win0, tokA, lenA);
+                            } else {
+                                or_bits32(M.window, off - win0, tokA, lenA);
+                                or_bits32(M.window, off - win0 + lenA, tokB, lenB);
+                            }
+                        }
+                        bits += __shfl_sync(0xffffffffu, incl, 31);
+                        carry_pos = __shfl_sync(0xffffffffu, pos, min(ntok - t0, 32u) - 1u);
+                    }
+                    tile_nnz += ntok;
+                    // sub-block strings follow one another: an empty one starts where the next one does
+                    {
+                        uint32_t s1 = __shfl_sync(0xffffffffu, my_start, 1);
+                        uint32_t s0 = __shfl_sync(0xffffffffu, my_start, 0);
+                        if (s1 == 0xFFFFFFFFu) s1 = bits;
+                        if (s0 == 0xFFFFFFFFu) s0 = s1;
+                        const uint32_t q = cb / kSB;                // first sub-block of this chunk
+                        if (lane == q) my_len = s1 - s0;
+                        if (lane == q + 1u) my_len = bits - s1;
+                    }
+                } else {
+                    bits = min(cb + kChunk, bl) * G.width;
+                }
+
+                // ---- flush the completed words of the window ------------------------------------------
+                __syncwarp();
+                {
+                    const uint32_t full = (bits >> 5) - flushed;
+                    for (uint32_t i = lane; i < full; i += 32) dst[flushed + i] = M.window[i];
+                    const uint32_t partial = M.window[full];
+                    __syncwarp();
+                    for (uint32_t i = lane; i < full + 3u; i += 32) M.window[i] = 0;
+                    __syncwarp();
+                    if (lane == 0) M.window[0] = partial;
+                    __syncwarp();
+                    flushed += full;
+                }
+            }
+
+            // ---- end of the block: last partial word, then the block's header ----------------------------
+            if (bits & 31u) {
+                if (lane == 0) {
+                    dst[flushed] = M.window[0];
+                    M.window[0] = 0;
+                }
+                __syncwarp();
+            }
+            if (MODE == kModeErc) {
+                uint32_t* hdr = slot + W;
+                if (lane == 0) hdr[0] = __float_as_uint(norm);
+                const uint32_t hi = __shfl_down_sync(0xffffffffu, my_len, 1);
+                if (!(lane & 1u) && lane < nsb) hdr[1u + lane / 2u] = my_len | (lane + 1u < nsb ? hi << 16 : 0u);
+                W += head_words + (bits + 31u) / 32u;
+                tile_code_bits += bits;
+            } else {
+                if (lane == 0 && (G.bucket <= kBLK || bib == 0))
+                    payload[G.bucket <= kBLK ? fixed_off + (uint64_t)bi * G.rec_words : bucket_idx * G.rec_words] =
+                        __float_as_uint(norm);
             }
         }
 
-        // ---- emit into the staging buffer -------------------------------------------
+        // ---- ERC: chain the tile to its predecessors, then move its image into the stream ---------------
         if (MODE == kModeErc) {
-            if (tid < nblk_tile) stage[s_blk_wordoff[tid]] = __float_as_uint(s_blk_norm[tid]);
-            if (tid < nsb_tile) {
-                uint32_t bi = tid / spb, sbi = tid - bi * spb;
-                atomicOr(stage + s_blk_wordoff[bi] + 1u + sbi / 2u, s_sb_bits[tid] << (16u * (sbi & 1u)));
-            }
-#pragma unroll
-            for (int j = 0; j < kSbPerWarp; ++j) {
-                const uint32_t sb = warp * kSbPerWarp + j;
-                uint32_t nz = q[j].masks & 0xffu;
-                // the previous nonzero position is needed again; recompute it (cheap)
-                uint32_t last_pos = nz ? lane * 8u + (31u - __clz(nz)) + 1u : 0u;
-                uint32_t any = __ballot_sync(0xffffffffu, nz != 0);
-                uint32_t lower = any & ((1u << lane) - 1u);
-                uint32_t prev = __shfl_sync(0xffffffffu, last_pos, lower ? 31 - __clz(lower) : 0);
-                if (!lower) prev = 0;
-                if (sb >= nsb_tile) continue;
-                uint32_t cursor = s_sb_bitoff[sb] + lane_off[j];
-                while (nz) {
-                    uint32_t e = __ffs(nz) - 1u;
-                    nz &= nz - 1u;
-                    uint32_t pos = lane * 8u + e + 1u;
-                    uint32_t gl = s_lut[pos - prev - 1u], ll = s_lut[sym_of(q[j], e) - 1u];
-                    uint32_t glen = gl >> 16, llen = ll >> 16;
-                    uint64_t sign = (q[j].masks >> (8u + e)) & 1u;
-                    uint64_t token = ((uint64_t)(gl & 0xffffu) << (1u + llen)) | (sign << llen) | (ll & 0xffffu);
-                    uint32_t tlen = glen + 1u + llen;
-                    stage_or(stage, cursor, token, tlen);
-                    cursor += tlen;
-                    prev = pos;
+            const uint32_t tile_words = W;
+            bool failed;
+            const uint64_t tile_off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
+            __syncwarp();
+            if (!failed) {
+                for (uint32_t i = lane; i < tile_words; i += 32) payload[tile_off + i] = __ldcg(slot + i);
+                if (lane < nblk_tile) table[first_block + lane] = 32ull * (tile_off + my_blk_wordoff);
+                if (tile == G.ntiles - 1 && lane == 0) {
+                    table[G.nblk] = 32ull * (tile_off + tile_words);
+                    P.ws->total_words = tile_off + tile_words;
                 }
             }
+            if (lane == 0 && tile_code_bits)
+                atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)tile_code_bits);
         } else {
-            if (G.bucket <= kBLK) {
-                if (tid < nblk_tile) stage[tid * G.rec_words] = __float_as_uint(s_blk_norm[tid]);
-            } else if (bib == 0 && tid == 0) {
-                payload[bucket_idx * G.rec_words] = __float_as_uint(s_blk_norm[0]);
-            }
-            const uint32_t wbits = G.width;
 #pragma unroll
-            for (int j = 0; j < kSbPerWarp; ++j) {
-                const uint32_t sb = warp * kSbPerWarp + j;
-                const uint32_t base = sb * kSB + lane * 8u;
-                if (base >= tile_len) continue;
-                uint32_t bi = G.bucket <= kBLK ? sb / spb : 0u;
-                uint32_t in_blk = base - bi * blk_elems;
-                uint32_t cursor = G.bucket <= kBLK ? 32u * (bi * G.rec_words + 1u) + in_blk * wbits : base * wbits;
-#pragma unroll
-                for (uint32_t e = 0; e < 8; ++e) {
-                    if (base + e >= tile_len) break;
-                    uint32_t field = 0;
-                    if ((q[j].masks >> e) & 1u) field = (((q[j].masks >> (8u + e)) & 1u) << (wbits - 1u)) | sym_of(q[j], e);
-                    if (field) stage_or(stage, cursor, field, wbits);
-                    cursor += wbits;
-                }
-            }
+            for (int o = 16; o > 0; o >>= 1) tile_nnz += __shfl_xor_sync(0xffffffffu, tile_nnz, o);
         }
-        __syncthreads();
 
-        // ---- copy the tile out -------------------------------------------------------
-        if (MODE == kModeErc) tile_off = s_tile_off;
-        const bool aborted = s_abort != 0;
-        for (uint32_t i = tid; i < tile_words; i += kEncThreads) {
-            if (!aborted) payload[tile_off + i] = stage[i];
-            stage[i] = 0;
-        }
-        if (MODE == kModeErc && !aborted) {
-            if (tid < nblk_tile) table[first_block + tid] = 32ull * (tile_off + s_blk_wordoff[tid]);
-            if (tile == G.ntiles - 1 && tid == 0) {
-                table[G.nblk] = 32ull * (tile_off + tile_words);
-                P.ws->total_words = tile_off + tile_words;
-            }
-        }
-        __syncthreads();
-
-        // ---- last tile to finish writes the header ------------------------------------
-        if (tid == 0) {
-            if (s_nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)s_nnz);
+        // ---- last tile to finish writes the header -------------------------------------------------------
+        __syncwarp();
+        if (lane == 0) {
+            if (tile_nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)tile_nnz);
             __threadfence();
             unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), 1ull);
             if (prev == G.ntiles - 1) {
@@ -562,26 +674,28 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
     return cudaGetLastError();
 }
 
+int encode_max_blocks(int sms) { return sms * kEncMinBlocks; }
+
 template <uint32_t L, uint32_t M>
-static cudaError_t launch_one(const EncodeParams& P, int sms, cudaStream_t stream) {
-    size_t smem = (size_t)P.stage_words * 4;
+static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
+    const size_t smem = (size_t)kEncWarps * P.warp_smem_words * 4u;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    uint64_t grid = P.geo.ntiles < (uint64_t)(2 * sms) ? P.geo.ntiles : (uint64_t)(2 * sms);
-    encode_kernel<L, M><<<(unsigned)grid, kEncThreads, smem, stream>>>(P);
+    if (smem > 96 * 1024 || P.grid == 0) return cudaErrorInvalidValue;
+    encode_kernel<L, M><<<P.grid, kEncThreads, smem, stream>>>(P);
     return cudaGetLastError();
 }
 
-cudaError_t launch_encode(const EncodeParams& P, int sms, cudaStream_t stream) {
+cudaError_t launch_encode(const EncodeParams& P, cudaStream_t stream) {
     const bool uni = P.geo.levelset == kLevelsUniform, fixed = P.geo.mode == kModeFixed;
-    if (!uni && !fixed) return launch_one<kLevelsExp, kModeErc>(P, sms, stream);
-    if (!uni && fixed) return launch_one<kLevelsExp, kModeFixed>(P, sms, stream);
-    if (uni && !fixed) return launch_one<kLevelsUniform, kModeErc>(P, sms, stream);
-    return launch_one<kLevelsUniform, kModeFixed>(P, sms, stream);
+    if (!uni && !fixed) return launch_one<kLevelsExp, kModeErc>(P, stream);
+    if (!uni && fixed) return launch_one<kLevelsExp, kModeFixed>(P, stream);
+    if (uni && !fixed) return launch_one<kLevelsUniform, kModeErc>(P, stream);
+    return launch_one<kLevelsUniform, kModeFixed>(P, stream);
 }
 
 }  // namespace nuq
