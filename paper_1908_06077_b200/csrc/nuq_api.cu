@@ -205,6 +205,10 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     P.slots = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + slots_offset(pl));
     P.seed = seed;
     P.offset = offset;
+    for (uint32_t r = 0; r < 10; ++r) {               // Philox key schedule (Weyl sequence)
+        P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
+        P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
+    }
     if (launch_encode(P, stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;
 }

@@ -72,6 +72,7 @@ struct EncodeParams {
     uint64_t* out_bits;
     Workspace* ws;
     uint64_t seed, offset;
+    uint32_t round_keys[20]; // Philox4x32-10 key schedule of `seed`: (k0, k1) of round 0, 1, ..., 9
     uint32_t* slots;         // ERC mode: grid * kEncWarps scratch slots of slot_words words
     uint32_t slot_words;     // capacity of one slot = largest possible tile image
     uint32_t window_words;   // shared-memory bit window of one warp

@@ -54,20 +54,20 @@ cudaError_t upload_erc_lut() {
 // ---------------------------------------------------------------------------
 // Philox4x32-10 (Salmon et al. 2011), one block = the draws of 4 consecutive elements.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
-                                               uint32_t k1) {
+// The ten round keys (key + r * Weyl constants) are precomputed on the host and sit in the
+// kernel's parameter block, so they cost no instructions here.
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const uint32_t (&rk)[20]) {
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         uint64_t p0 = (uint64_t)0xD2511F53u * c0;
         uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
-        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk[2 * r];
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk[2 * r + 1];
         c1 = (uint32_t)p1;
         c3 = (uint32_t)p0;
         c0 = n0;
         c2 = n2;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     return make_uint4(c0, c1, c2, c3);
 }
@@ -139,7 +139,7 @@ __device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile,
         uint64_t v = idx >= 0 ? ld_volatile_u64(state + idx) : kTilePrefix;   // before tile 0: prefix 0
         uint32_t polls = 0;
         while (__any_sync(0xffffffffu, (v >> 62) == 0)) {
-            if (++polls > (1u << 18)) {                    // ~tens of ms: give up, never hang
+            if (++polls > (1u << 16)) {                    // ~tens of ms: give up, never hang
                 if (lane == 0) {
                     latch_status(ws, kErrTimeout);
                     st_volatile_u64(state + tile, kTilePoison);
@@ -147,7 +147,7 @@ __device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile,
                 *failed = true;
                 return 0;
             }
-            __nanosleep(64);
+            __nanosleep(polls < 8 ? 200 : 1000);           // a waiting warp should not eat issue slots
             if ((v >> 62) == 0) v = ld_volatile_u64(state + idx);
         }
         if (__any_sync(0xffffffffu, (v >> 62) == 3)) {     // a predecessor gave up
@@ -216,7 +216,6 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
     uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
     uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
     const float top = __uint_as_float((127u + G.s) << 23);
-    const uint32_t k0 = (uint32_t)P.seed, k1 = (uint32_t)(P.seed >> 32);
     const uint32_t c2 = (uint32_t)P.offset, c3 = (uint32_t)(P.offset >> 32);
     const uint32_t lt_mask = (1u << lane) - 1u;
 
@@ -361,7 +360,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                             x.w = 0.0f;
                         }
                         const uint64_t ctr = (elem0 + blk_first + base) >> 2;
-                        const uint4 rnd = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, k0, k1);
+                        const uint4 rnd = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, P.round_keys);
                         uint32_t q0, q1, q2, q3;
                         if (LEVELSET == kLevelsExp) {
                             q0 = quantize_exp(x.x, inv, top, rnd.x);
