@@ -302,6 +302,7 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     }
     for (uint32_t k = K; k < kMaxK; ++k) P.streams[k] = nullptr;
     P.K = K;
+    P.group = K >= 8 ? 8u : K >= 3 ? 4u : K;            // 1, 2, 4 or 8 streams side by side
     P.acc = acc;
     Workspace* ws = nullptr;
     int dev = 0;

@@ -84,6 +84,7 @@ struct DecodeParams {
     Geometry geo;
     const uint32_t* streams[kMaxK];
     uint32_t K;
+    uint32_t group;          // streams decoded side by side = warps per CTA (1, 2, 4 or 8)
     float* acc;
     Workspace* ws;
 };

@@ -1,13 +1,39 @@
 // DECODE + aggregate (App. A decoding; Algorithm 1, aggregation line): the K
-// workers' containers are decoded and summed into one fp32 vector.  A warp owns
-// a tile of up to 8192 output elements held in shared memory; lane l walks the
-// token chain of sub-block l of the tile, stream after stream in ascending k, so
-// every output element receives its terms in the order k = 0, 1, ... and the
-// result is bit-reproducible.  The tile is written to HBM once.
+// workers' containers are decoded and summed into one fp32 vector.
+//
+// A CTA owns a tile of up to 8192 output elements (32 coding sub-blocks) whose
+// running sums live in shared memory; the tile is written to HBM once.  Streams
+// are taken G at a time (G = 8, or 1 / 2 / 4 when K is smaller); the CTA has G
+// warps and warp w owns the S = 32 / G sub-blocks w*S .. w*S+S-1 of the tile, for
+// every stream of the group.  Three steps per group:
+//
+//   set-up   warp j reads, for stream j of the group, the tile's block offsets,
+//            norms and sub-block token lengths, validates them and leaves one
+//            chain descriptor per sub-block in shared memory.
+//   decode   lane (j, q) of warp w walks the token chain of stream j, sub-block
+//            w*S+q: ERC^-1 gap, sign bit, ERC^-1 level index, by table look-up on
+//            a 32-bit window (12-bit prefix table; longer codes take the loop of
+//            Algorithm 2).  All 32 chains of a warp advance in lock step; the
+//            decoded (position, sign, index) triples go to a per-lane list.
+//   add      for j = 0 .. G-1 in order, the warp adds the listed values of
+//            stream j into its part of the tile.  Entries of one stream hit
+//            distinct elements, so the adds are plain shared-memory updates, and
+//            every element receives its terms in ascending stream order: the
+//            sum is bit-reproducible and equals ((0 + q_0) + q_1) + ... .
+//
+// Lists hold 2048 entries per warp.  If a chain has more tokens than its share,
+// the pass is redone with half as many streams (twice the share); with a single
+// stream left, the lists are filled and added in several rounds, which cannot
+// change the order in which an element receives its terms.  No warp waits on
+// another except at the two block barriers of a group; nothing spins.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 
 namespace nuq {
+
+constexpr uint32_t kLutBits = 12;                       // prefix bits resolved by the ERC^-1 table
+constexpr uint32_t kListEntries = 2048;                 // 16-bit list entries per warp
+constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
 // One Elias-recursive integer from the top of a 64-bit MSB-first window (Algorithm 2,
 // decoding): N = 1; while the next bit is 1, read that bit plus N more as the new N.
@@ -48,10 +74,50 @@ __device__ __forceinline__ float level_times_norm(float norm, uint32_t levelset,
     return __fmul_rn(norm, level);
 }
 
-__global__ void __launch_bounds__(32) decode_kernel(const __grid_constant__ DecodeParams P) {
-    extern __shared__ __align__(16) float tile_acc[];       // kBLK floats
+// ERC^-1 of a 12-bit prefix: value | length << 8, or 0 when the code is longer than the prefix
+// (or is not a code).  Obtained by running Algorithm 2's decoder on the prefix.
+__device__ __forceinline__ uint32_t erc_prefix_entry(uint32_t idx) {
+    uint32_t N = 1, pos = 0;
+    for (int it = 0; it < 6; ++it) {
+        if (pos >= kLutBits) return 0;
+        if (!((idx >> (kLutBits - 1u - pos)) & 1u)) return N | ((pos + 1u) << 8);
+        const uint32_t nb = N + 1u;
+        if (pos + nb > kLutBits) return 0;
+        N = (idx >> (kLutBits - pos - nb)) & ((1u << nb) - 1u);
+        pos += nb;
+    }
+    return 0;
+}
+
+// What the set-up step leaves for the lane that walks sub-block `sb` of one stream.
+struct Chain {
+    const uint32_t* tok;     // ERC: token words of the sub-block's coding block;  fixed: field words of its bucket
+    float norm;
+    uint32_t cur, end;       // ERC: first and past-the-end bit of the chain;  fixed: bit of the first field, unused
+    uint32_t last;           // last valid word index behind tok
+};
+
+// Per stream of the group.
+struct StreamInfo {
+    uint32_t ok, mode, levelset, nlev, width;
+};
+
+__global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_constant__ DecodeParams P) {
+    extern __shared__ __align__(16) unsigned char dsm[];
     const Geometry& G = P.geo;
-    const uint32_t lane = threadIdx.x;
+    const uint32_t NG = P.group;                            // streams per group = warps per CTA (1, 2, 4 or 8)
+    const uint32_t S = 32u / NG;                            // sub-blocks per warp
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    float* acc = reinterpret_cast<float*>(dsm);                                   // kBLK running sums
+    uint16_t* lut = reinterpret_cast<uint16_t*>(dsm + 4u * kBLK);                 // ERC^-1 of 12-bit prefixes
+    Chain* chains = reinterpret_cast<Chain*>(dsm + 4u * kBLK + 2u * (1u << kLutBits));   // [group][32]
+    StreamInfo* infos = reinterpret_cast<StreamInfo*>(chains + kMaxGroup * 32u);  // [group]
+    uint32_t* list = reinterpret_cast<uint32_t*>(infos + kMaxGroup) + warp * (kListEntries / 2u);
+    float* accw = acc + warp * S * kSB;                     // this warp's part of the tile
+
+    for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) lut[i] = (uint16_t)erc_prefix_entry(i);
+    for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
+        *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
 
     for (uint64_t tile = blockIdx.x; tile < G.ntiles; tile += gridDim.x) {
         // ---- tile geometry (same tiling as the encoder) ---------------------------
@@ -77,57 +143,55 @@ __global__ void __launch_bounds__(32) decode_kernel(const __grid_constant__ Deco
             blk_elems = kBLK;
         }
         const uint32_t nsb_tile = (tile_len + kSB - 1) / kSB;
-        const uint32_t sb = lane;
-        const uint32_t bi = sb / spb, sb0 = bi * spb, sbi = sb - sb0;
-        const uint32_t blk_len = min(blk_elems, tile_len - min(tile_len, bi * blk_elems));   // elements of my block
-        const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
-        const uint32_t sn = sb < nsb_tile ? min(kSB, tile_len - sb * kSB) : 0u;              // elements of my sub-block
-        float* mine = tile_acc + sb * kSB;
 
-        for (uint32_t i = lane * 4u; i < kBLK; i += 128u)
-            *reinterpret_cast<float4*>(tile_acc + i) = make_float4(0.f, 0.f, 0.f, 0.f);
-        __syncwarp();
+        for (uint32_t g0 = 0; g0 < P.K; g0 += NG) {
+            const uint32_t gcount = min(NG, P.K - g0);      // streams in this group
+            __syncthreads();                                // the previous descriptors are no longer read
 
-        for (uint32_t k = 0; k < P.K; ++k) {
-            const uint32_t* hdr = P.streams[k];
-            // ---- header validation against the call's arguments ---------------------
-            const uint32_t flags = __ldg(hdr + 6);
-            const uint32_t levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
-            const uint64_t hd = (uint64_t)__ldg(hdr + 2) | ((uint64_t)__ldg(hdr + 3) << 32);
-            const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
-            const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
-            bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
-                      __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
-                      (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
-            const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
-            const uint64_t cwords = cbits >> 5;
-
-            if (ok && mode == kModeErc) {
-                const uint64_t head = kHeaderWords + 2 * (G.nblk + 1);
-                ok = hnblk == G.nblk && cwords > head;
-                bool lane_ok = true;
-                uint32_t cur = 0, endb = 0, last = 0;
-                const uint32_t* tok = hdr;
-                float norm = 0.0f;
-                if (ok) {
-                    const uint64_t* table = reinterpret_cast<const uint64_t*>(hdr + kHeaderWords);
-                    const uint32_t* payload = hdr + head;
-                    const uint64_t payload_words = cwords - head;
+            // ================= set-up: warp j describes stream g0 + j =================
+            if (warp < gcount) {
+                const uint32_t* hdr = P.streams[g0 + warp];
+                const uint32_t sb = lane;
+                const uint32_t flags = __ldg(hdr + 6);
+                const uint32_t levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
+                const uint64_t hd = (uint64_t)__ldg(hdr + 2) | ((uint64_t)__ldg(hdr + 3) << 32);
+                const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
+                const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
+                bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
+                          __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
+                          (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
+                const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
+                const uint32_t width = 1u + (32u - __clz(nlev - 1u));           // fixed mode: sign bit + ceil(log2(levels))
+                const uint64_t cwords = cbits >> 5;
+                const uint32_t bi = sb / spb, sb0 = bi * spb, sbi = sb - sb0;
+                const uint32_t blk_len = min(blk_elems, tile_len - min(tile_len, bi * blk_elems));
+                const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
+                Chain ch;
+                ch.tok = hdr;
+                ch.norm = 0.0f;
+                ch.cur = ch.end = ch.last = 0;
+                if (ok && mode == kModeErc) {
+                    const uint64_t head = kHeaderWords + 2 * (G.nblk + 1);
+                    ok = hnblk == G.nblk && cwords > head;
+                    bool lane_ok = true;
                     uint32_t len = 0, head_words = 0, rec_words = 0;
-                    if (sb < nsb_tile) {
-                        uint64_t off = __ldg(table + first_block + bi), end = __ldg(table + first_block + bi + 1);
+                    if (ok && sb < nsb_tile) {
+                        const uint64_t* table = reinterpret_cast<const uint64_t*>(hdr + kHeaderWords);
+                        const uint32_t* payload = hdr + head;
+                        const uint64_t payload_words = cwords - head;
+                        const uint64_t off = __ldg(table + first_block + bi), end = __ldg(table + first_block + bi + 1);
                         head_words = 1u + (nsb_blk + 1u) / 2u;
                         lane_ok = (off & 31u) == 0 && (end & 31u) == 0 && off < end && (end >> 5) <= payload_words &&
                                   ((end - off) >> 5) >= head_words && ((end - off) >> 5) <= (1u << 20);
                         if (lane_ok) {
                             const uint32_t* rec = payload + (off >> 5);
                             rec_words = (uint32_t)((end - off) >> 5);
-                            norm = __uint_as_float(__ldg(rec));
+                            ch.norm = __uint_as_float(__ldg(rec));
                             len = (__ldg(rec + 1u + sbi / 2u) >> (16u * (sbi & 1u))) & 0xffffu;
-                            tok = rec + head_words;
+                            ch.tok = rec + head_words;
                         }
                     }
-                    // start of my chain = sum of the lengths of the earlier sub-blocks of my block
+                    // start of a chain = sum of the lengths of the earlier sub-blocks of its block
                     uint32_t incl = len;
 #pragma unroll
                     for (int o = 1; o < 32; o <<= 1) {
@@ -135,96 +199,213 @@ __global__ void __launch_bounds__(32) decode_kernel(const __grid_constant__ Deco
                         if (lane >= (uint32_t)o) incl += t;
                     }
                     const uint32_t excl0 = __shfl_sync(0xffffffffu, incl - len, sb0 & 31u);
-                    cur = incl - len - excl0;
-                    endb = cur + len;
-                    if (sb < nsb_tile && lane_ok) {
-                        uint32_t tok_words = rec_words - head_words;
-                        lane_ok = endb <= 32u * tok_words;
-                        last = tok_words ? tok_words - 1u : 0u;
+                    ch.cur = incl - len - excl0;
+                    ch.end = ch.cur + len;
+                    if (ok && sb < nsb_tile && lane_ok) {
+                        const uint32_t tok_words = rec_words - head_words;
+                        lane_ok = ch.end <= 32u * tok_words;
+                        ch.last = tok_words ? tok_words - 1u : 0u;
+                    }
+                    ok = __all_sync(0xffffffffu, ok && lane_ok);
+                } else if (ok) {
+                    const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
+                    const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
+                    ok = hnblk == G.nb &&
+                         cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
+                    if (ok && sb < nsb_tile) {
+                        const uint32_t* payload = hdr + kHeaderWords;
+                        const uint64_t bucket_of_sb = G.bucket <= kBLK ? first_block + bi : bucket_idx;
+                        const uint32_t* rec = payload + bucket_of_sb * rec_words;
+                        const uint64_t bucket_len = bucket_of_sb == G.nb - 1 ? last_len : G.bucket;
+                        ch.norm = __uint_as_float(__ldg(rec));
+                        ch.tok = rec + 1;
+                        ch.cur = (G.bucket <= kBLK ? sbi * kSB : bib * kBLK + sb * kSB) * width;   // bit of the first field
+                        ch.last = (uint32_t)((bucket_len * width + 31) / 32) - 1u;
                     }
                 }
-                if (!__all_sync(0xffffffffu, ok && lane_ok)) ok = false;
-                if (ok && sb < nsb_tile) {
-                    // ---- the token walk: ERC^-1 gap, sign bit, ERC^-1 level index ----------
-                    uint32_t pos = 0;
-                    while (cur < endb) {
-                        uint64_t win = window64(tok, cur, last);
-                        uint32_t used = 0, gap, sym;
-                        bool good = erc_read(win, used, gap);
-                        uint32_t negative = (uint32_t)(win >> 63);
-                        win <<= 1;
-                        used += 1;
-                        good = good && erc_read(win, used, sym);
-                        pos += gap;
-                        if (!good || used > endb - cur || pos > sn || sym == 0 || sym >= nlev) {
-                            ok = false;
-                            break;
-                        }
-                        float v = level_times_norm(norm, levelset, G.s, sym);
-                        mine[pos - 1u] += negative ? -v : v;
-                        cur += used;
-                    }
-                }
-            } else if (ok) {
-                // ---- fixed-width fields ------------------------------------------------------
-                const uint32_t w = 1u + (32u - __clz(nlev - 1u));           // sign bit + ceil(log2(levels))
-                const uint32_t rec_words = 1u + (G.bucket * w + 31u) / 32u;
-                const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
-                ok = hnblk == G.nb &&
-                     cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * w + 31) / 32;
-                if (ok && sb < nsb_tile) {
-                    const uint32_t* payload = hdr + kHeaderWords;
-                    uint64_t bucket_of_sb = G.bucket <= kBLK ? first_block + bi : bucket_idx;
-                    const uint32_t* rec = payload + bucket_of_sb * rec_words;
-                    uint32_t in_bucket = G.bucket <= kBLK ? sbi * kSB : bib * kBLK + sb * kSB;
-                    float norm = __uint_as_float(__ldg(rec));
-                    uint64_t bucket_len = bucket_of_sb == G.nb - 1 ? last_len : G.bucket;
-                    uint32_t lastw = (uint32_t)((bucket_len * w + 31) / 32) - 1u;
-                    const uint32_t* fields = rec + 1;
-                    for (uint32_t e = 0; e < sn; ++e) {
-                        uint32_t cur = (in_bucket + e) * w;
-                        uint32_t wi = cur >> 5, sh = cur & 31u;
-                        uint64_t two = (uint64_t)__ldg(fields + wi) << 32 | __ldg(fields + min(wi + 1u, lastw));
-                        uint32_t field = (uint32_t)((two << sh) >> (64u - w));
-                        uint32_t sym = field & ((1u << (w - 1u)) - 1u);
-                        if (sym >= nlev) { ok = false; break; }
-                        if (sym) {
-                            float v = level_times_norm(norm, levelset, G.s, sym);
-                            mine[e] += (field >> (w - 1u)) ? -v : v;
-                        }
-                    }
+                chains[warp * 32u + sb] = ch;
+                if (lane == 0) {
+                    StreamInfo si;
+                    si.ok = ok ? 1u : 0u;
+                    si.mode = mode;
+                    si.levelset = levelset;
+                    si.nlev = nlev;
+                    si.width = width;
+                    infos[warp] = si;
+                    if (!ok) latch_status(P.ws, kErrBadStream);
                 }
             }
-            if (!__all_sync(0xffffffffu, ok)) {
-                if (lane == 0) latch_status(P.ws, kErrBadStream);
+            __syncthreads();
+
+            // ================= decode + add, warp-local =================
+            // lane (j, q): stream g0 + j, sub-block warp * S + q
+            const uint32_t lj = lane / S, lq = lane - lj * S;
+            const uint32_t my_sb = warp * S + lq;
+            const uint32_t my_sn = my_sb < nsb_tile ? min(kSB, tile_len - my_sb * kSB) : 0u;   // elements of my sub-block
+            bool wide = false;                              // index - 1 does not fit 7 bits (uniform levels, s = 8)
+            for (uint32_t j = 0; j < gcount; ++j) wide = wide || (infos[j].ok && infos[j].nlev > 129u);
+            const uint32_t entries = wide ? kListEntries / 2u : kListEntries;
+            uint32_t width_now = 1;                         // streams decoded side by side; halves when a list overflows
+            while (width_now < gcount) width_now <<= 1;
+
+            for (uint32_t j0 = 0; j0 < gcount;) {
+                const uint32_t nact = width_now * S;        // lanes that own a chain in this pass
+                const uint32_t cap = entries / nact;        // list entries per chain
+                const bool mine = lj >= j0 && lj < j0 + width_now && lj < gcount;
+                const uint32_t a = (lj - j0) * S + lq;      // my column in the interleaved list
+                const StreamInfo si = infos[mine ? lj : 0];
+                const Chain ch = chains[(mine ? lj : 0) * 32u + my_sb];
+                bool running = mine && si.ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
+                bool bad = false, retry = false;
+                uint32_t cur = ch.cur, pos = 0;
+                // One round fills the lists and adds them.  More than one round happens only when a
+                // single stream is being decoded (width_now == 1), where the order of the rounds
+                // cannot change the order in which an element receives its terms.
+                for (uint32_t round = 0;; ++round) {
+                    uint32_t n = 0;
+                    bool full = false;
+                    while (__any_sync(0xffffffffu, running)) {
+                        if (running) {
+                            const uint32_t wi = cur >> 5;
+                            const uint32_t x0 = __ldg(ch.tok + min(wi, ch.last));
+                            const uint32_t x1 = __ldg(ch.tok + min(wi + 1u, ch.last));
+                            const uint32_t win = __funnelshift_l(x1, x0, cur);              // 32 bits from the cursor
+                            uint32_t gap = 0, sym = 0, negative = 0, used = 0;
+                            const uint32_t e1 = lut[win >> (32u - kLutBits)];
+                            uint32_t e2 = 0;
+                            if (e1) {
+                                const uint32_t t = win << (e1 >> 8);                        // the sign bit is on top
+                                e2 = lut[(t << 1) >> (32u - kLutBits)];
+                                gap = e1 & 0xffu;
+                                negative = t >> 31;
+                                sym = e2 & 0xffu;
+                                used = (e1 >> 8) + 1u + (e2 >> 8);
+                            }
+                            bool good = e2 != 0;
+                            if (!good) {                    // a code longer than 12 bits: Algorithm 2 as a loop
+                                uint64_t win64 = window64(ch.tok, cur, ch.last);
+                                used = 0;
+                                good = erc_read(win64, used, gap);
+                                negative = (uint32_t)(win64 >> 63);
+                                win64 <<= 1;
+                                used += 1;
+                                good = good && erc_read(win64, used, sym);
+                            }
+                            const uint32_t npos = pos + gap;
+                            if (!good || used > ch.end - cur || npos > my_sn || sym == 0 || sym >= si.nlev) {
+                                bad = true;
+                                running = false;
+                            } else if (n == cap) {          // list full: this token waits for the next round
+                                full = true;
+                                running = false;
+                            } else {
+                                const uint32_t e = (npos - 1u) | (negative << 8) | ((sym - 1u) << 9);
+                                if (wide) list[n * nact + a] = e;
+                                else reinterpret_cast<uint16_t*>(list)[n * nact + a] = (uint16_t)e;
+                                ++n;
+                                pos = npos;
+                                cur += used;
+                                running = cur < ch.end;
+                            }
+                        }
+                    }
+                    const bool any_full = __any_sync(0xffffffffu, full);
+                    if (any_full && width_now > 1u) {       // twice the list share per chain; start the pass again
+                        retry = true;
+                        break;
+                    }
+                    __syncwarp();
+
+                    // ---- add, one stream after the other ----
+                    const uint32_t per_chain = 32u / S;     // lanes that share one chain's list
+                    const uint32_t c = lane / per_chain, i0 = lane - c * per_chain;
+                    for (uint32_t j = j0; j < min(j0 + width_now, gcount); ++j) {
+                        const StreamInfo sj = infos[j];
+                        const uint32_t owner = j * S + c;   // the lane that decoded chain (j, c)
+                        const uint32_t n_c = __shfl_sync(0xffffffffu, n, owner);
+                        const float norm_c = __shfl_sync(0xffffffffu, ch.norm, owner);
+                        if (!sj.ok) continue;
+                        if (sj.mode == kModeErc) {
+                            const uint32_t col = (j - j0) * S + c;
+                            float* part = accw + c * kSB;
+                            for (uint32_t i = i0; i < n_c; i += per_chain) {
+                                const uint32_t e = wide ? list[i * nact + col]
+                                                        : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * nact + col];
+                                const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
+                                part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
+                            }
+                        } else if (round == 0) {
+                            // fixed-width fields: every element of the warp's sub-blocks has one
+                            bool field_bad = false;
+                            for (uint32_t idx = lane; idx < S * kSB; idx += 32) {
+                                const uint32_t q = idx >> 8, p = idx & 255u, sb = warp * S + q;
+                                if (sb >= nsb_tile || sb * kSB + p >= tile_len) continue;
+                                const Chain cf = chains[j * 32u + sb];
+                                const uint32_t bit = cf.cur + p * sj.width;
+                                const uint32_t wi = bit >> 5;
+                                const uint32_t x0 = __ldg(cf.tok + min(wi, cf.last));
+                                const uint32_t x1 = __ldg(cf.tok + min(wi + 1u, cf.last));
+                                const uint32_t field = __funnelshift_l(x1, x0, bit) >> (32u - sj.width);
+                                const uint32_t sym = field & ((1u << (sj.width - 1u)) - 1u);
+                                if (sym >= sj.nlev) { field_bad = true; continue; }
+                                if (sym) {
+                                    const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
+                                    accw[idx] += (field >> (sj.width - 1u)) ? -v : v;
+                                }
+                            }
+                            if (__any_sync(0xffffffffu, field_bad) && lane == 0) latch_status(P.ws, kErrBadStream);
+                        }
+                        __syncwarp();
+                    }
+                    if (!any_full) break;
+                    running = full;                         // the chains that stopped at a full list go on
+                }
+                if (__any_sync(0xffffffffu, bad) && lane == 0) latch_status(P.ws, kErrBadStream);
+                if (retry) {
+                    width_now >>= 1;
+                    continue;
+                }
+                j0 += width_now;
             }
         }
-        __syncwarp();
 
-        // ---- write the tile once ----------------------------------------------------------
-        float* dst = P.acc + elem0;
-        for (uint32_t i = lane * 4u; i < tile_len; i += 128u) {
-            if (i + 4u <= tile_len) {
-                *reinterpret_cast<float4*>(dst + i) = *reinterpret_cast<const float4*>(tile_acc + i);
-            } else {
-                for (uint32_t e = i; e < tile_len; ++e) dst[e] = tile_acc[e];
+        // ---- write this warp's part of the tile once, and clear it for the next tile ----
+        __syncwarp();
+        {
+            const uint32_t first = warp * S * kSB;
+            float* dst = P.acc + elem0 + first;
+            for (uint32_t i = lane * 4u; i < S * kSB; i += 128u) {
+                if (first + i + 4u <= tile_len) {
+                    *reinterpret_cast<float4*>(dst + i) = *reinterpret_cast<const float4*>(accw + i);
+                } else {
+                    for (uint32_t e = i; e < i + 4u && first + e < tile_len; ++e) dst[e] = accw[e];
+                }
+                *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
         __syncwarp();
     }
 }
 
+static size_t decode_smem_bytes(uint32_t group) {
+    return 4u * kBLK + 2u * (1u << kLutBits) + kMaxGroup * 32u * sizeof(Chain) + kMaxGroup * sizeof(StreamInfo) +
+           (size_t)group * kListEntries * 2u;
+}
+
 cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     static bool attr_set = false;
-    const size_t smem = kBLK * sizeof(float);
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    uint64_t cap = (uint64_t)sms * 6 * 4;
-    uint64_t grid = P.geo.ntiles < cap ? P.geo.ntiles : cap;
-    decode_kernel<<<(unsigned)grid, 32, smem, stream>>>(P);
+    const size_t smem = decode_smem_bytes(P.group);
+    uint64_t resident = 220u * 1024u / (smem + 1024u);                      // CTAs per SM by shared memory
+    if (resident < 1) resident = 1;
+    if (resident * P.group > 48) resident = 48 / P.group;                   // and by warps worth keeping resident
+    const uint64_t cap = (uint64_t)sms * resident;
+    const uint64_t grid = P.geo.ntiles < cap ? P.geo.ntiles : cap;
+    decode_kernel<<<(unsigned)grid, 32u * P.group, smem, stream>>>(P);
     return cudaGetLastError();
 }
 
