@@ -21,7 +21,7 @@
 //            every element receives its terms in ascending stream order: the
 //            sum is bit-reproducible and equals ((0 + q_0) + q_1) + ... .
 //
-// Lists hold 2048 entries per warp.  If a chain has more tokens than its share,
+// Lists hold 1792 entries per warp.  If a chain has more tokens than its share,
 // the pass is redone with half as many streams (twice the share); with a single
 // stream left, the lists are filled and added in several rounds, which cannot
 // change the order in which an element receives its terms.  No warp waits on
@@ -32,7 +32,7 @@
 namespace nuq {
 
 constexpr uint32_t kLutBits = 12;                       // prefix bits resolved by the ERC^-1 table
-constexpr uint32_t kListEntries = 2048;                 // 16-bit list entries per warp
+constexpr uint32_t kListEntries = 1792;                 // 16-bit list entries per warp (3 CTAs of 8 warps per SM)
 constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
 // One Elias-recursive integer from the top of a 64-bit MSB-first window (Algorithm 2,
@@ -264,25 +264,24 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 for (uint32_t round = 0;; ++round) {
                     uint32_t n = 0;
                     bool full = false;
+                    // Every lane executes every step (a lane whose chain has ended works on stale but
+                    // in-bounds data and commits nothing), so the loop body has no divergent branch
+                    // except the rare long-code path.
+                    uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + a;
+                    uint32_t* slot32 = list + a;
                     while (__any_sync(0xffffffffu, running)) {
-                        if (running) {
-                            const uint32_t wi = cur >> 5;
-                            const uint32_t x0 = __ldg(ch.tok + min(wi, ch.last));
-                            const uint32_t x1 = __ldg(ch.tok + min(wi + 1u, ch.last));
-                            const uint32_t win = __funnelshift_l(x1, x0, cur);              // 32 bits from the cursor
-                            uint32_t gap = 0, sym = 0, negative = 0, used = 0;
-                            const uint32_t e1 = lut[win >> (32u - kLutBits)];
-                            uint32_t e2 = 0;
-                            if (e1) {
-                                const uint32_t t = win << (e1 >> 8);                        // the sign bit is on top
-                                e2 = lut[(t << 1) >> (32u - kLutBits)];
-                                gap = e1 & 0xffu;
-                                negative = t >> 31;
-                                sym = e2 & 0xffu;
-                                used = (e1 >> 8) + 1u + (e2 >> 8);
-                            }
-                            bool good = e2 != 0;
-                            if (!good) {                    // a code longer than 12 bits: Algorithm 2 as a loop
+                        const uint32_t wi = cur >> 5;
+                        const uint32_t x0 = __ldg(ch.tok + min(wi, ch.last));
+                        const uint32_t x1 = __ldg(ch.tok + min(wi + 1u, ch.last));
+                        const uint32_t win = __funnelshift_l(x1, x0, cur);                  // 32 bits from the cursor
+                        const uint32_t e1 = lut[win >> (32u - kLutBits)];
+                        const uint32_t t = win << (e1 >> 8);                                // the sign bit is on top
+                        const uint32_t e2 = lut[(t << 1) >> (32u - kLutBits)];
+                        uint32_t gap = e1 & 0xffu, sym = e2 & 0xffu, negative = t >> 31;
+                        uint32_t used = (e1 >> 8) + 1u + (e2 >> 8);
+                        bool good = e1 != 0 && e2 != 0;
+                        if (__any_sync(0xffffffffu, running && !good)) {
+                            if (running && !good) {         // a code longer than 12 bits: Algorithm 2 as a loop
                                 uint64_t win64 = window64(ch.tok, cur, ch.last);
                                 used = 0;
                                 good = erc_read(win64, used, gap);
@@ -291,23 +290,22 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                                 used += 1;
                                 good = good && erc_read(win64, used, sym);
                             }
-                            const uint32_t npos = pos + gap;
-                            if (!good || used > ch.end - cur || npos > my_sn || sym == 0 || sym >= si.nlev) {
-                                bad = true;
-                                running = false;
-                            } else if (n == cap) {          // list full: this token waits for the next round
-                                full = true;
-                                running = false;
-                            } else {
-                                const uint32_t e = (npos - 1u) | (negative << 8) | ((sym - 1u) << 9);
-                                if (wide) list[n * nact + a] = e;
-                                else reinterpret_cast<uint16_t*>(list)[n * nact + a] = (uint16_t)e;
-                                ++n;
-                                pos = npos;
-                                cur += used;
-                                running = cur < ch.end;
-                            }
                         }
+                        const uint32_t npos = pos + gap;
+                        const bool valid = good && used <= ch.end - cur && npos <= my_sn && sym != 0 && sym < si.nlev;
+                        const bool room = n < cap;
+                        const bool commit = running && valid && room;
+                        bad = bad || (running && !valid);
+                        full = full || (running && valid && !room);      // this token waits for the next round
+                        if (commit) {
+                            const uint32_t e = (npos - 1u) | (negative << 8) | ((sym - 1u) << 9);
+                            if (wide) slot32[n * nact] = e;
+                            else slot16[n * nact] = (uint16_t)e;
+                            pos = npos;
+                            cur += used;
+                            ++n;
+                        }
+                        running = commit && cur < ch.end;
                     }
                     const bool any_full = __any_sync(0xffffffffu, full);
                     if (any_full && width_now > 1u) {       // twice the list share per chain; start the pass again
@@ -328,11 +326,23 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                         if (sj.mode == kModeErc) {
                             const uint32_t col = (j - j0) * S + c;
                             float* part = accw + c * kSB;
-                            for (uint32_t i = i0; i < n_c; i += per_chain) {
-                                const uint32_t e = wide ? list[i * nact + col]
-                                                        : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * nact + col];
-                                const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
-                                part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
+                            if (!wide && sj.levelset == kLevelsExp) {
+                                // value = +-norm * 2^(index - 1 - s): the exponent field is built from the entry
+                                const uint16_t* src = reinterpret_cast<const uint16_t*>(list) + col;
+                                const uint32_t ebias = 127u - G.s;              // (index - 1) + ebias = biased exponent
+                                for (uint32_t i = i0; i < n_c; i += per_chain) {
+                                    const uint32_t e = src[i * nact];
+                                    const float level = __uint_as_float(((e >> 9) + ebias) << 23);
+                                    const float v = __fmul_rn(norm_c, level);
+                                    part[e & 0xffu] += __uint_as_float(__float_as_uint(v) ^ ((e << 23) & 0x80000000u));
+                                }
+                            } else {
+                                for (uint32_t i = i0; i < n_c; i += per_chain) {
+                                    const uint32_t e = wide ? list[i * nact + col]
+                                                            : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * nact + col];
+                                    const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
+                                    part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
+                                }
                             }
                         } else if (round == 0) {
                             // fixed-width fields: every element of the warp's sub-blocks has one
