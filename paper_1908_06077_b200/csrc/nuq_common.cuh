@@ -41,7 +41,8 @@ struct Workspace {
     uint64_t code_bits;     // token bits of the whole call
     uint64_t nnz;           // nonzero symbols of the whole call
     uint64_t total_words;   // payload words of the whole call
-    uint64_t reserved[2];
+    uint64_t dec_ticket;    // decoder: next tile to hand out (cleared before each decode launch)
+    uint64_t reserved[1];
     // followed by: uint64_t tile_state[ntiles], float norms[nb] for wide buckets, then (16-byte
     // aligned) one scratch slot per encoder warp that holds the image of the tile it is working on
 };

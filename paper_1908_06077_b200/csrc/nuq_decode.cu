@@ -21,7 +21,7 @@
 //            every element receives its terms in ascending stream order: the
 //            sum is bit-reproducible and equals ((0 + q_0) + q_1) + ... .
 //
-// Lists hold 1792 entries per warp.  If a chain has more tokens than its share,
+// Lists hold 1536 entries per warp.  If a chain has more tokens than its share,
 // the pass is redone with half as many streams (twice the share); with a single
 // stream left, the lists are filled and added in several rounds, which cannot
 // change the order in which an element receives its terms.  No warp waits on
@@ -32,7 +32,7 @@
 namespace nuq {
 
 constexpr uint32_t kLutBits = 12;                       // prefix bits resolved by the ERC^-1 table
-constexpr uint32_t kListEntries = 1792;                 // 16-bit list entries per warp (3 CTAs of 8 warps per SM)
+constexpr uint32_t kListEntries = 1536;                 // 16-bit list entries per warp (3 CTAs of 8 warps per SM)
 constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
 // One Elias-recursive integer from the top of a 64-bit MSB-first window (Algorithm 2,
@@ -102,6 +102,13 @@ struct StreamInfo {
     uint32_t ok, mode, levelset, nlev, width;
 };
 
+// Per stream of the call: what its header says, checked once per CTA.
+struct StreamHead {
+    const uint32_t* hdr;
+    uint64_t cwords;         // container words the header declares
+    uint32_t ok, mode, levelset, nlev, width, pad;
+};
+
 __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
     const Geometry& G = P.geo;
@@ -112,14 +119,50 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
     uint16_t* lut = reinterpret_cast<uint16_t*>(dsm + 4u * kBLK);                 // ERC^-1 of 12-bit prefixes
     Chain* chains = reinterpret_cast<Chain*>(dsm + 4u * kBLK + 2u * (1u << kLutBits));   // [group][32]
     StreamInfo* infos = reinterpret_cast<StreamInfo*>(chains + kMaxGroup * 32u);  // [group]
-    uint32_t* list = reinterpret_cast<uint32_t*>(infos + kMaxGroup) + warp * (kListEntries / 2u);
+    StreamHead* heads = reinterpret_cast<StreamHead*>(infos + kMaxGroup);         // [kMaxK]
+    uint32_t* list = reinterpret_cast<uint32_t*>(heads + kMaxK) + warp * (kListEntries / 2u);
     float* accw = acc + warp * S * kSB;                     // this warp's part of the tile
 
     for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) lut[i] = (uint16_t)erc_prefix_entry(i);
+    // ---- header validation against the call's arguments, once per stream ----
+    for (uint32_t k = threadIdx.x; k < P.K; k += blockDim.x) {
+        const uint32_t* hdr = P.streams[k];
+        const uint32_t flags = __ldg(hdr + 6);
+        const uint32_t levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
+        const uint64_t hd = (uint64_t)__ldg(hdr + 2) | ((uint64_t)__ldg(hdr + 3) << 32);
+        const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
+        const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
+        bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
+                  __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
+                  (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
+        const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
+        const uint32_t width = 1u + (32u - __clz(nlev - 1u));                   // fixed mode: sign bit + ceil(log2(levels))
+        const uint64_t cwords = cbits >> 5;
+        if (ok && mode == kModeErc) {
+            ok = hnblk == G.nblk && cwords > kHeaderWords + 2 * (G.nblk + 1);
+        } else if (ok) {
+            const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
+            const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
+            ok = hnblk == G.nb &&
+                 cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
+        }
+        StreamHead h;
+        h.hdr = hdr; h.cwords = cwords; h.ok = ok ? 1u : 0u; h.mode = mode; h.levelset = levelset;
+        h.nlev = nlev; h.width = width; h.pad = 0;
+        heads[k] = h;
+        if (!ok) latch_status(P.ws, kErrBadStream);
+    }
     for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
         *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    for (uint64_t tile = blockIdx.x; tile < G.ntiles; tile += gridDim.x) {
+    __shared__ unsigned long long s_tile;
+    for (;;) {
+        // tiles are handed out one at a time: their cost varies with the density of the streams
+        __syncthreads();
+        if (threadIdx.x == 0) s_tile = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        __syncthreads();
+        const uint64_t tile = s_tile;
+        if (tile >= G.ntiles) break;
         // ---- tile geometry (same tiling as the encoder) ---------------------------
         uint64_t elem0, first_block, bucket_idx = 0;
         uint32_t tile_len, spb, blk_elems, bib = 0;
@@ -150,19 +193,12 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
 
             // ================= set-up: warp j describes stream g0 + j =================
             if (warp < gcount) {
-                const uint32_t* hdr = P.streams[g0 + warp];
+                const StreamHead hd = heads[g0 + warp];
+                const uint32_t* hdr = hd.hdr;
                 const uint32_t sb = lane;
-                const uint32_t flags = __ldg(hdr + 6);
-                const uint32_t levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
-                const uint64_t hd = (uint64_t)__ldg(hdr + 2) | ((uint64_t)__ldg(hdr + 3) << 32);
-                const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
-                const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
-                bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
-                          __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
-                          (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
-                const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
-                const uint32_t width = 1u + (32u - __clz(nlev - 1u));           // fixed mode: sign bit + ceil(log2(levels))
-                const uint64_t cwords = cbits >> 5;
+                bool ok = hd.ok != 0;
+                const uint32_t levelset = hd.levelset, mode = hd.mode, nlev = hd.nlev, width = hd.width;
+                const uint64_t cwords = hd.cwords;
                 const uint32_t bi = sb / spb, sb0 = bi * spb, sbi = sb - sb0;
                 const uint32_t blk_len = min(blk_elems, tile_len - min(tile_len, bi * blk_elems));
                 const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
@@ -172,7 +208,6 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 ch.cur = ch.end = ch.last = 0;
                 if (ok && mode == kModeErc) {
                     const uint64_t head = kHeaderWords + 2 * (G.nblk + 1);
-                    ok = hnblk == G.nblk && cwords > head;
                     bool lane_ok = true;
                     uint32_t len = 0, head_words = 0, rec_words = 0;
                     if (ok && sb < nsb_tile) {
@@ -210,9 +245,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 } else if (ok) {
                     const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
                     const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
-                    ok = hnblk == G.nb &&
-                         cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
-                    if (ok && sb < nsb_tile) {
+                    if (sb < nsb_tile) {
                         const uint32_t* payload = hdr + kHeaderWords;
                         const uint64_t bucket_of_sb = G.bucket <= kBLK ? first_block + bi : bucket_idx;
                         const uint32_t* rec = payload + bucket_of_sb * rec_words;
@@ -232,7 +265,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                     si.nlev = nlev;
                     si.width = width;
                     infos[warp] = si;
-                    if (!ok) latch_status(P.ws, kErrBadStream);
+                    if (!ok && hd.ok) latch_status(P.ws, kErrBadStream);
                 }
             }
             __syncthreads();
@@ -398,7 +431,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
 }
 
 static size_t decode_smem_bytes(uint32_t group) {
-    return 4u * kBLK + 2u * (1u << kLutBits) + kMaxGroup * 32u * sizeof(Chain) + kMaxGroup * sizeof(StreamInfo) +
+    return 4u * kBLK + 2u * (1u << kLutBits) + kMaxGroup * 32u * sizeof(Chain) + kMaxGroup * sizeof(StreamInfo) + kMaxK * sizeof(StreamHead) +
            (size_t)group * kListEntries * 2u;
 }
 
@@ -410,9 +443,10 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
         attr_set = true;
     }
     const size_t smem = decode_smem_bytes(P.group);
-    uint64_t resident = 220u * 1024u / (smem + 1024u);                      // CTAs per SM by shared memory
+    uint64_t resident = 228u * 1024u / (smem + 1024u);                      // CTAs per SM by shared memory
     if (resident < 1) resident = 1;
     if (resident * P.group > 48) resident = 48 / P.group;                   // and by warps worth keeping resident
+    if (cudaMemsetAsync(&P.ws->dec_ticket, 0, sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;
     const uint64_t cap = (uint64_t)sms * resident;
     const uint64_t grid = P.geo.ntiles < cap ? P.geo.ntiles : cap;
     decode_kernel<<<(unsigned)grid, 32u * P.group, smem, stream>>>(P);
