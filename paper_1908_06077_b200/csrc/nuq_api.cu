@@ -151,7 +151,6 @@ using namespace nuq;
 struct EncodePlan {
     size_t state_bytes;      // control block + one look-back word per tile
     size_t norms_bytes;      // bucket norms for buckets wider than a tile
-    size_t slot_bytes;       // one warp's tile image (ERC mode), 0 in the fixed-width mode
     uint32_t want_grid;      // CTAs that give every SM its full share
 };
 
@@ -160,23 +159,21 @@ static EncodePlan plan_encode(EncodeParams& P, int sms) {
     EncodePlan pl;
     pl.state_bytes = sizeof(Workspace) + 8 * G.ntiles;
     pl.norms_bytes = G.bucket > kBLK ? 4 * G.nb : 0;
-    P.slot_words = G.mode == kModeErc ? (stage_words_for(G) + 3u) & ~3u : 0u;
-    pl.slot_bytes = 4u * (size_t)P.slot_words;
-    const uint32_t bits_per_elem = G.mode == kModeErc ? 2u + max_level_code_bits(G) : G.width;
-    P.window_words = (kEncChunk * bits_per_elem + 31u) / 32u + 4u;
-    const uint32_t group_words = G.levelset == kLevelsExp ? 2u : 3u;
-    P.warp_smem_words = P.window_words + (G.mode == kModeErc ? kEncChunk + (kEncChunk / 4u) * group_words : 0u);
-    P.warp_smem_words = (P.warp_smem_words + 3u) & ~3u;
-    const uint64_t need = (G.ntiles + kEncWarps - 1) / kEncWarps;
-    const uint64_t cap = (uint64_t)encode_max_blocks(sms);
-    pl.want_grid = (uint32_t)(need < cap ? need : cap);
+    P.stage_words = (stage_words_for(G) + 3u) & ~3u;
+    if (G.mode == kModeErc) {
+        P.window_words = (kBLK / kEncWarps * (2u + max_level_code_bits(G)) + 31u) / 32u + 4u;
+        P.warp_smem_words = (P.window_words + kEncChunk + 3u) & ~3u;
+    } else {
+        P.window_words = 0;
+        P.warp_smem_words = 0;
+    }
+    const uint64_t cap = (uint64_t)encode_max_blocks(sms, encode_smem_bytes(P));
+    pl.want_grid = (uint32_t)(G.ntiles < cap ? G.ntiles : cap);
     return pl;
 }
 
-static size_t slots_offset(const EncodePlan& pl) { return (pl.state_bytes + pl.norms_bytes + 15) & ~(size_t)15; }
-
 // Shared tail of the two encode entry points: clears the call's scan state in `ws` and
-// enqueues the kernels.  `ws` must hold slots_offset(pl) + P.grid * kEncWarps * pl.slot_bytes.
+// enqueues the kernels.  `ws` must hold pl.state_bytes + pl.norms_bytes.
 static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const float* g, uint32_t norm_kind,
                                  uint64_t seed, uint64_t offset, void* out, uint64_t* out_bits, Workspace* ws,
                                  int dev, cudaStream_t stream) {
@@ -202,7 +199,6 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     P.out = static_cast<uint32_t*>(out);
     P.out_bits = out_bits;
     P.ws = ws;
-    P.slots = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(ws) + slots_offset(pl));
     P.seed = seed;
     P.offset = offset;
     for (uint32_t r = 0; r < 10; ++r) {               // Philox key schedule (Weyl sequence)
@@ -250,7 +246,7 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     const EncodePlan pl = plan_encode(P, device_sms(dev));
     P.grid = pl.want_grid;
     Workspace* ws = nullptr;
-    nuq_status st = get_workspace(stream, slots_offset(pl) + (size_t)P.grid * kEncWarps * pl.slot_bytes, &ws, &dev);
+    nuq_status st = get_workspace(stream, pl.state_bytes + pl.norms_bytes, &ws, &dev);
     if (st != NUQ_OK) return st;
     return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, dev, stream);
 }
@@ -265,15 +261,8 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
     const EncodePlan pl = plan_encode(P, device_sms(dev));
-    // the fixed array must hold the scan state and the tile images of at least one CTA's warps;
-    // fewer CTAs than the device could run are launched when it cannot hold more
-    const size_t fixed_part = slots_offset(pl), per_cta = (size_t)kEncWarps * pl.slot_bytes;
-    if (fixed_part + per_cta > kStaticScratchBytes) return NUQ_ERR_CAPACITY;
+    if (pl.state_bytes + pl.norms_bytes > kStaticScratchBytes) return NUQ_ERR_CAPACITY;   // vector too long for the array
     P.grid = pl.want_grid;
-    if (per_cta) {
-        const size_t fit = (kStaticScratchBytes - fixed_part) / per_cta;
-        if (fit < P.grid) P.grid = (uint32_t)fit;
-    }
     auto it = g_static_ws.find(dev);
     if (it == g_static_ws.end()) {
         // first call on this device: ask the runtime where this device keeps the array

@@ -13,10 +13,10 @@ constexpr uint32_t kBLK = 32 * kSB;       // elements per coding block / per til
 constexpr uint32_t kHeaderWords = 16;
 constexpr uint32_t kMaxK = 64;
 
-constexpr int kEncThreads = 256;          // 8 independent warps, each takes whole tiles
+constexpr int kEncThreads = 256;          // 8 warps share a tile, 1024 elements each
 constexpr int kEncWarps = kEncThreads / 32;
-constexpr int kEncMinBlocks = 4;          // resident CTAs per SM the encoder is compiled for
-constexpr uint32_t kEncChunk = 512;       // elements a warp quantizes per step
+constexpr int kEncMinBlocks = 3;          // resident CTAs per SM the encoder is compiled for
+constexpr uint32_t kEncChunk = 512;       // elements a warp quantizes before it generates their tokens
 
 enum : uint32_t { kNormL2 = 0, kNormLinf = 1 };
 enum : uint32_t { kLevelsExp = 0, kLevelsUniform = 1 };
@@ -43,8 +43,7 @@ struct Workspace {
     uint64_t total_words;   // payload words of the whole call
     uint64_t dec_ticket;    // decoder: next tile to hand out (cleared before each decode launch)
     uint64_t reserved[1];
-    // followed by: uint64_t tile_state[ntiles], float norms[nb] for wide buckets, then (16-byte
-    // aligned) one scratch slot per encoder warp that holds the image of the tile it is working on
+    // followed by: uint64_t tile_state[ntiles], then float norms[nb] for wide buckets
 };
 constexpr size_t kWorkspaceClearFrom = 8;
 
@@ -74,10 +73,9 @@ struct EncodeParams {
     Workspace* ws;
     uint64_t seed, offset;
     uint32_t round_keys[20]; // Philox4x32-10 key schedule of `seed`: (k0, k1) of round 0, 1, ..., 9
-    uint32_t* slots;         // ERC mode: grid * kEncWarps scratch slots of slot_words words
-    uint32_t slot_words;     // capacity of one slot = largest possible tile image
-    uint32_t window_words;   // shared-memory bit window of one warp
-    uint32_t warp_smem_words;// shared memory of one warp (window, token list, group list)
+    uint32_t stage_words;    // shared-memory image of a tile's records (multiple of 4)
+    uint32_t window_words;   // shared-memory token string of one warp
+    uint32_t warp_smem_words;// shared memory of one warp (token string, token list)
     uint32_t grid;           // CTAs to launch
 };
 

@@ -1,28 +1,27 @@
 // ENCODE of NUQSGD (App. A) for one gradient vector: bucket norm, stochastic
-// quantization (Definition 1) and Elias-recursive token packing in one kernel.
+// quantization (Definition 1) and Elias-recursive token packing in one kernel
+// that reads the gradient from HBM exactly once.
 //
-// ONE WARP owns a tile of up to 8192 consecutive elements (whole buckets, or one
-// 8192-element coding block of a wider bucket) and there is no block-level
-// barrier anywhere: warps of a CTA only share two read-only code tables.  For
-// each bucket of its tile a warp
-//   1. reads the bucket once and reduces its norm (fp64 sums of exact squares);
-//   2. walks the bucket again in chunks of 512 elements (the second read is
-//      served by L2/L1): a lane handles 4 consecutive elements per 128-element
-//      row with one 128-bit load and one Philox block;
-//   3. keeps only the groups of 4 elements that hold a nonzero symbol (ballot /
-//      popc compaction into a shared-memory list), expands those groups to one
-//      entry per nonzero symbol (second compaction), and generates the tokens
-//      from that dense list, 32 tokens per step, OR-ing them into a small
-//      shared-memory bit window behind a running bit cursor;
-//   4. flushes the completed words of the window to the warp's scratch slot in
-//      global memory, which ends up holding the exact image of the tile
-//      (norm word, sub-block lengths, token strings, per bucket).
-// The tile's size is then chained to its predecessors by a decoupled look-back
-// scan, and the image is copied from the slot (still in L2) to its place in the
-// packed stream.  In the fixed-width mode the place is known in advance and the
-// window is flushed straight into the stream.
+// A persistent CTA of 8 warps takes tiles of up to 8192 consecutive elements
+// (whole buckets, or one 8192-element coding block of a wider bucket) by ticket.
+// The tile's bytes are brought into shared memory by one bulk asynchronous copy
+// (TMA, completion on an mbarrier); the copy of the next tile is started as soon
+// as the current tile has been quantized, so HBM latency hides behind the packing
+// of the current tile and behind the other CTAs of the SM.  Per tile:
+//   1. each warp reduces the squares (fp64) of its 1024 elements per sub-block;
+//      after one barrier every warp derives the bucket norms it needs;
+//   2. each warp quantizes its elements 512 at a time (one 128-bit shared-memory
+//      load and one Philox block per lane and 128-element row), compacts the
+//      nonzero symbols with ballots into a dense list, and turns that list into
+//      tokens, 32 per step, appended to the warp's own bit string;
+//   3. after a second barrier every warp runs the same small scan over the 32
+//      sub-block lengths, which gives the layout of the tile's records, and
+//      shifts its strings to their place in the staged tile;
+//   4. one warp chains the tile's size to its predecessors (decoupled look-back,
+//      bounded waits) and the CTA copies the staged tile to the packed stream.
+// In the fixed-width mode the fields go straight to their known place.
 //
-// The kernel is bound by instruction issue, not by HBM; the quantizer is branch
+// The kernel is bound by instruction issue, not by HBM: the quantizer is branch
 // free and all per-symbol work runs on dense lists.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
@@ -168,8 +167,43 @@ __device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile,
     return exclusive;
 }
 
-constexpr uint32_t kChunk = 512;                 // elements quantized per step of a warp (2 sub-blocks, 4 rows)
-constexpr uint32_t kChunkRows = kChunk / 128;
+// ---------------------------------------------------------------------------
+// Bulk asynchronous copy (TMA, untiled form) and its mbarrier.  One CTA-local
+// barrier, never a cluster multicast.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// Announces `bytes` to the barrier and starts the copy global -> shared.  Both addresses
+// 16-byte aligned, `bytes` a positive multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic writes to dst are ordered first
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst_smem)),
+                 "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+// Waits until the phase with the given parity has completed.  Bounded: false after ~tens of ms.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t polls = 0; polls < (1u << 20); ++polls) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (polls > 64) __nanosleep(100);
+    }
+    return false;
+}
 
 // Symbols travel as small fields: level index in the low bits, sign above it.
 template <uint32_t LEVELSET>
@@ -178,52 +212,95 @@ struct Sym {
     static constexpr uint32_t kMask = (1u << kBits) - 1u;
 };
 
-// OR `nbits` (1..32) right-aligned bits of `value` into the MSB-first bit string `dst` at `bitpos`.
+// OR `nbits` (0..32) right-aligned bits of `value` into the MSB-first bit string `dst` at `bitpos`.
+// Two words are touched unconditionally (a zero is OR-ed when there is nothing to add).
 __device__ __forceinline__ void or_bits32(uint32_t* dst, uint32_t bitpos, uint32_t value, uint32_t nbits) {
-    const uint32_t a = value << (32u - nbits);
+    const uint32_t a = nbits ? value << (32u - nbits) : 0u;
     const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
-    const uint32_t w0 = a >> sh;
-    const uint32_t w1 = __funnelshift_r(0u, a, sh);
-    if (w0) atomicOr(dst + w, w0);
-    if (w1) atomicOr(dst + w + 1, w1);
+    atomicOr(dst + w, a >> sh);
+    atomicOr(dst + w + 1, __funnelshift_r(0u, a, sh));
 }
 
-// Shared memory of one warp.
-struct WarpMem {
-    uint32_t* window;     // bit window behind the cursor
-    uint32_t* tokens;     // kChunk entries: position | field << 10
-    uint32_t* groups;     // kChunk / 4 entries of 2 (exponential) or 3 (uniform) words
-};
+// 32 bits of the MSB-first bit string `src` starting at bit `sbit` (>= -31); bits before
+// the string read as garbage and must be masked by the caller.
+__device__ __forceinline__ uint32_t bits_at(const uint32_t* src, int sbit) {
+    if (sbit < 0) return src[0] >> (uint32_t)(-sbit);
+    const uint32_t w = (uint32_t)sbit >> 5;
+    return __funnelshift_l(src[w + 1], src[w], (uint32_t)sbit);
+}
+
+constexpr uint32_t kWarpElems = kBLK / kEncWarps;   // 1024 elements of a tile per warp (4 sub-blocks)
+constexpr uint32_t kChunk = 512;                    // elements quantized before their tokens are generated
+constexpr uint32_t kChunkRows = kChunk / 128;
 
 template <uint32_t LEVELSET, uint32_t MODE>
 __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(const __grid_constant__ EncodeParams P) {
-    extern __shared__ __align__(16) uint32_t smem[];
+    extern __shared__ __align__(128) uint32_t smem[];
+    __shared__ __align__(8) uint64_t s_bar;                // completes when the tile's bytes have landed
     __shared__ uint32_t s_lut[256];                        // ERC(N), N = 1..256: code | len << 16
-    __shared__ uint32_t s_lut_signed[256];                 // exponential levels: sign bit + ERC(index) by field
+    __shared__ uint32_t s_lut_signed[256];                 // exponential levels: sign bit + ERC(index), by field
+    __shared__ double s_partial[32];                       // per sub-block (or per warp) sums of squares
+    __shared__ uint32_t s_maxbits[32];                     // ... or max |x| bit patterns
+    __shared__ uint32_t s_sb_bits[32];                     // token bits of each sub-block
+    __shared__ uint32_t s_sb_src[32];                      // where they start in the owning warp's window
+    __shared__ uint32_t s_start[32];                       // scratch: first token offset of a sub-block (per warp 4)
+    __shared__ unsigned long long s_tile[2], s_tile_off;
+    __shared__ uint32_t s_abort, s_nnz, s_code_bits;
 
     using S = Sym<LEVELSET>;
-    constexpr uint32_t kGroupWords = LEVELSET == kLevelsExp ? 2u : 3u;
     const Geometry& G = P.geo;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    const uint32_t gwarp = blockIdx.x * kEncWarps + warp;
-    uint32_t* wmem = smem + warp * P.warp_smem_words;
-    WarpMem M;
-    M.window = wmem;
-    M.tokens = wmem + P.window_words;
-    M.groups = M.tokens + kChunk;
+    float* data = reinterpret_cast<float*>(smem);                               // kBLK floats: the tile
+    uint32_t* stage = smem + kBLK;                                              // image of the tile's records
+    uint32_t* wmem = stage + P.stage_words + warp * P.warp_smem_words;
+    uint32_t* window = wmem;                                                    // this warp's token string
+    uint32_t* tokens = wmem + P.window_words;                                   // kChunk entries: position | field << 10
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
-    uint32_t* slot = P.slots + (uint64_t)gwarp * P.slot_words;
     uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
     uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
     const float top = __uint_as_float((127u + G.s) << 23);
     const uint32_t c2 = (uint32_t)P.offset, c3 = (uint32_t)(P.offset >> 32);
     const uint32_t lt_mask = (1u << lane) - 1u;
+    const bool coarse = G.bucket % kWarpElems == 0;         // a warp's four sub-blocks always share one bucket
+    const uint32_t spb = G.bucket <= kBLK ? G.sb_per_block : 32u;       // sub-blocks per coding block
+    uint32_t bi_q[4];                                       // block (within a tile) of the warp's four sub-blocks
+#pragma unroll
+    for (int q = 0; q < 4; ++q) bi_q[q] = (warp * 4u + q) / spb;
+    const uint32_t bi_lane = lane / spb;                    // block of sub-block `lane`
+
+    // where tile `t` starts and how long it is
+    auto tile_span = [&](uint64_t t, uint64_t& elem0, uint32_t& tile_len) {
+        if (G.bucket <= kBLK) {
+            elem0 = t * G.blocks_per_tile * G.bucket;
+            const uint64_t left = G.d - elem0;
+            tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
+        } else {
+            const uint64_t bucket_idx = t / G.blk_per_bucket;
+            const uint32_t bib = (uint32_t)(t % G.blk_per_bucket);
+            const uint64_t b0 = bucket_idx * G.bucket;
+            const uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
+            elem0 = b0 + (uint64_t)bib * kBLK;
+            const uint64_t left = blen - (uint64_t)bib * kBLK;
+            tile_len = left < kBLK ? (uint32_t)left : kBLK;
+        }
+    };
+    // thread 0: take a ticket and start the copy of that tile into `data`
+    auto fetch_tile = [&](uint32_t slot) {
+        const uint64_t t = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        s_tile[slot] = t;
+        if (t < G.ntiles) {
+            uint64_t elem0;
+            uint32_t tile_len;
+            tile_span(t, elem0, tile_len);
+            const uint32_t bytes = (tile_len * 4u) & ~15u;
+            if (bytes) bulk_load(data, P.g + elem0, bytes, &s_bar);
+        }
+    };
 
     {
         const uint32_t e = c_erc_lut[tid];
         s_lut[tid] = e;
-        // field = sign << 7 | index: the sign bit followed by ERC(index)
-        const uint32_t idx = tid & 0x7Fu;
+        const uint32_t idx = tid & 0x7Fu;                   // field = sign << 7 | index: sign bit, then ERC(index)
         uint32_t v = 0;
         if (idx >= 1) {
             const uint32_t l = c_erc_lut[idx - 1u], len = l >> 16;
@@ -231,367 +308,411 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
         }
         s_lut_signed[tid] = v;
     }
-    for (uint32_t i = lane; i < P.window_words; i += 32) M.window[i] = 0;
+    for (uint32_t i = tid; i < P.stage_words; i += kEncThreads) stage[i] = 0;
+    for (uint32_t i = lane; i < P.window_words; i += 32) window[i] = 0;
+    if (tid == 0) {
+        mbar_init(&s_bar, 1);
+        s_abort = 0;
+        s_nnz = 0;
+        s_code_bits = 0;
+    }
+    __syncthreads();
+    if (tid == 0) fetch_tile(0);
     __syncthreads();
 
-    for (;;) {
-        uint64_t tile = 0;
-        if (lane == 0) tile = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
-        tile = __shfl_sync(0xffffffffu, tile, 0);
+    uint32_t parity = 0;
+    for (uint32_t it = 0;; ++it) {
+        const uint64_t tile = s_tile[it & 1u];
         if (tile >= G.ntiles) break;
 
         // ---- tile geometry ------------------------------------------------------
-        uint64_t elem0, first_block;
-        uint32_t tile_len, nblk_tile, blk_elems;
-        uint64_t bucket_idx = 0;
-        uint32_t bib = 0;                                   // block within a wide bucket
+        uint64_t elem0, first_block, bucket_idx = 0;
+        uint32_t tile_len, nblk_tile, blk_elems, bib = 0;
+        tile_span(tile, elem0, tile_len);
         if (G.bucket <= kBLK) {
             first_block = tile * G.blocks_per_tile;
-            elem0 = first_block * G.bucket;
-            const uint64_t left = G.d - elem0;
-            tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
             blk_elems = G.bucket;
             nblk_tile = (tile_len + G.bucket - 1) / G.bucket;
         } else {
             bucket_idx = tile / G.blk_per_bucket;
             bib = (uint32_t)(tile % G.blk_per_bucket);
             first_block = tile;
-            const uint64_t b0 = bucket_idx * G.bucket;
-            const uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
-            elem0 = b0 + (uint64_t)bib * kBLK;
-            const uint64_t left = blen - (uint64_t)bib * kBLK;
-            tile_len = left < kBLK ? (uint32_t)left : kBLK;
             blk_elems = kBLK;
             nblk_tile = 1;
         }
-        const float* gt = P.g + elem0;
+        const uint32_t nsb_tile = (tile_len + kSB - 1) / kSB;
+        const uint32_t wbase = warp * kWarpElems;           // first element of the warp within the tile
 
-        uint32_t W = 0;                                     // ERC: words of the tile image so far
-        uint32_t my_blk_wordoff = 0;                        // ERC: lane bi keeps the word offset of block bi
-        uint32_t tile_code_bits = 0, tile_nnz = 0;
-        uint64_t fixed_off = 0;                             // fixed mode: word offset of the tile's first record
-        if (MODE == kModeFixed)
-            fixed_off = G.bucket <= kBLK ? first_block * G.rec_words
-                                         : bucket_idx * G.rec_words + 1u + (uint64_t)bib * (kBLK * G.width / 32u);
-
-        for (uint32_t bi = 0; bi < nblk_tile; ++bi) {
-            const uint32_t blk_first = bi * blk_elems;
-            const uint32_t bl = min(blk_elems, tile_len - blk_first);
-            const uint32_t nsb = (bl + kSB - 1) / kSB;
-            const uint32_t head_words = 1u + (nsb + 1u) / 2u;
-            const float* gb = gt + blk_first;
-
-            // ---- bucket norm: fp64 sum of exact squares (or max |x|), one rounding to fp32 ----
-            float norm;
-            if (P.norms_in != nullptr) {
-                norm = P.norms_in[G.bucket <= kBLK ? first_block + bi : bucket_idx];
-            } else {
-                double acc = 0.0;
-                uint32_t mx = 0;
-#pragma unroll 4
-                for (uint32_t base = lane * 4u; base < bl; base += 128u) {
-                    float4 x;
-                    if (base + 4u <= bl) {
-                        x = __ldg(reinterpret_cast<const float4*>(gb + base));
-                    } else {
-                        x.x = __ldg(gb + base);
-                        x.y = base + 1u < bl ? __ldg(gb + base + 1u) : 0.0f;
-                        x.z = base + 2u < bl ? __ldg(gb + base + 2u) : 0.0f;
-                        x.w = 0.0f;
+        // ---- the tile's bytes: wait for the bulk copy, fetch the ragged end, zero the rest ----
+        {
+            const uint32_t bulk_elems = ((tile_len * 4u) & ~15u) / 4u;
+            if (bulk_elems) {
+                if (!mbar_wait(&s_bar, parity)) {           // never seen in practice; do not hang
+                    if (tid == 0) {
+                        latch_status(P.ws, kErrTimeout);
+                        s_abort = 1;
                     }
+                }
+                parity ^= 1u;
+            }
+            if (tile_len < kBLK) {
+                for (uint32_t i = bulk_elems + tid; i < kBLK; i += kEncThreads)
+                    data[i] = i < tile_len ? __ldg(P.g + elem0 + i) : 0.0f;
+                __syncthreads();
+            }
+        }
+        const float4* rows = reinterpret_cast<const float4*>(data + wbase) + lane;   // row j at rows[32 * j]
+
+        // ---- bucket norms: fp64 sums of exact squares (or max |x|), one rounding to fp32 ----
+        if (P.norms_in == nullptr) {
+            double acc = 0.0;
+            uint32_t mx = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const float4 x = rows[32 * (2 * q + h)];
                     if (G.norm_kind == kNormL2) {
                         acc = fma((double)x.x, (double)x.x, acc);
                         acc = fma((double)x.y, (double)x.y, acc);
                         acc = fma((double)x.z, (double)x.z, acc);
                         acc = fma((double)x.w, (double)x.w, acc);
-                    } else {                                // max |x| on the bit patterns: NaN sorts above inf
+                    } else {                                // on the bit patterns: NaN sorts above inf
                         mx = max(max(mx, __float_as_uint(fabsf(x.x))), __float_as_uint(fabsf(x.y)));
                         mx = max(max(mx, __float_as_uint(fabsf(x.z))), __float_as_uint(fabsf(x.w)));
                     }
                 }
-                if (G.norm_kind == kNormL2) {
+                if (!coarse || q == 3) {                    // one partial per sub-block, or one per warp
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-                    norm = (float)sqrt(acc);
+                    for (int o = 16; o > 0; o >>= 1) {
+                        acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                    }
+                    if (lane == 0) {
+                        s_partial[warp * 4 + q] = acc;
+                        s_maxbits[warp * 4 + q] = mx;
+                    }
+                    acc = 0.0;
+                    mx = 0;
+                } else if (lane == 0) {
+                    s_partial[warp * 4 + q] = 0.0;
+                    s_maxbits[warp * 4 + q] = 0;
+                }
+            }
+        }
+        __syncthreads();                                    // B1: partials visible
+
+        // every warp derives the norms of the buckets its own sub-blocks belong to (same
+        // reduction tree in every warp, so all agree bit for bit)
+        float inv_q[4], norm_q[4];
+        {
+            const double my_part = s_partial[lane];
+            const uint32_t my_max = s_maxbits[lane];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (q > 0 && (coarse || bi_q[q] == bi_q[q - 1])) {            // same bucket as the previous sub-block
+                    inv_q[q] = inv_q[q - 1];
+                    norm_q[q] = norm_q[q - 1];
+                    continue;
+                }
+                const uint32_t bi = bi_q[q], sb0 = bi * spb;
+                float norm;
+                if (P.norms_in != nullptr) {
+                    const uint64_t nb_idx = G.bucket <= kBLK ? first_block + bi : bucket_idx;
+                    norm = nb_idx < G.nb ? P.norms_in[nb_idx] : 0.0f;
                 } else {
+                    const bool in = lane >= sb0 && lane < sb0 + spb;
+                    double a = in ? my_part : 0.0;
+                    uint32_t m = in ? my_max : 0u;
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-                    norm = __uint_as_float(mx);
-                }
-            }
-            if (norm != norm) norm = __uint_as_float(0x7fc00000u);     // one NaN pattern in the stream
-            float inv = 0.0f;                                           // 0: the bucket is not quantized
-            if (norm > 0.0f && norm < __uint_as_float(0x7f800000u)) {
-                inv = __fdiv_rn(top, norm);                             // one IEEE division per bucket
-                if (!(inv < __uint_as_float(0x7f800000u))) inv = 0.0f;
-            }
-
-            // ---- where this block's bits go -----------------------------------------------
-            uint32_t* dst;                                  // words of the block's bit string are flushed here
-            if (MODE == kModeErc) {
-                if (lane == bi) my_blk_wordoff = W;
-                dst = slot + W + head_words;
-            } else if (G.bucket <= kBLK) {
-                dst = payload + fixed_off + (uint64_t)bi * G.rec_words + 1u;
-            } else {
-                dst = payload + fixed_off;
-            }
-            uint32_t bits = 0;                              // bits of the block's string so far
-            uint32_t flushed = 0;                           // whole words already written to dst
-            uint32_t my_len = 0;                            // ERC: lane q keeps the token bits of sub-block q
-
-            for (uint32_t cb = 0; cb < bl; cb += kChunk) {
-                const uint32_t win0 = 32u * flushed;        // bit of the block string at window bit 0
-                uint32_t ngroups = 0, ntok = 0;
-
-                // ---- quantize (Definition 1), 128 elements per step ---------------------------
-                if (inv != 0.0f) {
-#pragma unroll 1
-                    for (uint32_t r = 0; r < kChunkRows; ++r) {
-                        const uint32_t base = cb + r * 128u + lane * 4u;        // element within the block
-                        if (cb + r * 128u >= bl) break;
-                        float4 x;
-                        if (base + 4u <= bl) {
-                            x = __ldg(reinterpret_cast<const float4*>(gb + base));
-                        } else {
-                            x.x = base + 0u < bl ? __ldg(gb + base + 0u) : 0.0f;
-                            x.y = base + 1u < bl ? __ldg(gb + base + 1u) : 0.0f;
-                            x.z = base + 2u < bl ? __ldg(gb + base + 2u) : 0.0f;
-                            x.w = 0.0f;
-                        }
-                        const uint64_t ctr = (elem0 + blk_first + base) >> 2;
-                        const uint4 rnd = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, P.round_keys);
-                        uint32_t q0, q1, q2, q3;
-                        if (LEVELSET == kLevelsExp) {
-                            q0 = quantize_exp(x.x, inv, top, rnd.x);
-                            q1 = quantize_exp(x.y, inv, top, rnd.y);
-                            q2 = quantize_exp(x.z, inv, top, rnd.z);
-                            q3 = quantize_exp(x.w, inv, top, rnd.w);
-                        } else {
-                            q0 = quantize_uniform(x.x, inv, top, rnd.x);
-                            q1 = quantize_uniform(x.y, inv, top, rnd.y);
-                            q2 = quantize_uniform(x.z, inv, top, rnd.z);
-                            q3 = quantize_uniform(x.w, inv, top, rnd.w);
-                        }
-                        const uint32_t b0 = __float_as_uint(x.x), b1 = __float_as_uint(x.y);
-                        const uint32_t b2 = __float_as_uint(x.z), b3 = __float_as_uint(x.w);
-                        // fields (index | sign << kBits) of the 4 elements, packed; a zero symbol has no sign
-                        uint32_t f01, f23;                   // exponential: f01 holds all four bytes
-                        bool any;
-                        if (LEVELSET == kLevelsExp) {
-                            const uint32_t syms = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
-                            const uint32_t tops =
-                                __byte_perm(__byte_perm(b0, b1, 0x0073), __byte_perm(b2, b3, 0x0073), 0x5410);
-                            const uint32_t nzb = (syms + 0x7F7F7F7Fu) & 0x80808080u;   // bit 7 of a byte: symbol != 0
-                            f01 = syms | (tops & nzb);
-                            f23 = 0;
-                            any = syms != 0;
-                        } else {
-                            f01 = (q0 | (q0 ? (b0 >> 16) & 0x8000u : 0u)) | ((q1 | (q1 ? (b1 >> 16) & 0x8000u : 0u)) << 16);
-                            f23 = (q2 | (q2 ? (b2 >> 16) & 0x8000u : 0u)) | ((q3 | (q3 ? (b3 >> 16) & 0x8000u : 0u)) << 16);
-                            any = (f01 | f23) != 0;
-                        }
-                        if (MODE == kModeErc) {
-                            // keep the groups that hold a nonzero symbol
-                            const uint32_t vote = __ballot_sync(0xffffffffu, any);
-                            if (any) {
-                                uint32_t* ge = M.groups + (ngroups + __popc(vote & lt_mask)) * kGroupWords;
-                                ge[0] = f01;
-                                if (LEVELSET == kLevelsExp) {
-                                    ge[1] = r * 32u + lane;
-                                } else {
-                                    ge[1] = f23;
-                                    ge[2] = r * 32u + lane;
-                                }
-                            }
-                            ngroups += __popc(vote);
-                        } else if (any) {
-                            // fixed-width fields, MSB first, straight into the window
-                            const uint32_t wbits = G.width;
-                            uint32_t f[4];
-                            if (LEVELSET == kLevelsExp) {
-                                f[0] = f01 & 0xFFu; f[1] = (f01 >> 8) & 0xFFu; f[2] = (f01 >> 16) & 0xFFu; f[3] = f01 >> 24;
-                            } else {
-                                f[0] = f01 & 0xFFFFu; f[1] = f01 >> 16; f[2] = f23 & 0xFFFFu; f[3] = f23 >> 16;
-                            }
-                            uint64_t str = 0;
-#pragma unroll
-                            for (int c = 0; c < 4; ++c) {
-                                str = (str << wbits) | ((f[c] & S::kMask) | ((f[c] >> S::kBits) << (wbits - 1u)));
-                                tile_nnz += (f[c] & S::kMask) != 0;
-                            }
-                            or_bits(M.window, base * wbits - win0, str, 4u * wbits);
-                        }
+                    for (int o = 16; o > 0; o >>= 1) {
+                        a += __shfl_xor_sync(0xffffffffu, a, o);
+                        m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
                     }
+                    norm = G.norm_kind == kNormL2 ? (float)sqrt(a) : __uint_as_float(m);
                 }
-
-                if (MODE == kModeErc) {
-                    __syncwarp();
-                    // ---- expand the kept groups to one entry per nonzero symbol ---------------------
-                    for (uint32_t g0 = 0; g0 < ngroups; g0 += 32) {
-                        const bool valid = g0 + lane < ngroups;
-                        uint32_t f01 = 0, f23 = 0, gpos = 0;
-                        if (valid) {
-                            const uint32_t* ge = M.groups + (g0 + lane) * kGroupWords;
-                            f01 = ge[0];
-                            if (LEVELSET == kLevelsExp) { gpos = ge[1]; } else { f23 = ge[1]; gpos = ge[2]; }
-                        }
-                        uint32_t f[4];
-                        if (LEVELSET == kLevelsExp) {
-                            f[0] = f01 & 0xFFu; f[1] = (f01 >> 8) & 0xFFu; f[2] = (f01 >> 16) & 0xFFu; f[3] = f01 >> 24;
-                        } else {
-                            f[0] = f01 & 0xFFFFu; f[1] = f01 >> 16; f[2] = f23 & 0xFFFFu; f[3] = f23 >> 16;
-                        }
-                        const uint32_t cnt = (f[0] != 0) + (f[1] != 0) + (f[2] != 0) + (f[3] != 0);
-                        uint32_t incl = cnt;
-#pragma unroll
-                        for (int o = 1; o < 32; o <<= 1) {
-                            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                            if (lane >= (uint32_t)o) incl += t;
-                        }
-                        uint32_t at = ntok + incl - cnt;
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            if (f[c]) M.tokens[at++] = (gpos * 4u + (uint32_t)c) | (f[c] << 10);
-                        }
-                        ntok += __shfl_sync(0xffffffffu, incl, 31);
-                    }
-                    __syncwarp();
-
-                    // ---- tokens ERC(gap) sign ERC(index), 32 per step, behind the bit cursor ----------
-                    int carry_pos = -1;                     // position (within the chunk) of the last nonzero so far
-                    uint32_t my_start = 0xFFFFFFFFu;        // lane q < 2: where sub-block q's string starts
-                    for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
-                        const bool valid = t0 + lane < ntok;
-                        const uint32_t e = valid ? M.tokens[t0 + lane] : 0u;
-                        const int pos = (int)(e & 1023u);
-                        const uint32_t field = e >> 10;
-                        int prev = __shfl_up_sync(0xffffffffu, pos, 1);
-                        if (lane == 0) prev = carry_pos;
-                        const bool first_of_sb = (prev >> 8) != (pos >> 8);      // also when there is no predecessor
-                        if (first_of_sb) prev = (pos & ~255) - 1;                  // the run restarts: t_0 = 0
-                        uint32_t tlen = 0, tokA = 0, lenA = 0, tokB = 0, lenB = 0;
-                        if (valid) {
-                            const uint32_t gl = s_lut[pos - prev - 1];
-                            if (LEVELSET == kLevelsExp) {
-                                const uint32_t ll = s_lut_signed[field];
-                                lenB = ll >> 16;
-                                tokA = ((gl & 0xffffu) << lenB) | (ll & 0xffffu);                  // <= 16 + 8 bits
-                                lenA = (gl >> 16) + lenB;
-                                tlen = lenA;
-                            } else {
-                                const uint32_t ll = s_lut[(field & S::kMask) - 1u];
-                                tokA = gl & 0xffffu;
-                                lenA = gl >> 16;
-                                lenB = (ll >> 16) + 1u;                                           // sign + ERC(index) <= 17
-                                tokB = ((field >> S::kBits) << (lenB - 1u)) | (ll & 0xffffu);
-                                tlen = lenA + lenB;
-                            }
-                        }
-                        uint32_t incl = tlen;
-#pragma unroll
-                        for (int o = 1; o < 32; o <<= 1) {
-                            const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                            if (lane >= (uint32_t)o) incl += t;
-                        }
-                        const uint32_t off = bits + incl - tlen;    // bit of the block string where my token starts
-                        // the first token of a sub-block marks where that sub-block's string starts
-                        uint32_t starts = __ballot_sync(0xffffffffu, valid && first_of_sb);
-                        while (starts) {
-                            const int src = __ffs(starts) - 1;
-                            starts &= starts - 1;
-                            const uint32_t q = (uint32_t)__shfl_sync(0xffffffffu, pos, src) >> 8;
-                            const uint32_t o = __shfl_sync(0xffffffffu, off, src);
-                            if (lane == q) my_start = o;
-                        }
-                        if (valid) {
-                            if (LEVELSET == kLevelsExp) {
-                                or_bits32(M.window, off - win0, tokA, lenA);
-                            } else {
-                                or_bits32(M.window, off - win0, tokA, lenA);
-                                or_bits32(M.window, off - win0 + lenA, tokB, lenB);
-                            }
-                        }
-                        bits += __shfl_sync(0xffffffffu, incl, 31);
-                        carry_pos = __shfl_sync(0xffffffffu, pos, min(ntok - t0, 32u) - 1u);
-                    }
-                    tile_nnz += ntok;
-                    // sub-block strings follow one another: an empty one starts where the next one does
-                    {
-                        uint32_t s1 = __shfl_sync(0xffffffffu, my_start, 1);
-                        uint32_t s0 = __shfl_sync(0xffffffffu, my_start, 0);
-                        if (s1 == 0xFFFFFFFFu) s1 = bits;
-                        if (s0 == 0xFFFFFFFFu) s0 = s1;
-                        const uint32_t q = cb / kSB;                // first sub-block of this chunk
-                        if (lane == q) my_len = s1 - s0;
-                        if (lane == q + 1u) my_len = bits - s1;
-                    }
-                } else {
-                    bits = min(cb + kChunk, bl) * G.width;
+                if (norm != norm) norm = __uint_as_float(0x7fc00000u);     // one NaN pattern in the stream
+                float inv = 0.0f;                                           // 0: the bucket is not quantized
+                if (norm > 0.0f && norm < __uint_as_float(0x7f800000u)) {
+                    inv = __fdiv_rn(top, norm);                             // one IEEE division per bucket
+                    if (!(inv < __uint_as_float(0x7f800000u))) inv = 0.0f;
                 }
-
-                // ---- flush the completed words of the window ------------------------------------------
-                __syncwarp();
-                {
-                    const uint32_t full = (bits >> 5) - flushed;
-                    for (uint32_t i = lane; i < full; i += 32) dst[flushed + i] = M.window[i];
-                    const uint32_t partial = M.window[full];
-                    __syncwarp();
-                    for (uint32_t i = lane; i < full + 3u; i += 32) M.window[i] = 0;
-                    __syncwarp();
-                    if (lane == 0) M.window[0] = partial;
-                    __syncwarp();
-                    flushed += full;
-                }
-            }
-
-            // ---- end of the block: last partial word, then the block's header ----------------------------
-            if (bits & 31u) {
-                if (lane == 0) {
-                    dst[flushed] = M.window[0];
-                    M.window[0] = 0;
-                }
-                __syncwarp();
-            }
-            if (MODE == kModeErc) {
-                uint32_t* hdr = slot + W;
-                if (lane == 0) hdr[0] = __float_as_uint(norm);
-                const uint32_t hi = __shfl_down_sync(0xffffffffu, my_len, 1);
-                if (!(lane & 1u) && lane < nsb) hdr[1u + lane / 2u] = my_len | (lane + 1u < nsb ? hi << 16 : 0u);
-                W += head_words + (bits + 31u) / 32u;
-                tile_code_bits += bits;
-            } else {
-                if (lane == 0 && (G.bucket <= kBLK || bib == 0))
-                    payload[G.bucket <= kBLK ? fixed_off + (uint64_t)bi * G.rec_words : bucket_idx * G.rec_words] =
-                        __float_as_uint(norm);
+                inv_q[q] = inv;
+                norm_q[q] = norm;
             }
         }
 
-        // ---- ERC: chain the tile to its predecessors, then move its image into the stream ---------------
-        if (MODE == kModeErc) {
-            const uint32_t tile_words = W;
-            bool failed;
-            const uint64_t tile_off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
-            __syncwarp();
-            if (!failed) {
-                for (uint32_t i = lane; i < tile_words; i += 32) payload[tile_off + i] = __ldcg(slot + i);
-                if (lane < nblk_tile) table[first_block + lane] = 32ull * (tile_off + my_blk_wordoff);
-                if (tile == G.ntiles - 1 && lane == 0) {
-                    table[G.nblk] = 32ull * (tile_off + tile_words);
-                    P.ws->total_words = tile_off + tile_words;
+        // ---- quantize (Definition 1) and generate tokens, 512 elements at a time -------------
+        uint32_t bits = 0;                                  // ERC: bits in this warp's window so far
+        uint32_t my_nnz = 0;
+        if (MODE == kModeErc && lane < 4) s_start[warp * 4 + lane] = 0xFFFFFFFFu;
+#pragma unroll 1
+        for (uint32_t half = 0; half < 2; ++half) {
+            uint32_t ntok = 0;
+#pragma unroll
+            for (uint32_t r = 0; r < kChunkRows; ++r) {
+                const uint32_t j = half * kChunkRows + r;   // row of the warp
+                const float inv = inv_q[j >> 1];
+                if (inv == 0.0f) continue;                  // bucket not quantized (warp uniform)
+                const float4 x = rows[32 * j];
+                const uint32_t base = wbase + j * 128u + lane * 4u;             // element within the tile
+                const uint64_t ctr = (elem0 + base) >> 2;
+                const uint4 rnd = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, P.round_keys);
+                uint32_t q0, q1, q2, q3;
+                if (LEVELSET == kLevelsExp) {
+                    q0 = quantize_exp(x.x, inv, top, rnd.x);
+                    q1 = quantize_exp(x.y, inv, top, rnd.y);
+                    q2 = quantize_exp(x.z, inv, top, rnd.z);
+                    q3 = quantize_exp(x.w, inv, top, rnd.w);
+                } else {
+                    q0 = quantize_uniform(x.x, inv, top, rnd.x);
+                    q1 = quantize_uniform(x.y, inv, top, rnd.y);
+                    q2 = quantize_uniform(x.z, inv, top, rnd.z);
+                    q3 = quantize_uniform(x.w, inv, top, rnd.w);
+                }
+                // fields (index | sign << kBits); a zero symbol has no sign
+                uint32_t f0, f1, f2, f3;
+                if (LEVELSET == kLevelsExp) {
+                    const uint32_t syms = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
+                    const uint32_t tops = __byte_perm(__byte_perm(__float_as_uint(x.x), __float_as_uint(x.y), 0x0073),
+                                                      __byte_perm(__float_as_uint(x.z), __float_as_uint(x.w), 0x0073), 0x5410);
+                    const uint32_t nzb = (syms + 0x7F7F7F7Fu) & 0x80808080u;   // bit 7 of a byte: symbol != 0
+                    const uint32_t f = syms | (tops & nzb);
+                    f0 = f & 0xFFu; f1 = (f >> 8) & 0xFFu; f2 = (f >> 16) & 0xFFu; f3 = f >> 24;
+                } else {
+                    f0 = q0 | (q0 ? (__float_as_uint(x.x) >> 16) & 0x8000u : 0u);
+                    f1 = q1 | (q1 ? (__float_as_uint(x.y) >> 16) & 0x8000u : 0u);
+                    f2 = q2 | (q2 ? (__float_as_uint(x.z) >> 16) & 0x8000u : 0u);
+                    f3 = q3 | (q3 ? (__float_as_uint(x.w) >> 16) & 0x8000u : 0u);
+                }
+                if (MODE == kModeErc) {
+                    // keep the nonzero symbols, in element order: rank = nonzeros in lower lanes + own earlier ones
+                    const uint32_t v0 = __ballot_sync(0xffffffffu, q0 != 0), v1 = __ballot_sync(0xffffffffu, q1 != 0);
+                    const uint32_t v2 = __ballot_sync(0xffffffffu, q2 != 0), v3 = __ballot_sync(0xffffffffu, q3 != 0);
+                    uint32_t at = ntok + __popc(v0 & lt_mask) + __popc(v1 & lt_mask) + __popc(v2 & lt_mask) +
+                                  __popc(v3 & lt_mask);
+                    const uint32_t pos = r * 128u + lane * 4u;                  // position within the 512-element chunk
+                    if (q0) tokens[at++] = pos | (f0 << 10);
+                    if (q1) tokens[at++] = (pos + 1u) | (f1 << 10);
+                    if (q2) tokens[at++] = (pos + 2u) | (f2 << 10);
+                    if (q3) tokens[at++] = (pos + 3u) | (f3 << 10);
+                    ntok += __popc(v0) + __popc(v1) + __popc(v2) + __popc(v3);
+                } else if (q0 | q1 | q2 | q3) {
+                    // fixed-width fields, MSB first, straight into the staged tile
+                    const uint32_t wbits = G.width;
+                    const uint32_t ff[4] = {f0, f1, f2, f3};
+                    uint64_t str = 0;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        str = (str << wbits) | ((ff[c] & S::kMask) | ((ff[c] >> S::kBits) << (wbits - 1u)));
+                        my_nnz += (ff[c] & S::kMask) != 0;
+                    }
+                    uint32_t cursor;
+                    if (G.bucket <= kBLK) {
+                        const uint32_t bi = bi_q[j >> 1];
+                        cursor = 32u * (bi * G.rec_words + 1u) + (base - bi * blk_elems) * wbits;
+                    } else {
+                        cursor = base * wbits;
+                    }
+                    or_bits(stage, cursor, str, 4u * wbits);
                 }
             }
-            if (lane == 0 && tile_code_bits)
-                atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)tile_code_bits);
+
+            if (MODE == kModeErc) {
+                __syncwarp();
+                // ---- tokens ERC(gap) sign ERC(index), 32 per step, appended to the warp's window ----
+                int carry_pos = -1;                         // position (within the chunk) of the last nonzero so far
+                for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
+                    const bool valid = t0 + lane < ntok;
+                    const uint32_t e = valid ? tokens[t0 + lane] : 0u;
+                    const int pos = (int)(e & 1023u);
+                    const uint32_t field = e >> 10;
+                    int prev = __shfl_up_sync(0xffffffffu, pos, 1);
+                    if (lane == 0) prev = carry_pos;
+                    const bool first_of_sb = (prev >> 8) != (pos >> 8);      // also when there is no predecessor
+                    if (first_of_sb) prev = (pos & ~255) - 1;                  // the run restarts: t_0 = 0
+                    const uint32_t gl = s_lut[(pos - prev - 1) & 255];
+                    uint32_t tlen, tokA, lenA, tokB = 0, lenB;
+                    if (LEVELSET == kLevelsExp) {
+                        const uint32_t ll = s_lut_signed[field & 255u];
+                        lenB = ll >> 16;
+                        tokA = ((gl & 0xffffu) << lenB) | (ll & 0xffffu);     // <= 16 + 8 bits
+                        lenA = valid ? (gl >> 16) + lenB : 0u;
+                        tlen = lenA;
+                    } else {
+                        const uint32_t ll = s_lut[((field & S::kMask) - 1u) & 255u];
+                        tokA = gl & 0xffffu;
+                        lenA = valid ? gl >> 16 : 0u;
+                        lenB = valid ? (ll >> 16) + 1u : 0u;                  // sign + ERC(index) <= 17 bits
+                        tokB = ((field >> S::kBits) << (ll >> 16)) | (ll & 0xffffu);
+                        tlen = lenA + lenB;
+                    }
+                    uint32_t incl = tlen;
+#pragma unroll
+                    for (int o = 1; o < 32; o <<= 1) {
+                        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                        if (lane >= (uint32_t)o) incl += t;
+                    }
+                    const uint32_t off = bits + incl - tlen;    // bit of the window where my token starts
+                    // the first token of a sub-block marks where that sub-block's string starts
+                    if (valid && first_of_sb) s_start[warp * 4u + half * 2u + ((uint32_t)pos >> 8)] = off;
+                    or_bits32(window, off, tokA, lenA);
+                    if (LEVELSET != kLevelsExp) or_bits32(window, off + lenA, tokB, lenB);
+                    bits += __shfl_sync(0xffffffffu, incl, 31);
+                    carry_pos = __shfl_sync(0xffffffffu, pos, min(ntok - t0, 32u) - 1u);
+                }
+                my_nnz += ntok;                             // warp uniform: counted once below
+                __syncwarp();
+            }
+        }
+        if (MODE == kModeErc) {
+            // sub-block strings follow one another: an empty one starts where the next one does
+            uint32_t st = lane < 4 ? s_start[warp * 4u + lane] : 0xFFFFFFFFu;
+            uint32_t s3 = __shfl_sync(0xffffffffu, st, 3), s2 = __shfl_sync(0xffffffffu, st, 2);
+            uint32_t s1 = __shfl_sync(0xffffffffu, st, 1), s0 = __shfl_sync(0xffffffffu, st, 0);
+            if (s3 == 0xFFFFFFFFu) s3 = bits;
+            if (s2 == 0xFFFFFFFFu) s2 = s3;
+            if (s1 == 0xFFFFFFFFu) s1 = s2;
+            if (s0 == 0xFFFFFFFFu) s0 = s1;
+            if (lane < 4) {
+                const uint32_t begin = lane == 0 ? s0 : lane == 1 ? s1 : lane == 2 ? s2 : s3;
+                const uint32_t end = lane == 0 ? s1 : lane == 1 ? s2 : lane == 2 ? s3 : bits;
+                s_sb_src[warp * 4u + lane] = begin;
+                s_sb_bits[warp * 4u + lane] = end - begin;
+            }
+            if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
         } else {
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) tile_nnz += __shfl_xor_sync(0xffffffffu, tile_nnz, o);
+            for (int o = 16; o > 0; o >>= 1) my_nnz += __shfl_xor_sync(0xffffffffu, my_nnz, o);
+            if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
+        }
+        __syncthreads();                                    // B2: the tile's data is no longer read; lengths visible
+        if (tid == 0) fetch_tile((it + 1u) & 1u);           // the next tile's bytes arrive while this one is packed
+
+        // ---- layout of the tile's records ---------------------------------------------
+        uint64_t tile_off = 0;
+        uint32_t tile_words = 0;
+        uint32_t my_blk_wordoff = 0;                        // lane bi: word offset of block bi within the tile
+        if (MODE == kModeErc) {
+            // every warp runs the same scan over the 32 sub-block lengths
+            const uint32_t sb = lane;
+            const uint32_t v = sb < nsb_tile ? s_sb_bits[sb] : 0u;
+            uint32_t incl = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= (uint32_t)o) incl += t;
+            }
+            const uint32_t excl = incl - v;
+            const uint32_t bi = bi_lane, sb0 = bi * spb;
+            const uint32_t sb_last = min(sb0 + spb, nsb_tile) - 1u;         // meaningful when sb < nsb_tile
+            const uint32_t excl0 = __shfl_sync(0xffffffffu, excl, sb0 & 31u);
+            const uint32_t incl_last = __shfl_sync(0xffffffffu, incl, sb_last & 31u);
+            const uint32_t nsb_blk = sb_last - sb0 + 1u;
+            const uint32_t head_words = 1u + (nsb_blk + 1u) / 2u;
+            const bool leader = sb < nsb_tile && sb == sb0;
+            const uint32_t blk_words = leader ? head_words + (incl_last - excl0 + 31u) / 32u : 0u;
+            uint32_t wincl = blk_words;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(0xffffffffu, wincl, o);
+                if (lane >= (uint32_t)o) wincl += t;
+            }
+            const uint32_t wexcl = wincl - blk_words;
+            const uint32_t blk_off = __shfl_sync(0xffffffffu, wexcl, sb0 & 31u);    // words before my block
+            const uint32_t my_bitoff = 32u * (blk_off + head_words) + (excl - excl0);   // where sub-block `lane` goes
+            tile_words = __shfl_sync(0xffffffffu, wincl, 31);
+            const uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
+            // lane bi keeps the offset of block bi (held by the lane of the block's first sub-block)
+            my_blk_wordoff = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
+            // header words of the blocks: norm, then the u16 lengths two per word.  Lanes 4w .. 4w+3
+            // of warp w stand for the warp's own sub-blocks, whose norms it holds.
+            if ((lane >> 2) == warp && sb < nsb_tile) {
+                const uint32_t q = lane & 3u;
+                const float nq = q == 0 ? norm_q[0] : q == 1 ? norm_q[1] : q == 2 ? norm_q[2] : norm_q[3];
+                if (leader) stage[blk_off] = __float_as_uint(nq);
+                const uint32_t sbi = sb - sb0;
+                atomicOr(stage + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
+            }
+            if (tid == 0) s_code_bits = code_bits;
+
+            // ---- every warp moves its sub-block strings to their place in the staged tile ----
+            __syncwarp();
+#pragma unroll 1
+            for (uint32_t q = 0; q < 4; ++q) {
+                const uint32_t sbq = warp * 4u + q;
+                if (sbq >= nsb_tile) break;
+                const uint32_t len = s_sb_bits[sbq], src = s_sb_src[sbq];
+                const uint32_t dst = __shfl_sync(0xffffffffu, my_bitoff, sbq);
+                if (len == 0) continue;
+                const uint32_t w_first = dst >> 5, w_last = (dst + len - 1u) >> 5;
+                for (uint32_t w = w_first + lane; w <= w_last; w += 32) {
+                    const int sbit = (int)src + (int)(32u * w) - (int)dst;
+                    uint32_t val = bits_at(window, sbit);
+                    const uint32_t head = 32u * w < dst ? dst - 32u * w : 0u;     // bits of this word before the string
+                    const uint32_t tail_end = min(dst + len - 32u * w, 32u);      // bits of this word up to its end
+                    uint32_t mask = 0xFFFFFFFFu >> head;
+                    if (tail_end < 32u) mask &= ~(0xFFFFFFFFu >> tail_end);
+                    val &= mask;
+                    if (val) atomicOr(stage + w, val);
+                }
+            }
+            __syncwarp();
+            for (uint32_t i = lane; i < (bits + 31u) / 32u + 2u; i += 32) window[i] = 0;   // ready for the next tile
+        } else {
+            if (G.bucket <= kBLK) {
+                tile_off = first_block * G.rec_words;
+                tile_words = (nblk_tile - 1u) * G.rec_words + 1u +
+                             ((tile_len - (nblk_tile - 1u) * G.bucket) * G.width + 31u) / 32u;
+                // norm words: lanes 4w .. 4w+3 of warp w stand for the warp's own sub-blocks
+                if ((lane >> 2) == warp && lane < nsb_tile && lane == bi_lane * spb) {
+                    const uint32_t q = lane & 3u;
+                    const float nq = q == 0 ? norm_q[0] : q == 1 ? norm_q[1] : q == 2 ? norm_q[2] : norm_q[3];
+                    stage[bi_lane * G.rec_words] = __float_as_uint(nq);
+                }
+            } else {
+                tile_off = bucket_idx * G.rec_words + 1u + (uint64_t)bib * (kBLK * G.width / 32u);
+                tile_words = (tile_len * G.width + 31u) / 32u;
+                if (bib == 0 && tid == 0) payload[bucket_idx * G.rec_words] = __float_as_uint(norm_q[0]);
+            }
+        }
+        __syncthreads();                                    // B3: the staged tile is complete
+
+        if (MODE == kModeErc) {
+            if (warp == 0) {                                // chain the tile to its predecessors
+                bool failed;
+                const uint64_t off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
+                if (lane == 0) {
+                    s_tile_off = off;
+                    if (failed) s_abort = 1;
+                }
+            }
+            __syncthreads();                                // B4
+            tile_off = s_tile_off;
         }
 
-        // ---- last tile to finish writes the header -------------------------------------------------------
-        __syncwarp();
-        if (lane == 0) {
-            if (tile_nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)tile_nnz);
+        // ---- copy the tile out ---------------------------------------------------------
+        const bool aborted = s_abort != 0;
+        for (uint32_t i = tid; i < tile_words; i += kEncThreads) {
+            if (!aborted) payload[tile_off + i] = stage[i];
+            stage[i] = 0;
+        }
+        if (MODE == kModeErc && !aborted && warp == 0) {
+            if (lane < nblk_tile) table[first_block + lane] = 32ull * (tile_off + my_blk_wordoff);
+            if (tile == G.ntiles - 1 && lane == 0) {
+                table[G.nblk] = 32ull * (tile_off + tile_words);
+                P.ws->total_words = tile_off + tile_words;
+            }
+        }
+        __syncthreads();                                    // B5: stage is clean, counters are final
+
+        // ---- last tile to finish writes the header -------------------------------------
+        if (tid == 0) {
+            if (s_nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)s_nnz);
+            if (MODE == kModeErc && s_code_bits)
+                atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)s_code_bits);
+            s_nnz = 0;
+            s_code_bits = 0;
             __threadfence();
             unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), 1ull);
             if (prev == G.ntiles - 1) {
@@ -622,6 +743,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             }
         }
     }
+    // a copy that was started for a tile nobody will pack must land before the CTA may exit
+    // (fetch_tile only starts copies for valid tiles, and every valid tile is waited for above)
 }
 
 // ---------------------------------------------------------------------------
@@ -673,18 +796,28 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
     return cudaGetLastError();
 }
 
-int encode_max_blocks(int sms) { return sms * kEncMinBlocks; }
+// shared memory of one CTA: the tile, its staged image, and per warp a bit window and a token list
+size_t encode_smem_bytes(const EncodeParams& P) {
+    return 4u * ((size_t)kBLK + P.stage_words + (size_t)kEncWarps * P.warp_smem_words);
+}
+
+int encode_max_blocks(int sms, size_t smem_bytes) {
+    size_t per_sm = (227u * 1024u) / (smem_bytes + 1024u + 3u * 1024u);     // + static shared memory and the per-CTA reserve
+    if (per_sm > (size_t)kEncMinBlocks) per_sm = kEncMinBlocks;
+    if (per_sm < 1) per_sm = 1;
+    return sms * (int)per_sm;
+}
 
 template <uint32_t L, uint32_t M>
 static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
-    const size_t smem = (size_t)kEncWarps * P.warp_smem_words * 4u;
+    const size_t smem = encode_smem_bytes(P);
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    if (smem > 96 * 1024 || P.grid == 0) return cudaErrorInvalidValue;
+    if (smem > 112 * 1024 || P.grid == 0) return cudaErrorInvalidValue;
     encode_kernel<L, M><<<P.grid, kEncThreads, smem, stream>>>(P);
     return cudaGetLastError();
 }
