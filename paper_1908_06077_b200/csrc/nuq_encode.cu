@@ -635,6 +635,15 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 atomicOr(stage + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
             }
             if (tid == 0) s_code_bits = code_bits;
+            if (warp == 0) {
+                // chain the tile to its predecessors while the other warps move their strings
+                bool failed;
+                const uint64_t off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
+                if (lane == 0) {
+                    s_tile_off = off;
+                    if (failed) s_abort = 1;
+                }
+            }
 
             // ---- every warp moves its sub-block strings to their place in the staged tile ----
             __syncwarp();
@@ -676,20 +685,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 if (bib == 0 && tid == 0) payload[bucket_idx * G.rec_words] = __float_as_uint(norm_q[0]);
             }
         }
-        __syncthreads();                                    // B3: the staged tile is complete
-
-        if (MODE == kModeErc) {
-            if (warp == 0) {                                // chain the tile to its predecessors
-                bool failed;
-                const uint64_t off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
-                if (lane == 0) {
-                    s_tile_off = off;
-                    if (failed) s_abort = 1;
-                }
-            }
-            __syncthreads();                                // B4
-            tile_off = s_tile_off;
-        }
+        __syncthreads();                                    // B3: the staged tile is complete, its place is known
+        if (MODE == kModeErc) tile_off = s_tile_off;
 
         // ---- copy the tile out ---------------------------------------------------------
         const bool aborted = s_abort != 0;
@@ -704,8 +701,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 P.ws->total_words = tile_off + tile_words;
             }
         }
-        __syncthreads();                                    // B5: stage is clean, counters are final
 
+        // (no barrier here: the next tile's first barrier orders the clean stage and the counters)
         // ---- last tile to finish writes the header -------------------------------------
         if (tid == 0) {
             if (s_nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)s_nnz);
