@@ -124,20 +124,63 @@ __device__ __forceinline__ void st_volatile_u64(uint64_t* p, uint64_t v) {
 
 // Decoupled look-back over tile payload sizes, run by one warp.  Returns the
 // exclusive prefix (words) of `tile`, or sets *failed.  Every wait is bounded.
+//
+// All CTAs of a wave reach this point at about the same time, so a tile usually finds
+// its ~450 running predecessors in the "aggregate" state and has to sum all of them.
+// A step therefore looks at 256 predecessors at once (8 independent loads per lane):
+// the walk costs a couple of L2 round trips instead of one per 32 tiles.
+constexpr int kLookPerLane = 8;
+// The caller has already stored kTileAggregate | aggregate (kTilePrefix for tile 0) in state[tile].
 __device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile, uint64_t aggregate, bool* failed) {
     const uint32_t lane = lane_id();
     *failed = false;
-    if (tile == 0) {
-        if (lane == 0) st_volatile_u64(state, kTilePrefix | aggregate);
-        return 0;
-    }
-    if (lane == 0) st_volatile_u64(state + tile, kTileAggregate | aggregate);
+    if (tile == 0) return 0;                               // announced as a prefix by the caller
     uint64_t exclusive = 0;
-    int64_t idx = (int64_t)tile - 1 - (int64_t)lane;
+    int64_t base = (int64_t)tile - 1;                      // nearest predecessor not yet accounted for
+    uint32_t polls = 0;
     for (;;) {
-        uint64_t v = idx >= 0 ? ld_volatile_u64(state + idx) : kTilePrefix;   // before tile 0: prefix 0
-        uint32_t polls = 0;
-        while (__any_sync(0xffffffffu, (v >> 62) == 0)) {
+        // lane l looks at predecessors base - 8 l, base - 8 l - 1, ..., nearest first
+        uint64_t v[kLookPerLane];
+#pragma unroll
+        for (int k = 0; k < kLookPerLane; ++k) {
+            const int64_t idx = base - (int64_t)(lane * kLookPerLane + k);
+            v[k] = idx >= 0 ? ld_volatile_u64(state + idx) : kTilePrefix;     // before tile 0: prefix 0
+        }
+        uint64_t sum = 0;
+        uint32_t stop = 0;                                  // 0 none, 1 not ready, 2 prefix found, 3 poisoned
+#pragma unroll
+        for (int k = 0; k < kLookPerLane; ++k) {
+            const uint32_t flag = (uint32_t)(v[k] >> 62);
+            if (stop == 0) {
+                if (flag == 0) stop = 1;
+                else if (flag == 3) stop = 3;
+                else {
+                    sum += v[k] & kTileValueMask;
+                    if (flag == 2) stop = 2;
+                }
+            }
+        }
+        const uint32_t stops = __ballot_sync(0xffffffffu, stop != 0);
+        const uint32_t first = stops ? (uint32_t)__ffs(stops) - 1u : 32u;      // lanes below it are all aggregates
+        const uint32_t how = __shfl_sync(0xffffffffu, stop, first & 31u);
+        uint64_t contrib = lane <= first ? sum : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
+        if (stops && how == 3) {                            // a predecessor gave up
+            if (lane == 0) st_volatile_u64(state + tile, kTilePoison);
+            *failed = true;
+            return 0;
+        }
+        if (stops && how == 1) {
+            // the states up to the first one that is not ready are final: take them, wait, look again
+            exclusive += contrib;
+            // how many states of lane `first` were taken before the unready one
+            uint32_t taken = kLookPerLane;
+#pragma unroll
+            for (int k = kLookPerLane - 1; k >= 0; --k)
+                if ((uint32_t)(v[k] >> 62) == 0) taken = (uint32_t)k;
+            taken = __shfl_sync(0xffffffffu, taken, first & 31u);
+            base -= (int64_t)(first * kLookPerLane + taken);
             if (++polls > (1u << 16)) {                    // ~tens of ms: give up, never hang
                 if (lane == 0) {
                     latch_status(ws, kErrTimeout);
@@ -146,22 +189,12 @@ __device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile,
                 *failed = true;
                 return 0;
             }
-            __nanosleep(polls < 8 ? 200 : 1000);           // a waiting warp should not eat issue slots
-            if ((v >> 62) == 0) v = ld_volatile_u64(state + idx);
+            __nanosleep(polls < 16 ? 100 : 1000);          // a waiting warp should not eat issue slots
+            continue;
         }
-        if (__any_sync(0xffffffffu, (v >> 62) == 3)) {     // a predecessor gave up
-            if (lane == 0) st_volatile_u64(state + tile, kTilePoison);
-            *failed = true;
-            return 0;
-        }
-        uint32_t prefix_mask = __ballot_sync(0xffffffffu, (v >> 62) == 2);
-        uint32_t first = prefix_mask ? (uint32_t)__ffs(prefix_mask) - 1u : 31u;
-        uint64_t contrib = lane <= first ? (v & kTileValueMask) : 0;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
         exclusive += contrib;
-        if (prefix_mask) break;
-        idx -= 32;
+        if (stops) break;                                   // how == 2: reached a tile that knows its prefix
+        base -= 32 * kLookPerLane;
     }
     if (lane == 0) st_volatile_u64(state + tile, kTilePrefix | (exclusive + aggregate));
     return exclusive;
@@ -230,8 +263,82 @@ __device__ __forceinline__ uint32_t bits_at(const uint32_t* src, int sbit) {
 }
 
 constexpr uint32_t kWarpElems = kBLK / kEncWarps;   // 1024 elements of a tile per warp (4 sub-blocks)
-constexpr uint32_t kChunk = 512;                    // elements quantized before their tokens are generated
+constexpr uint32_t kChunk = kEncChunk;              // elements quantized before their tokens are generated
 constexpr uint32_t kChunkRows = kChunk / 128;
+
+// A tile whose records are staged in shared memory and whose place in the stream is not
+// yet known.
+struct Pending {
+    unsigned long long tile;
+    uint32_t words, nblk, code_bits, nnz, valid, pad;
+    uint32_t blk_wordoff[32];                              // word offset of block bi within the tile
+};
+
+// Bookkeeping when a tile has been written: counters, and the container header by whichever
+// tile finishes last.  One thread.
+template <uint32_t MODE>
+__device__ void finish_tile(const EncodeParams& P, uint32_t nnz, uint32_t code_bits) {
+    const Geometry& G = P.geo;
+    if (nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)nnz);
+    if (code_bits) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)code_bits);
+    __threadfence();
+    const unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), 1ull);
+    if (prev != G.ntiles - 1) return;
+    __threadfence();
+    uint64_t code_total, words;
+    const uint64_t nnz_total = ld_volatile_u64(&P.ws->nnz);
+    const uint64_t nrec = MODE == kModeErc ? G.nblk : G.nb;
+    if (MODE == kModeErc) {
+        code_total = ld_volatile_u64(&P.ws->code_bits);
+        words = kHeaderWords + 2 * (G.nblk + 1) + ld_volatile_u64(&P.ws->total_words);
+    } else {
+        code_total = G.d * G.width;
+        const uint64_t last = G.d - (G.nb - 1) * G.bucket;
+        words = kHeaderWords + (G.nb - 1) * G.rec_words + 1 + (last * G.width + 31) / 32;
+    }
+    const uint64_t container_bits = 32 * words;
+    uint32_t* h = P.out;
+    h[0] = kMagic; h[1] = kVersion;
+    h[2] = (uint32_t)G.d; h[3] = (uint32_t)(G.d >> 32);
+    h[4] = G.bucket; h[5] = G.s;
+    h[6] = G.norm_kind | (G.levelset << 8) | (G.mode << 16);
+    h[7] = kSB;
+    h[8] = (uint32_t)nrec; h[9] = (uint32_t)(nrec >> 32);
+    h[10] = (uint32_t)container_bits; h[11] = (uint32_t)(container_bits >> 32);
+    h[12] = (uint32_t)code_total; h[13] = (uint32_t)(code_total >> 32);
+    h[14] = (uint32_t)nnz_total; h[15] = (uint32_t)(nnz_total >> 32);
+    if (P.out_bits) *P.out_bits = container_bits;
+}
+
+// One warp: find the place of a staged tile (its predecessors announced their sizes an
+// iteration ago, so the walk rarely waits), copy the image to the stream, clear the stage.
+__device__ void flush_pending(const EncodeParams& P, Pending& pd, uint32_t* stg, uint64_t* tile_state, uint64_t* table,
+                              uint32_t* payload, uint32_t lane) {
+    const Geometry& G = P.geo;
+    const uint64_t tile = pd.tile;
+    const uint32_t words = pd.words;
+    bool failed;
+    const uint64_t off = tile_lookback(P.ws, tile_state, tile, words, &failed);
+    for (uint32_t i = lane; i < words; i += 32) {
+        if (!failed) payload[off + i] = stg[i];
+        stg[i] = 0;
+    }
+    if (!failed) {
+        const uint64_t first_block = G.bucket <= kBLK ? tile * G.blocks_per_tile : tile;
+        if (lane < pd.nblk) table[first_block + lane] = 32ull * (off + pd.blk_wordoff[lane]);
+        if (tile == G.ntiles - 1 && lane == 0) {
+            table[G.nblk] = 32ull * (off + words);
+            P.ws->total_words = off + words;
+        }
+    }
+    __syncwarp();
+    if (lane == 0) {
+        pd.valid = 0;
+        finish_tile<kModeErc>(P, pd.nnz, pd.code_bits);
+    }
+    __syncwarp();
+}
+
 
 template <uint32_t LEVELSET, uint32_t MODE>
 __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(const __grid_constant__ EncodeParams P) {
@@ -244,15 +351,16 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
     __shared__ uint32_t s_sb_bits[32];                     // token bits of each sub-block
     __shared__ uint32_t s_sb_src[32];                      // where they start in the owning warp's window
     __shared__ uint32_t s_start[32];                       // scratch: first token offset of a sub-block (per warp 4)
-    __shared__ unsigned long long s_tile[2], s_tile_off;
-    __shared__ uint32_t s_abort, s_nnz, s_code_bits;
+    __shared__ unsigned long long s_tile[2];
+    __shared__ uint32_t s_abort, s_nnz;
+    __shared__ Pending s_pend[2];                          // ERC: the two staged tiles (current, previous)
 
     using S = Sym<LEVELSET>;
     const Geometry& G = P.geo;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     float* data = reinterpret_cast<float*>(smem);                               // kBLK floats: the tile
     uint32_t* stage = smem + kBLK;                                              // image of the tile's records
-    uint32_t* wmem = stage + P.stage_words + warp * P.warp_smem_words;
+    uint32_t* wmem = stage + (MODE == kModeErc ? 2u : 1u) * P.stage_words + warp * P.warp_smem_words;
     uint32_t* window = wmem;                                                    // this warp's token string
     uint32_t* tokens = wmem + P.window_words;                                   // kChunk entries: position | field << 10
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
@@ -284,10 +392,13 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             tile_len = left < kBLK ? (uint32_t)left : kBLK;
         }
     };
-    // thread 0: take a ticket and start the copy of that tile into `data`
-    auto fetch_tile = [&](uint32_t slot) {
-        const uint64_t t = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
-        s_tile[slot] = t;
+    // thread 0: take a ticket ...
+    auto take_ticket = [&](uint32_t slot) {
+        s_tile[slot] = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+    };
+    // ... and start the copy of that tile into `data` once nobody reads the previous one
+    auto start_copy = [&](uint32_t slot) {
+        const uint64_t t = s_tile[slot];
         if (t < G.ntiles) {
             uint64_t elem0;
             uint32_t tile_len;
@@ -308,16 +419,20 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
         }
         s_lut_signed[tid] = v;
     }
-    for (uint32_t i = tid; i < P.stage_words; i += kEncThreads) stage[i] = 0;
+    for (uint32_t i = tid; i < (MODE == kModeErc ? 2u : 1u) * P.stage_words; i += kEncThreads) stage[i] = 0;
     for (uint32_t i = lane; i < P.window_words; i += 32) window[i] = 0;
     if (tid == 0) {
         mbar_init(&s_bar, 1);
         s_abort = 0;
         s_nnz = 0;
-        s_code_bits = 0;
+        s_pend[0].valid = 0;
+        s_pend[1].valid = 0;
     }
     __syncthreads();
-    if (tid == 0) fetch_tile(0);
+    if (tid == 0) {
+        take_ticket(0);
+        start_copy(0);
+    }
     __syncthreads();
 
     uint32_t parity = 0;
@@ -401,6 +516,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             }
         }
         __syncthreads();                                    // B1: partials visible
+        if (tid == 0) take_ticket((it + 1u) & 1u);          // visible to all after the next barrier
 
         // every warp derives the norms of the buckets its own sub-blocks belong to (same
         // reduction tree in every warp, so all agree bit for bit)
@@ -442,17 +558,21 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             }
         }
 
-        // ---- quantize (Definition 1) and generate tokens, 512 elements at a time -------------
+        // ---- quantize (Definition 1) and generate tokens, one chunk of elements at a time ------
         uint32_t bits = 0;                                  // ERC: bits in this warp's window so far
         uint32_t my_nnz = 0;
         if (MODE == kModeErc && lane < 4) s_start[warp * 4 + lane] = 0xFFFFFFFFu;
+        // lane q < 4 keeps 2^s / norm and the block of the warp's sub-block q for the loop below
+        const float inv_own = (lane & 3u) == 0 ? inv_q[0] : (lane & 3u) == 1 ? inv_q[1] : (lane & 3u) == 2 ? inv_q[2] : inv_q[3];
+        const uint32_t bi_own = (lane & 3u) == 0 ? bi_q[0] : (lane & 3u) == 1 ? bi_q[1] : (lane & 3u) == 2 ? bi_q[2] : bi_q[3];
 #pragma unroll 1
-        for (uint32_t half = 0; half < 2; ++half) {
+        for (uint32_t part = 0; part < kWarpElems / kChunk; ++part) {
             uint32_t ntok = 0;
 #pragma unroll
             for (uint32_t r = 0; r < kChunkRows; ++r) {
-                const uint32_t j = half * kChunkRows + r;   // row of the warp
-                const float inv = inv_q[j >> 1];
+                const uint32_t j = part * kChunkRows + r;   // row of the warp
+                const float inv = __shfl_sync(0xffffffffu, inv_own, j >> 1);
+                const uint32_t bi_row = __shfl_sync(0xffffffffu, bi_own, j >> 1);   // block of this row's sub-block
                 if (inv == 0.0f) continue;                  // bucket not quantized (warp uniform)
                 const float4 x = rows[32 * j];
                 const uint32_t base = wbase + j * 128u + lane * 4u;             // element within the tile
@@ -509,7 +629,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                     }
                     uint32_t cursor;
                     if (G.bucket <= kBLK) {
-                        const uint32_t bi = bi_q[j >> 1];
+                        const uint32_t bi = bi_row;
                         cursor = 32u * (bi * G.rec_words + 1u) + (base - bi * blk_elems) * wbits;
                     } else {
                         cursor = base * wbits;
@@ -555,7 +675,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                     }
                     const uint32_t off = bits + incl - tlen;    // bit of the window where my token starts
                     // the first token of a sub-block marks where that sub-block's string starts
-                    if (valid && first_of_sb) s_start[warp * 4u + half * 2u + ((uint32_t)pos >> 8)] = off;
+                    if (valid && first_of_sb) s_start[warp * 4u + part * (kChunk / kSB) + ((uint32_t)pos >> 8)] = off;
                     or_bits32(window, off, tokA, lenA);
                     if (LEVELSET != kLevelsExp) or_bits32(window, off + lenA, tokB, lenB);
                     bits += __shfl_sync(0xffffffffu, incl, 31);
@@ -587,13 +707,11 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
         }
         __syncthreads();                                    // B2: the tile's data is no longer read; lengths visible
-        if (tid == 0) fetch_tile((it + 1u) & 1u);           // the next tile's bytes arrive while this one is packed
+        if (tid == 0) start_copy((it + 1u) & 1u);           // the next tile's bytes arrive while this one is packed
 
         // ---- layout of the tile's records ---------------------------------------------
-        uint64_t tile_off = 0;
-        uint32_t tile_words = 0;
-        uint32_t my_blk_wordoff = 0;                        // lane bi: word offset of block bi within the tile
         if (MODE == kModeErc) {
+            uint32_t* stg = stage + (it & 1u) * P.stage_words;              // this tile's image; the other one is pending
             // every warp runs the same scan over the 32 sub-block lengths
             const uint32_t sb = lane;
             const uint32_t v = sb < nsb_tile ? s_sb_bits[sb] : 0u;
@@ -621,27 +739,31 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             const uint32_t wexcl = wincl - blk_words;
             const uint32_t blk_off = __shfl_sync(0xffffffffu, wexcl, sb0 & 31u);    // words before my block
             const uint32_t my_bitoff = 32u * (blk_off + head_words) + (excl - excl0);   // where sub-block `lane` goes
-            tile_words = __shfl_sync(0xffffffffu, wincl, 31);
+            const uint32_t tile_words = __shfl_sync(0xffffffffu, wincl, 31);
             const uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
-            // lane bi keeps the offset of block bi (held by the lane of the block's first sub-block)
-            my_blk_wordoff = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
             // header words of the blocks: norm, then the u16 lengths two per word.  Lanes 4w .. 4w+3
             // of warp w stand for the warp's own sub-blocks, whose norms it holds.
             if ((lane >> 2) == warp && sb < nsb_tile) {
                 const uint32_t q = lane & 3u;
                 const float nq = q == 0 ? norm_q[0] : q == 1 ? norm_q[1] : q == 2 ? norm_q[2] : norm_q[3];
-                if (leader) stage[blk_off] = __float_as_uint(nq);
+                if (leader) stg[blk_off] = __float_as_uint(nq);
                 const uint32_t sbi = sb - sb0;
-                atomicOr(stage + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
+                atomicOr(stg + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
             }
-            if (tid == 0) s_code_bits = code_bits;
             if (warp == 0) {
-                // chain the tile to its predecessors while the other warps move their strings
-                bool failed;
-                const uint64_t off = tile_lookback(P.ws, tile_state, tile, tile_words, &failed);
+                // announce the tile's size to its successors now; its own place is looked up one
+                // iteration later, when the predecessors have long announced theirs
+                Pending& pd = s_pend[it & 1u];
+                pd.blk_wordoff[lane] = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
                 if (lane == 0) {
-                    s_tile_off = off;
-                    if (failed) s_abort = 1;
+                    st_volatile_u64(tile_state + tile, (tile == 0 ? kTilePrefix : kTileAggregate) | tile_words);
+                    pd.tile = tile;
+                    pd.words = tile_words;
+                    pd.nblk = nblk_tile;
+                    pd.code_bits = code_bits;
+                    pd.nnz = s_nnz;
+                    pd.valid = 1;
+                    s_nnz = 0;
                 }
             }
 
@@ -663,12 +785,19 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                     uint32_t mask = 0xFFFFFFFFu >> head;
                     if (tail_end < 32u) mask &= ~(0xFFFFFFFFu >> tail_end);
                     val &= mask;
-                    if (val) atomicOr(stage + w, val);
+                    if (val) atomicOr(stg + w, val);
                 }
             }
             __syncwarp();
             for (uint32_t i = lane; i < (bits + 31u) / 32u + 2u; i += 32) window[i] = 0;   // ready for the next tile
+
+            // ---- one warp (they take turns) writes out the tile staged one iteration ago ----
+            if (warp == (it & 7u) && s_pend[(it & 1u) ^ 1u].valid)
+                flush_pending(P, s_pend[(it & 1u) ^ 1u], stage + ((it & 1u) ^ 1u) * P.stage_words, tile_state, table,
+                              payload, lane);
         } else {
+            uint64_t tile_off;
+            uint32_t tile_words;
             if (G.bucket <= kBLK) {
                 tile_off = first_block * G.rec_words;
                 tile_words = (nblk_tile - 1u) * G.rec_words + 1u +
@@ -684,64 +813,28 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 tile_words = (tile_len * G.width + 31u) / 32u;
                 if (bib == 0 && tid == 0) payload[bucket_idx * G.rec_words] = __float_as_uint(norm_q[0]);
             }
-        }
-        __syncthreads();                                    // B3: the staged tile is complete, its place is known
-        if (MODE == kModeErc) tile_off = s_tile_off;
-
-        // ---- copy the tile out ---------------------------------------------------------
-        const bool aborted = s_abort != 0;
-        for (uint32_t i = tid; i < tile_words; i += kEncThreads) {
-            if (!aborted) payload[tile_off + i] = stage[i];
-            stage[i] = 0;
-        }
-        if (MODE == kModeErc && !aborted && warp == 0) {
-            if (lane < nblk_tile) table[first_block + lane] = 32ull * (tile_off + my_blk_wordoff);
-            if (tile == G.ntiles - 1 && lane == 0) {
-                table[G.nblk] = 32ull * (tile_off + tile_words);
-                P.ws->total_words = tile_off + tile_words;
+            __syncthreads();                                // the staged fields are complete
+            for (uint32_t i = tid; i < tile_words; i += kEncThreads) {
+                payload[tile_off + i] = stage[i];
+                stage[i] = 0;
             }
-        }
-
-        // (no barrier here: the next tile's first barrier orders the clean stage and the counters)
-        // ---- last tile to finish writes the header -------------------------------------
-        if (tid == 0) {
-            if (s_nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)s_nnz);
-            if (MODE == kModeErc && s_code_bits)
-                atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)s_code_bits);
-            s_nnz = 0;
-            s_code_bits = 0;
-            __threadfence();
-            unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), 1ull);
-            if (prev == G.ntiles - 1) {
-                __threadfence();
-                uint64_t code_bits, words;
-                uint64_t nnz = ld_volatile_u64(&P.ws->nnz);
-                uint64_t nrec = MODE == kModeErc ? G.nblk : G.nb;
-                if (MODE == kModeErc) {
-                    code_bits = ld_volatile_u64(&P.ws->code_bits);
-                    words = kHeaderWords + 2 * (G.nblk + 1) + ld_volatile_u64(&P.ws->total_words);
-                } else {
-                    code_bits = G.d * G.width;
-                    uint64_t last = G.d - (G.nb - 1) * G.bucket;
-                    words = kHeaderWords + (G.nb - 1) * G.rec_words + 1 + (last * G.width + 31) / 32;
-                }
-                uint64_t container_bits = 32 * words;
-                uint32_t* h = P.out;
-                h[0] = kMagic; h[1] = kVersion;
-                h[2] = (uint32_t)G.d; h[3] = (uint32_t)(G.d >> 32);
-                h[4] = G.bucket; h[5] = G.s;
-                h[6] = G.norm_kind | (G.levelset << 8) | (G.mode << 16);
-                h[7] = kSB;
-                h[8] = (uint32_t)nrec; h[9] = (uint32_t)(nrec >> 32);
-                h[10] = (uint32_t)container_bits; h[11] = (uint32_t)(container_bits >> 32);
-                h[12] = (uint32_t)code_bits; h[13] = (uint32_t)(code_bits >> 32);
-                h[14] = (uint32_t)nnz; h[15] = (uint32_t)(nnz >> 32);
-                if (P.out_bits) *P.out_bits = container_bits;
+            if (tid == 0) {
+                const uint32_t nnz = s_nnz;
+                s_nnz = 0;
+                finish_tile<kModeFixed>(P, nnz, 0);
             }
         }
     }
-    // a copy that was started for a tile nobody will pack must land before the CTA may exit
-    // (fetch_tile only starts copies for valid tiles, and every valid tile is waited for above)
+
+    // ---- the tile staged in the last iteration is still pending ----
+    if (MODE == kModeErc) {
+        __syncthreads();
+        if (warp == 0) {
+            for (uint32_t b = 0; b < 2; ++b)
+                if (s_pend[b].valid)
+                    flush_pending(P, s_pend[b], stage + b * P.stage_words, tile_state, table, payload, lane);
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -795,7 +888,8 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
 
 // shared memory of one CTA: the tile, its staged image, and per warp a bit window and a token list
 size_t encode_smem_bytes(const EncodeParams& P) {
-    return 4u * ((size_t)kBLK + P.stage_words + (size_t)kEncWarps * P.warp_smem_words);
+    const size_t stages = P.geo.mode == kModeErc ? 2 : 1;   // ERC: the current tile and the one awaiting its place
+    return 4u * ((size_t)kBLK + stages * P.stage_words + (size_t)kEncWarps * P.warp_smem_words);
 }
 
 int encode_max_blocks(int sms, size_t smem_bytes) {
