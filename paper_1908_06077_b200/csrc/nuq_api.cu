@@ -162,7 +162,8 @@ static EncodePlan plan_encode(EncodeParams& P, int sms) {
     P.stage_words = (stage_words_for(G) + 3u) & ~3u;
     if (G.mode == kModeErc) {
         P.window_words = (kBLK / kEncWarps * (2u + max_level_code_bits(G)) + 31u) / 32u + 4u;
-        P.warp_smem_words = (P.window_words + kEncChunk + 3u) & ~3u;
+        const uint32_t list_words = G.levelset == kLevelsExp ? kEncChunk / 2u : kEncChunk;   // 16- or 32-bit entries
+        P.warp_smem_words = (P.window_words + list_words + 3u) & ~3u;
     } else {
         P.window_words = 0;
         P.warp_smem_words = 0;

@@ -362,7 +362,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
     uint32_t* stage = smem + kBLK;                                              // image of the tile's records
     uint32_t* wmem = stage + (MODE == kModeErc ? 2u : 1u) * P.stage_words + warp * P.warp_smem_words;
     uint32_t* window = wmem;                                                    // this warp's token string
-    uint32_t* tokens = wmem + P.window_words;                                   // kChunk entries: position | field << 10
+    uint32_t* tokens = wmem + P.window_words;               // kChunk entries: position | field << 10 (uniform levels)
+    uint16_t* tokens16 = reinterpret_cast<uint16_t*>(tokens);   //                position | field << 8  (exponential levels)
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
     uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
     uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
@@ -590,15 +591,16 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                     q2 = quantize_uniform(x.z, inv, top, rnd.z);
                     q3 = quantize_uniform(x.w, inv, top, rnd.w);
                 }
-                // fields (index | sign << kBits); a zero symbol has no sign
-                uint32_t f0, f1, f2, f3;
+                // fields (index | sign << kBits); in the fixed-width mode a zero symbol must carry no sign
+                uint32_t f = 0, f0 = 0, f1 = 0, f2 = 0, f3 = 0;
                 if (LEVELSET == kLevelsExp) {
                     const uint32_t syms = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
-                    const uint32_t tops = __byte_perm(__byte_perm(__float_as_uint(x.x), __float_as_uint(x.y), 0x0073),
-                                                      __byte_perm(__float_as_uint(x.z), __float_as_uint(x.w), 0x0073), 0x5410);
-                    const uint32_t nzb = (syms + 0x7F7F7F7Fu) & 0x80808080u;   // bit 7 of a byte: symbol != 0
-                    const uint32_t f = syms | (tops & nzb);
-                    f0 = f & 0xFFu; f1 = (f >> 8) & 0xFFu; f2 = (f >> 16) & 0xFFu; f3 = f >> 24;
+                    // top bytes of the four inputs: their sign bits at bits 7, 15, 23, 31
+                    uint32_t tops = __byte_perm(__byte_perm(__float_as_uint(x.x), __float_as_uint(x.y), 0x0073),
+                                                __byte_perm(__float_as_uint(x.z), __float_as_uint(x.w), 0x0073), 0x5410);
+                    if (MODE == kModeFixed) tops &= syms + 0x7F7F7F7Fu;        // bit 7 of a byte: symbol != 0
+                    f = syms | (tops & 0x80808080u);
+                    if (MODE == kModeFixed) { f0 = f & 0xFFu; f1 = (f >> 8) & 0xFFu; f2 = (f >> 16) & 0xFFu; f3 = f >> 24; }
                 } else {
                     f0 = q0 | (q0 ? (__float_as_uint(x.x) >> 16) & 0x8000u : 0u);
                     f1 = q1 | (q1 ? (__float_as_uint(x.y) >> 16) & 0x8000u : 0u);
@@ -612,10 +614,20 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                     uint32_t at = ntok + __popc(v0 & lt_mask) + __popc(v1 & lt_mask) + __popc(v2 & lt_mask) +
                                   __popc(v3 & lt_mask);
                     const uint32_t pos = r * 128u + lane * 4u;                  // position within the 512-element chunk
-                    if (q0) tokens[at++] = pos | (f0 << 10);
-                    if (q1) tokens[at++] = (pos + 1u) | (f1 << 10);
-                    if (q2) tokens[at++] = (pos + 2u) | (f2 << 10);
-                    if (q3) tokens[at++] = (pos + 3u) | (f3 << 10);
+                    if (LEVELSET == kLevelsExp) {
+                        // 16-bit entries position | field << 8, two at a time by byte permutation
+                        const uint32_t pb = pos * 0x01010101u + 0x03020100u;    // the four positions, one per byte
+                        const uint32_t e01 = __byte_perm(pb, f, 0x5140), e23 = __byte_perm(pb, f, 0x7362);
+                        if (q0) tokens16[at++] = (uint16_t)e01;
+                        if (q1) tokens16[at++] = (uint16_t)(e01 >> 16);
+                        if (q2) tokens16[at++] = (uint16_t)e23;
+                        if (q3) tokens16[at++] = (uint16_t)(e23 >> 16);
+                    } else {
+                        if (q0) tokens[at++] = pos | (f0 << 10);
+                        if (q1) tokens[at++] = (pos + 1u) | (f1 << 10);
+                        if (q2) tokens[at++] = (pos + 2u) | (f2 << 10);
+                        if (q3) tokens[at++] = (pos + 3u) | (f3 << 10);
+                    }
                     ntok += __popc(v0) + __popc(v1) + __popc(v2) + __popc(v3);
                 } else if (q0 | q1 | q2 | q3) {
                     // fixed-width fields, MSB first, straight into the staged tile
@@ -644,9 +656,10 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 int carry_pos = -1;                         // position (within the chunk) of the last nonzero so far
                 for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
                     const bool valid = t0 + lane < ntok;
-                    const uint32_t e = valid ? tokens[t0 + lane] : 0u;
-                    const int pos = (int)(e & 1023u);
-                    const uint32_t field = e >> 10;
+                    uint32_t e = 0;
+                    if (valid) e = LEVELSET == kLevelsExp ? (uint32_t)tokens16[t0 + lane] : tokens[t0 + lane];
+                    const int pos = (int)(e & (LEVELSET == kLevelsExp ? 255u : 1023u));
+                    const uint32_t field = e >> (LEVELSET == kLevelsExp ? 8 : 10);
                     int prev = __shfl_up_sync(0xffffffffu, pos, 1);
                     if (lane == 0) prev = carry_pos;
                     const bool first_of_sb = (prev >> 8) != (pos >> 8);      // also when there is no predecessor
@@ -770,10 +783,12 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             // ---- every warp moves its sub-block strings to their place in the staged tile ----
             __syncwarp();
 #pragma unroll 1
-            for (uint32_t q = 0; q < 4; ++q) {
+            for (uint32_t q = 0; q < 4; q += coarse ? 4u : 1u) {
+                // the strings of sub-blocks of one block follow one another in the window and in the
+                // tile alike, so a warp whose four sub-blocks share a block moves them in one piece
                 const uint32_t sbq = warp * 4u + q;
                 if (sbq >= nsb_tile) break;
-                const uint32_t len = s_sb_bits[sbq], src = s_sb_src[sbq];
+                const uint32_t len = coarse ? bits : s_sb_bits[sbq], src = coarse ? 0u : s_sb_src[sbq];
                 const uint32_t dst = __shfl_sync(0xffffffffu, my_bitoff, sbq);
                 if (len == 0) continue;
                 const uint32_t w_first = dst >> 5, w_last = (dst + len - 1u) >> 5;
