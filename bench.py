@@ -106,6 +106,24 @@ class ClockSampler:
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons)}
 
 
+def max_over_ranks(values, device):
+    """element-wise maximum of a list of floats over all ranks (the timing of a multi-rank run is the
+    slowest rank's); a no-op without a process group.  The only collective in this benchmark: the path
+    itself has no exchange step, every rank runs an independent replica."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.tolist()]
+
+
+def aggregate_value(world, K, d, t_step_ms):
+    """whole-job GB/s (fp32 in): every rank moves (K + 1) * 4 * d bytes per step"""
+    return world * (K + 1) * 4.0 * d / (t_step_ms / 1e3) / 1e9
+
+
 def oracle_step(workload, steps, warmup):
     """the CPU oracle on the same workload: K encodes + one decode_accumulate per step, single thread"""
     import oracle as O
@@ -227,15 +245,10 @@ def run_gpu(args):
                "d2h_bytes_per_step": 4 * d, "ms_per_step": t_e2e * 1e3}
 
     # ---- max over ranks ---------------------------------------------------------------------
-    if world > 1:
-        tt = torch.tensor([t_step, t_enc, t_dec], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        t_step, t_enc, t_dec = [float(x) for x in tt.tolist()]
-        if e2e is not None:
-            te = torch.tensor([e2e["ms_per_step"]], device="cuda", dtype=torch.float64)
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-            e2e["ms_per_step"] = float(te.item())
-            e2e["value"] = world * (K + 1) * 4.0 * d / (e2e["ms_per_step"] / 1e3) / 1e9
+    t_step, t_enc, t_dec = max_over_ranks([t_step, t_enc, t_dec], "cuda")
+    if e2e is not None:
+        e2e["ms_per_step"] = max_over_ranks([e2e["ms_per_step"]], "cuda")[0]
+        e2e["value"] = aggregate_value(world, K, d, e2e["ms_per_step"])
 
     if rank == 0:
         peak, peak_kind = measured_peak()
@@ -247,7 +260,7 @@ def run_gpu(args):
         dec_achieved = dec_bytes / (t_dec / 1e3) / 1e9
         line = {
             "metric": METRIC,
-            "value": world * (K + 1) * 4.0 * d / (t_step / 1e3) / 1e9,
+            "value": aggregate_value(world, K, d, t_step),
             "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": t_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": desc, "d": d, "bucket": bucket, "s": s, "K": K,
@@ -263,7 +276,7 @@ def run_gpu(args):
             "roofline_decode": {"kernel": "decode_kernel", "bound": "hbm", "achieved": dec_achieved, "peak": peak,
                                 "unit": "GB/s", "frac": dec_achieved / peak, "peak_kind": f"of {peak_kind}",
                                 "traffic": DECODE_TRAFFIC_BYTES.get(args.workload)},
-            "gpu_launches": steps * (K * (2 if wide else 1) + 1),
+            "gpu_launches": steps * (K * (2 if wide else 1) + 1),      # encode (+ bucket norms) per worker, one decode
             "clocks": clocks,
         }
         if e2e is not None:
@@ -277,9 +290,11 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/
-ENCODE_TRAFFIC_BYTES = {}
-DECODE_TRAFFIC_BYTES = {}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures
+# summarised under profiles/ (the decoder's write count is short under ncu: its write-back
+# drains after the kernel has ended)
+ENCODE_TRAFFIC_BYTES = {"c3": 102.31e6 + 3.72e6}
+DECODE_TRAFFIC_BYTES = {"c3": 24.65e6 + 44.35e6}
 
 
 def main():
