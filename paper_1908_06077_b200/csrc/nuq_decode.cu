@@ -280,6 +280,18 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
             const uint32_t entries = wide ? kListEntries / 2u : kListEntries;
             uint32_t width_now = 1;                         // streams decoded side by side; halves when a list overflows
             while (width_now < gcount) width_now <<= 1;
+            {
+                // start narrow enough for the longest chain of this warp: a token of dense data takes
+                // about 5 bits (3 at least), so bits / 5 tokens is a fair guess; a wrong guess only costs
+                // the retry below
+                uint32_t guess = 0;
+                if (lj < gcount && infos[lj].ok && infos[lj].mode == kModeErc) {
+                    const Chain c = chains[lj * 32u + my_sb];
+                    guess = (c.end - c.cur) / 5u + 2u;
+                }
+                guess = __reduce_max_sync(0xffffffffu, guess);
+                while (width_now > 1u && entries / (width_now * S) < guess) width_now >>= 1;
+            }
 
             for (uint32_t j0 = 0; j0 < gcount;) {
                 const uint32_t nact = width_now * S;        // lanes that own a chain in this pass
@@ -378,23 +390,37 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                                 }
                             }
                         } else if (round == 0) {
-                            // fixed-width fields: every element of the warp's sub-blocks has one
+                            // fixed-width fields: every element of the warp's sub-blocks has one.  A lane
+                            // takes 4 consecutive elements at a time: two words hold their 4 * width <= 40 bits
                             bool field_bad = false;
-                            for (uint32_t idx = lane; idx < S * kSB; idx += 32) {
-                                const uint32_t q = idx >> 8, p = idx & 255u, sb = warp * S + q;
+                            const uint32_t wd = sj.width, smask = (1u << (wd - 1u)) - 1u;
+                            for (uint32_t grp = lane; grp < S * (kSB / 4u); grp += 32) {
+                                const uint32_t q = grp >> 6, p = (grp & 63u) * 4u, sb = warp * S + q;
                                 if (sb >= nsb_tile || sb * kSB + p >= tile_len) continue;
+                                const uint32_t nel = min(4u, tile_len - (sb * kSB + p));
                                 const Chain cf = chains[j * 32u + sb];
-                                const uint32_t bit = cf.cur + p * sj.width;
+                                const uint32_t bit = cf.cur + p * wd;
                                 const uint32_t wi = bit >> 5;
                                 const uint32_t x0 = __ldg(cf.tok + min(wi, cf.last));
                                 const uint32_t x1 = __ldg(cf.tok + min(wi + 1u, cf.last));
-                                const uint32_t field = __funnelshift_l(x1, x0, bit) >> (32u - sj.width);
-                                const uint32_t sym = field & ((1u << (sj.width - 1u)) - 1u);
-                                if (sym >= sj.nlev) { field_bad = true; continue; }
-                                if (sym) {
-                                    const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
-                                    accw[idx] += (field >> (sj.width - 1u)) ? -v : v;
+                                const uint32_t x2 = __ldg(cf.tok + min(wi + 2u, cf.last));
+                                // 64 bits from the first field on
+                                const uint64_t win = ((uint64_t)__funnelshift_l(x1, x0, bit) << 32) | __funnelshift_l(x2, x1, bit);
+                                float4 a = *reinterpret_cast<float4*>(accw + grp * 4u);
+                                float* av = reinterpret_cast<float*>(&a);
+#pragma unroll
+                                for (uint32_t c = 0; c < 4; ++c) {
+                                    const uint32_t field = (uint32_t)(win >> (64u - (c + 1u) * wd)) & ((1u << wd) - 1u);
+                                    const uint32_t sym = field & smask;
+                                    if (c < nel) {
+                                        if (sym >= sj.nlev) field_bad = true;
+                                        else if (sym) {
+                                            const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
+                                            av[c] += (field >> (wd - 1u)) ? -v : v;
+                                        }
+                                    }
                                 }
+                                *reinterpret_cast<float4*>(accw + grp * 4u) = a;
                             }
                             if (__any_sync(0xffffffffu, field_bad) && lane == 0) latch_status(P.ws, kErrBadStream);
                         }
