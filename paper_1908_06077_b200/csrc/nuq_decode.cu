@@ -21,11 +21,12 @@
 //            every element receives its terms in ascending stream order: the
 //            sum is bit-reproducible and equals ((0 + q_0) + q_1) + ... .
 //
-// Lists hold 1536 entries per warp.  If a chain has more tokens than its share,
-// the pass is redone with half as many streams (twice the share); with a single
-// stream left, the lists are filled and added in several rounds, which cannot
-// change the order in which an element receives its terms.  No warp waits on
-// another except at the two block barriers of a group; nothing spins.
+// Lists hold 48 entries per chain.  Sparse streams need one decode / add round per
+// tile; when a chain may have more tokens than that, the rounds advance through
+// the sub-block 48 positions at a time (a chain has at most 48 tokens there), and
+// since all terms of an element fall into the same round the order of its adds
+// is unchanged.  No warp waits on another except at the two block barriers of a
+// group; nothing spins.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 
@@ -277,165 +278,160 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
             const uint32_t my_sn = my_sb < nsb_tile ? min(kSB, tile_len - my_sb * kSB) : 0u;   // elements of my sub-block
             bool wide = false;                              // index - 1 does not fit 7 bits (uniform levels, s = 8)
             for (uint32_t j = 0; j < gcount; ++j) wide = wide || (infos[j].ok && infos[j].nlev > 129u);
-            const uint32_t entries = wide ? kListEntries / 2u : kListEntries;
-            uint32_t width_now = 1;                         // streams decoded side by side; halves when a list overflows
-            while (width_now < gcount) width_now <<= 1;
-            {
-                // start narrow enough for the longest chain of this warp: a token of dense data takes
-                // about 5 bits (3 at least), so bits / 5 tokens is a fair guess; a wrong guess only costs
-                // the retry below
-                uint32_t guess = 0;
-                if (lj < gcount && infos[lj].ok && infos[lj].mode == kModeErc) {
-                    const Chain c = chains[lj * 32u + my_sb];
-                    guess = (c.end - c.cur) / 5u + 2u;
-                }
-                guess = __reduce_max_sync(0xffffffffu, guess);
-                while (width_now > 1u && entries / (width_now * S) < guess) width_now >>= 1;
-            }
+            const uint32_t cap = (wide ? kListEntries / 2u : kListEntries) / 32u;   // list entries per chain
+            const bool mine = lj < gcount;
+            const StreamInfo si = infos[mine ? lj : 0];
+            const Chain ch = chains[(mine ? lj : 0) * 32u + my_sb];
+            const bool has_chain = mine && si.ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
 
-            for (uint32_t j0 = 0; j0 < gcount;) {
-                const uint32_t nact = width_now * S;        // lanes that own a chain in this pass
-                const uint32_t cap = entries / nact;        // list entries per chain
-                const bool mine = lj >= j0 && lj < j0 + width_now && lj < gcount;
-                const uint32_t a = (lj - j0) * S + lq;      // my column in the interleaved list
-                const StreamInfo si = infos[mine ? lj : 0];
-                const Chain ch = chains[(mine ? lj : 0) * 32u + my_sb];
-                bool running = mine && si.ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
-                bool bad = false, retry = false;
-                uint32_t cur = ch.cur, pos = 0;
-                // One round fills the lists and adds them.  More than one round happens only when a
-                // single stream is being decoded (width_now == 1), where the order of the rounds
-                // cannot change the order in which an element receives its terms.
-                for (uint32_t round = 0;; ++round) {
-                    uint32_t n = 0;
-                    bool full = false;
-                    // Every lane executes every step (a lane whose chain has ended works on stale but
-                    // in-bounds data and commits nothing), so the loop body has no divergent branch
-                    // except the rare long-code path.
-                    uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + a;
-                    uint32_t* slot32 = list + a;
-                    while (__any_sync(0xffffffffu, running)) {
-                        const uint32_t wi = cur >> 5;
-                        const uint32_t x0 = __ldg(ch.tok + min(wi, ch.last));
-                        const uint32_t x1 = __ldg(ch.tok + min(wi + 1u, ch.last));
-                        const uint32_t win = __funnelshift_l(x1, x0, cur);                  // 32 bits from the cursor
-                        const uint32_t e1 = lut[win >> (32u - kLutBits)];
-                        const uint32_t t = win << (e1 >> 8);                                // the sign bit is on top
-                        const uint32_t e2 = lut[(t << 1) >> (32u - kLutBits)];
-                        uint32_t gap = e1 & 0xffu, sym = e2 & 0xffu, negative = t >> 31;
-                        uint32_t used = (e1 >> 8) + 1u + (e2 >> 8);
-                        bool good = e1 != 0 && e2 != 0;
-                        if (__any_sync(0xffffffffu, running && !good)) {
-                            if (running && !good) {         // a code longer than 12 bits: Algorithm 2 as a loop
-                                uint64_t win64 = window64(ch.tok, cur, ch.last);
-                                used = 0;
-                                good = erc_read(win64, used, gap);
-                                negative = (uint32_t)(win64 >> 63);
-                                win64 <<= 1;
-                                used += 1;
-                                good = good && erc_read(win64, used, sym);
-                            }
+            // A round decodes, for all 32 chains at once, the tokens whose position lies below a limit,
+            // and then adds them stream after stream.  Sparse data takes one round (limit = the whole
+            // sub-block).  When the lists could overflow, the limit advances by `cap` positions per
+            // round: a chain then has at most `cap` tokens per round, and every element still receives
+            // its terms in ascending stream order because all of its terms fall into the same round.
+            // a chain of t tokens in 256 positions takes about t (2 log2(256 / t) + 4) bits: 48 tokens ~ 400 bits
+            uint32_t guess = has_chain ? (ch.end - ch.cur) / 8u + 1u : 0u;
+            guess = __reduce_max_sync(0xffffffffu, guess);
+            uint32_t step = guess <= cap ? kSB : cap;
+            bool alive = has_chain, bad = false, fixed_done = false;
+            uint32_t cur = ch.cur, pos = 0;
+            uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
+            uint32_t* slot32 = list + lane;
+            for (uint32_t limit = step;; limit += step) {
+                uint32_t n = 0;
+                bool full = false, running = alive;
+                // Every lane executes every step (a lane that has stopped works on stale but in-bounds
+                // data and commits nothing): no divergent branch except the rare long-code path.
+                while (__any_sync(0xffffffffu, running)) {
+                    const uint32_t wi = cur >> 5;
+                    const uint32_t x0 = __ldg(ch.tok + min(wi, ch.last));
+                    const uint32_t x1 = __ldg(ch.tok + min(wi + 1u, ch.last));
+                    const uint32_t win = __funnelshift_l(x1, x0, cur);                      // 32 bits from the cursor
+                    const uint32_t e1 = lut[win >> (32u - kLutBits)];
+                    const uint32_t t = win << (e1 >> 8);                                    // the sign bit is on top
+                    const uint32_t e2 = lut[(t << 1) >> (32u - kLutBits)];
+                    uint32_t gap = e1 & 0xffu, sym = e2 & 0xffu, negative = t >> 31;
+                    uint32_t used = (e1 >> 8) + 1u + (e2 >> 8);
+                    bool good = e1 != 0 && e2 != 0;
+                    if (__any_sync(0xffffffffu, running && !good)) {
+                        if (running && !good) {             // a code longer than 12 bits: Algorithm 2 as a loop
+                            uint64_t win64 = window64(ch.tok, cur, ch.last);
+                            used = 0;
+                            good = erc_read(win64, used, gap);
+                            negative = (uint32_t)(win64 >> 63);
+                            win64 <<= 1;
+                            used += 1;
+                            good = good && erc_read(win64, used, sym);
                         }
-                        const uint32_t npos = pos + gap;
-                        const bool valid = good && used <= ch.end - cur && npos <= my_sn && sym != 0 && sym < si.nlev;
-                        const bool room = n < cap;
-                        const bool commit = running && valid && room;
-                        bad = bad || (running && !valid);
-                        full = full || (running && valid && !room);      // this token waits for the next round
-                        if (commit) {
-                            const uint32_t e = (npos - 1u) | (negative << 8) | ((sym - 1u) << 9);
-                            if (wide) slot32[n * nact] = e;
-                            else slot16[n * nact] = (uint16_t)e;
-                            pos = npos;
-                            cur += used;
-                            ++n;
-                        }
-                        running = commit && cur < ch.end;
                     }
-                    const bool any_full = __any_sync(0xffffffffu, full);
-                    if (any_full && width_now > 1u) {       // twice the list share per chain; start the pass again
-                        retry = true;
+                    const uint32_t npos = pos + gap;
+                    const bool valid = good && used <= ch.end - cur && npos <= my_sn && sym != 0 && sym < si.nlev;
+                    const bool inside = npos <= limit;      // else the token belongs to a later round
+                    const bool room = n < cap;
+                    const bool commit = running && valid && inside && room;
+                    if (running && !valid) {
+                        bad = true;
+                        alive = false;
+                    }
+                    full = full || (running && valid && inside && !room);
+                    if (commit) {
+                        const uint32_t e = (npos - 1u) | (negative << 8) | ((sym - 1u) << 9);
+                        if (wide) slot32[n * 32u] = e;
+                        else slot16[n * 32u] = (uint16_t)e;
+                        pos = npos;
+                        cur += used;
+                        ++n;
+                        alive = cur < ch.end;
+                    }
+                    running = commit && alive;
+                }
+                if (__any_sync(0xffffffffu, full)) {
+                    if (step == cap) {                      // cannot happen: at most `cap` positions per round
+                        bad = true;
                         break;
                     }
-                    __syncwarp();
-
-                    // ---- add, one stream after the other ----
-                    const uint32_t per_chain = 32u / S;     // lanes that share one chain's list
-                    const uint32_t c = lane / per_chain, i0 = lane - c * per_chain;
-                    for (uint32_t j = j0; j < min(j0 + width_now, gcount); ++j) {
-                        const StreamInfo sj = infos[j];
-                        const uint32_t owner = j * S + c;   // the lane that decoded chain (j, c)
-                        const uint32_t n_c = __shfl_sync(0xffffffffu, n, owner);
-                        const float norm_c = __shfl_sync(0xffffffffu, ch.norm, owner);
-                        if (!sj.ok) continue;
-                        if (sj.mode == kModeErc) {
-                            const uint32_t col = (j - j0) * S + c;
-                            float* part = accw + c * kSB;
-                            if (!wide && sj.levelset == kLevelsExp) {
-                                // value = +-norm * 2^(index - 1 - s): the exponent field is built from the entry
-                                const uint16_t* src = reinterpret_cast<const uint16_t*>(list) + col;
-                                const uint32_t ebias = 127u - G.s;              // (index - 1) + ebias = biased exponent
-                                for (uint32_t i = i0; i < n_c; i += per_chain) {
-                                    const uint32_t e = src[i * nact];
-                                    const float level = __uint_as_float(((e >> 9) + ebias) << 23);
-                                    const float v = __fmul_rn(norm_c, level);
-                                    part[e & 0xffu] += __uint_as_float(__float_as_uint(v) ^ ((e << 23) & 0x80000000u));
-                                }
-                            } else {
-                                for (uint32_t i = i0; i < n_c; i += per_chain) {
-                                    const uint32_t e = wide ? list[i * nact + col]
-                                                            : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * nact + col];
-                                    const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
-                                    part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
-                                }
-                            }
-                        } else if (round == 0) {
-                            // fixed-width fields: every element of the warp's sub-blocks has one.  A lane
-                            // takes 4 consecutive elements at a time: two words hold their 4 * width <= 40 bits
-                            bool field_bad = false;
-                            const uint32_t wd = sj.width, smask = (1u << (wd - 1u)) - 1u;
-                            for (uint32_t grp = lane; grp < S * (kSB / 4u); grp += 32) {
-                                const uint32_t q = grp >> 6, p = (grp & 63u) * 4u, sb = warp * S + q;
-                                if (sb >= nsb_tile || sb * kSB + p >= tile_len) continue;
-                                const uint32_t nel = min(4u, tile_len - (sb * kSB + p));
-                                const Chain cf = chains[j * 32u + sb];
-                                const uint32_t bit = cf.cur + p * wd;
-                                const uint32_t wi = bit >> 5;
-                                const uint32_t x0 = __ldg(cf.tok + min(wi, cf.last));
-                                const uint32_t x1 = __ldg(cf.tok + min(wi + 1u, cf.last));
-                                const uint32_t x2 = __ldg(cf.tok + min(wi + 2u, cf.last));
-                                // 64 bits from the first field on
-                                const uint64_t win = ((uint64_t)__funnelshift_l(x1, x0, bit) << 32) | __funnelshift_l(x2, x1, bit);
-                                float4 a = *reinterpret_cast<float4*>(accw + grp * 4u);
-                                float* av = reinterpret_cast<float*>(&a);
-#pragma unroll
-                                for (uint32_t c = 0; c < 4; ++c) {
-                                    const uint32_t field = (uint32_t)(win >> (64u - (c + 1u) * wd)) & ((1u << wd) - 1u);
-                                    const uint32_t sym = field & smask;
-                                    if (c < nel) {
-                                        if (sym >= sj.nlev) field_bad = true;
-                                        else if (sym) {
-                                            const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
-                                            av[c] += (field >> (wd - 1u)) ? -v : v;
-                                        }
-                                    }
-                                }
-                                *reinterpret_cast<float4*>(accw + grp * 4u) = a;
-                            }
-                            if (__any_sync(0xffffffffu, field_bad) && lane == 0) latch_status(P.ws, kErrBadStream);
-                        }
-                        __syncwarp();
-                    }
-                    if (!any_full) break;
-                    running = full;                         // the chains that stopped at a full list go on
-                }
-                if (__any_sync(0xffffffffu, bad) && lane == 0) latch_status(P.ws, kErrBadStream);
-                if (retry) {
-                    width_now >>= 1;
+                    // the guess was too low (only possible in a one-round attempt): nothing has been
+                    // added yet, start over with the window that cannot overflow
+                    step = cap;
+                    limit = 0;
+                    alive = has_chain;
+                    bad = false;
+                    cur = ch.cur;
+                    pos = 0;
                     continue;
                 }
-                j0 += width_now;
+                __syncwarp();
+
+                // ---- add, one stream after the other ----
+                const uint32_t per_chain = 32u / S;         // lanes that share one chain's list
+                const uint32_t c = lane / per_chain, i0 = lane - c * per_chain;
+                for (uint32_t j = 0; j < gcount; ++j) {
+                    const StreamInfo sj = infos[j];
+                    const uint32_t owner = j * S + c;       // the lane that decoded chain (j, c)
+                    const uint32_t n_c = __shfl_sync(0xffffffffu, n, owner);
+                    const float norm_c = __shfl_sync(0xffffffffu, ch.norm, owner);
+                    if (!sj.ok) continue;
+                    if (sj.mode == kModeErc) {
+                        float* part = accw + c * kSB;
+                        if (!wide && sj.levelset == kLevelsExp) {
+                            // value = +-norm * 2^(index - 1 - s): the exponent field is built from the entry
+                            const uint16_t* src = reinterpret_cast<const uint16_t*>(list) + owner;
+                            const uint32_t ebias = 127u - G.s;              // (index - 1) + ebias = biased exponent
+                            for (uint32_t i = i0; i < n_c; i += per_chain) {
+                                const uint32_t e = src[i * 32u];
+                                const float level = __uint_as_float(((e >> 9) + ebias) << 23);
+                                const float v = __fmul_rn(norm_c, level);
+                                part[e & 0xffu] += __uint_as_float(__float_as_uint(v) ^ ((e << 23) & 0x80000000u));
+                            }
+                        } else {
+                            for (uint32_t i = i0; i < n_c; i += per_chain) {
+                                const uint32_t e = wide ? list[i * 32u + owner]
+                                                        : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * 32u + owner];
+                                const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
+                                part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
+                            }
+                        }
+                    } else if (!fixed_done) {
+                        // fixed-width fields: every element of the warp's sub-blocks has one.  A lane
+                        // takes 4 consecutive elements at a time: two words hold their 4 * width <= 40 bits
+                        bool field_bad = false;
+                        const uint32_t wd = sj.width, smask = (1u << (wd - 1u)) - 1u;
+                        for (uint32_t grp = lane; grp < S * (kSB / 4u); grp += 32) {
+                            const uint32_t q = grp >> 6, p = (grp & 63u) * 4u, sb = warp * S + q;
+                            if (sb >= nsb_tile || sb * kSB + p >= tile_len) continue;
+                            const uint32_t nel = min(4u, tile_len - (sb * kSB + p));
+                            const Chain cf = chains[j * 32u + sb];
+                            const uint32_t bit = cf.cur + p * wd;
+                            const uint32_t wi = bit >> 5;
+                            const uint32_t x0 = __ldg(cf.tok + min(wi, cf.last));
+                            const uint32_t x1 = __ldg(cf.tok + min(wi + 1u, cf.last));
+                            const uint32_t x2 = __ldg(cf.tok + min(wi + 2u, cf.last));
+                            // 64 bits from the first field on
+                            const uint64_t win = ((uint64_t)__funnelshift_l(x1, x0, bit) << 32) | __funnelshift_l(x2, x1, bit);
+                            float4 a = *reinterpret_cast<float4*>(accw + grp * 4u);
+                            float* av = reinterpret_cast<float*>(&a);
+#pragma unroll
+                            for (uint32_t c = 0; c < 4; ++c) {
+                                const uint32_t field = (uint32_t)(win >> (64u - (c + 1u) * wd)) & ((1u << wd) - 1u);
+                                const uint32_t sym = field & smask;
+                                if (c < nel) {
+                                    if (sym >= sj.nlev) field_bad = true;
+                                    else if (sym) {
+                                        const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
+                                        av[c] += (field >> (wd - 1u)) ? -v : v;
+                                    }
+                                }
+                            }
+                            *reinterpret_cast<float4*>(accw + grp * 4u) = a;
+                        }
+                            if (__any_sync(0xffffffffu, field_bad) && lane == 0) latch_status(P.ws, kErrBadStream);
+                    }
+                    __syncwarp();
+                }
+                fixed_done = true;
+                if (!__any_sync(0xffffffffu, alive)) break;
             }
+            if (__any_sync(0xffffffffu, bad) && lane == 0) latch_status(P.ws, kErrBadStream);
         }
 
         // ---- write this warp's part of the tile once, and clear it for the next tile ----
