@@ -110,6 +110,66 @@ struct StreamHead {
     uint32_t ok, mode, levelset, nlev, width, pad;
 };
 
+// Where a tile lies in the vector and in the containers.
+struct TileGeo {
+    uint64_t elem0, first_block, bucket_idx;
+    uint32_t tile_len, spb, blk_elems, bib, nsb_tile;
+};
+
+// Descriptor of sub-block `sb` of the tile in stream `hd` (header already validated): block offsets
+// from the table, norm, the chain's place from the sub-block lengths; everything is range-checked.
+// Returns false when the container is malformed there.
+__device__ bool describe_chain(const Geometry& G, const TileGeo& T, const StreamHead& hd, uint32_t sb, Chain* out) {
+    Chain ch;
+    ch.tok = hd.hdr;
+    ch.norm = 0.0f;
+    ch.cur = ch.end = ch.last = 0;
+    *out = ch;
+    if (sb >= T.nsb_tile) return true;
+    const uint32_t bi = sb / T.spb, sb0 = bi * T.spb, sbi = sb - sb0;
+    const uint32_t blk_len = min(T.blk_elems, T.tile_len - min(T.tile_len, bi * T.blk_elems));
+    const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
+    if (hd.mode == kModeErc) {
+        const uint64_t head = kHeaderWords + 2 * (G.nblk + 1);
+        const uint64_t* table = reinterpret_cast<const uint64_t*>(hd.hdr + kHeaderWords);
+        const uint32_t* payload = hd.hdr + head;
+        const uint64_t payload_words = hd.cwords - head;
+        const uint64_t off = __ldg(table + T.first_block + bi), end = __ldg(table + T.first_block + bi + 1);
+        const uint32_t head_words = 1u + (nsb_blk + 1u) / 2u;
+        if (!((off & 31u) == 0 && (end & 31u) == 0 && off < end && (end >> 5) <= payload_words &&
+              ((end - off) >> 5) >= head_words && ((end - off) >> 5) <= (1u << 20)))
+            return false;
+        const uint32_t* rec = payload + (off >> 5);
+        const uint32_t tok_words = (uint32_t)((end - off) >> 5) - head_words;
+        // start of the chain = sum of the lengths of the earlier sub-blocks of its block
+        uint32_t cur = 0, len = 0;
+        for (uint32_t w = 0; 2u * w <= sbi; ++w) {
+            const uint32_t word = __ldg(rec + 1u + w), lo = word & 0xffffu, hi = word >> 16;
+            if (2u * w < sbi) cur += lo; else len = lo;
+            if (2u * w + 1u < sbi) cur += hi; else if (2u * w + 1u == sbi) len = hi;
+        }
+        if (cur + len > 32u * tok_words) return false;
+        ch.norm = __uint_as_float(__ldg(rec));
+        ch.tok = rec + head_words;
+        ch.cur = cur;
+        ch.end = cur + len;
+        ch.last = tok_words ? tok_words - 1u : 0u;
+    } else {
+        const uint32_t rec_words = 1u + (G.bucket * hd.width + 31u) / 32u;
+        const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
+        const uint32_t* payload = hd.hdr + kHeaderWords;
+        const uint64_t bucket_of_sb = G.bucket <= kBLK ? T.first_block + bi : T.bucket_idx;
+        const uint32_t* rec = payload + bucket_of_sb * rec_words;
+        const uint64_t bucket_len = bucket_of_sb == G.nb - 1 ? last_len : G.bucket;
+        ch.norm = __uint_as_float(__ldg(rec));
+        ch.tok = rec + 1;
+        ch.cur = (G.bucket <= kBLK ? sbi * kSB : T.bib * kBLK + sb * kSB) * hd.width;   // bit of the first field
+        ch.last = (uint32_t)((bucket_len * hd.width + 31) / 32) - 1u;
+    }
+    *out = ch;
+    return true;
+}
+
 __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
     const Geometry& G = P.geo;
@@ -118,9 +178,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     float* acc = reinterpret_cast<float*>(dsm);                                   // kBLK running sums
     uint16_t* lut = reinterpret_cast<uint16_t*>(dsm + 4u * kBLK);                 // ERC^-1 of 12-bit prefixes
-    Chain* chains = reinterpret_cast<Chain*>(dsm + 4u * kBLK + 2u * (1u << kLutBits));   // [group][32]
-    StreamInfo* infos = reinterpret_cast<StreamInfo*>(chains + kMaxGroup * 32u);  // [group]
-    StreamHead* heads = reinterpret_cast<StreamHead*>(infos + kMaxGroup);         // [kMaxK]
+    StreamHead* heads = reinterpret_cast<StreamHead*>(dsm + 4u * kBLK + 2u * (1u << kLutBits));   // [kMaxK]
     uint32_t* list = reinterpret_cast<uint32_t*>(heads + kMaxK) + warp * (kListEntries / 2u);
     float* accw = acc + warp * S * kSB;                     // this warp's part of the tile
 
@@ -156,133 +214,60 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
     for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
         *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    __shared__ unsigned long long s_tile;
+    __syncthreads();                                        // table and headers are ready; from here on warps run alone
+
     for (;;) {
-        // tiles are handed out one at a time: their cost varies with the density of the streams
-        __syncthreads();
-        if (threadIdx.x == 0) s_tile = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
-        __syncthreads();
-        const uint64_t tile = s_tile;
+        // work is handed out one warp-sized unit at a time (S sub-blocks of one tile, all streams)
+        unsigned long long unit = 0;
+        if (lane == 0) unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        unit = __shfl_sync(0xffffffffu, unit, 0);
+        const uint64_t tile = unit / NG;
+        const uint32_t part = (uint32_t)(unit % NG);        // which S sub-blocks of the tile
         if (tile >= G.ntiles) break;
         // ---- tile geometry (same tiling as the encoder) ---------------------------
-        uint64_t elem0, first_block, bucket_idx = 0;
-        uint32_t tile_len, spb, blk_elems, bib = 0;
+        TileGeo T;
+        T.bucket_idx = 0;
+        T.bib = 0;
         if (G.bucket <= kBLK) {
-            first_block = tile * G.blocks_per_tile;
-            elem0 = first_block * G.bucket;
-            uint64_t left = G.d - elem0;
-            tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
-            spb = G.sb_per_block;
-            blk_elems = G.bucket;
+            T.first_block = tile * G.blocks_per_tile;
+            T.elem0 = T.first_block * G.bucket;
+            const uint64_t left = G.d - T.elem0;
+            T.tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
+            T.spb = G.sb_per_block;
+            T.blk_elems = G.bucket;
         } else {
-            bucket_idx = tile / G.blk_per_bucket;
-            bib = (uint32_t)(tile % G.blk_per_bucket);
-            first_block = tile;
-            uint64_t b0 = bucket_idx * G.bucket;
-            uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
-            elem0 = b0 + (uint64_t)bib * kBLK;
-            uint64_t left = blen - (uint64_t)bib * kBLK;
-            tile_len = left < kBLK ? (uint32_t)left : kBLK;
-            spb = 32;
-            blk_elems = kBLK;
+            T.bucket_idx = tile / G.blk_per_bucket;
+            T.bib = (uint32_t)(tile % G.blk_per_bucket);
+            T.first_block = tile;
+            const uint64_t b0 = T.bucket_idx * G.bucket;
+            const uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
+            T.elem0 = b0 + (uint64_t)T.bib * kBLK;
+            const uint64_t left = blen - (uint64_t)T.bib * kBLK;
+            T.tile_len = left < kBLK ? (uint32_t)left : kBLK;
+            T.spb = 32;
+            T.blk_elems = kBLK;
         }
-        const uint32_t nsb_tile = (tile_len + kSB - 1) / kSB;
+        T.nsb_tile = (T.tile_len + kSB - 1) / kSB;
+        const uint32_t tile_len = T.tile_len, nsb_tile = T.nsb_tile;
+        const uint64_t elem0 = T.elem0;
 
         for (uint32_t g0 = 0; g0 < P.K; g0 += NG) {
             const uint32_t gcount = min(NG, P.K - g0);      // streams in this group
-            __syncthreads();                                // the previous descriptors are no longer read
-
-            // ================= set-up: warp j describes stream g0 + j =================
-            if (warp < gcount) {
-                const StreamHead hd = heads[g0 + warp];
-                const uint32_t* hdr = hd.hdr;
-                const uint32_t sb = lane;
-                bool ok = hd.ok != 0;
-                const uint32_t levelset = hd.levelset, mode = hd.mode, nlev = hd.nlev, width = hd.width;
-                const uint64_t cwords = hd.cwords;
-                const uint32_t bi = sb / spb, sb0 = bi * spb, sbi = sb - sb0;
-                const uint32_t blk_len = min(blk_elems, tile_len - min(tile_len, bi * blk_elems));
-                const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
-                Chain ch;
-                ch.tok = hdr;
-                ch.norm = 0.0f;
-                ch.cur = ch.end = ch.last = 0;
-                if (ok && mode == kModeErc) {
-                    const uint64_t head = kHeaderWords + 2 * (G.nblk + 1);
-                    bool lane_ok = true;
-                    uint32_t len = 0, head_words = 0, rec_words = 0;
-                    if (ok && sb < nsb_tile) {
-                        const uint64_t* table = reinterpret_cast<const uint64_t*>(hdr + kHeaderWords);
-                        const uint32_t* payload = hdr + head;
-                        const uint64_t payload_words = cwords - head;
-                        const uint64_t off = __ldg(table + first_block + bi), end = __ldg(table + first_block + bi + 1);
-                        head_words = 1u + (nsb_blk + 1u) / 2u;
-                        lane_ok = (off & 31u) == 0 && (end & 31u) == 0 && off < end && (end >> 5) <= payload_words &&
-                                  ((end - off) >> 5) >= head_words && ((end - off) >> 5) <= (1u << 20);
-                        if (lane_ok) {
-                            const uint32_t* rec = payload + (off >> 5);
-                            rec_words = (uint32_t)((end - off) >> 5);
-                            ch.norm = __uint_as_float(__ldg(rec));
-                            len = (__ldg(rec + 1u + sbi / 2u) >> (16u * (sbi & 1u))) & 0xffffu;
-                            ch.tok = rec + head_words;
-                        }
-                    }
-                    // start of a chain = sum of the lengths of the earlier sub-blocks of its block
-                    uint32_t incl = len;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= (uint32_t)o) incl += t;
-                    }
-                    const uint32_t excl0 = __shfl_sync(0xffffffffu, incl - len, sb0 & 31u);
-                    ch.cur = incl - len - excl0;
-                    ch.end = ch.cur + len;
-                    if (ok && sb < nsb_tile && lane_ok) {
-                        const uint32_t tok_words = rec_words - head_words;
-                        lane_ok = ch.end <= 32u * tok_words;
-                        ch.last = tok_words ? tok_words - 1u : 0u;
-                    }
-                    ok = __all_sync(0xffffffffu, ok && lane_ok);
-                } else if (ok) {
-                    const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
-                    const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
-                    if (sb < nsb_tile) {
-                        const uint32_t* payload = hdr + kHeaderWords;
-                        const uint64_t bucket_of_sb = G.bucket <= kBLK ? first_block + bi : bucket_idx;
-                        const uint32_t* rec = payload + bucket_of_sb * rec_words;
-                        const uint64_t bucket_len = bucket_of_sb == G.nb - 1 ? last_len : G.bucket;
-                        ch.norm = __uint_as_float(__ldg(rec));
-                        ch.tok = rec + 1;
-                        ch.cur = (G.bucket <= kBLK ? sbi * kSB : bib * kBLK + sb * kSB) * width;   // bit of the first field
-                        ch.last = (uint32_t)((bucket_len * width + 31) / 32) - 1u;
-                    }
-                }
-                chains[warp * 32u + sb] = ch;
-                if (lane == 0) {
-                    StreamInfo si;
-                    si.ok = ok ? 1u : 0u;
-                    si.mode = mode;
-                    si.levelset = levelset;
-                    si.nlev = nlev;
-                    si.width = width;
-                    infos[warp] = si;
-                    if (!ok && hd.ok) latch_status(P.ws, kErrBadStream);
-                }
-            }
-            __syncthreads();
 
             // ================= decode + add, warp-local =================
-            // lane (j, q): stream g0 + j, sub-block warp * S + q
+            // lane (j, q): stream g0 + j, sub-block part * S + q
             const uint32_t lj = lane / S, lq = lane - lj * S;
-            const uint32_t my_sb = warp * S + lq;
+            const uint32_t my_sb = part * S + lq;
             const uint32_t my_sn = my_sb < nsb_tile ? min(kSB, tile_len - my_sb * kSB) : 0u;   // elements of my sub-block
             bool wide = false;                              // index - 1 does not fit 7 bits (uniform levels, s = 8)
-            for (uint32_t j = 0; j < gcount; ++j) wide = wide || (infos[j].ok && infos[j].nlev > 129u);
+            for (uint32_t j = 0; j < gcount; ++j) wide = wide || (heads[g0 + j].ok && heads[g0 + j].nlev > 129u);
             const uint32_t cap = (wide ? kListEntries / 2u : kListEntries) / 32u;   // list entries per chain
             const bool mine = lj < gcount;
-            const StreamInfo si = infos[mine ? lj : 0];
-            const Chain ch = chains[(mine ? lj : 0) * 32u + my_sb];
-            const bool has_chain = mine && si.ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
+            const StreamHead si = heads[g0 + (mine ? lj : 0)];
+            Chain ch;                                       // each lane describes the chain it walks
+            const bool chain_ok = describe_chain(G, T, si, mine && si.ok ? my_sb : 32u, &ch);
+            if (__any_sync(0xffffffffu, !chain_ok) && lane == 0) latch_status(P.ws, kErrBadStream);
+            const bool has_chain = mine && si.ok && chain_ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
 
             // A round decodes, for all 32 chains at once, the tokens whose position lies below a limit,
             // and then adds them stream after stream.  Sparse data takes one round (limit = the whole
@@ -366,7 +351,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 const uint32_t per_chain = 32u / S;         // lanes that share one chain's list
                 const uint32_t c = lane / per_chain, i0 = lane - c * per_chain;
                 for (uint32_t j = 0; j < gcount; ++j) {
-                    const StreamInfo sj = infos[j];
+                    const StreamHead sj = heads[g0 + j];
                     const uint32_t owner = j * S + c;       // the lane that decoded chain (j, c)
                     const uint32_t n_c = __shfl_sync(0xffffffffu, n, owner);
                     const float norm_c = __shfl_sync(0xffffffffu, ch.norm, owner);
@@ -396,11 +381,13 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                         // takes 4 consecutive elements at a time: two words hold their 4 * width <= 40 bits
                         bool field_bad = false;
                         const uint32_t wd = sj.width, smask = (1u << (wd - 1u)) - 1u;
+                        Chain cf;
+                        cf.tok = sj.hdr; cf.norm = 0.0f; cf.cur = cf.end = cf.last = 0;
                         for (uint32_t grp = lane; grp < S * (kSB / 4u); grp += 32) {
-                            const uint32_t q = grp >> 6, p = (grp & 63u) * 4u, sb = warp * S + q;
+                            const uint32_t q = grp >> 6, p = (grp & 63u) * 4u, sb = part * S + q;
+                            if ((grp & 32u) == 0) describe_chain(G, T, sj, sb, &cf);   // a sub-block lasts two steps
                             if (sb >= nsb_tile || sb * kSB + p >= tile_len) continue;
                             const uint32_t nel = min(4u, tile_len - (sb * kSB + p));
-                            const Chain cf = chains[j * 32u + sb];
                             const uint32_t bit = cf.cur + p * wd;
                             const uint32_t wi = bit >> 5;
                             const uint32_t x0 = __ldg(cf.tok + min(wi, cf.last));
@@ -437,7 +424,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
         // ---- write this warp's part of the tile once, and clear it for the next tile ----
         __syncwarp();
         {
-            const uint32_t first = warp * S * kSB;
+            const uint32_t first = part * S * kSB;
             float* dst = P.acc + elem0 + first;
             for (uint32_t i = lane * 4u; i < S * kSB; i += 128u) {
                 if (first + i + 4u <= tile_len) {
@@ -453,7 +440,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
 }
 
 static size_t decode_smem_bytes(uint32_t group) {
-    return 4u * kBLK + 2u * (1u << kLutBits) + kMaxGroup * 32u * sizeof(Chain) + kMaxGroup * sizeof(StreamInfo) + kMaxK * sizeof(StreamHead) +
+    return 4u * kBLK + 2u * (1u << kLutBits) + kMaxK * sizeof(StreamHead) +
            (size_t)group * kListEntries * 2u;
 }
 
