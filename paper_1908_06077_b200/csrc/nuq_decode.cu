@@ -279,7 +279,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
             guess = __reduce_max_sync(0xffffffffu, guess);
             uint32_t step = guess <= cap ? kSB : cap;
             bool alive = has_chain, bad = false, fixed_done = false;
-            uint32_t cur = ch.cur, pos = 0;
+            uint32_t cur = ch.cur, pos = 0, max_sym = 0;
             uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
             uint32_t* slot32 = list + lane;
             for (uint32_t limit = step;; limit += step) {
@@ -309,18 +309,21 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                             good = good && erc_read(win64, used, sym);
                         }
                     }
+                    // Range checks are made once per chain, after the walk (see below): a token of a
+                    // malformed chain may be committed, but its position is masked to the sub-block
+                    // when it is added, so nothing is written out of bounds.
                     const uint32_t npos = pos + gap;
-                    const bool valid = good && used <= ch.end - cur && npos <= my_sn && sym != 0 && sym < si.nlev;
                     const bool inside = npos <= limit;      // else the token belongs to a later round
                     const bool room = n < cap;
-                    const bool commit = running && valid && inside && room;
-                    if (running && !valid) {
+                    const bool commit = running && good && inside && room;
+                    if (running && !good) {
                         bad = true;
                         alive = false;
                     }
-                    full = full || (running && valid && inside && !room);
+                    full = full || (running && good && inside && !room);
                     if (commit) {
-                        const uint32_t e = (npos - 1u) | (negative << 8) | ((sym - 1u) << 9);
+                        max_sym = max(max_sym, sym);
+                        const uint32_t e = ((npos - 1u) & 0xffu) | (negative << 8) | ((sym - 1u) << 9);
                         if (wide) slot32[n * 32u] = e;
                         else slot16[n * 32u] = (uint16_t)e;
                         pos = npos;
@@ -343,6 +346,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                     bad = false;
                     cur = ch.cur;
                     pos = 0;
+                    max_sym = 0;
                     continue;
                 }
                 __syncwarp();
@@ -418,6 +422,8 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 fixed_done = true;
                 if (!__any_sync(0xffffffffu, alive)) break;
             }
+            // a well-formed chain ends exactly at its declared length, inside its sub-block, with known indices
+            if (has_chain && !bad) bad = cur != ch.end || pos > my_sn || max_sym >= si.nlev;
             if (__any_sync(0xffffffffu, bad) && lane == 0) latch_status(P.ws, kErrBadStream);
         }
 
