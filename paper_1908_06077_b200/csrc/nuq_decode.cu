@@ -1,32 +1,31 @@
 // DECODE + aggregate (App. A decoding; Algorithm 1, aggregation line): the K
 // workers' containers are decoded and summed into one fp32 vector.
 //
-// A CTA owns a tile of up to 8192 output elements (32 coding sub-blocks) whose
-// running sums live in shared memory; the tile is written to HBM once.  Streams
-// are taken G at a time (G = 8, or 1 / 2 / 4 when K is smaller); the CTA has G
-// warps and warp w owns the S = 32 / G sub-blocks w*S .. w*S+S-1 of the tile, for
-// every stream of the group.  Three steps per group:
+// Work is handed out by ticket in warp-sized units: S consecutive sub-blocks of a
+// tile of up to 8192 output elements (32 coding sub-blocks), for G streams at a
+// time (G = 8, or 1 / 2 / 4 when K is smaller; S = 32 / G).  A warp keeps the
+// running sums of its S * 256 elements in shared memory and writes them to HBM
+// once; warps never wait for one another.  Per unit and group of streams:
 //
-//   set-up   warp j reads, for stream j of the group, the tile's block offsets,
-//            norms and sub-block token lengths, validates them and leaves one
-//            chain descriptor per sub-block in shared memory.
-//   decode   lane (j, q) of warp w walks the token chain of stream j, sub-block
-//            w*S+q: ERC^-1 gap, sign bit, ERC^-1 level index, by table look-up on
-//            a 32-bit window (12-bit prefix table; longer codes take the loop of
-//            Algorithm 2).  All 32 chains of a warp advance in lock step; the
-//            decoded (position, sign, index) triples go to a per-lane list.
+//   describe lane (j, q) reads, for stream j and sub-block q of the unit, the block
+//            offset, the norm and the sub-block token lengths, range-checks them and
+//            so knows where its chain of tokens starts and ends.
+//   decode   the lane walks that chain: ERC^-1 gap, sign bit, ERC^-1 level index, by
+//            table look-up on a 32-bit window (12-bit prefix table; longer codes take
+//            the loop of Algorithm 2).  All 32 chains of a warp advance in lock
+//            step; the decoded (position, sign, index) triples go to a per-lane list.
 //   add      for j = 0 .. G-1 in order, the warp adds the listed values of
-//            stream j into its part of the tile.  Entries of one stream hit
-//            distinct elements, so the adds are plain shared-memory updates, and
-//            every element receives its terms in ascending stream order: the
-//            sum is bit-reproducible and equals ((0 + q_0) + q_1) + ... .
+//            stream j into its sums.  Entries of one stream hit distinct elements,
+//            so the adds are plain shared-memory updates, and every element receives
+//            its terms in ascending stream order: the sum is bit-reproducible and
+//            equals ((0 + q_0) + q_1) + ... .
 //
 // Lists hold 48 entries per chain.  Sparse streams need one decode / add round per
-// tile; when a chain may have more tokens than that, the rounds advance through
+// unit; when a chain may have more tokens than that, the rounds advance through
 // the sub-block 48 positions at a time (a chain has at most 48 tokens there), and
 // since all terms of an element fall into the same round the order of its adds
-// is unchanged.  No warp waits on another except at the two block barriers of a
-// group; nothing spins.
+// is unchanged.  Streams in the fixed-width mode are added field by field in
+// their turn.  Nothing spins.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 
@@ -90,17 +89,12 @@ __device__ __forceinline__ uint32_t erc_prefix_entry(uint32_t idx) {
     return 0;
 }
 
-// What the set-up step leaves for the lane that walks sub-block `sb` of one stream.
+// What a lane needs to know to walk sub-block `sb` of one stream.
 struct Chain {
     const uint32_t* tok;     // ERC: token words of the sub-block's coding block;  fixed: field words of its bucket
     float norm;
     uint32_t cur, end;       // ERC: first and past-the-end bit of the chain;  fixed: bit of the first field, unused
     uint32_t last;           // last valid word index behind tok
-};
-
-// Per stream of the group.
-struct StreamInfo {
-    uint32_t ok, mode, levelset, nlev, width;
 };
 
 // Per stream of the call: what its header says, checked once per CTA.

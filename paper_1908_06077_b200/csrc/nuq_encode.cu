@@ -10,15 +10,19 @@
 // of the current tile and behind the other CTAs of the SM.  Per tile:
 //   1. each warp reduces the squares (fp64) of its 1024 elements per sub-block;
 //      after one barrier every warp derives the bucket norms it needs;
-//   2. each warp quantizes its elements 512 at a time (one 128-bit shared-memory
+//   2. each warp quantizes its elements 256 at a time (one 128-bit shared-memory
 //      load and one Philox block per lane and 128-element row), compacts the
 //      nonzero symbols with ballots into a dense list, and turns that list into
 //      tokens, 32 per step, appended to the warp's own bit string;
 //   3. after a second barrier every warp runs the same small scan over the 32
 //      sub-block lengths, which gives the layout of the tile's records, and
-//      shifts its strings to their place in the staged tile;
-//   4. one warp chains the tile's size to its predecessors (decoupled look-back,
-//      bounded waits) and the CTA copies the staged tile to the packed stream.
+//      shifts its strings to their place in the staged tile; the tile's size is
+//      announced to the tiles behind it at once;
+//   4. one iteration later (two staged tiles exist), one warp looks up the tile's
+//      place in the stream (decoupled look-back over the sizes announced by its
+//      predecessors, bounded waits) and copies the staged tile there.  Looking
+//      the place up later matters: the predecessors, which started at the same
+//      time, have all announced their sizes by then, so nobody waits.
 // In the fixed-width mode the fields go straight to their known place.
 //
 // The kernel is bound by instruction issue, not by HBM: the quantizer is branch
