@@ -294,7 +294,7 @@ def run_gpu(args):
 # summarised under profiles/ (the decoder's write count is short under ncu: its write-back
 # drains after the kernel has ended)
 ENCODE_TRAFFIC_BYTES = {"c3": 102.31e6 + 3.72e6}
-DECODE_TRAFFIC_BYTES = {"c3": 24.65e6 + 44.35e6}
+DECODE_TRAFFIC_BYTES = {"c3": 24.60e6 + 49.12e6}
 
 
 def main():
