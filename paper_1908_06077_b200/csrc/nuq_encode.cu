@@ -85,16 +85,15 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 //   0x7FFFFF - (word >> 9) to the bit pattern of y carries into the exponent field
 //   exactly in that case, so (bits + 0x7FFFFF - (word >> 9)) >> 23 - 126 is the level
 //   index e + 1 + [u < p].  For y < 1 the same expression is at most 1, and it is 1
-//   only if u < y as well, so the maximum with [u < y] is the index in every case.
-// y < 1 (r in [0, 2^-s]): p = y, and u < y  <=>  float(m) - y 2^24 < 0 (both terms
-//   exact, the sign of a rounded difference is the sign of the exact one).
+//   only if u < y as well.
+// y < 1 (r in [0, 2^-s]): p = y, and u < y  <=>  float(m) < y 2^24 (both sides exact).
+// With up = [float(m) < y 2^24] (always true for y >= 1) the index is max(hi, 1) if up, else 0.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t quantize_exp(float v, float inv, float top, uint32_t word) {
     const float y = fminf(__fmul_rn(fabsf(v), inv), top);
     const int hi = (int)(__float_as_uint(y) + (0x007FFFFFu - 0x3F000000u) - (word >> 9)) >> 23;
-    const float diff = __fsub_rn(__uint2float_rn(word >> 8), __fmul_rn(y, 16777216.0f));
-    const int up = (int)(__float_as_uint(diff) >> 31);
-    return (uint32_t)max(hi, up);
+    const bool up = __uint2float_rn(word >> 8) < __fmul_rn(y, 16777216.0f);
+    return up ? (uint32_t)max(hi, 1) : 0u;                  // no round-up: y < 1 and the index is 0
 }
 
 // Uniform levels k / 2^s:  p = y - floor(y).
@@ -632,7 +631,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                         if (q2) tokens[at++] = (pos + 2u) | (f2 << 10);
                         if (q3) tokens[at++] = (pos + 3u) | (f3 << 10);
                     }
-                    ntok += __popc(v0) + __popc(v1) + __popc(v2) + __popc(v3);
+                    ntok = __shfl_sync(0xffffffffu, at, 31);                     // lane 31 ends behind the last entry
                 } else if (q0 | q1 | q2 | q3) {
                     // fixed-width fields, MSB first, straight into the staged tile
                     const uint32_t wbits = G.width;
