@@ -91,11 +91,27 @@ uint32_t max_level_code_bits(const Geometry& G) {
     return best;
 }
 
+// Most token bits that `elems` consecutive elements lying in at most `buckets` buckets can produce.
+// Always true: a token has at most |ERC(1)| + 1 + L bits per position it consumes (L = longest
+// level code), i.e. 2 + L bits per element.  With the Euclidean norm computed by the encoder
+// itself a much smaller bound holds: a symbol above the lowest level needs r > 2^-s, and at most
+// 4^s coordinates of a bucket can have that (the counting step of the paper's sparsity lemma,
+// Lemma 10); all others cost at most |ERC(1)| + 1 + |ERC(1)| = 3 bits per consumed position.
+uint32_t token_bits_bound(const Geometry& G, uint32_t elems, uint32_t buckets, bool norms_are_ours) {
+    const uint32_t L = max_level_code_bits(G);
+    const uint32_t safe = elems * (2u + L);
+    if (!norms_are_ours || G.norm_kind != kNormL2 || G.s > 7u) return safe;
+    const uint64_t high = (uint64_t)buckets * ((1ull << (2u * G.s)) + 8u);      // + slack for the rounding of the norm
+    const uint32_t nhigh = high < elems ? (uint32_t)high : elems;
+    const uint32_t tight = 3u * elems + nhigh * (L - 1u);
+    return tight < safe ? tight : safe;
+}
+
 // words of shared-memory staging one tile can need
-uint32_t stage_words_for(const Geometry& G) {
+uint32_t stage_words_for(const Geometry& G, bool norms_are_ours) {
     if (G.mode == kModeFixed) return G.bucket <= kBLK ? G.blocks_per_tile * G.rec_words : kBLK * G.width / 32u;
     uint32_t head = 1u + (G.sb_per_block + 1u) / 2u + 1u;          // norm, lengths, padding
-    return G.blocks_per_tile * head + (kBLK * (2u + max_level_code_bits(G)) + 31u) / 32u;
+    return G.blocks_per_tile * head + (token_bits_bound(G, kBLK, G.blocks_per_tile, norms_are_ours) + 31u) / 32u;
 }
 
 uint64_t bound_bytes(const Geometry& G) {
@@ -154,14 +170,17 @@ struct EncodePlan {
     uint32_t want_grid;      // CTAs that give every SM its full share
 };
 
-static EncodePlan plan_encode(EncodeParams& P, int sms) {
+static EncodePlan plan_encode(EncodeParams& P, int sms, bool norms_are_ours) {
     const Geometry& G = P.geo;
     EncodePlan pl;
     pl.state_bytes = sizeof(Workspace) + 8 * G.ntiles;
     pl.norms_bytes = G.bucket > kBLK ? 4 * G.nb : 0;
-    P.stage_words = (stage_words_for(G) + 3u) & ~3u;
+    P.stage_words = (stage_words_for(G, norms_are_ours) + 3u) & ~3u;
     if (G.mode == kModeErc) {
-        P.window_words = (kBLK / kEncWarps * (2u + max_level_code_bits(G)) + 31u) / 32u + 4u;
+        // a warp's 1024 elements lie in at most this many buckets
+        const uint32_t warp_elems = kBLK / kEncWarps;
+        const uint32_t warp_buckets = G.bucket >= warp_elems ? 2u : warp_elems / G.bucket + 1u;
+        P.window_words = (token_bits_bound(G, warp_elems, warp_buckets, norms_are_ours) + 31u) / 32u + 4u;
         const uint32_t list_words = G.levelset == kLevelsExp ? kEncChunk / 2u : kEncChunk;   // 16- or 32-bit entries
         P.warp_smem_words = (P.window_words + list_words + 3u) & ~3u;
     } else {
@@ -244,7 +263,7 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
-    const EncodePlan pl = plan_encode(P, device_sms(dev));
+    const EncodePlan pl = plan_encode(P, device_sms(dev), (norm_kind & NUQ_TEST_NORMS) == 0);
     P.grid = pl.want_grid;
     Workspace* ws = nullptr;
     nuq_status st = get_workspace(stream, pl.state_bytes + pl.norms_bytes, &ws, &dev);
@@ -261,7 +280,7 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
     if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
-    const EncodePlan pl = plan_encode(P, device_sms(dev));
+    const EncodePlan pl = plan_encode(P, device_sms(dev), (norm_kind & NUQ_TEST_NORMS) == 0);
     if (pl.state_bytes + pl.norms_bytes > kStaticScratchBytes) return NUQ_ERR_CAPACITY;   // vector too long for the array
     P.grid = pl.want_grid;
     auto it = g_static_ws.find(dev);

@@ -15,7 +15,7 @@ constexpr uint32_t kMaxK = 64;
 
 constexpr int kEncThreads = 256;          // 8 warps share a tile, 1024 elements each
 constexpr int kEncWarps = kEncThreads / 32;
-constexpr int kEncMinBlocks = 3;          // resident CTAs per SM the encoder is compiled for
+constexpr int kEncMinBlocks = 4;          // resident CTAs per SM the encoder is compiled for
 constexpr uint32_t kEncChunk = 256;       // elements a warp quantizes before it generates their tokens
 
 enum : uint32_t { kNormL2 = 0, kNormLinf = 1 };
