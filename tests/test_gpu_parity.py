@@ -175,3 +175,25 @@ def test_degenerate_buckets():
         acc = gpu_decode([got], d, bucket, 4)
         assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([want], d, bucket, 4)[1].view(np.uint32))
         assert not acc[:4096].any()
+
+
+@pytest.mark.parametrize("d,bucket,s", [(40000, 256, 4), (70000, 1024, 5), (50000, 4096, 6), (33000, 256, 2),
+                                        (100000, 8192, 4)])
+def test_dense_inputs_stay_inside_the_staging_buffers(d, bucket, s):
+    """Vectors whose coordinates all have r = 2^-s (every coordinate becomes a token) or are as
+    dense as the norm allows: the encoder sizes its shared-memory staging by the sparsity bound of
+    the paper (at most 4^s coordinates of a bucket above the lowest level, Lemma 10), so the
+    free-running path must still equal the oracle here."""
+    rng = np.random.default_rng(d + s)
+    flat = np.where(rng.random(d) < 0.5, -1.0, 1.0).astype(np.float32)         # r = 1/sqrt(bucket) everywhere
+    spiky = flat.copy()
+    spiky[:: max(1, bucket // (4 ** s))] *= 3.0                                # about 4^s larger coordinates per bucket
+    noisy = (rng.standard_normal(d) * 1.0).astype(np.float32)
+    for g in (flat, spiky, noisy):
+        got, bits = gpu_encode(g, bucket, s, 0, seed=3, offset=1)
+        nbad, rel = compare_symbols(g, bucket, s, 0, 3, 1, got)
+        if nbad == 0 and rel == 0.0:
+            want, want_bits = O.encode(g, bucket, s, 0, 3, 1)
+            assert bits == want_bits and np.array_equal(got, want)
+        acc = gpu_decode([got], d, bucket, s)
+        assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([got], d, bucket, s)[1].view(np.uint32))
