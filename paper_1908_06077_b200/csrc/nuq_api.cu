@@ -165,7 +165,7 @@ using namespace nuq;
 
 // What one encode call needs from its workspace and from shared memory.
 struct EncodePlan {
-    size_t state_bytes;      // control block + one look-back word per tile
+    size_t state_bytes;      // control block + one look-back word per tile and per group of 32 tiles
     size_t norms_bytes;      // bucket norms for buckets wider than a tile
     uint32_t want_grid;      // CTAs that give every SM its full share
 };
@@ -173,7 +173,7 @@ struct EncodePlan {
 static EncodePlan plan_encode(EncodeParams& P, int sms, bool norms_are_ours) {
     const Geometry& G = P.geo;
     EncodePlan pl;
-    pl.state_bytes = sizeof(Workspace) + 8 * G.ntiles;
+    pl.state_bytes = sizeof(Workspace) + 8 * (G.ntiles + (G.ntiles + 31) / 32);
     pl.norms_bytes = G.bucket > kBLK ? 4 * G.nb : 0;
     P.stage_words = (stage_words_for(G, norms_are_ours) + 3u) & ~3u;
     if (G.mode == kModeErc) {

@@ -43,7 +43,7 @@ struct Workspace {
     uint64_t total_words;   // payload words of the whole call
     uint64_t dec_ticket;    // decoder: next tile to hand out (cleared before each decode launch)
     uint64_t reserved[1];
-    // followed by: uint64_t tile_state[ntiles], then float norms[nb] for wide buckets
+    // followed by: uint64_t tile_state[ntiles], group_state[ceil(ntiles / 32)], then float norms[nb] for wide buckets
 };
 constexpr size_t kWorkspaceClearFrom = 8;
 

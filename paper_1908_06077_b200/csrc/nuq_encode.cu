@@ -125,81 +125,103 @@ __device__ __forceinline__ void st_volatile_u64(uint64_t* p, uint64_t v) {
     *reinterpret_cast<volatile uint64_t*>(p) = v;
 }
 
-// Decoupled look-back over tile payload sizes, run by one warp.  Returns the
+// Two-level decoupled look-back over tile payload sizes, run by one warp.  Returns the
 // exclusive prefix (words) of `tile`, or sets *failed.  Every wait is bounded.
 //
-// All CTAs of a wave reach this point at about the same time, so a tile usually finds
-// its ~450 running predecessors in the "aggregate" state and has to sum all of them.
-// A step therefore looks at 256 predecessors at once (8 independent loads per lane):
-// the walk costs a couple of L2 round trips instead of one per 32 tiles.
-constexpr int kLookPerLane = 8;
-// The caller has already stored kTileAggregate | aggregate (kTilePrefix for tile 0) in state[tile].
-__device__ uint64_t tile_lookback(Workspace* ws, uint64_t* state, uint64_t tile, uint64_t aggregate, bool* failed) {
+// As many tiles as there are resident CTAs (several hundred) are under way at any time and
+// none of them knows its place yet, so a walk over single tiles would have to sum all of
+// them.  Sizes are therefore also accumulated per group of 32 consecutive tiles:
+//   tile_state[t]   kTileAggregate | words          once tile t has been encoded
+//   group_state[g]  count << 48 | words so far      while tiles of the group announce themselves
+//                   kTilePrefix | words before the end of the group, written by whoever places
+//                   the group's last tile
+// A tile sums the sizes of the tiles before it in its own group (one load per lane), then
+// walks back over whole groups, 64 per step, to the nearest one that knows its prefix.
+constexpr uint32_t kGroupTiles = 32;
+constexpr uint32_t kGroupCountShift = 48;
+constexpr uint64_t kGroupSumMask = (1ull << kGroupCountShift) - 1;
+
+// The workers' side: tile `tile` takes `words` words.
+__device__ __forceinline__ void announce_tile(uint64_t* tile_state, uint64_t* group_state, uint64_t tile, uint32_t words) {
+    st_volatile_u64(tile_state + tile, kTileAggregate | words);
+    atomicAdd(reinterpret_cast<unsigned long long*>(group_state + tile / kGroupTiles),
+              (1ull << kGroupCountShift) | (unsigned long long)words);
+}
+
+// One more poll of a look-back wait; false when the patience is used up (tens of ms).
+__device__ __forceinline__ bool lookback_backoff(Workspace* ws, uint32_t& polls) {
+    if (++polls > (1u << 16)) {
+        if (lane_id() == 0) latch_status(ws, kErrTimeout);
+        return false;
+    }
+    __nanosleep(polls < 64 ? 250 : 1000);                   // a waiting warp should not eat issue slots
+    return true;
+}
+
+__device__ uint64_t tile_lookback(Workspace* ws, const uint64_t* tile_state, uint64_t* group_state, uint64_t tile,
+                                  uint64_t ntiles, uint32_t words, bool* failed) {
     const uint32_t lane = lane_id();
-    *failed = false;
-    if (tile == 0) return 0;                               // announced as a prefix by the caller
-    uint64_t exclusive = 0;
-    int64_t base = (int64_t)tile - 1;                      // nearest predecessor not yet accounted for
+    const uint64_t grp = tile / kGroupTiles;
+    const uint32_t r = (uint32_t)(tile % kGroupTiles);      // tiles of the group before this one
     uint32_t polls = 0;
+    uint64_t exclusive = 0;
+    *failed = true;
+    // ---- the tiles before this one in its own group ----
     for (;;) {
-        // lane l looks at predecessors base - 8 l, base - 8 l - 1, ..., nearest first
-        uint64_t v[kLookPerLane];
-#pragma unroll
-        for (int k = 0; k < kLookPerLane; ++k) {
-            const int64_t idx = base - (int64_t)(lane * kLookPerLane + k);
-            v[k] = idx >= 0 ? ld_volatile_u64(state + idx) : kTilePrefix;     // before tile 0: prefix 0
+        const uint64_t v = lane < r ? ld_volatile_u64(tile_state + grp * kGroupTiles + lane) : kTileAggregate;
+        const uint32_t missing = __ballot_sync(0xffffffffu, (v >> 62) != 1);
+        if (!missing) {
+            exclusive = __reduce_add_sync(0xffffffffu, (uint32_t)v);           // a tile has far fewer than 2^27 words
+            break;
         }
-        uint64_t sum = 0;
-        uint32_t stop = 0;                                  // 0 none, 1 not ready, 2 prefix found, 3 poisoned
-#pragma unroll
-        for (int k = 0; k < kLookPerLane; ++k) {
-            const uint32_t flag = (uint32_t)(v[k] >> 62);
-            if (stop == 0) {
-                if (flag == 0) stop = 1;
-                else if (flag == 3) stop = 3;
-                else {
-                    sum += v[k] & kTileValueMask;
-                    if (flag == 2) stop = 2;
-                }
+        // wait for the first missing one alone, then look at all of them again
+        const uint64_t* p = tile_state + grp * kGroupTiles + (__ffs(missing) - 1);
+        while ((ld_volatile_u64(p) >> 62) != 1)
+            if (!lookback_backoff(ws, polls)) return 0;
+    }
+    // ---- whole groups, nearest first: lane l looks at groups base - l and base - 32 - l ----
+    int64_t base = (int64_t)grp - 1;
+    while (base >= 0) {
+        const int64_t i0 = base - (int64_t)lane, i1 = i0 - 32;
+        const uint64_t v0 = i0 >= 0 ? ld_volatile_u64(group_state + i0) : kTilePrefix;    // before group 0: prefix 0
+        const uint64_t v1 = i1 >= 0 ? ld_volatile_u64(group_state + i1) : kTilePrefix;
+        const bool p0 = (v0 >> 62) == 2, p1 = (v1 >> 62) == 2;                    // knows its prefix
+        const bool n0 = !p0 && (v0 >> kGroupCountShift) != kGroupTiles;           // still collecting (earlier groups are full ones)
+        const bool n1 = !p1 && (v1 >> kGroupCountShift) != kGroupTiles;
+        const uint64_t pm = (uint64_t)__ballot_sync(0xffffffffu, p0) | ((uint64_t)__ballot_sync(0xffffffffu, p1) << 32);
+        const uint64_t nm = (uint64_t)__ballot_sync(0xffffffffu, n0) | ((uint64_t)__ballot_sync(0xffffffffu, n1) << 32);
+        const uint32_t first_p = pm ? (uint32_t)__ffsll((long long)pm) - 1u : 64u;
+        const uint32_t first_n = nm ? (uint32_t)__ffsll((long long)nm) - 1u : 64u;
+        if (first_n < first_p) {
+            // a group on the way is not complete yet: wait for it alone, then look at all of them again
+            const uint64_t* p = group_state + (base - (int64_t)first_n);
+            for (;;) {
+                const uint64_t v = ld_volatile_u64(p);
+                if ((v >> 62) == 2 || (v >> kGroupCountShift) == kGroupTiles) break;
+                if (!lookback_backoff(ws, polls)) return 0;
             }
-        }
-        const uint32_t stops = __ballot_sync(0xffffffffu, stop != 0);
-        const uint32_t first = stops ? (uint32_t)__ffs(stops) - 1u : 32u;      // lanes below it are all aggregates
-        const uint32_t how = __shfl_sync(0xffffffffu, stop, first & 31u);
-        uint64_t contrib = lane <= first ? sum : 0;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xffffffffu, contrib, o);
-        if (stops && how == 3) {                            // a predecessor gave up
-            if (lane == 0) st_volatile_u64(state + tile, kTilePoison);
-            *failed = true;
-            return 0;
-        }
-        if (stops && how == 1) {
-            // the states up to the first one that is not ready are final: take them, wait, look again
-            exclusive += contrib;
-            // how many states of lane `first` were taken before the unready one
-            uint32_t taken = kLookPerLane;
-#pragma unroll
-            for (int k = kLookPerLane - 1; k >= 0; --k)
-                if ((uint32_t)(v[k] >> 62) == 0) taken = (uint32_t)k;
-            taken = __shfl_sync(0xffffffffu, taken, first & 31u);
-            base -= (int64_t)(first * kLookPerLane + taken);
-            if (++polls > (1u << 16)) {                    // ~tens of ms: give up, never hang
-                if (lane == 0) {
-                    latch_status(ws, kErrTimeout);
-                    st_volatile_u64(state + tile, kTilePoison);
-                }
-                *failed = true;
-                return 0;
-            }
-            __nanosleep(polls < 16 ? 100 : 1000);          // a waiting warp should not eat issue slots
             continue;
         }
-        exclusive += contrib;
-        if (stops) break;                                   // how == 2: reached a tile that knows its prefix
-        base -= 32 * kLookPerLane;
+        uint64_t c = 0;
+        if (lane <= first_p) c += p0 ? v0 & kTileValueMask : v0 & kGroupSumMask;
+        if (lane + 32u <= first_p) c += p1 ? v1 & kTileValueMask : v1 & kGroupSumMask;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+        exclusive += c;
+        if (first_p < 64u) break;
+        base -= 64;
     }
-    if (lane == 0) st_volatile_u64(state + tile, kTilePrefix | (exclusive + aggregate));
+    // ---- whoever places the last tile of a group tells the later groups where it ends ----
+    if (r == kGroupTiles - 1u || tile == ntiles - 1) {
+        const uint64_t members = tile == ntiles - 1 ? r + 1u : kGroupTiles;
+        for (;;) {                                          // every member's size has been added (they were all seen above)
+            const uint64_t v = ld_volatile_u64(group_state + grp);
+            if ((v >> kGroupCountShift) == members) break;
+            if (!lookback_backoff(ws, polls)) return 0;
+        }
+        if (lane == 0) st_volatile_u64(group_state + grp, kTilePrefix | (exclusive + words));
+    }
+    *failed = false;
     return exclusive;
 }
 
@@ -269,6 +291,30 @@ constexpr uint32_t kWarpElems = kBLK / kEncWarps;   // 1024 elements of a tile p
 constexpr uint32_t kChunk = kEncChunk;              // elements quantized before their tokens are generated
 constexpr uint32_t kChunkRows = kChunk / 128;
 
+// Named CTA barriers.  The 8 worker warps meet at kBarWork; the writer warp (ERC mode) and the
+// workers hand the two staged tiles back and forth through kBarStaged + b (workers arrive, the
+// writer waits) and kBarFree + b (the writer arrives, workers wait).
+constexpr uint32_t kBarWork = 1, kBarStaged = 2, kBarFree = 4;
+constexpr uint32_t kEncAllThreads = kEncThreads + 32;      // ERC mode: workers + the writer warp
+template <uint32_t ID, uint32_t COUNT>
+__device__ __forceinline__ void bar_sync() {
+    asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
+}
+template <uint32_t ID, uint32_t COUNT>
+__device__ __forceinline__ void bar_arrive() {
+    __threadfence_block();
+    asm volatile("bar.arrive %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
+}
+// the pair of barriers of stage b (0 or 1); immediate barrier numbers, so that the kernel claims only those it uses
+template <uint32_t BASE>
+__device__ __forceinline__ void stage_sync(uint32_t b) {
+    if (b) bar_sync<BASE + 1, kEncAllThreads>(); else bar_sync<BASE, kEncAllThreads>();
+}
+template <uint32_t BASE>
+__device__ __forceinline__ void stage_arrive(uint32_t b) {
+    if (b) bar_arrive<BASE + 1, kEncAllThreads>(); else bar_arrive<BASE, kEncAllThreads>();
+}
+
 // A tile whose records are staged in shared memory and whose place in the stream is not
 // yet known.
 struct Pending {
@@ -277,16 +323,23 @@ struct Pending {
     uint32_t blk_wordoff[32];                              // word offset of block bi within the tile
 };
 
-// Bookkeeping when a tile has been written: counters, and the container header by whichever
-// tile finishes last.  One thread.
+// What a CTA has written so far (shared memory; updated by one thread at a time, CTA barriers in between).
+struct CtaTotals {
+    uint64_t nnz, code_bits;
+    uint32_t tiles, stop;                                  // stop: iterations the workers ran (set when they leave)
+};
+
+// Bookkeeping of a CTA that has written all its tiles: counters, and the container header by
+// whichever CTA finishes last.  One thread, after a CTA barrier behind the last write.
 template <uint32_t MODE>
-__device__ void finish_tile(const EncodeParams& P, uint32_t nnz, uint32_t code_bits) {
+__device__ void finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, uint64_t code_bits) {
     const Geometry& G = P.geo;
+    if (tiles == 0) return;
     if (nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)nnz);
     if (code_bits) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)code_bits);
     __threadfence();
-    const unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), 1ull);
-    if (prev != G.ntiles - 1) return;
+    const unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), (unsigned long long)tiles);
+    if (prev + tiles != G.ntiles) return;
     __threadfence();
     uint64_t code_total, words;
     const uint64_t nnz_total = ld_volatile_u64(&P.ws->nnz);
@@ -315,13 +368,13 @@ __device__ void finish_tile(const EncodeParams& P, uint32_t nnz, uint32_t code_b
 
 // One warp: find the place of a staged tile (its predecessors announced their sizes an
 // iteration ago, so the walk rarely waits), copy the image to the stream, clear the stage.
-__device__ void flush_pending(const EncodeParams& P, Pending& pd, uint32_t* stg, uint64_t* tile_state, uint64_t* table,
-                              uint32_t* payload, uint32_t lane) {
+__device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot, uint32_t* stg, const uint64_t* tile_state,
+                              uint64_t* group_state, uint64_t* table, uint32_t* payload, uint32_t lane) {
     const Geometry& G = P.geo;
     const uint64_t tile = pd.tile;
     const uint32_t words = pd.words;
     bool failed;
-    const uint64_t off = tile_lookback(P.ws, tile_state, tile, words, &failed);
+    const uint64_t off = tile_lookback(P.ws, tile_state, group_state, tile, G.ntiles, words, &failed);
     for (uint32_t i = lane; i < words; i += 32) {
         if (!failed) payload[off + i] = stg[i];
         stg[i] = 0;
@@ -337,14 +390,15 @@ __device__ void flush_pending(const EncodeParams& P, Pending& pd, uint32_t* stg,
     __syncwarp();
     if (lane == 0) {
         pd.valid = 0;
-        finish_tile<kModeErc>(P, pd.nnz, pd.code_bits);
+        tot.tiles += 1;
+        tot.nnz += pd.nnz;
+        tot.code_bits += pd.code_bits;
     }
     __syncwarp();
 }
 
-
 template <uint32_t LEVELSET, uint32_t MODE>
-__global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(const __grid_constant__ EncodeParams P) {
+__global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(const __grid_constant__ EncodeParams P) {
     extern __shared__ __align__(128) uint32_t smem[];
     __shared__ __align__(8) uint64_t s_bar;                // completes when the tile's bytes have landed
     __shared__ uint32_t s_lut[256];                        // ERC(N), N = 1..256: code | len << 16
@@ -357,6 +411,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
     __shared__ unsigned long long s_tile[2];
     __shared__ uint32_t s_abort, s_nnz;
     __shared__ Pending s_pend[2];                          // ERC: the two staged tiles (current, previous)
+    __shared__ CtaTotals s_tot;
 
     using S = Sym<LEVELSET>;
     const Geometry& G = P.geo;
@@ -368,6 +423,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
     uint32_t* tokens = wmem + P.window_words;               // kChunk entries: position | field << 10 (uniform levels)
     uint16_t* tokens16 = reinterpret_cast<uint16_t*>(tokens);   //                position | field << 8  (exponential levels)
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
+    uint64_t* group_state = tile_state + G.ntiles;
     uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
     uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
     const float top = __uint_as_float((127u + G.s) << 23);
@@ -397,9 +453,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
         }
     };
     // thread 0: take a ticket ...
-    auto take_ticket = [&](uint32_t slot) {
-        s_tile[slot] = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
-    };
+    auto take_ticket = [&]() { return atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull); };
     // ... and start the copy of that tile into `data` once nobody reads the previous one
     auto start_copy = [&](uint32_t slot) {
         const uint64_t t = s_tile[slot];
@@ -412,7 +466,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
         }
     };
 
-    {
+    if (tid < 256u) {
         const uint32_t e = c_erc_lut[tid];
         s_lut[tid] = e;
         const uint32_t idx = tid & 0x7Fu;                   // field = sign << 7 | index: sign bit, then ERC(index)
@@ -423,24 +477,43 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
         }
         s_lut_signed[tid] = v;
     }
-    for (uint32_t i = tid; i < (MODE == kModeErc ? 2u : 1u) * P.stage_words; i += kEncThreads) stage[i] = 0;
-    for (uint32_t i = lane; i < P.window_words; i += 32) window[i] = 0;
+    for (uint32_t i = tid; i < (MODE == kModeErc ? 2u : 1u) * P.stage_words; i += blockDim.x) stage[i] = 0;
+    if (warp < (uint32_t)kEncWarps)
+        for (uint32_t i = lane; i < P.window_words; i += 32) window[i] = 0;
     if (tid == 0) {
         mbar_init(&s_bar, 1);
         s_abort = 0;
         s_nnz = 0;
         s_pend[0].valid = 0;
         s_pend[1].valid = 0;
+        s_tot.nnz = 0;
+        s_tot.code_bits = 0;
+        s_tot.tiles = 0;
+        s_tot.stop = 0xFFFFFFFFu;
     }
     __syncthreads();
     if (tid == 0) {
-        take_ticket(0);
+        s_tile[0] = take_ticket();
         start_copy(0);
     }
     __syncthreads();
 
+    const bool writer = MODE == kModeErc && warp == (uint32_t)kEncWarps;
+    if (writer) {
+        // ---- the writer warp: finds the place of every staged tile (look-back), copies it to the
+        // stream and hands the stage back; the workers never wait for it unless it falls two tiles behind
+        for (uint32_t k = 0;; ++k) {
+            stage_sync<kBarStaged>(k & 1u);                    // tile k of this CTA is staged
+            if (k >= *reinterpret_cast<volatile uint32_t*>(&s_tot.stop)) break;
+            flush_pending(P, s_pend[k & 1u], s_tot, stage + (k & 1u) * P.stage_words, tile_state, group_state, table,
+                          payload, lane);
+            stage_arrive<kBarFree>(k & 1u);
+        }
+    }
+
     uint32_t parity = 0;
-    for (uint32_t it = 0;; ++it) {
+    uint32_t it = 0;
+    for (; !writer; ++it) {                                 // the 8 worker warps
         const uint64_t tile = s_tile[it & 1u];
         if (tile >= G.ntiles) break;
 
@@ -477,7 +550,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             if (tile_len < kBLK) {
                 for (uint32_t i = bulk_elems + tid; i < kBLK; i += kEncThreads)
                     data[i] = i < tile_len ? __ldg(P.g + elem0 + i) : 0.0f;
-                __syncthreads();
+                bar_sync<kBarWork, kEncThreads>();
             }
         }
         const float4* rows = reinterpret_cast<const float4*>(data + wbase) + lane;   // row j at rows[32 * j]
@@ -519,8 +592,11 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 }
             }
         }
-        __syncthreads();                                    // B1: partials visible
-        if (tid == 0) take_ticket((it + 1u) & 1u);          // visible to all after the next barrier
+        bar_sync<kBarWork, kEncThreads>();                    // B1: partials visible
+        // the next ticket is asked for now and stored just before the next barrier: the round trip
+        // of the atomic is over by then
+        unsigned long long next_ticket = 0;
+        if (tid == 0) next_ticket = take_ticket();
 
         // every warp derives the norms of the buckets its own sub-blocks belong to (same
         // reduction tree in every warp, so all agree bit for bit)
@@ -722,7 +798,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             for (int o = 16; o > 0; o >>= 1) my_nnz += __shfl_xor_sync(0xffffffffu, my_nnz, o);
             if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
         }
-        __syncthreads();                                    // B2: the tile's data is no longer read; lengths visible
+        if (tid == 0) s_tile[(it + 1u) & 1u] = next_ticket;
+        bar_sync<kBarWork, kEncThreads>();                    // B2: the tile's data is no longer read; lengths visible
         if (tid == 0) start_copy((it + 1u) & 1u);           // the next tile's bytes arrive while this one is packed
 
         // ---- layout of the tile's records ---------------------------------------------
@@ -757,6 +834,10 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             const uint32_t my_bitoff = 32u * (blk_off + head_words) + (excl - excl0);   // where sub-block `lane` goes
             const uint32_t tile_words = __shfl_sync(0xffffffffu, wincl, 31);
             const uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
+            // announce the tile's size to its successors at once; the writer warp looks up its place
+            if (tid == 0) announce_tile(tile_state, group_state, tile, tile_words);
+            // this stage held the tile of two iterations ago: the writer must be done with it
+            if (it >= 2u) stage_sync<kBarFree>(it & 1u);
             // header words of the blocks: norm, then the u16 lengths two per word.  Lanes 4w .. 4w+3
             // of warp w stand for the warp's own sub-blocks, whose norms it holds.
             if ((lane >> 2) == warp && sb < nsb_tile) {
@@ -767,12 +848,9 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 atomicOr(stg + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
             }
             if (warp == 0) {
-                // announce the tile's size to its successors now; its own place is looked up one
-                // iteration later, when the predecessors have long announced theirs
                 Pending& pd = s_pend[it & 1u];
                 pd.blk_wordoff[lane] = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
                 if (lane == 0) {
-                    st_volatile_u64(tile_state + tile, (tile == 0 ? kTilePrefix : kTileAggregate) | tile_words);
                     pd.tile = tile;
                     pd.words = tile_words;
                     pd.nblk = nblk_tile;
@@ -808,11 +886,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
             }
             __syncwarp();
             for (uint32_t i = lane; i < (bits + 31u) / 32u + 2u; i += 32) window[i] = 0;   // ready for the next tile
-
-            // ---- one warp (they take turns) writes out the tile staged one iteration ago ----
-            if (warp == (it & 7u) && s_pend[(it & 1u) ^ 1u].valid)
-                flush_pending(P, s_pend[(it & 1u) ^ 1u], stage + ((it & 1u) ^ 1u) * P.stage_words, tile_state, table,
-                              payload, lane);
+            stage_arrive<kBarStaged>(it & 1u);     // the writer may take the tile
         } else {
             uint64_t tile_off;
             uint32_t tile_words;
@@ -831,28 +905,29 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_kernel(cons
                 tile_words = (tile_len * G.width + 31u) / 32u;
                 if (bib == 0 && tid == 0) payload[bucket_idx * G.rec_words] = __float_as_uint(norm_q[0]);
             }
-            __syncthreads();                                // the staged fields are complete
+            bar_sync<kBarWork, kEncThreads>();                // the staged fields are complete
             for (uint32_t i = tid; i < tile_words; i += kEncThreads) {
                 payload[tile_off + i] = stage[i];
                 stage[i] = 0;
             }
             if (tid == 0) {
-                const uint32_t nnz = s_nnz;
+                s_tot.nnz += s_nnz;
+                s_tot.tiles += 1;
                 s_nnz = 0;
-                finish_tile<kModeFixed>(P, nnz, 0);
             }
         }
     }
 
-    // ---- the tile staged in the last iteration is still pending ----
-    if (MODE == kModeErc) {
-        __syncthreads();
-        if (warp == 0) {
-            for (uint32_t b = 0; b < 2; ++b)
-                if (s_pend[b].valid)
-                    flush_pending(P, s_pend[b], stage + b * P.stage_words, tile_state, table, payload, lane);
-        }
+    if (MODE == kModeErc && !writer) {
+        // ---- the workers ran `it` iterations: wait until the writer has written the last two tiles,
+        // telling it in between that no further one comes ----
+        if (it >= 2u) stage_sync<kBarFree>(it & 1u);
+        if (tid == 0) s_tot.stop = it;
+        stage_arrive<kBarStaged>(it & 1u);
+        if (it >= 1u) stage_sync<kBarFree>((it + 1u) & 1u);
     }
+    __syncthreads();                                        // every write of this CTA lies behind this barrier
+    if (tid == 0) finish_cta<MODE>(P, s_tot.tiles, s_tot.nnz, s_tot.code_bits);
 }
 
 // ---------------------------------------------------------------------------
@@ -927,7 +1002,7 @@ static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
         attr_set = true;
     }
     if (smem > 112 * 1024 || P.grid == 0) return cudaErrorInvalidValue;
-    encode_kernel<L, M><<<P.grid, kEncThreads, smem, stream>>>(P);
+    encode_kernel<L, M><<<P.grid, M == kModeErc ? kEncAllThreads : (uint32_t)kEncThreads, smem, stream>>>(P);
     return cudaGetLastError();
 }
 
