@@ -250,15 +250,16 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src_gmem, 
 // Waits until the phase with the given parity has completed.  Bounded: false after ~tens of ms.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_u32(bar);
-    for (uint32_t polls = 0; polls < (1u << 20); ++polls) {
+    // the hardware parks the thread for up to the hinted time (ns), so a wait costs a handful of
+    // instructions; the number of tries bounds the wait (a fraction of a second at most)
+    for (uint32_t polls = 0; polls < (1u << 17); ++polls) {
         uint32_t done;
         asm volatile(
-            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+            "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(2000u)
             : "memory");
         if (done) return true;
-        if (polls > 64) __nanosleep(100);
     }
     return false;
 }
