@@ -32,7 +32,10 @@
 namespace nuq {
 
 constexpr uint32_t kLutBits = 12;                       // prefix bits resolved by the ERC^-1 table
-constexpr uint32_t kListEntries = 1536;                 // 16-bit list entries per warp (3 CTAs of 8 warps per SM)
+constexpr uint32_t kWarpWords = 1152;                   // shared-memory words a warp has for lists and staged tokens
+constexpr uint32_t kStageWords = 12;                    // token words per chain copied to shared memory before the walk
+constexpr uint32_t kStagedListWords = kWarpWords - 32u * kStageWords;   // what is left for the lists then (48 entries per chain)
+constexpr uint32_t kDecMaxWarps = 12;                   // warps per CTA (they share the table and the stream heads only)
 constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
 // One Elias-recursive integer from the top of a 64-bit MSB-first window (Algorithm 2,
@@ -56,12 +59,13 @@ __device__ __forceinline__ bool erc_read(uint64_t& win, uint32_t& used, uint32_t
     return false;
 }
 
-// 64 bits of the MSB-first bit string `words` starting at bit `cur`; word indices are clamped to `last`.
-__device__ __forceinline__ uint64_t window64(const uint32_t* __restrict__ words, uint32_t cur, uint32_t last) {
+// 64 bits of the MSB-first bit string `words` (word i at words[i * stride], global or shared memory) starting at
+// bit `cur`; word indices are clamped to `last`.
+__device__ __forceinline__ uint64_t window64(const uint32_t* words, uint32_t stride, uint32_t cur, uint32_t last) {
     uint32_t wi = cur >> 5, sh = cur & 31u;
-    uint32_t w0 = __ldg(words + min(wi, last));
-    uint32_t w1 = __ldg(words + min(wi + 1u, last));
-    uint32_t w2 = __ldg(words + min(wi + 2u, last));
+    uint32_t w0 = words[min(wi, last) * stride];
+    uint32_t w1 = words[min(wi + 1u, last) * stride];
+    uint32_t w2 = words[min(wi + 2u, last) * stride];
     uint64_t win = ((uint64_t)w0 << 32 | w1) << sh;
     if (sh) win |= (uint64_t)w2 >> (32u - sh);
     return win;
@@ -164,17 +168,25 @@ __device__ bool describe_chain(const Geometry& G, const TileGeo& T, const Stream
     return true;
 }
 
-__global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_constant__ DecodeParams P) {
+// shared memory: the ERC^-1 table, the stream heads, then per warp the running sums of its S sub-blocks
+// and kWarpWords for lists and staged tokens
+__host__ __device__ inline size_t decode_warp_offset(uint32_t K) {
+    return (2u * (1u << kLutBits) + (size_t)K * sizeof(StreamHead) + 15u) & ~(size_t)15u;
+}
+__host__ __device__ inline size_t decode_warp_bytes(uint32_t group) {
+    return 4u * ((32u / group) * kSB + kWarpWords);
+}
+
+__global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
     const Geometry& G = P.geo;
-    const uint32_t NG = P.group;                            // streams per group = warps per CTA (1, 2, 4 or 8)
+    const uint32_t NG = P.group;                            // streams decoded side by side (1, 2, 4 or 8)
     const uint32_t S = 32u / NG;                            // sub-blocks per warp
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    float* acc = reinterpret_cast<float*>(dsm);                                   // kBLK running sums
-    uint16_t* lut = reinterpret_cast<uint16_t*>(dsm + 4u * kBLK);                 // ERC^-1 of 12-bit prefixes
-    StreamHead* heads = reinterpret_cast<StreamHead*>(dsm + 4u * kBLK + 2u * (1u << kLutBits));   // [kMaxK]
-    uint32_t* list = reinterpret_cast<uint32_t*>(heads + kMaxK) + warp * (kListEntries / 2u);
-    float* accw = acc + warp * S * kSB;                     // this warp's part of the tile
+    uint16_t* lut = reinterpret_cast<uint16_t*>(dsm);                             // ERC^-1 of 12-bit prefixes
+    StreamHead* heads = reinterpret_cast<StreamHead*>(dsm + 2u * (1u << kLutBits));   // [K]
+    float* accw = reinterpret_cast<float*>(dsm + decode_warp_offset(P.K) + warp * decode_warp_bytes(NG));   // S * 256 running sums
+    uint32_t* list = reinterpret_cast<uint32_t*>(accw + S * kSB);
 
     for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) lut[i] = (uint16_t)erc_prefix_entry(i);
     // ---- header validation against the call's arguments, once per stream ----
@@ -255,7 +267,6 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
             const uint32_t my_sn = my_sb < nsb_tile ? min(kSB, tile_len - my_sb * kSB) : 0u;   // elements of my sub-block
             bool wide = false;                              // index - 1 does not fit 7 bits (uniform levels, s = 8)
             for (uint32_t j = 0; j < gcount; ++j) wide = wide || (heads[g0 + j].ok && heads[g0 + j].nlev > 129u);
-            const uint32_t cap = (wide ? kListEntries / 2u : kListEntries) / 32u;   // list entries per chain
             const bool mine = lj < gcount;
             const StreamHead si = heads[g0 + (mine ? lj : 0)];
             Chain ch;                                       // each lane describes the chain it walks
@@ -271,9 +282,31 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
             // a chain of t tokens in 256 positions takes about t (2 log2(256 / t) + 4) bits: 48 tokens ~ 400 bits
             uint32_t guess = has_chain ? (ch.end - ch.cur) / 8u + 1u : 0u;
             guess = __reduce_max_sync(0xffffffffu, guess);
+            // Short chains (the usual case) are first copied to shared memory, a word per lane and step, with
+            // all loads in flight at once: the walk below is a chain of dependent reads, and from global
+            // memory every step of it would wait for the cache.  Long chains are walked in place.
+            const uint32_t nw = has_chain ? ((ch.end - 1u) >> 5) - (ch.cur >> 5) + 1u : 0u;     // words my chain touches
+            const bool staged = !wide && guess <= 2u * kStagedListWords / 32u &&
+                                __reduce_max_sync(0xffffffffu, nw) <= kStageWords;
+            const uint32_t cap = staged ? 2u * kStagedListWords / 32u : (wide ? kWarpWords : 2u * kWarpWords) / 32u;   // list entries per chain
+            const uint32_t* tokp = ch.tok;                  // word i of the chain's string at tokp[i * stride]
+            uint32_t stride = 1, last = ch.last, cur0 = ch.cur, end = ch.end;
+            if (staged) {
+                uint32_t* st = list + kStagedListWords + lane;
+                const uint32_t* src = ch.tok + (ch.cur >> 5);
+#pragma unroll
+                for (uint32_t i = 0; i < kStageWords; ++i)
+                    if (i < nw) st[i * 32u] = __ldg(src + i);
+                tokp = st;
+                stride = 32;
+                last = nw ? nw - 1u : 0u;
+                cur0 = ch.cur & 31u;
+                end = ch.end - (ch.cur & ~31u);
+            }
+            __syncwarp();
             uint32_t step = guess <= cap ? kSB : cap;
             bool alive = has_chain, bad = false, fixed_done = false;
-            uint32_t cur = ch.cur, pos = 0, max_sym = 0;
+            uint32_t cur = cur0, pos = 0, max_sym = 0;
             uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
             uint32_t* slot32 = list + lane;
             for (uint32_t limit = step;; limit += step) {
@@ -283,8 +316,8 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 // data and commits nothing): no divergent branch except the rare long-code path.
                 while (__any_sync(0xffffffffu, running)) {
                     const uint32_t wi = cur >> 5;
-                    const uint32_t x0 = __ldg(ch.tok + min(wi, ch.last));
-                    const uint32_t x1 = __ldg(ch.tok + min(wi + 1u, ch.last));
+                    const uint32_t x0 = tokp[min(wi, last) * stride];
+                    const uint32_t x1 = tokp[min(wi + 1u, last) * stride];
                     const uint32_t win = __funnelshift_l(x1, x0, cur);                      // 32 bits from the cursor
                     const uint32_t e1 = lut[win >> (32u - kLutBits)];
                     const uint32_t t = win << (e1 >> 8);                                    // the sign bit is on top
@@ -294,7 +327,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                     bool good = e1 != 0 && e2 != 0;
                     if (__any_sync(0xffffffffu, running && !good)) {
                         if (running && !good) {             // a code longer than 12 bits: Algorithm 2 as a loop
-                            uint64_t win64 = window64(ch.tok, cur, ch.last);
+                            uint64_t win64 = window64(tokp, stride, cur, last);
                             used = 0;
                             good = erc_read(win64, used, gap);
                             negative = (uint32_t)(win64 >> 63);
@@ -323,7 +356,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                         pos = npos;
                         cur += used;
                         ++n;
-                        alive = cur < ch.end;
+                        alive = cur < end;
                     }
                     running = commit && alive;
                 }
@@ -338,7 +371,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                     limit = 0;
                     alive = has_chain;
                     bad = false;
-                    cur = ch.cur;
+                    cur = cur0;
                     pos = 0;
                     max_sym = 0;
                     continue;
@@ -417,7 +450,7 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
                 if (!__any_sync(0xffffffffu, alive)) break;
             }
             // a well-formed chain ends exactly at its declared length, inside its sub-block, with known indices
-            if (has_chain && !bad) bad = cur != ch.end || pos > my_sn || max_sym >= si.nlev;
+            if (has_chain && !bad) bad = cur != end || pos > my_sn || max_sym >= si.nlev;
             if (__any_sync(0xffffffffu, bad) && lane == 0) latch_status(P.ws, kErrBadStream);
         }
 
@@ -439,26 +472,38 @@ __global__ void __launch_bounds__(32 * kMaxGroup) decode_kernel(const __grid_con
     }
 }
 
-static size_t decode_smem_bytes(uint32_t group) {
-    return 4u * kBLK + 2u * (1u << kLutBits) + kMaxK * sizeof(StreamHead) +
-           (size_t)group * kListEntries * 2u;
+static size_t decode_smem_bytes(uint32_t group, uint32_t K, uint32_t warps) {
+    return decode_warp_offset(K) + (size_t)warps * decode_warp_bytes(group);
 }
 
 cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
+    constexpr size_t kSmemPerSm = 227u * 1024u, kSmemMaxCta = 227u * 1024u;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMaxCta);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    const size_t smem = decode_smem_bytes(P.group);
-    uint64_t resident = 228u * 1024u / (smem + 1024u);                      // CTAs per SM by shared memory
+    // warps per CTA: up to 12, two such CTAs per SM when the warps' sums are small enough (8 streams side by
+    // side: 8.5 KB per warp), else as many warps as one CTA per SM can hold
+    const size_t fixed = decode_warp_offset(P.K) + 1024u, per_warp = decode_warp_bytes(P.group);
+    uint32_t warps = kDecMaxWarps;
+    while (warps > 1 && 2u * (fixed + warps * per_warp) > kSmemPerSm) --warps;
+    if (warps < 6) {                                        // one CTA per SM with all the warps that fit
+        warps = kDecMaxWarps;
+        while (warps > 1 && fixed + warps * per_warp > kSmemPerSm) --warps;
+    }
+    const size_t smem = decode_smem_bytes(P.group, P.K, warps);
+    if (smem > kSmemMaxCta) return cudaErrorInvalidValue;
+    uint64_t resident = kSmemPerSm / (smem + 1024u);                        // CTAs per SM by shared memory
     if (resident < 1) resident = 1;
-    if (resident * P.group > 48) resident = 48 / P.group;                   // and by warps worth keeping resident
+    if (resident * warps > 48) resident = 48 / warps;                       // and by warps worth keeping resident
     if (cudaMemsetAsync(&P.ws->dec_ticket, 0, sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;
+    const uint64_t units = P.geo.ntiles * P.group;                          // warp-sized units of work
     const uint64_t cap = (uint64_t)sms * resident;
-    const uint64_t grid = P.geo.ntiles < cap ? P.geo.ntiles : cap;
-    decode_kernel<<<(unsigned)grid, 32u * P.group, smem, stream>>>(P);
+    const uint64_t want = (units + warps - 1) / warps;
+    const uint64_t grid = want < cap ? want : cap;
+    decode_kernel<<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
     return cudaGetLastError();
 }
 
