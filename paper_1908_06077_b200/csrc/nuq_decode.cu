@@ -35,7 +35,7 @@ constexpr uint32_t kLutBits = 12;                       // prefix bits resolved 
 constexpr uint32_t kWarpWords = 1152;                   // shared-memory words a warp has for lists and staged tokens
 constexpr uint32_t kStageWords = 12;                    // token words per chain copied to shared memory before the walk
 constexpr uint32_t kStagedListWords = kWarpWords - 32u * kStageWords;   // what is left for the lists then (48 entries per chain)
-constexpr uint32_t kDecMaxWarps = 12;                   // warps per CTA (they share the table and the stream heads only)
+constexpr uint32_t kDecMaxWarps = 25;                   // warps per CTA = per SM (they share the table and the stream heads only)
 constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
 // One Elias-recursive integer from the top of a 64-bit MSB-first window (Algorithm 2,
@@ -484,25 +484,33 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    // warps per CTA: up to 12, two such CTAs per SM when the warps' sums are small enough (8 streams side by
-    // side: 8.5 KB per warp), else as many warps as one CTA per SM can hold
+    // One CTA per SM with as many warps as its shared memory holds (25 at most: 80 registers per thread).
+    // The warps take equal units of work by ticket, so the kernel lasts ceil(units / warps in flight)
+    // rounds, and a round takes about as long as there are warps on the SM (the kernel is bound by
+    // instruction issue): among the five largest warp counts take the one with the least rounds * warps.
     const size_t fixed = decode_warp_offset(P.K) + 1024u, per_warp = decode_warp_bytes(P.group);
-    uint32_t warps = kDecMaxWarps;
-    while (warps > 1 && 2u * (fixed + warps * per_warp) > kSmemPerSm) --warps;
-    if (warps < 6) {                                        // one CTA per SM with all the warps that fit
-        warps = kDecMaxWarps;
-        while (warps > 1 && fixed + warps * per_warp > kSmemPerSm) --warps;
+    uint32_t wmax = kDecMaxWarps;
+    while (wmax > 1 && fixed + wmax * per_warp > kSmemPerSm) --wmax;
+    const uint64_t units = P.geo.ntiles * P.group;                          // warp-sized units of work
+    uint32_t warps = wmax;
+    uint64_t best = ~0ull;
+    if (units <= (uint64_t)sms * wmax) {                                    // one round: spread it over all SMs
+        warps = (uint32_t)((units + sms - 1) / sms);
+        best = 0;
+    }
+    for (uint32_t w = wmax; best && w >= 1 && w + 4 >= wmax; --w) {
+        const uint64_t in_flight = (uint64_t)sms * w;
+        const uint64_t cost = ((units + in_flight - 1) / in_flight) * w;
+        if (cost < best) {
+            best = cost;
+            warps = w;
+        }
     }
     const size_t smem = decode_smem_bytes(P.group, P.K, warps);
     if (smem > kSmemMaxCta) return cudaErrorInvalidValue;
-    uint64_t resident = kSmemPerSm / (smem + 1024u);                        // CTAs per SM by shared memory
-    if (resident < 1) resident = 1;
-    if (resident * warps > 48) resident = 48 / warps;                       // and by warps worth keeping resident
     if (cudaMemsetAsync(&P.ws->dec_ticket, 0, sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;
-    const uint64_t units = P.geo.ntiles * P.group;                          // warp-sized units of work
-    const uint64_t cap = (uint64_t)sms * resident;
     const uint64_t want = (units + warps - 1) / warps;
-    const uint64_t grid = want < cap ? want : cap;
+    const uint64_t grid = want < (uint64_t)sms ? want : (uint64_t)sms;
     decode_kernel<<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
     return cudaGetLastError();
 }
