@@ -59,13 +59,14 @@ __device__ __forceinline__ bool erc_read(uint64_t& win, uint32_t& used, uint32_t
     return false;
 }
 
-// 64 bits of the MSB-first bit string `words` (word i at words[i * stride], global or shared memory) starting at
-// bit `cur`; word indices are clamped to `last`.
-__device__ __forceinline__ uint64_t window64(const uint32_t* words, uint32_t stride, uint32_t cur, uint32_t last) {
+// 64 bits of the MSB-first bit string whose word i is word(i), starting at bit `cur`; word indices are
+// clamped to `last`.
+template <class Fetch>
+__device__ __forceinline__ uint64_t window64(Fetch word, uint32_t cur, uint32_t last) {
     uint32_t wi = cur >> 5, sh = cur & 31u;
-    uint32_t w0 = words[min(wi, last) * stride];
-    uint32_t w1 = words[min(wi + 1u, last) * stride];
-    uint32_t w2 = words[min(wi + 2u, last) * stride];
+    uint32_t w0 = word(min(wi, last));
+    uint32_t w1 = word(min(wi + 1u, last));
+    uint32_t w2 = word(min(wi + 2u, last));
     uint64_t win = ((uint64_t)w0 << 32 | w1) << sh;
     if (sh) win |= (uint64_t)w2 >> (32u - sh);
     return win;
@@ -289,16 +290,13 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             const bool staged = !wide && guess <= 2u * kStagedListWords / 32u &&
                                 __reduce_max_sync(0xffffffffu, nw) <= kStageWords;
             const uint32_t cap = staged ? 2u * kStagedListWords / 32u : (wide ? kWarpWords : 2u * kWarpWords) / 32u;   // list entries per chain
-            const uint32_t* tokp = ch.tok;                  // word i of the chain's string at tokp[i * stride]
-            uint32_t stride = 1, last = ch.last, cur0 = ch.cur, end = ch.end;
+            uint32_t last = ch.last, cur0 = ch.cur, end = ch.end;
+            uint32_t* st = list + kStagedListWords + lane;   // word i of a staged chain at st[32 i]
             if (staged) {
-                uint32_t* st = list + kStagedListWords + lane;
                 const uint32_t* src = ch.tok + (ch.cur >> 5);
 #pragma unroll
                 for (uint32_t i = 0; i < kStageWords; ++i)
                     if (i < nw) st[i * 32u] = __ldg(src + i);
-                tokp = st;
-                stride = 32;
                 last = nw ? nw - 1u : 0u;
                 cur0 = ch.cur & 31u;
                 end = ch.end - (ch.cur & ~31u);
@@ -309,15 +307,17 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             uint32_t cur = cur0, pos = 0, max_sym = 0;
             uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
             uint32_t* slot32 = list + lane;
-            for (uint32_t limit = step;; limit += step) {
-                uint32_t n = 0;
-                bool full = false, running = alive;
+            uint32_t n = 0, limit = step;
+            bool full = false, running = false;
+            // One round of the walk; `word(i)` fetches word i of the lane's chain (two instances: from
+            // shared memory for staged chains, from global memory otherwise).
+            auto walk = [&](auto word) {
                 // Every lane executes every step (a lane that has stopped works on stale but in-bounds
                 // data and commits nothing): no divergent branch except the rare long-code path.
                 while (__any_sync(0xffffffffu, running)) {
                     const uint32_t wi = cur >> 5;
-                    const uint32_t x0 = tokp[min(wi, last) * stride];
-                    const uint32_t x1 = tokp[min(wi + 1u, last) * stride];
+                    const uint32_t x0 = word(min(wi, last));
+                    const uint32_t x1 = word(min(wi + 1u, last));
                     const uint32_t win = __funnelshift_l(x1, x0, cur);                      // 32 bits from the cursor
                     const uint32_t e1 = lut[win >> (32u - kLutBits)];
                     const uint32_t t = win << (e1 >> 8);                                    // the sign bit is on top
@@ -327,7 +327,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     bool good = e1 != 0 && e2 != 0;
                     if (__any_sync(0xffffffffu, running && !good)) {
                         if (running && !good) {             // a code longer than 12 bits: Algorithm 2 as a loop
-                            uint64_t win64 = window64(tokp, stride, cur, last);
+                            uint64_t win64 = window64(word, cur, last);
                             used = 0;
                             good = erc_read(win64, used, gap);
                             negative = (uint32_t)(win64 >> 63);
@@ -360,6 +360,13 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     }
                     running = commit && alive;
                 }
+            };
+            for (;; limit += step) {
+                n = 0;
+                full = false;
+                running = alive;
+                if (staged) walk([st](uint32_t i) { return st[32u * i]; });
+                else walk([&ch](uint32_t i) { return __ldg(ch.tok + i); });
                 if (__any_sync(0xffffffffu, full)) {
                     if (step == cap) {                      // cannot happen: at most `cap` positions per round
                         bad = true;
