@@ -10,6 +10,10 @@
 //   describe lane (j, q) reads, for stream j and sub-block q of the unit, the block
 //            offset, the norm and the sub-block token lengths, range-checks them and
 //            so knows where its chain of tokens starts and ends.
+//   stage    chains of at most 12 words (the usual case) are copied to shared memory, all
+//            loads in flight at once: the walk is a chain of dependent reads, which from
+//            global memory would wait for the cache at every step.  Longer chains are
+//            walked in place.
 //   decode   the lane walks that chain: ERC^-1 gap, sign bit, ERC^-1 level index, by
 //            table look-up on a 32-bit window (12-bit prefix table; longer codes take
 //            the loop of Algorithm 2).  All 32 chains of a warp advance in lock
@@ -20,12 +24,13 @@
 //            its terms in ascending stream order: the sum is bit-reproducible and
 //            equals ((0 + q_0) + q_1) + ... .
 //
-// Lists hold 48 entries per chain.  Sparse streams need one decode / add round per
-// unit; when a chain may have more tokens than that, the rounds advance through
-// the sub-block 48 positions at a time (a chain has at most 48 tokens there), and
-// since all terms of an element fall into the same round the order of its adds
-// is unchanged.  Streams in the fixed-width mode are added field by field in
-// their turn.  Nothing spins.
+// Lists hold 48 entries per staged chain (72 when nothing is staged).  Sparse streams
+// need one decode / add round per unit; when a chain may have more tokens than that,
+// the rounds advance through the sub-block that many positions at a time (a chain has
+// at most as many tokens there), and since all terms of an element fall into the same
+// round the order of its adds is unchanged.  Streams in the fixed-width mode are added
+// field by field in their turn.  One CTA per SM holds up to 25 such warps; they share
+// only the table and the validated stream headers.  Nothing spins.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 

@@ -2,8 +2,10 @@
 // quantization (Definition 1) and Elias-recursive token packing in one kernel
 // that reads the gradient from HBM exactly once.
 //
-// A persistent CTA of 8 warps takes tiles of up to 8192 consecutive elements
-// (whole buckets, or one 8192-element coding block of a wider bucket) by ticket.
+// A persistent CTA takes tiles of up to 8192 consecutive elements (whole buckets, or
+// one 8192-element coding block of a wider bucket) by ticket.  Eight worker warps
+// encode the tile; in the ERC mode a ninth warp, the writer, finds the tile's place
+// in the stream and copies it out, so the workers never wait for other CTAs.
 // The tile's bytes are brought into shared memory by one bulk asynchronous copy
 // (TMA, completion on an mbarrier); the copy of the next tile is started as soon
 // as the current tile has been quantized, so HBM latency hides behind the packing
@@ -16,14 +18,17 @@
 //      tokens, 32 per step, appended to the warp's own bit string;
 //   3. after a second barrier every warp runs the same small scan over the 32
 //      sub-block lengths, which gives the layout of the tile's records, and
-//      shifts its strings to their place in the staged tile; the tile's size is
-//      announced to the tiles behind it at once;
-//   4. one iteration later (two staged tiles exist), one warp looks up the tile's
-//      place in the stream (decoupled look-back over the sizes announced by its
-//      predecessors, bounded waits) and copies the staged tile there.  Looking
-//      the place up later matters: the predecessors, which started at the same
-//      time, have all announced their sizes by then, so nobody waits.
-// In the fixed-width mode the fields go straight to their known place.
+//      shifts its strings to their place in one of two staged tile images; the
+//      tile's size is announced to the tiles behind it at once;
+//   4. the writer warp, woken through a named barrier, sums the sizes announced
+//      by the tile's predecessors (two-level decoupled look-back: single tiles
+//      within a group of 32, whole groups before that; bounded waits), copies the
+//      staged image to its place, writes the block offsets and hands the stage
+//      back through a second named barrier.  The workers meet the writer again
+//      only two tiles later, when they need that stage.
+// In the fixed-width mode the fields go straight to their known place and there
+// is no writer warp.  Counters and the container header are written once per CTA,
+// the header by whichever CTA finishes last.
 //
 // The kernel is bound by instruction issue, not by HBM: the quantizer is branch
 // free and all per-symbol work runs on dense lists.
