@@ -286,7 +286,9 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             // round: a chain then has at most `cap` tokens per round, and every element still receives
             // its terms in ascending stream order because all of its terms fall into the same round.
             // a chain of t tokens in 256 positions takes about t (2 log2(256 / t) + 4) bits: 48 tokens ~ 400 bits
-            uint32_t guess = has_chain ? (ch.end - ch.cur) / 8u + 1u : 0u;
+            // (a token of a dense chain, gaps of 1 to 3, takes about 5 bits)
+            const uint32_t chain_bits = has_chain ? ch.end - ch.cur : 0u;
+            uint32_t guess = chain_bits <= 384u ? (chain_bits + 7u) / 8u : chain_bits / 5u;
             guess = __reduce_max_sync(0xffffffffu, guess);
             // Short chains (the usual case) are first copied to shared memory, a word per lane and step, with
             // all loads in flight at once: the walk below is a chain of dependent reads, and from global
@@ -307,12 +309,19 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                 end = ch.end - (ch.cur & ~31u);
             }
             __syncwarp();
-            uint32_t step = guess <= cap ? kSB : cap;
+            // positions per round: the whole sub-block when the longest chain should fit its list, else
+            // an even split into as many rounds as the guess asks for (at least `cap` positions, which
+            // can never overflow)
+            uint32_t step = kSB;
+            if (guess > cap) {
+                const uint32_t rounds = (guess + guess / 3u + cap - 1u) / cap;     // a third of slack: 32 chains must all fit
+                step = max(cap, (kSB + rounds - 1u) / rounds);
+            }
             bool alive = has_chain, bad = false, fixed_done = false;
             uint32_t cur = cur0, pos = 0, max_sym = 0;
             uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
             uint32_t* slot32 = list + lane;
-            uint32_t n = 0, limit = step;
+            uint32_t n = 0, limit = 0;
             bool full = false, running = false;
             // One round of the walk; `word(i)` fetches word i of the lane's chain (two instances: from
             // shared memory for staged chains, from global memory otherwise).
@@ -366,7 +375,11 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     running = commit && alive;
                 }
             };
-            for (;; limit += step) {
+            for (;;) {
+                const uint32_t done_pos = limit;            // positions below this have been added
+                const uint32_t cur_s = cur, pos_s = pos, max_sym_s = max_sym;
+                const bool alive_s = alive, bad_s = bad;
+                limit = done_pos + step;
                 n = 0;
                 full = false;
                 running = alive;
@@ -377,15 +390,15 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                         bad = true;
                         break;
                     }
-                    // the guess was too low (only possible in a one-round attempt): nothing has been
-                    // added yet, start over with the window that cannot overflow
+                    // the guess was too low: nothing of this round has been added yet, so take the round
+                    // again from where it started, with the window that cannot overflow
                     step = cap;
-                    limit = 0;
-                    alive = has_chain;
-                    bad = false;
-                    cur = cur0;
-                    pos = 0;
-                    max_sym = 0;
+                    limit = done_pos;
+                    alive = alive_s;
+                    bad = bad_s;
+                    cur = cur_s;
+                    pos = pos_s;
+                    max_sym = max_sym_s;
                     continue;
                 }
                 __syncwarp();
