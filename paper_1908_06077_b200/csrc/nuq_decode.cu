@@ -31,6 +31,8 @@
 // round the order of its adds is unchanged.  Streams in the fixed-width mode are added
 // field by field in their turn.  One CTA per SM holds up to 25 such warps; they share
 // only the table and the validated stream headers.  Nothing spins.
+#include <type_traits>
+
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 
@@ -325,7 +327,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             bool full = false, running = false;
             // One round of the walk; `word(i)` fetches word i of the lane's chain (two instances: from
             // shared memory for staged chains, from global memory otherwise).
-            auto walk = [&](auto word) {
+            auto walk = [&](auto word, auto wide_entries) {
                 // Every lane executes every step (a lane that has stopped works on stale but in-bounds
                 // data and commits nothing): no divergent branch except the rare long-code path.
                 while (__any_sync(0xffffffffu, running)) {
@@ -348,25 +350,23 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                             win64 <<= 1;
                             used += 1;
                             good = good && erc_read(win64, used, sym);
+                            if (!good) {                    // not a code at all: the chain is malformed
+                                bad = true;
+                                alive = false;
+                            }
                         }
                     }
                     // Range checks are made once per chain, after the walk (see below): a token of a
                     // malformed chain may be committed, but its position is masked to the sub-block
                     // when it is added, so nothing is written out of bounds.
                     const uint32_t npos = pos + gap;
-                    const bool inside = npos <= limit;      // else the token belongs to a later round
-                    const bool room = n < cap;
-                    const bool commit = running && good && inside && room;
-                    if (running && !good) {
-                        bad = true;
-                        alive = false;
-                    }
-                    full = full || (running && good && inside && !room);
+                    const bool commit = running && good && npos <= limit;   // beyond the limit: a later round's token
                     if (commit) {
                         max_sym = max(max_sym, sym);
                         const uint32_t e = ((npos - 1u) & 0xffu) | (negative << 8) | ((sym - 1u) << 9);
-                        if (wide) slot32[n * 32u] = e;
-                        else slot16[n * 32u] = (uint16_t)e;
+                        const uint32_t at = min(n, cap - 1u) * 32u;     // a list that runs over is noticed after the round
+                        if (decltype(wide_entries)::value) slot32[at] = e;
+                        else slot16[at] = (uint16_t)e;
                         pos = npos;
                         cur += used;
                         ++n;
@@ -383,8 +383,10 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                 n = 0;
                 full = false;
                 running = alive;
-                if (staged) walk([st](uint32_t i) { return st[32u * i]; });
-                else walk([&ch](uint32_t i) { return __ldg(ch.tok + i); });
+                if (staged) walk([st](uint32_t i) { return st[32u * i]; }, std::false_type());
+                else if (!wide) walk([&ch](uint32_t i) { return __ldg(ch.tok + i); }, std::false_type());
+                else walk([&ch](uint32_t i) { return __ldg(ch.tok + i); }, std::true_type());
+                full = n > cap;
                 if (__any_sync(0xffffffffu, full)) {
                     if (step == cap) {                      // cannot happen: at most `cap` positions per round
                         bad = true;
