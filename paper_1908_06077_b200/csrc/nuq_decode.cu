@@ -42,6 +42,7 @@ constexpr uint32_t kLutBits = 12;                       // prefix bits resolved 
 constexpr uint32_t kWarpWords = 1152;                   // shared-memory words a warp has for lists and staged tokens
 constexpr uint32_t kStageWords = 12;                    // token words per chain copied to shared memory before the walk
 constexpr uint32_t kStagedListWords = kWarpWords - 32u * kStageWords;   // what is left for the lists then (48 entries per chain)
+constexpr uint32_t kStageSoftBits = 32u * (kStageWords - 2u);   // a lane stops here when its chain goes on behind the staged words
 constexpr uint32_t kDecMaxWarps = 25;                   // warps per CTA = per SM (they share the table and the stream heads only)
 constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
@@ -86,19 +87,29 @@ __device__ __forceinline__ float level_times_norm(float norm, uint32_t levelset,
     return __fmul_rn(norm, level);
 }
 
-// ERC^-1 of a 12-bit prefix: value | length << 8, or 0 when the code is longer than the prefix
+// ERC^-1 of an nbits-bit prefix: value | length << 8, or 0 when the code is longer than the prefix
 // (or is not a code).  Obtained by running Algorithm 2's decoder on the prefix.
-__device__ __forceinline__ uint32_t erc_prefix_entry(uint32_t idx) {
+__device__ __forceinline__ uint32_t erc_prefix_entry(uint32_t idx, uint32_t nbits) {
     uint32_t N = 1, pos = 0;
     for (int it = 0; it < 6; ++it) {
-        if (pos >= kLutBits) return 0;
-        if (!((idx >> (kLutBits - 1u - pos)) & 1u)) return N | ((pos + 1u) << 8);
+        if (pos >= nbits) return 0;
+        if (!((idx >> (nbits - 1u - pos)) & 1u)) return N | ((pos + 1u) << 8);
         const uint32_t nb = N + 1u;
-        if (pos + nb > kLutBits) return 0;
-        N = (idx >> (kLutBits - pos - nb)) & ((1u << nb) - 1u);
+        if (pos + nb > nbits) return 0;
+        N = (idx >> (nbits - pos - nb)) & ((1u << nb) - 1u);
         pos += nb;
     }
     return 0;
+}
+
+// Sign and level index of a token from its next 8 bits (sign bit, then ERC(index) of at most 7 bits,
+// i.e. index <= 15): the upper byte of the token's list entry, (index - 1) << 9 | sign << 8, and in
+// the low byte the bits consumed; 0 when the code is longer.
+constexpr uint32_t kSignedBits = 8;
+__device__ __forceinline__ uint32_t signed_index_entry(uint32_t idx) {
+    const uint32_t r = erc_prefix_entry(idx & 0x7fu, kSignedBits - 1u);
+    if (r == 0) return 0;
+    return (((r & 0xffu) - 1u) << 9) | ((idx >> 7) << 8) | ((r >> 8) + 1u);
 }
 
 // What a lane needs to know to walk sub-block `sb` of one stream.
@@ -176,10 +187,10 @@ __device__ bool describe_chain(const Geometry& G, const TileGeo& T, const Stream
     return true;
 }
 
-// shared memory: the ERC^-1 table, the stream heads, then per warp the running sums of its S sub-blocks
+// shared memory: the two ERC^-1 tables, the stream heads, then per warp the running sums of its S sub-blocks
 // and kWarpWords for lists and staged tokens
 __host__ __device__ inline size_t decode_warp_offset(uint32_t K) {
-    return (2u * (1u << kLutBits) + (size_t)K * sizeof(StreamHead) + 15u) & ~(size_t)15u;
+    return (2u * ((1u << kLutBits) + (1u << kSignedBits)) + (size_t)K * sizeof(StreamHead) + 15u) & ~(size_t)15u;
 }
 __host__ __device__ inline size_t decode_warp_bytes(uint32_t group) {
     return 4u * ((32u / group) * kSB + kWarpWords);
@@ -192,11 +203,13 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     const uint32_t S = 32u / NG;                            // sub-blocks per warp
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     uint16_t* lut = reinterpret_cast<uint16_t*>(dsm);                             // ERC^-1 of 12-bit prefixes
-    StreamHead* heads = reinterpret_cast<StreamHead*>(dsm + 2u * (1u << kLutBits));   // [K]
+    uint16_t* lut2 = lut + (1u << kLutBits);                                      // sign + ERC^-1 of 7-bit prefixes
+    StreamHead* heads = reinterpret_cast<StreamHead*>(lut2 + (1u << kSignedBits));   // [K]
     float* accw = reinterpret_cast<float*>(dsm + decode_warp_offset(P.K) + warp * decode_warp_bytes(NG));   // S * 256 running sums
     uint32_t* list = reinterpret_cast<uint32_t*>(accw + S * kSB);
 
-    for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) lut[i] = (uint16_t)erc_prefix_entry(i);
+    for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) lut[i] = (uint16_t)erc_prefix_entry(i, kLutBits);
+    for (uint32_t i = threadIdx.x; i < (1u << kSignedBits); i += blockDim.x) lut2[i] = (uint16_t)signed_index_entry(i);
     // ---- header validation against the call's arguments, once per stream ----
     for (uint32_t k = threadIdx.x; k < P.K; k += blockDim.x) {
         const uint32_t* hdr = P.streams[k];
@@ -274,7 +287,11 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             const uint32_t my_sb = part * S + lq;
             const uint32_t my_sn = my_sb < nsb_tile ? min(kSB, tile_len - my_sb * kSB) : 0u;   // elements of my sub-block
             bool wide = false;                              // index - 1 does not fit 7 bits (uniform levels, s = 8)
-            for (uint32_t j = 0; j < gcount; ++j) wide = wide || (heads[g0 + j].ok && heads[g0 + j].nlev > 129u);
+            bool small_index = true;                        // exponential levels, index <= 15: sign and index from one look-up
+            for (uint32_t j = 0; j < gcount; ++j) {
+                wide = wide || (heads[g0 + j].ok && heads[g0 + j].nlev > 129u);
+                small_index = small_index && (!heads[g0 + j].ok || (heads[g0 + j].levelset == kLevelsExp && heads[g0 + j].nlev <= 16u));
+            }
             const bool mine = lj < gcount;
             const StreamHead si = heads[g0 + (mine ? lj : 0)];
             Chain ch;                                       // each lane describes the chain it walks
@@ -283,73 +300,69 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             const bool has_chain = mine && si.ok && chain_ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
 
             // A round decodes, for all 32 chains at once, the tokens whose position lies below a limit,
-            // and then adds them stream after stream.  Sparse data takes one round (limit = the whole
-            // sub-block).  When the lists could overflow, the limit advances by `cap` positions per
-            // round: a chain then has at most `cap` tokens per round, and every element still receives
-            // its terms in ascending stream order because all of its terms fall into the same round.
-            // a chain of t tokens in 256 positions takes about t (2 log2(256 / t) + 4) bits: 48 tokens ~ 400 bits
-            // (a token of a dense chain, gaps of 1 to 3, takes about 5 bits)
-            const uint32_t chain_bits = has_chain ? ch.end - ch.cur : 0u;
-            uint32_t guess = chain_bits <= 384u ? (chain_bits + 7u) / 8u : chain_bits / 5u;
-            guess = __reduce_max_sync(0xffffffffu, guess);
-            // Short chains (the usual case) are first copied to shared memory, a word per lane and step, with
-            // all loads in flight at once: the walk below is a chain of dependent reads, and from global
-            // memory every step of it would wait for the cache.  Long chains are walked in place.
-            const uint32_t nw = has_chain ? ((ch.end - 1u) >> 5) - (ch.cur >> 5) + 1u : 0u;     // words my chain touches
-            const bool staged = !wide && guess <= 2u * kStagedListWords / 32u &&
-                                __reduce_max_sync(0xffffffffu, nw) <= kStageWords;
-            const uint32_t cap = staged ? 2u * kStagedListWords / 32u : (wide ? kWarpWords : 2u * kWarpWords) / 32u;   // list entries per chain
-            uint32_t last = ch.last, cur0 = ch.cur, end = ch.end;
-            uint32_t* st = list + kStagedListWords + lane;   // word i of a staged chain at st[32 i]
-            if (staged) {
-                const uint32_t* src = ch.tok + (ch.cur >> 5);
-#pragma unroll
-                for (uint32_t i = 0; i < kStageWords; ++i)
-                    if (i < nw) st[i * 32u] = __ldg(src + i);
-                last = nw ? nw - 1u : 0u;
-                cur0 = ch.cur & 31u;
-                end = ch.end - (ch.cur & ~31u);
-            }
-            __syncwarp();
-            // positions per round: the whole sub-block when the longest chain should fit its list, else
-            // an even split into as many rounds as the guess asks for (at least `cap` positions, which
-            // can never overflow)
+            // and then adds them stream after stream; every element still receives its terms in ascending
+            // stream order because all of its terms fall into the same round.  The walk reads the chain
+            // from shared memory: every lane copies the next kStageWords words of its chain there, all
+            // loads in flight at once (the walk is a chain of dependent reads, which from global memory
+            // would wait for the cache at every step), and again whenever it has used them up.
+            // Sparse data takes one round (limit = the whole sub-block).  When the longest chain is
+            // expected to hold more tokens than a list (a chain of t tokens in 256 positions takes about
+            // t (2 log2(256 / t) + 4) bits, 5 bits per token when it is dense), the sub-block is split
+            // evenly into rounds, with a third of slack; a round in which a list runs over is taken again
+            // with half the positions.
+            const uint32_t cap = (wide ? kStagedListWords : 2u * kStagedListWords) / 32u;   // list entries per chain
+            const uint32_t chain_bits = __reduce_max_sync(0xffffffffu, has_chain ? ch.end - ch.cur : 0u);
             uint32_t step = kSB;
-            if (guess > cap) {
-                const uint32_t rounds = (guess + guess / 3u + cap - 1u) / cap;     // a third of slack: 32 chains must all fit
+            if (chain_bits > 9u * cap) {                    // 9 bits per token is what sparse chains take
+                const uint32_t guess = chain_bits <= 512u ? chain_bits / 8u : chain_bits / 5u;
+                const uint32_t rounds = max(2u, (guess + guess / 3u + cap - 1u) / cap);
                 step = max(cap, (kSB + rounds - 1u) / rounds);
             }
+            const uint32_t end = ch.end;
             bool alive = has_chain, bad = false, fixed_done = false;
-            uint32_t cur = cur0, pos = 0, max_sym = 0;
+            uint32_t cur = ch.cur, pos = 0, max_hi = 0;    // max_hi: the largest entry part (index - 1) << 9 | sign << 8 so far
+            uint32_t* st = list + kStagedListWords + lane;   // word i of the staged part of my chain at st[32 i]
             uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
             uint32_t* slot32 = list + lane;
             uint32_t n = 0, limit = 0;
-            bool full = false, running = false;
-            // One round of the walk; `word(i)` fetches word i of the lane's chain (two instances: from
-            // shared memory for staged chains, from global memory otherwise).
-            auto walk = [&](auto word, auto wide_entries) {
+            uint32_t rbase = 0, rcur = 0, rlast = 0, rstop = 0;   // first staged bit; cursor, last word and stopping bit relative to it
+            bool running = false;
+            // One round of the walk over the staged words.
+            auto walk = [&](auto wide_entries, auto one_lookup) {
+                auto word = [st](uint32_t i) { return st[32u * i]; };
                 // Every lane executes every step (a lane that has stopped works on stale but in-bounds
                 // data and commits nothing): no divergent branch except the rare long-code path.
                 while (__any_sync(0xffffffffu, running)) {
-                    const uint32_t wi = cur >> 5;
-                    const uint32_t x0 = word(min(wi, last));
-                    const uint32_t x1 = word(min(wi + 1u, last));
-                    const uint32_t win = __funnelshift_l(x1, x0, cur);                      // 32 bits from the cursor
+                    const uint32_t wi = rcur >> 5;
+                    const uint32_t x0 = word(min(wi, rlast));
+                    const uint32_t x1 = word(min(wi + 1u, rlast));
+                    const uint32_t win = __funnelshift_l(x1, x0, rcur);                     // 32 bits from the cursor
                     const uint32_t e1 = lut[win >> (32u - kLutBits)];
                     const uint32_t t = win << (e1 >> 8);                                    // the sign bit is on top
-                    const uint32_t e2 = lut[(t << 1) >> (32u - kLutBits)];
-                    uint32_t gap = e1 & 0xffu, sym = e2 & 0xffu, negative = t >> 31;
-                    uint32_t used = (e1 >> 8) + 1u + (e2 >> 8);
-                    bool good = e1 != 0 && e2 != 0;
+                    uint32_t gap = e1 & 0xffu, used, hi;    // hi: (index - 1) << 9 | sign << 8
+                    bool good;
+                    if (decltype(one_lookup)::value) {
+                        const uint32_t e2 = lut2[t >> (32u - kSignedBits)];
+                        used = (e1 >> 8) + (e2 & 0xffu);
+                        hi = e2 & 0xff00u;
+                        good = e1 != 0 && e2 != 0;
+                    } else {
+                        const uint32_t e2 = lut[(t << 1) >> (32u - kLutBits)];
+                        used = (e1 >> 8) + 1u + (e2 >> 8);
+                        hi = ((t >> 31) << 8) | (((e2 & 0xffu) - 1u) << 9);
+                        good = e1 != 0 && e2 != 0;
+                    }
                     if (__any_sync(0xffffffffu, running && !good)) {
-                        if (running && !good) {             // a code longer than 12 bits: Algorithm 2 as a loop
-                            uint64_t win64 = window64(word, cur, last);
+                        if (running && !good) {             // a code longer than the table's prefix: Algorithm 2 as a loop
+                            uint64_t win64 = window64(word, rcur, rlast);
+                            uint32_t sym = 1;
                             used = 0;
                             good = erc_read(win64, used, gap);
-                            negative = (uint32_t)(win64 >> 63);
+                            const uint32_t negative = (uint32_t)(win64 >> 63);
                             win64 <<= 1;
                             used += 1;
                             good = good && erc_read(win64, used, sym);
+                            hi = (negative << 8) | ((min(sym, 0x10000u) - 1u) << 9);
                             if (!good) {                    // not a code at all: the chain is malformed
                                 bad = true;
                                 alive = false;
@@ -362,45 +375,66 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     const uint32_t npos = pos + gap;
                     const bool commit = running && good && npos <= limit;   // beyond the limit: a later round's token
                     if (commit) {
-                        max_sym = max(max_sym, sym);
-                        const uint32_t e = ((npos - 1u) & 0xffu) | (negative << 8) | ((sym - 1u) << 9);
+                        max_hi = max(max_hi, hi);
+                        const uint32_t e = ((npos - 1u) & 0xffu) | hi;
                         const uint32_t at = min(n, cap - 1u) * 32u;     // a list that runs over is noticed after the round
                         if (decltype(wide_entries)::value) slot32[at] = e;
                         else slot16[at] = (uint16_t)e;
                         pos = npos;
-                        cur += used;
+                        rcur += used;
                         ++n;
-                        alive = cur < end;
                     }
-                    running = commit && alive;
+                    running = commit && rcur < rstop;
                 }
             };
             for (;;) {
                 const uint32_t done_pos = limit;            // positions below this have been added
-                const uint32_t cur_s = cur, pos_s = pos, max_sym_s = max_sym;
+                const uint32_t cur_s = cur, pos_s = pos, max_hi_s = max_hi;
                 const bool alive_s = alive, bad_s = bad;
                 limit = done_pos + step;
                 n = 0;
-                full = false;
-                running = alive;
-                if (staged) walk([st](uint32_t i) { return st[32u * i]; }, std::false_type());
-                else if (!wide) walk([&ch](uint32_t i) { return __ldg(ch.tok + i); }, std::false_type());
-                else walk([&ch](uint32_t i) { return __ldg(ch.tok + i); }, std::true_type());
-                full = n > cap;
-                if (__any_sync(0xffffffffu, full)) {
-                    if (step == cap) {                      // cannot happen: at most `cap` positions per round
+                bool refill = alive;                        // lanes that stage the next words of their chain
+                for (;;) {
+                    // ---- stage, then walk until every lane has reached the limit, its chain's end or the
+                    // end of its staged words; lanes of the last kind stage again and go on alone ----
+                    if (refill) {
+                        const uint32_t w0 = cur >> 5;
+                        const uint32_t nws = min(kStageWords, ((end - 1u) >> 5) - w0 + 1u);     // up to the word that holds the chain's last bit
+                        const uint32_t* src = ch.tok + w0;
+#pragma unroll
+                        for (uint32_t i = 0; i < kStageWords; ++i)
+                            if (i < nws) st[i * 32u] = __ldg(src + i);
+                        rbase = 32u * w0;
+                        rcur = cur - rbase;
+                        rlast = nws - 1u;
+                        // go on while the cursor is before the chain's end or, when the chain is longer than
+                        // the staged words, while two more words lie behind it (the long-code path looks that far)
+                        rstop = end - rbase <= 32u * nws ? end - rbase : kStageSoftBits;
+                    }
+                    __syncwarp();
+                    running = refill;
+                    if (small_index) walk(std::false_type(), std::true_type());
+                    else if (!wide) walk(std::false_type(), std::false_type());
+                    else walk(std::true_type(), std::false_type());
+                    cur = rbase + rcur;
+                    alive = alive && !bad && cur < end;
+                    refill = alive && rcur >= rstop && n <= cap;
+                    if (!__any_sync(0xffffffffu, refill) || __any_sync(0xffffffffu, n > cap)) break;
+                }
+                // a list ran over: nothing of this round has been added yet, so take the round again from
+                // where it started with half the positions (`cap` positions cannot run over)
+                if (__any_sync(0xffffffffu, n > cap)) {
+                    if (step <= cap) {                      // cannot happen
                         bad = true;
                         break;
                     }
-                    // the guess was too low: nothing of this round has been added yet, so take the round
-                    // again from where it started, with the window that cannot overflow
-                    step = cap;
+                    step = max(cap, step / 2u);
                     limit = done_pos;
                     alive = alive_s;
                     bad = bad_s;
                     cur = cur_s;
                     pos = pos_s;
-                    max_sym = max_sym_s;
+                    max_hi = max_hi_s;
                     continue;
                 }
                 __syncwarp();
@@ -477,7 +511,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                 if (!__any_sync(0xffffffffu, alive)) break;
             }
             // a well-formed chain ends exactly at its declared length, inside its sub-block, with known indices
-            if (has_chain && !bad) bad = cur != end || pos > my_sn || max_sym >= si.nlev;
+            if (has_chain && !bad) bad = cur != end || pos > my_sn || (max_hi >> 9) + 1u >= si.nlev;
             if (__any_sync(0xffffffffu, bad) && lane == 0) latch_status(P.ws, kErrBadStream);
         }
 
