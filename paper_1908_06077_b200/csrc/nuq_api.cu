@@ -179,7 +179,9 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, bool norms_are_ours) {
     if (G.mode == kModeErc) {
         // a warp's 1024 elements lie in at most this many buckets
         const uint32_t warp_elems = kBLK / kEncWarps;
-        const uint32_t warp_buckets = G.bucket >= warp_elems ? 2u : warp_elems / G.bucket + 1u;
+        // (tiles start at bucket boundaries and a warp's part at a multiple of 1024 elements)
+        const uint32_t warp_buckets = G.bucket >= warp_elems ? (G.bucket % warp_elems == 0 ? 1u : 2u)
+                                                             : (warp_elems % G.bucket == 0 ? warp_elems / G.bucket : warp_elems / G.bucket + 1u);
         P.window_words = (token_bits_bound(G, warp_elems, warp_buckets, norms_are_ours) + 31u) / 32u + 4u;
         const uint32_t list_words = G.levelset == kLevelsExp ? kEncChunk / 2u : kEncChunk;   // 16- or 32-bit entries
         P.warp_smem_words = (P.window_words + list_words + 3u) & ~3u;
@@ -187,7 +189,16 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, bool norms_are_ours) {
         P.window_words = 0;
         P.warp_smem_words = 0;
     }
-    const uint64_t cap = (uint64_t)encode_max_blocks(sms, encode_smem_bytes(P));
+    // two staged tiles let the writer warp lag one tile behind the workers; a third one, taken when
+    // it costs no resident CTA, lets it lag two
+    P.stages = G.mode == kModeErc ? 2u : 1u;
+    int per_sm = encode_blocks_per_sm(P);
+    if (G.mode == kModeErc) {
+        P.stages = 3;
+        if (encode_blocks_per_sm(P) < per_sm) P.stages = 2;
+    }
+    if (per_sm < 1) per_sm = 1;
+    const uint64_t cap = (uint64_t)sms * (uint64_t)per_sm;
     pl.want_grid = (uint32_t)(G.ntiles < cap ? G.ntiles : cap);
     return pl;
 }

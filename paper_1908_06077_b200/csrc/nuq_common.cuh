@@ -74,6 +74,7 @@ struct EncodeParams {
     uint64_t seed, offset;
     uint32_t round_keys[20]; // Philox4x32-10 key schedule of `seed`: (k0, k1) of round 0, 1, ..., 9
     uint32_t stage_words;    // shared-memory image of a tile's records (multiple of 4)
+    uint32_t stages;         // staged tile images per CTA (ERC: 2 or 3; fixed width: 1)
     uint32_t window_words;   // shared-memory token string of one warp
     uint32_t warp_smem_words;// shared memory of one warp (token string, token list)
     uint32_t grid;           // CTAs to launch

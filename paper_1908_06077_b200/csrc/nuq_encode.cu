@@ -300,7 +300,7 @@ constexpr uint32_t kChunkRows = kChunk / 128;
 // Named CTA barriers.  The 8 worker warps meet at kBarWork; the writer warp (ERC mode) and the
 // workers hand the two staged tiles back and forth through kBarStaged + b (workers arrive, the
 // writer waits) and kBarFree + b (the writer arrives, workers wait).
-constexpr uint32_t kBarWork = 1, kBarStaged = 2, kBarFree = 4;
+constexpr uint32_t kBarWork = 1, kBarStaged = 2, kBarFree = 5;     // kBarStaged + b, kBarFree + b for stage b < 3
 constexpr uint32_t kEncAllThreads = kEncThreads + 32;      // ERC mode: workers + the writer warp
 template <uint32_t ID, uint32_t COUNT>
 __device__ __forceinline__ void bar_sync() {
@@ -311,14 +311,18 @@ __device__ __forceinline__ void bar_arrive() {
     __threadfence_block();
     asm volatile("bar.arrive %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
 }
-// the pair of barriers of stage b (0 or 1); immediate barrier numbers, so that the kernel claims only those it uses
+// the pair of barriers of stage b (0, 1 or 2); immediate barrier numbers, so that the kernel claims only those it uses
 template <uint32_t BASE>
 __device__ __forceinline__ void stage_sync(uint32_t b) {
-    if (b) bar_sync<BASE + 1, kEncAllThreads>(); else bar_sync<BASE, kEncAllThreads>();
+    if (b == 0) bar_sync<BASE, kEncAllThreads>();
+    else if (b == 1) bar_sync<BASE + 1, kEncAllThreads>();
+    else bar_sync<BASE + 2, kEncAllThreads>();
 }
 template <uint32_t BASE>
 __device__ __forceinline__ void stage_arrive(uint32_t b) {
-    if (b) bar_arrive<BASE + 1, kEncAllThreads>(); else bar_arrive<BASE, kEncAllThreads>();
+    if (b == 0) bar_arrive<BASE, kEncAllThreads>();
+    else if (b == 1) bar_arrive<BASE + 1, kEncAllThreads>();
+    else bar_arrive<BASE + 2, kEncAllThreads>();
 }
 
 // A tile whose records are staged in shared memory and whose place in the stream is not
@@ -416,7 +420,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
     __shared__ uint32_t s_start[32];                       // scratch: first token offset of a sub-block (per warp 4)
     __shared__ unsigned long long s_tile[2];
     __shared__ uint32_t s_abort, s_nnz;
-    __shared__ Pending s_pend[2];                          // ERC: the two staged tiles (current, previous)
+    __shared__ Pending s_pend[3];                          // ERC: the staged tiles (current and up to two earlier ones)
     __shared__ CtaTotals s_tot;
 
     using S = Sym<LEVELSET>;
@@ -424,7 +428,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     float* data = reinterpret_cast<float*>(smem);                               // kBLK floats: the tile
     uint32_t* stage = smem + kBLK;                                              // image of the tile's records
-    uint32_t* wmem = stage + (MODE == kModeErc ? 2u : 1u) * P.stage_words + warp * P.warp_smem_words;
+    uint32_t* wmem = stage + P.stages * P.stage_words + warp * P.warp_smem_words;
     uint32_t* window = wmem;                                                    // this warp's token string
     uint32_t* tokens = wmem + P.window_words;               // kChunk entries: position | field << 10 (uniform levels)
     uint16_t* tokens16 = reinterpret_cast<uint16_t*>(tokens);   //                position | field << 8  (exponential levels)
@@ -483,7 +487,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
         }
         s_lut_signed[tid] = v;
     }
-    for (uint32_t i = tid; i < (MODE == kModeErc ? 2u : 1u) * P.stage_words; i += blockDim.x) stage[i] = 0;
+    for (uint32_t i = tid; i < P.stages * P.stage_words; i += blockDim.x) stage[i] = 0;
     if (warp < (uint32_t)kEncWarps)
         for (uint32_t i = lane; i < P.window_words; i += 32) window[i] = 0;
     if (tid == 0) {
@@ -492,6 +496,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
         s_nnz = 0;
         s_pend[0].valid = 0;
         s_pend[1].valid = 0;
+        s_pend[2].valid = 0;
         s_tot.nnz = 0;
         s_tot.code_bits = 0;
         s_tot.tiles = 0;
@@ -508,18 +513,19 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
     if (writer) {
         // ---- the writer warp: finds the place of every staged tile (look-back), copies it to the
         // stream and hands the stage back; the workers never wait for it unless it falls two tiles behind
+        uint32_t b = 0;                                     // stage of tile k: k mod P.stages
         for (uint32_t k = 0;; ++k) {
-            stage_sync<kBarStaged>(k & 1u);                    // tile k of this CTA is staged
+            stage_sync<kBarStaged>(b);                      // tile k of this CTA is staged
             if (k >= *reinterpret_cast<volatile uint32_t*>(&s_tot.stop)) break;
-            flush_pending(P, s_pend[k & 1u], s_tot, stage + (k & 1u) * P.stage_words, tile_state, group_state, table,
-                          payload, lane);
-            stage_arrive<kBarFree>(k & 1u);
+            flush_pending(P, s_pend[b], s_tot, stage + b * P.stage_words, tile_state, group_state, table, payload, lane);
+            stage_arrive<kBarFree>(b);
+            b = b + 1u == P.stages ? 0u : b + 1u;
         }
     }
 
     uint32_t parity = 0;
-    uint32_t it = 0;
-    for (; !writer; ++it) {                                 // the 8 worker warps
+    uint32_t it = 0, sg = 0;                                // sg: stage of iteration it, it mod P.stages
+    for (; !writer; ++it, sg = sg + 1u == P.stages ? 0u : sg + 1u) {           // the 8 worker warps
         const uint64_t tile = s_tile[it & 1u];
         if (tile >= G.ntiles) break;
 
@@ -810,7 +816,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
 
         // ---- layout of the tile's records ---------------------------------------------
         if (MODE == kModeErc) {
-            uint32_t* stg = stage + (it & 1u) * P.stage_words;              // this tile's image; the other one is pending
+            uint32_t* stg = stage + sg * P.stage_words;                      // this tile's image; the others are pending
             // every warp runs the same scan over the 32 sub-block lengths
             const uint32_t sb = lane;
             const uint32_t v = sb < nsb_tile ? s_sb_bits[sb] : 0u;
@@ -842,8 +848,8 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
             const uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
             // announce the tile's size to its successors at once; the writer warp looks up its place
             if (tid == 0) announce_tile(tile_state, group_state, tile, tile_words);
-            // this stage held the tile of two iterations ago: the writer must be done with it
-            if (it >= 2u) stage_sync<kBarFree>(it & 1u);
+            // this stage held the tile of P.stages iterations ago: the writer must be done with it
+            if (it >= P.stages) stage_sync<kBarFree>(sg);
             // header words of the blocks: norm, then the u16 lengths two per word.  Lanes 4w .. 4w+3
             // of warp w stand for the warp's own sub-blocks, whose norms it holds.
             if ((lane >> 2) == warp && sb < nsb_tile) {
@@ -854,7 +860,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
                 atomicOr(stg + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
             }
             if (warp == 0) {
-                Pending& pd = s_pend[it & 1u];
+                Pending& pd = s_pend[sg];
                 pd.blk_wordoff[lane] = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
                 if (lane == 0) {
                     pd.tile = tile;
@@ -892,7 +898,7 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
             }
             __syncwarp();
             for (uint32_t i = lane; i < (bits + 31u) / 32u + 2u; i += 32) window[i] = 0;   // ready for the next tile
-            stage_arrive<kBarStaged>(it & 1u);     // the writer may take the tile
+            stage_arrive<kBarStaged>(sg);                  // the writer may take the tile
         } else {
             uint64_t tile_off;
             uint32_t tile_words;
@@ -925,12 +931,17 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
     }
 
     if (MODE == kModeErc && !writer) {
-        // ---- the workers ran `it` iterations: wait until the writer has written the last two tiles,
-        // telling it in between that no further one comes ----
-        if (it >= 2u) stage_sync<kBarFree>(it & 1u);
+        // ---- the workers ran `it` iterations (the next one would use stage sg): wait until the writer
+        // has written the last tiles, telling it in between that no further one comes ----
+        if (it >= P.stages) stage_sync<kBarFree>(sg);       // tile it - stages: its barriers are used again below
         if (tid == 0) s_tot.stop = it;
-        stage_arrive<kBarStaged>(it & 1u);
-        if (it >= 1u) stage_sync<kBarFree>((it + 1u) & 1u);
+        stage_arrive<kBarStaged>(sg);
+        for (uint32_t back = P.stages - 1u; back >= 1u; --back) {   // tiles it - stages + 1 .. it - 1
+            if (it >= back) {
+                const uint32_t bb = (sg + P.stages - back) % P.stages;
+                stage_sync<kBarFree>(bb);
+            }
+        }
     }
     __syncthreads();                                        // every write of this CTA lies behind this barrier
     if (tid == 0) finish_cta<MODE>(P, s_tot.tiles, s_tot.nnz, s_tot.code_bits);
@@ -987,27 +998,45 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
 
 // shared memory of one CTA: the tile, its staged image, and per warp a bit window and a token list
 size_t encode_smem_bytes(const EncodeParams& P) {
-    const size_t stages = P.geo.mode == kModeErc ? 2 : 1;   // ERC: the current tile and the one awaiting its place
-    return 4u * ((size_t)kBLK + stages * P.stage_words + (size_t)kEncWarps * P.warp_smem_words);
+    return 4u * ((size_t)kBLK + (size_t)P.stages * P.stage_words + (size_t)kEncWarps * P.warp_smem_words);
 }
 
-int encode_max_blocks(int sms, size_t smem_bytes) {
-    size_t per_sm = (227u * 1024u) / (smem_bytes + 1024u + 3u * 1024u);     // + static shared memory and the per-CTA reserve
-    if (per_sm > (size_t)kEncMinBlocks) per_sm = kEncMinBlocks;
-    if (per_sm < 1) per_sm = 1;
-    return sms * (int)per_sm;
+constexpr int kEncMaxDynSmem = 112 * 1024;
+
+template <uint32_t L, uint32_t M>
+static cudaError_t prepare_kernel() {
+    static bool attr_set = false;
+    if (attr_set) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncMaxDynSmem);
+    if (e == cudaSuccess) attr_set = true;
+    return e;
+}
+
+template <uint32_t L, uint32_t M>
+static int blocks_per_sm(const EncodeParams& P) {
+    if (prepare_kernel<L, M>() != cudaSuccess) return 0;
+    int n = 0;
+    const int threads = M == kModeErc ? (int)kEncAllThreads : kEncThreads;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, encode_kernel<L, M>, threads, encode_smem_bytes(P)) != cudaSuccess)
+        return 0;
+    return n < kEncMinBlocks ? n : kEncMinBlocks;
+}
+
+int encode_blocks_per_sm(const EncodeParams& P) {
+    const bool uni = P.geo.levelset == kLevelsUniform, fixed = P.geo.mode == kModeFixed;
+    if (encode_smem_bytes(P) > (size_t)kEncMaxDynSmem) return 0;
+    if (!uni && !fixed) return blocks_per_sm<kLevelsExp, kModeErc>(P);
+    if (!uni && fixed) return blocks_per_sm<kLevelsExp, kModeFixed>(P);
+    if (uni && !fixed) return blocks_per_sm<kLevelsUniform, kModeErc>(P);
+    return blocks_per_sm<kLevelsUniform, kModeFixed>(P);
 }
 
 template <uint32_t L, uint32_t M>
 static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
     const size_t smem = encode_smem_bytes(P);
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, 112 * 1024);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
-    }
-    if (smem > 112 * 1024 || P.grid == 0) return cudaErrorInvalidValue;
+    cudaError_t e = prepare_kernel<L, M>();
+    if (e != cudaSuccess) return e;
+    if (smem > (size_t)kEncMaxDynSmem || P.grid == 0) return cudaErrorInvalidValue;
     encode_kernel<L, M><<<P.grid, M == kModeErc ? kEncAllThreads : (uint32_t)kEncThreads, smem, stream>>>(P);
     return cudaGetLastError();
 }

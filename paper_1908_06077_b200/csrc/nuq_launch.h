@@ -12,7 +12,7 @@ cudaError_t upload_erc_lut();                         // into the current device
 cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uint32_t norm_kind, float* norms,
                                 uint64_t nb, cudaStream_t stream);
 size_t encode_smem_bytes(const EncodeParams& P);      // dynamic shared memory of one encoder CTA
-int encode_max_blocks(int sms, size_t smem_bytes);    // CTAs that can be resident at once
+int encode_blocks_per_sm(const EncodeParams& P);      // encoder CTAs one SM holds at once (0 on error)
 cudaError_t launch_encode(const EncodeParams& P, cudaStream_t stream);
 cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream);
 
