@@ -243,14 +243,22 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
 
     __syncthreads();                                        // table and headers are ready; from here on warps run alone
 
+    // Work is handed out one warp-sized unit at a time (S sub-blocks of one tile, all streams).  The
+    // ticket of the next unit is asked for while the current one is decoded, except near the end: a
+    // unit reserved by a warp that is busy with a long one would be started late.
+    const uint64_t nunits = G.ntiles * NG;
+    const uint64_t in_flight = 3ull * gridDim.x * (blockDim.x >> 5);
+    const uint64_t reserve_until = nunits > in_flight ? nunits - in_flight : 0;
+    unsigned long long next_unit = 0;
+    bool have_next = false;
     for (;;) {
-        // work is handed out one warp-sized unit at a time (S sub-blocks of one tile, all streams)
-        unsigned long long unit = 0;
-        if (lane == 0) unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
-        unit = __shfl_sync(0xffffffffu, unit, 0);
+        if (!have_next && lane == 0) next_unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        const unsigned long long unit = __shfl_sync(0xffffffffu, next_unit, 0);
+        if (unit >= nunits) break;
         const uint64_t tile = unit / NG;
         const uint32_t part = (uint32_t)(unit % NG);        // which S sub-blocks of the tile
-        if (tile >= G.ntiles) break;
+        have_next = unit < reserve_until;
+        if (have_next && lane == 0) next_unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
         // ---- tile geometry (same tiling as the encoder) ---------------------------
         TileGeo T;
         T.bucket_idx = 0;
