@@ -163,6 +163,9 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
 
 using namespace nuq;
 
+// Mode of the containers this process has encoded, by address (see enqueue_encode).  Guarded by g_mu.
+static std::map<const void*, uint32_t> g_container_mode;
+
 // What one encode call needs from its workspace and from shared memory.
 struct EncodePlan {
     size_t state_bytes;      // control block + one look-back word per tile and per group of 32 tiles
@@ -237,6 +240,10 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
     }
     if (launch_encode(P, stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    // remember the mode of the container at this address: a hint for the decoder's choice of kernels,
+    // checked against the header on the device
+    if (g_container_mode.size() > 4096) g_container_mode.clear();
+    g_container_mode[out] = G.mode;
     return NUQ_OK;
 }
 
@@ -323,6 +330,11 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     for (uint32_t k = K; k < kMaxK; ++k) P.streams[k] = nullptr;
     P.K = K;
     P.group = K >= 8 ? 8u : K >= 3 ? 4u : K;            // 1, 2, 4 or 8 streams side by side
+    P.after_fixed = 1;                                  // all streams believed to be in the fixed-width mode?
+    for (uint32_t k = 0; k < K; ++k) {
+        auto it = g_container_mode.find(streams[k]);
+        if (it == g_container_mode.end() || it->second != kModeFixed) P.after_fixed = 0;
+    }
     P.acc = acc;
     Workspace* ws = nullptr;
     int dev = 0;

@@ -84,7 +84,8 @@ struct DecodeParams {
     Geometry geo;
     const uint32_t* streams[kMaxK];
     uint32_t K;
-    uint32_t group;          // streams decoded side by side = warps per CTA (1, 2, 4 or 8)
+    uint32_t group;          // streams decoded side by side (1, 2, 4 or 8)
+    uint32_t after_fixed;    // the fixed-width kernel runs first; the general kernel returns if it did the work
     float* acc;
     Workspace* ws;
 };

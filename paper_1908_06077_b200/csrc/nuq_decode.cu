@@ -187,6 +187,128 @@ __device__ bool describe_chain(const Geometry& G, const TileGeo& T, const Stream
     return true;
 }
 
+// A container's header checked against the call's arguments.
+__device__ StreamHead read_head(const Geometry& G, const uint32_t* hdr) {
+    const uint32_t flags = __ldg(hdr + 6);
+    const uint32_t levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
+    const uint64_t hd = (uint64_t)__ldg(hdr + 2) | ((uint64_t)__ldg(hdr + 3) << 32);
+    const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
+    const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
+    bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
+              __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
+              (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
+    const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
+    const uint32_t width = 1u + (32u - __clz(nlev - 1u));                   // fixed mode: sign bit + ceil(log2(levels))
+    const uint64_t cwords = cbits >> 5;
+    if (ok && mode == kModeErc) {
+        ok = hnblk == G.nblk && cwords > kHeaderWords + 2 * (G.nblk + 1);
+    } else if (ok) {
+        const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
+        const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
+        ok = hnblk == G.nb &&
+             cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
+    }
+    StreamHead h;
+    h.hdr = hdr; h.cwords = cwords; h.ok = ok ? 1u : 0u; h.mode = mode; h.levelset = levelset;
+    h.nlev = nlev; h.width = width; h.pad = 0;
+    return h;
+}
+
+// All streams in the fixed-width mode with the same field width W (sign bit + level index, MSB first):
+// no tokens to walk, so a thread takes 32 consecutive elements (W words of every stream, never across a
+// bucket: buckets are multiples of 256 elements), adds the K dequantized values of each element in
+// stream order in registers and stores the 32 sums.  Same arithmetic and order as the general path.
+template <uint32_t W>
+__device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const StreamHead* heads) {
+    const Geometry& G = P.geo;
+    const uint64_t ngroups = (G.d + 31) / 32;
+    const uint32_t levelset = heads[0].levelset, nlev = heads[0].nlev;
+    const uint32_t rec_words = 1u + G.bucket * W / 32u;
+    const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
+    constexpr uint32_t fmask = (1u << W) - 1u, smask = (1u << (W - 1u)) - 1u;
+    bool bad = false;
+    for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += (uint64_t)gridDim.x * blockDim.x) {
+        const uint64_t e0 = 32 * grp, b = e0 / G.bucket;
+        const uint32_t eb = (uint32_t)(e0 - b * G.bucket);                         // first element within its bucket
+        const uint32_t nel = G.d - e0 < 32 ? (uint32_t)(G.d - e0) : 32u;
+        const uint32_t bucket_len = b == G.nb - 1 ? (uint32_t)last_len : G.bucket;
+        const uint32_t avail = (bucket_len * W + 31u) / 32u - (eb / 32u) * W;      // field words of the record from here on
+        float* dst = P.acc + e0;
+#pragma unroll
+        for (uint32_t half = 0; half < 2; ++half) {         // 16 elements at a time: the sums stay in few registers
+            float acc[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+            for (uint32_t k = 0; k < P.K; ++k) {
+                const uint32_t* rec = heads[k].hdr + kHeaderWords + b * rec_words;
+                const float norm = __uint_as_float(__ldg(rec));
+                const uint32_t* fw = rec + 1u + (eb / 32u) * W;
+                // the words that hold fields 16 * half .. 16 * half + 15
+                constexpr uint32_t kHalfWords = (16u * W + 31u) / 32u + 1u;
+                const uint32_t w0 = (16u * half * W) >> 5;
+                uint32_t words[kHalfWords + 1];
+#pragma unroll
+                for (uint32_t j = 0; j < kHalfWords; ++j) words[j] = w0 + j < avail ? __ldg(fw + w0 + j) : 0u;
+                words[kHalfWords] = 0;
+#pragma unroll
+                for (uint32_t i = 0; i < 16; ++i) {
+                    const uint32_t bit = (16u * half + i) * W - 32u * w0, a = bit >> 5, sh = bit & 31u;
+                    const uint32_t field = sh + W <= 32u ? (words[a] >> (32u - sh - W)) & fmask
+                                                         : __funnelshift_l(words[a + 1], words[a], sh) >> (32u - W);
+                    const uint32_t sym = field & smask;
+                    if (16u * half + i < nel) {
+                        if (sym >= nlev) bad = true;
+                        else if (sym) {
+                            const float v = level_times_norm(norm, levelset, G.s, sym);
+                            acc[i] += (field >> (W - 1u)) ? -v : v;
+                        }
+                    }
+                }
+            }
+            if (nel == 32u) {
+#pragma unroll
+                for (int i = 0; i < 16; i += 4)
+                    *reinterpret_cast<float4*>(dst + 16 * half + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (16u * half + (uint32_t)i < nel) dst[16 * half + i] = acc[i];
+            }
+        }
+    }
+    if (bad) latch_status(P.ws, kErrBadStream);
+}
+
+// The kernel of that path.  It is launched when the library believes that all streams are in the
+// fixed-width mode (it wrote them itself); it checks the headers like the general kernel and, if they
+// say otherwise, leaves everything to the general kernel, which is launched behind it in any case and
+// returns at once when this one has done the work.
+__global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant__ DecodeParams P) {
+    __shared__ StreamHead heads[kMaxK];
+    __shared__ uint32_t s_width;
+    for (uint32_t k = threadIdx.x; k < P.K; k += blockDim.x) heads[k] = read_head(P.geo, P.streams[k]);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool same = true;
+        for (uint32_t k = 0; k < P.K; ++k)
+            same = same && heads[k].ok && heads[k].mode == kModeFixed && heads[k].levelset == heads[0].levelset;
+        s_width = same ? heads[0].width : 0u;
+        if (same && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0]) = 1;   // tell the general kernel
+    }
+    __syncthreads();
+    switch (s_width) {
+        case 3: decode_all_fixed<3>(P, heads); break;
+        case 4: decode_all_fixed<4>(P, heads); break;
+        case 5: decode_all_fixed<5>(P, heads); break;
+        case 6: decode_all_fixed<6>(P, heads); break;
+        case 7: decode_all_fixed<7>(P, heads); break;
+        case 8: decode_all_fixed<8>(P, heads); break;
+        case 9: decode_all_fixed<9>(P, heads); break;
+        case 10: decode_all_fixed<10>(P, heads); break;
+        default: break;
+    }
+}
+
 // shared memory: the two ERC^-1 tables, the stream heads, then per warp the running sums of its S sub-blocks
 // and kWarpWords for lists and staged tokens
 __host__ __device__ inline size_t decode_warp_offset(uint32_t K) {
@@ -198,6 +320,7 @@ __host__ __device__ inline size_t decode_warp_bytes(uint32_t group) {
 
 __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
+    if (P.after_fixed && *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0])) return;   // the fixed-width kernel did it all
     const Geometry& G = P.geo;
     const uint32_t NG = P.group;                            // streams decoded side by side (1, 2, 4 or 8)
     const uint32_t S = 32u / NG;                            // sub-blocks per warp
@@ -212,31 +335,8 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     for (uint32_t i = threadIdx.x; i < (1u << kSignedBits); i += blockDim.x) lut2[i] = (uint16_t)signed_index_entry(i);
     // ---- header validation against the call's arguments, once per stream ----
     for (uint32_t k = threadIdx.x; k < P.K; k += blockDim.x) {
-        const uint32_t* hdr = P.streams[k];
-        const uint32_t flags = __ldg(hdr + 6);
-        const uint32_t levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
-        const uint64_t hd = (uint64_t)__ldg(hdr + 2) | ((uint64_t)__ldg(hdr + 3) << 32);
-        const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
-        const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
-        bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
-                  __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
-                  (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
-        const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
-        const uint32_t width = 1u + (32u - __clz(nlev - 1u));                   // fixed mode: sign bit + ceil(log2(levels))
-        const uint64_t cwords = cbits >> 5;
-        if (ok && mode == kModeErc) {
-            ok = hnblk == G.nblk && cwords > kHeaderWords + 2 * (G.nblk + 1);
-        } else if (ok) {
-            const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
-            const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
-            ok = hnblk == G.nb &&
-                 cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
-        }
-        StreamHead h;
-        h.hdr = hdr; h.cwords = cwords; h.ok = ok ? 1u : 0u; h.mode = mode; h.levelset = levelset;
-        h.nlev = nlev; h.width = width; h.pad = 0;
-        heads[k] = h;
-        if (!ok) latch_status(P.ws, kErrBadStream);
+        heads[k] = read_head(G, P.streams[k]);
+        if (!heads[k].ok) latch_status(P.ws, kErrBadStream);
     }
     for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
         *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -327,7 +427,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                 step = max(cap, (kSB + rounds - 1u) / rounds);
             }
             const uint32_t end = ch.end;
-            bool alive = has_chain, bad = false, fixed_done = false;
+            bool alive = has_chain, bad = false;
             uint32_t cur = ch.cur, pos = 0, max_hi = 0;    // max_hi: the largest entry part (index - 1) << 9 | sign << 8 so far
             uint32_t* st = list + kStagedListWords + lane;   // word i of the staged part of my chain at st[32 i]
             uint16_t* slot16 = reinterpret_cast<uint16_t*>(list) + lane;
@@ -448,6 +548,10 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                 __syncwarp();
 
                 // ---- add, one stream after the other ----
+                // Streams in the fixed-width mode have a term for every element; they add, in their turn,
+                // those of the positions this round covers (all the remaining ones when no chain goes on).
+                const bool more = __any_sync(0xffffffffu, alive);
+                const uint32_t fixed_lo = done_pos, fixed_hi = more ? limit : kSB;
                 const uint32_t per_chain = 32u / S;         // lanes that share one chain's list
                 const uint32_t c = lane / per_chain, i0 = lane - c * per_chain;
                 for (uint32_t j = 0; j < gcount; ++j) {
@@ -476,7 +580,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                                 part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
                             }
                         }
-                    } else if (!fixed_done) {
+                    } else {
                         // fixed-width fields: every element of the warp's sub-blocks has one.  A lane
                         // takes 4 consecutive elements at a time: two words hold their 4 * width <= 40 bits
                         bool field_bad = false;
@@ -486,7 +590,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                         for (uint32_t grp = lane; grp < S * (kSB / 4u); grp += 32) {
                             const uint32_t q = grp >> 6, p = (grp & 63u) * 4u, sb = part * S + q;
                             if ((grp & 32u) == 0) describe_chain(G, T, sj, sb, &cf);   // a sub-block lasts two steps
-                            if (sb >= nsb_tile || sb * kSB + p >= tile_len) continue;
+                            if (sb >= nsb_tile || sb * kSB + p >= tile_len || p + 4u <= fixed_lo || p >= fixed_hi) continue;
                             const uint32_t nel = min(4u, tile_len - (sb * kSB + p));
                             const uint32_t bit = cf.cur + p * wd;
                             const uint32_t wi = bit >> 5;
@@ -501,7 +605,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                             for (uint32_t c = 0; c < 4; ++c) {
                                 const uint32_t field = (uint32_t)(win >> (64u - (c + 1u) * wd)) & ((1u << wd) - 1u);
                                 const uint32_t sym = field & smask;
-                                if (c < nel) {
+                                if (c < nel && p + c >= fixed_lo && p + c < fixed_hi) {
                                     if (sym >= sj.nlev) field_bad = true;
                                     else if (sym) {
                                         const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
@@ -515,8 +619,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     }
                     __syncwarp();
                 }
-                fixed_done = true;
-                if (!__any_sync(0xffffffffu, alive)) break;
+                if (!more) break;
             }
             // a well-formed chain ends exactly at its declared length, inside its sub-block, with known indices
             if (has_chain && !bad) bad = cur != end || pos > my_sn || (max_hi >> 9) + 1u >= si.nlev;
@@ -577,7 +680,12 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     }
     const size_t smem = decode_smem_bytes(P.group, P.K, warps);
     if (smem > kSmemMaxCta) return cudaErrorInvalidValue;
-    if (cudaMemsetAsync(&P.ws->dec_ticket, 0, sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;
+    if (cudaMemsetAsync(&P.ws->dec_ticket, 0, 2 * sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;   // ticket and the flag behind it
+    if (P.after_fixed) {
+        const uint64_t groups = (P.geo.d + 31) / 32, want_fixed = (groups + 255) / 256, cap_fixed = (uint64_t)sms * 4u;
+        decode_fixed_kernel<<<(unsigned)(want_fixed < cap_fixed ? want_fixed : cap_fixed), 256, 0, stream>>>(P);
+        if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
+    }
     const uint64_t want = (units + warps - 1) / warps;
     const uint64_t grid = want < (uint64_t)sms ? want : (uint64_t)sms;
     decode_kernel<<<(unsigned)grid, 32u * warps, smem, stream>>>(P);

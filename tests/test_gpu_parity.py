@@ -197,3 +197,55 @@ def test_dense_inputs_stay_inside_the_staging_buffers(d, bucket, s):
             assert bits == want_bits and np.array_equal(got, want)
         acc = gpu_decode([got], d, bucket, s)
         assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([got], d, bucket, s)[1].view(np.uint32))
+
+
+@pytest.mark.parametrize("d,bucket,s,ls", [(70001, 1024, 4, O.LEVELS_EXP), (8192 * 3 + 17, 8192, 2, O.LEVELS_EXP),
+                                           (200000, 65536, 4, O.LEVELS_EXP), (50000, 512, 7, O.LEVELS_EXP),
+                                           (33333, 256, 3, O.LEVELS_UNIFORM), (40000, 2048, 8, O.LEVELS_UNIFORM)])
+def test_fixed_width_streams_decoded_where_they_were_encoded(d, bucket, s, ls):
+    """Containers that stay on the device where the library wrote them: the decoder then knows (and
+    checks) that all of them are in the fixed-width mode and takes its simple path.  The sums must
+    equal the oracle's bit for bit, also when a buffer's content no longer is what the library wrote
+    there (an ERC container copied over a fixed-width one)."""
+    torch, nuq = require_cuda()
+    K = 3
+    flags_fixed = O.make_flags(O.NORM_L2, ls, O.MODE_FIXED)
+    flags_erc = O.make_flags(O.NORM_L2, ls, O.MODE_ERC)
+    gs = [_input(d, 100 + k) for k in range(K)]
+    nbytes = max(nuq.encode_bound(d, bucket, s, flags_fixed), nuq.encode_bound(d, bucket, s, flags_erc))
+    outs, host = [], []
+    for k in range(K):
+        out = torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda")
+        _, bits = nuq.encode(torch.from_numpy(gs[k]).cuda(), bucket, s, flags_fixed, 11 + k, 0, out=out)
+        outs.append(out)
+        host.append(out.cpu().numpy().view(np.uint32)[: int(bits.item()) // 32].copy())
+    acc = nuq.decode_accumulate(outs, d, bucket, s)
+    assert nuq.last_status() == 0
+    want = O.decode_accumulate(host, d, bucket, s)[1]
+    assert np.array_equal(acc.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    # same buffers, but the middle one now holds an ERC container of the same vector
+    erc, _ = gpu_encode(gs[1], bucket, s, flags_erc, seed=12, offset=0)
+    outs[1].zero_()
+    outs[1][: erc.size] = torch.from_numpy(erc.view(np.int32)).cuda()
+    host[1] = erc
+    acc = nuq.decode_accumulate(outs, d, bucket, s)
+    assert nuq.last_status() == 0
+    want = O.decode_accumulate(host, d, bucket, s)[1]
+    assert np.array_equal(acc.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("modes", [(O.MODE_ERC, O.MODE_FIXED, O.MODE_ERC), (O.MODE_FIXED, O.MODE_ERC, O.MODE_FIXED)])
+@pytest.mark.parametrize("d,bucket,s", [(20000, 256, 4), (50000, 1024, 5)])
+def test_mixed_modes_keep_the_stream_order_when_chains_take_several_rounds(modes, d, bucket, s):
+    """Dense ERC streams (every coordinate a token) are decoded in several rounds of positions; the
+    fixed-width streams of the same call must add their terms round by round too, or an element
+    would receive its terms out of stream order and the fp32 sum would differ."""
+    rng = np.random.default_rng(d)
+    streams = []
+    for k, mode in enumerate(modes):
+        g = np.where(rng.random(d) < 0.5, -1.0, 1.0).astype(np.float32) * (1.0 + 0.25 * rng.random(d).astype(np.float32))
+        streams.append(O.encode(g, bucket, s, O.make_flags(O.NORM_L2, O.LEVELS_EXP, mode), seed=k + 1, offset=0)[0])
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
