@@ -5,18 +5,20 @@
 // tile of up to 8192 output elements (32 coding sub-blocks), for G streams at a
 // time (G = 8, or 1 / 2 / 4 when K is smaller; S = 32 / G).  A warp keeps the
 // running sums of its S * 256 elements in shared memory and writes them to HBM
-// once; warps never wait for one another.  Per unit and group of streams:
+// once; warps never wait for one another, and the ticket of the next unit is
+// asked for while the current one is decoded.  Per unit and group of streams:
 //
 //   describe lane (j, q) reads, for stream j and sub-block q of the unit, the block
 //            offset, the norm and the sub-block token lengths, range-checks them and
 //            so knows where its chain of tokens starts and ends.
-//   stage    chains of at most 12 words (the usual case) are copied to shared memory, all
-//            loads in flight at once: the walk is a chain of dependent reads, which from
-//            global memory would wait for the cache at every step.  Longer chains are
-//            walked in place.
-//   decode   the lane walks that chain: ERC^-1 gap, sign bit, ERC^-1 level index, by
-//            table look-up on a 32-bit window (12-bit prefix table; longer codes take
-//            the loop of Algorithm 2).  All 32 chains of a warp advance in lock
+//   stage    every lane copies the next 12 words of its chain to shared memory, all
+//            loads in flight at once: the walk is a chain of dependent reads, which
+//            from global memory would wait for the cache at every step.  A lane that
+//            uses its words up stages the next ones and goes on.
+//   decode   the lane walks that chain: ERC^-1 gap by table look-up on a 32-bit window
+//            (12-bit prefix table), then sign and ERC^-1 level index (one 8-bit
+//            look-up for exponential levels, else the 12-bit table again; longer codes
+//            take the loop of Algorithm 2).  All 32 chains of a warp advance in lock
 //            step; the decoded (position, sign, index) triples go to a per-lane list.
 //   add      for j = 0 .. G-1 in order, the warp adds the listed values of
 //            stream j into its sums.  Entries of one stream hit distinct elements,
@@ -24,13 +26,16 @@
 //            its terms in ascending stream order: the sum is bit-reproducible and
 //            equals ((0 + q_0) + q_1) + ... .
 //
-// Lists hold 48 entries per staged chain (72 when nothing is staged).  Sparse streams
-// need one decode / add round per unit; when a chain may have more tokens than that,
-// the rounds advance through the sub-block that many positions at a time (a chain has
-// at most as many tokens there), and since all terms of an element fall into the same
-// round the order of its adds is unchanged.  Streams in the fixed-width mode are added
-// field by field in their turn.  One CTA per SM holds up to 25 such warps; they share
-// only the table and the validated stream headers.  Nothing spins.
+// Lists hold 48 entries per chain.  Sparse streams need one decode / add round per
+// unit; when the longest chain is expected to hold more tokens, the sub-block is split
+// evenly into rounds of positions, and a round whose list runs over is taken again with
+// half the positions.  All terms of an element fall into the same round, so the order
+// of its adds is unchanged; streams in the fixed-width mode add, in their turn, the
+// fields of the positions the round covers.  One CTA per SM holds up to 25 such warps;
+// they share only the tables and the validated stream headers.  Nothing spins.
+//
+// Calls whose streams are all in the fixed-width mode have no chains to walk; they are
+// served by a kernel of their own (decode_fixed_kernel below).
 #include <type_traits>
 
 #include "nuq_common.cuh"
