@@ -223,15 +223,17 @@ __device__ StreamHead read_head(const Geometry& G, const uint32_t* hdr) {
 // no tokens to walk, so a thread takes 32 consecutive elements (W words of every stream, never across a
 // bucket: buckets are multiples of 256 elements), adds the K dequantized values of each element in
 // stream order in registers and stores the 32 sums.  Same arithmetic and order as the general path.
-template <uint32_t W>
+template <uint32_t W, uint32_t LEVELSET>
 __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const StreamHead* heads) {
     const Geometry& G = P.geo;
     const uint64_t ngroups = (G.d + 31) / 32;
-    const uint32_t levelset = heads[0].levelset, nlev = heads[0].nlev;
+    const uint32_t nlev = heads[0].nlev;
+    const uint32_t exp_bias = (126u - G.s) << 23;           // exponent field of 2^(-1-s)
+    const float uni_scale = __uint_as_float((127u - G.s) << 23);
+    uint32_t max_sym = 0;
     const uint32_t rec_words = 1u + G.bucket * W / 32u;
     const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
     constexpr uint32_t fmask = (1u << W) - 1u, smask = (1u << (W - 1u)) - 1u;
-    bool bad = false;
     for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += (uint64_t)gridDim.x * blockDim.x) {
         const uint64_t e0 = 32 * grp, b = e0 / G.bucket;
         const uint32_t eb = (uint32_t)(e0 - b * G.bucket);                         // first element within its bucket
@@ -239,49 +241,57 @@ __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const St
         const uint32_t bucket_len = b == G.nb - 1 ? (uint32_t)last_len : G.bucket;
         const uint32_t avail = (bucket_len * W + 31u) / 32u - (eb / 32u) * W;      // field words of the record from here on
         float* dst = P.acc + e0;
+        // branch free: a zero symbol adds +0 (the sums never are -0, so that changes nothing), the
+        // largest symbol seen is checked once at the end; `whole`: all 32 elements exist
+        auto body = [&](auto whole) {
 #pragma unroll
-        for (uint32_t half = 0; half < 2; ++half) {         // 16 elements at a time: the sums stay in few registers
-            float acc[16];
+            for (uint32_t half = 0; half < 2; ++half) {     // 16 elements at a time: the sums stay in few registers
+                float acc[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
-            for (uint32_t k = 0; k < P.K; ++k) {
-                const uint32_t* rec = heads[k].hdr + kHeaderWords + b * rec_words;
-                const float norm = __uint_as_float(__ldg(rec));
-                const uint32_t* fw = rec + 1u + (eb / 32u) * W;
-                // the words that hold fields 16 * half .. 16 * half + 15
-                constexpr uint32_t kHalfWords = (16u * W + 31u) / 32u + 1u;
-                const uint32_t w0 = (16u * half * W) >> 5;
-                uint32_t words[kHalfWords + 1];
+                for (int i = 0; i < 16; ++i) acc[i] = 0.0f;
+                for (uint32_t k = 0; k < P.K; ++k) {
+                    const uint32_t* rec = heads[k].hdr + kHeaderWords + b * rec_words;
+                    const float norm = __uint_as_float(__ldg(rec));
+                    const uint32_t* fw = rec + 1u + (eb / 32u) * W;
+                    // the words that hold fields 16 * half .. 16 * half + 15
+                    constexpr uint32_t kHalfWords = (16u * W + 31u) / 32u + 1u;
+                    const uint32_t w0 = (16u * half * W) >> 5;
+                    uint32_t words[kHalfWords + 1];
 #pragma unroll
-                for (uint32_t j = 0; j < kHalfWords; ++j) words[j] = w0 + j < avail ? __ldg(fw + w0 + j) : 0u;
-                words[kHalfWords] = 0;
+                    for (uint32_t j = 0; j < kHalfWords; ++j) words[j] = w0 + j < avail ? __ldg(fw + w0 + j) : 0u;
+                    words[kHalfWords] = 0;
 #pragma unroll
-                for (uint32_t i = 0; i < 16; ++i) {
-                    const uint32_t bit = (16u * half + i) * W - 32u * w0, a = bit >> 5, sh = bit & 31u;
-                    const uint32_t field = sh + W <= 32u ? (words[a] >> (32u - sh - W)) & fmask
-                                                         : __funnelshift_l(words[a + 1], words[a], sh) >> (32u - W);
-                    const uint32_t sym = field & smask;
-                    if (16u * half + i < nel) {
-                        if (sym >= nlev) bad = true;
-                        else if (sym) {
-                            const float v = level_times_norm(norm, levelset, G.s, sym);
-                            acc[i] += (field >> (W - 1u)) ? -v : v;
+                    for (uint32_t i = 0; i < 16; ++i) {
+                        const uint32_t bit = (16u * half + i) * W - 32u * w0, a = bit >> 5, sh = bit & 31u;
+                        const uint32_t field = sh + W <= 32u ? (words[a] >> (32u - sh - W)) & fmask
+                                                             : __funnelshift_l(words[a + 1], words[a], sh) >> (32u - W);
+                        const uint32_t sym = field & smask;
+                        // exponential: l_j = 2^(j-1-s) (exact scaling);  uniform: l_k = k / 2^s
+                        const float level = LEVELSET == kLevelsExp ? __uint_as_float((sym << 23) + exp_bias)
+                                                                   : __fmul_rn((float)sym, uni_scale);
+                        const float mag = sym ? __fmul_rn(norm, level) : 0.0f;
+                        const float v = __uint_as_float(__float_as_uint(mag) ^ ((field << (32u - W)) & 0x80000000u));
+                        if (decltype(whole)::value || 16u * half + i < nel) {
+                            max_sym = max(max_sym, sym);
+                            acc[i] += v;
                         }
                     }
                 }
-            }
-            if (nel == 32u) {
+                if (decltype(whole)::value) {
 #pragma unroll
-                for (int i = 0; i < 16; i += 4)
-                    *reinterpret_cast<float4*>(dst + 16 * half + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
-            } else {
+                    for (int i = 0; i < 16; i += 4)
+                        *reinterpret_cast<float4*>(dst + 16 * half + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+                } else {
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (16u * half + (uint32_t)i < nel) dst[16 * half + i] = acc[i];
+                    for (int i = 0; i < 16; ++i)
+                        if (16u * half + (uint32_t)i < nel) dst[16 * half + i] = acc[i];
+                }
             }
-        }
+        };
+        if (nel == 32u) body(std::true_type());
+        else body(std::false_type());
     }
-    if (bad) latch_status(P.ws, kErrBadStream);
+    if (max_sym >= nlev) latch_status(P.ws, kErrBadStream);
 }
 
 // The kernel of that path.  It is launched when the library believes that all streams are in the
@@ -301,15 +311,24 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
         if (same && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0]) = 1;   // tell the general kernel
     }
     __syncthreads();
+    if (heads[0].levelset == kLevelsExp) {                  // s <= 14: at most 16 levels, 5 bits
+        switch (s_width) {
+            case 3: decode_all_fixed<3, kLevelsExp>(P, heads); break;
+            case 4: decode_all_fixed<4, kLevelsExp>(P, heads); break;
+            case 5: decode_all_fixed<5, kLevelsExp>(P, heads); break;
+            default: break;
+        }
+        return;
+    }
     switch (s_width) {
-        case 3: decode_all_fixed<3>(P, heads); break;
-        case 4: decode_all_fixed<4>(P, heads); break;
-        case 5: decode_all_fixed<5>(P, heads); break;
-        case 6: decode_all_fixed<6>(P, heads); break;
-        case 7: decode_all_fixed<7>(P, heads); break;
-        case 8: decode_all_fixed<8>(P, heads); break;
-        case 9: decode_all_fixed<9>(P, heads); break;
-        case 10: decode_all_fixed<10>(P, heads); break;
+        case 3: decode_all_fixed<3, kLevelsUniform>(P, heads); break;
+        case 4: decode_all_fixed<4, kLevelsUniform>(P, heads); break;
+        case 5: decode_all_fixed<5, kLevelsUniform>(P, heads); break;
+        case 6: decode_all_fixed<6, kLevelsUniform>(P, heads); break;
+        case 7: decode_all_fixed<7, kLevelsUniform>(P, heads); break;
+        case 8: decode_all_fixed<8, kLevelsUniform>(P, heads); break;
+        case 9: decode_all_fixed<9, kLevelsUniform>(P, heads); break;
+        case 10: decode_all_fixed<10, kLevelsUniform>(P, heads); break;
         default: break;
     }
 }
