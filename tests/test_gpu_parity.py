@@ -249,3 +249,19 @@ def test_mixed_modes_keep_the_stream_order_when_chains_take_several_rounds(modes
     assert rc == 0
     got = gpu_decode(streams, d, bucket, s)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("K", [9, 17])
+def test_more_streams_than_one_group(K):
+    """More than 8 streams are decoded in groups of 8, one group after the other, the last one
+    partly filled; the order of the adds is still the stream order across groups."""
+    d, bucket, s = 30000, 1024, 4
+    streams = []
+    for k in range(K):
+        mode = O.MODE_FIXED if k == 10 else O.MODE_ERC
+        streams.append(O.encode(_input(d, 7000 + k), bucket, s, O.make_flags(O.NORM_L2, O.LEVELS_EXP, mode),
+                                seed=k + 1, offset=0)[0])
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
