@@ -338,10 +338,18 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
 __host__ __device__ inline size_t decode_warp_offset(uint32_t K) {
     return (2u * ((1u << kLutBits) + (1u << kSignedBits)) + (size_t)K * sizeof(StreamHead) + 15u) & ~(size_t)15u;
 }
-__host__ __device__ inline size_t decode_warp_bytes(uint32_t group) {
-    return 4u * ((32u / group) * kSB + kWarpWords);
+// `sums_in_l2`: the running sums of a unit live in the output vector itself (see decode_kernel)
+__host__ __device__ inline size_t decode_warp_bytes(uint32_t group, bool sums_in_l2) {
+    return 4u * ((sums_in_l2 ? 0u : (32u / group) * kSB) + kWarpWords);
 }
 
+// SUMS_IN_L2 = false: a warp keeps the running sums of its S * 256 elements in shared memory and
+// stores them once (8 streams side by side: 4 KB per warp).  true: it zeroes its part of the output
+// vector and adds into it there, in the L2, with cache-global loads and stores; taken for fewer than
+// 8 streams, where the sums of a warp would need 8 to 32 KB of shared memory and only a few warps
+// would fit an SM, too few to hide the latency of the walk.  The order of the adds is the same.
+// (Taken for one or two streams side by side; with four, 17 warps fit and shared memory is faster.)
+template <bool SUMS_IN_L2>
 __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
     if (P.after_fixed && *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0])) return;   // the fixed-width kernel did it all
@@ -352,8 +360,8 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     uint16_t* lut = reinterpret_cast<uint16_t*>(dsm);                             // ERC^-1 of 12-bit prefixes
     uint16_t* lut2 = lut + (1u << kLutBits);                                      // sign + ERC^-1 of 7-bit prefixes
     StreamHead* heads = reinterpret_cast<StreamHead*>(lut2 + (1u << kSignedBits));   // [K]
-    float* accw = reinterpret_cast<float*>(dsm + decode_warp_offset(P.K) + warp * decode_warp_bytes(NG));   // S * 256 running sums
-    uint32_t* list = reinterpret_cast<uint32_t*>(accw + S * kSB);
+    float* accw = reinterpret_cast<float*>(dsm + decode_warp_offset(P.K) + warp * decode_warp_bytes(NG, SUMS_IN_L2));   // S * 256 running sums
+    uint32_t* list = reinterpret_cast<uint32_t*>(accw + (SUMS_IN_L2 ? 0u : S * kSB));
 
     for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) lut[i] = (uint16_t)erc_prefix_entry(i, kLutBits);
     for (uint32_t i = threadIdx.x; i < (1u << kSignedBits); i += blockDim.x) lut2[i] = (uint16_t)signed_index_entry(i);
@@ -362,8 +370,9 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
         heads[k] = read_head(G, P.streams[k]);
         if (!heads[k].ok) latch_status(P.ws, kErrBadStream);
     }
-    for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
-        *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (!SUMS_IN_L2)
+        for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
+            *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
 
     __syncthreads();                                        // table and headers are ready; from here on warps run alone
 
@@ -409,6 +418,25 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
         T.nsb_tile = (T.tile_len + kSB - 1) / kSB;
         const uint32_t tile_len = T.tile_len, nsb_tile = T.nsb_tile;
         const uint64_t elem0 = T.elem0;
+
+        // the unit's part of the output vector and how many of its S * 256 elements exist
+        float* const gsum = P.acc + elem0 + part * S * kSB;
+        const uint32_t unit_len = tile_len > part * S * kSB ? min(S * kSB, tile_len - part * S * kSB) : 0u;
+        if (SUMS_IN_L2) {
+            for (uint32_t i = lane * 4u; i < unit_len; i += 128u) {
+                if (i + 4u <= unit_len) __stcg(reinterpret_cast<float4*>(gsum + i), make_float4(0.f, 0.f, 0.f, 0.f));
+                else for (uint32_t e = i; e < unit_len; ++e) __stcg(gsum + e, 0.0f);
+            }
+            __syncwarp();
+        }
+        // sum[idx] += v for element idx of the unit (a malformed chain may name an element that does not exist)
+        auto add_to = [&](uint32_t idx, float v) {
+            if (SUMS_IN_L2) {
+                if (idx < unit_len) __stcg(gsum + idx, __ldcg(gsum + idx) + v);
+            } else {
+                accw[idx] += v;
+            }
+        };
 
         for (uint32_t g0 = 0; g0 < P.K; g0 += NG) {
             const uint32_t gcount = min(NG, P.K - g0);      // streams in this group
@@ -585,23 +613,44 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     const float norm_c = __shfl_sync(0xffffffffu, ch.norm, owner);
                     if (!sj.ok) continue;
                     if (sj.mode == kModeErc) {
-                        float* part = accw + c * kSB;
+                        const uint32_t part0 = c * kSB;      // first element of chain c's sub-block within the unit
                         if (!wide && sj.levelset == kLevelsExp) {
                             // value = +-norm * 2^(index - 1 - s): the exponent field is built from the entry
                             const uint16_t* src = reinterpret_cast<const uint16_t*>(list) + owner;
                             const uint32_t ebias = 127u - G.s;              // (index - 1) + ebias = biased exponent
-                            for (uint32_t i = i0; i < n_c; i += per_chain) {
-                                const uint32_t e = src[i * 32u];
-                                const float level = __uint_as_float(((e >> 9) + ebias) << 23);
-                                const float v = __fmul_rn(norm_c, level);
-                                part[e & 0xffu] += __uint_as_float(__float_as_uint(v) ^ ((e << 23) & 0x80000000u));
+                            if (SUMS_IN_L2) {
+                                // four entries at a time, loads before stores: the entries of one stream name
+                                // distinct elements, and an add in the L2 is a round trip
+                                for (uint32_t i = i0; i < n_c; i += 4u * per_chain) {
+                                    uint32_t idx[4];
+                                    float val[4], old[4];
+#pragma unroll
+                                    for (uint32_t u = 0; u < 4; ++u) {
+                                        const uint32_t ii = i + u * per_chain;
+                                        const uint32_t e = ii < n_c ? src[ii * 32u] : 0u;
+                                        const float v = __fmul_rn(norm_c, __uint_as_float(((e >> 9) + ebias) << 23));
+                                        val[u] = __uint_as_float(__float_as_uint(v) ^ ((e << 23) & 0x80000000u));
+                                        idx[u] = ii < n_c ? part0 + (e & 0xffu) : 0xFFFFFFFFu;
+                                        old[u] = idx[u] < unit_len ? __ldcg(gsum + idx[u]) : 0.0f;
+                                    }
+#pragma unroll
+                                    for (uint32_t u = 0; u < 4; ++u)
+                                        if (idx[u] < unit_len) __stcg(gsum + idx[u], old[u] + val[u]);
+                                }
+                            } else {
+                                for (uint32_t i = i0; i < n_c; i += per_chain) {
+                                    const uint32_t e = src[i * 32u];
+                                    const float level = __uint_as_float(((e >> 9) + ebias) << 23);
+                                    const float v = __fmul_rn(norm_c, level);
+                                    add_to(part0 + (e & 0xffu), __uint_as_float(__float_as_uint(v) ^ ((e << 23) & 0x80000000u)));
+                                }
                             }
                         } else {
                             for (uint32_t i = i0; i < n_c; i += per_chain) {
                                 const uint32_t e = wide ? list[i * 32u + owner]
                                                         : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * 32u + owner];
                                 const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
-                                part[e & 0xffu] += (e >> 8) & 1u ? -v : v;
+                                add_to(part0 + (e & 0xffu), (e >> 8) & 1u ? -v : v);
                             }
                         }
                     } else {
@@ -623,8 +672,6 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                             const uint32_t x2 = __ldg(cf.tok + min(wi + 2u, cf.last));
                             // 64 bits from the first field on
                             const uint64_t win = ((uint64_t)__funnelshift_l(x1, x0, bit) << 32) | __funnelshift_l(x2, x1, bit);
-                            float4 a = *reinterpret_cast<float4*>(accw + grp * 4u);
-                            float* av = reinterpret_cast<float*>(&a);
 #pragma unroll
                             for (uint32_t c = 0; c < 4; ++c) {
                                 const uint32_t field = (uint32_t)(win >> (64u - (c + 1u) * wd)) & ((1u << wd) - 1u);
@@ -633,11 +680,10 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                                     if (sym >= sj.nlev) field_bad = true;
                                     else if (sym) {
                                         const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
-                                        av[c] += (field >> (wd - 1u)) ? -v : v;
+                                        add_to(grp * 4u + c, (field >> (wd - 1u)) ? -v : v);
                                     }
                                 }
                             }
-                            *reinterpret_cast<float4*>(accw + grp * 4u) = a;
                         }
                             if (__any_sync(0xffffffffu, field_bad) && lane == 0) latch_status(P.ws, kErrBadStream);
                     }
@@ -652,7 +698,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
 
         // ---- write this warp's part of the tile once, and clear it for the next tile ----
         __syncwarp();
-        {
+        if (!SUMS_IN_L2) {
             const uint32_t first = part * S * kSB;
             float* dst = P.acc + elem0 + first;
             for (uint32_t i = lane * 4u; i < S * kSB; i += 128u) {
@@ -668,15 +714,17 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     }
 }
 
-static size_t decode_smem_bytes(uint32_t group, uint32_t K, uint32_t warps) {
-    return decode_warp_offset(K) + (size_t)warps * decode_warp_bytes(group);
+static size_t decode_smem_bytes(uint32_t group, uint32_t K, uint32_t warps, bool sums_in_l2) {
+    return decode_warp_offset(K) + (size_t)warps * decode_warp_bytes(group, sums_in_l2);
 }
 
 cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     constexpr size_t kSmemPerSm = 227u * 1024u, kSmemMaxCta = 227u * 1024u;
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMaxCta);
+        cudaError_t e = cudaFuncSetAttribute(decode_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMaxCta);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(decode_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemMaxCta);
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
@@ -685,7 +733,8 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     // rounds, and a round takes about as long as there are warps on the SM (the kernel is bound by
     // instruction issue): among the five largest warp counts take the one with the least rounds * warps,
     // the largest unless a smaller one saves 6 % or more.
-    const size_t fixed = decode_warp_offset(P.K) + 1024u, per_warp = decode_warp_bytes(P.group);
+    const bool sums_in_l2 = P.group < 4u;                  // 1 or 2 streams side by side
+    const size_t fixed = decode_warp_offset(P.K) + 1024u, per_warp = decode_warp_bytes(P.group, sums_in_l2);
     uint32_t wmax = kDecMaxWarps;
     while (wmax > 1 && fixed + wmax * per_warp > kSmemPerSm) --wmax;
     const uint64_t units = P.geo.ntiles * P.group;                          // warp-sized units of work
@@ -703,7 +752,7 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
             warps = w;
         }
     }
-    const size_t smem = decode_smem_bytes(P.group, P.K, warps);
+    const size_t smem = decode_smem_bytes(P.group, P.K, warps, sums_in_l2);
     if (smem > kSmemMaxCta) return cudaErrorInvalidValue;
     if (cudaMemsetAsync(&P.ws->dec_ticket, 0, 2 * sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;   // ticket and the flag behind it
     if (P.after_fixed) {
@@ -713,7 +762,8 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     }
     const uint64_t want = (units + warps - 1) / warps;
     const uint64_t grid = want < (uint64_t)sms ? want : (uint64_t)sms;
-    decode_kernel<<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
+    if (sums_in_l2) decode_kernel<true><<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
+    else decode_kernel<false><<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
     return cudaGetLastError();
 }
 
