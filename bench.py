@@ -301,8 +301,8 @@ def run_gpu(args):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures
 # summarised under profiles/ (the decoder's write count is short under ncu: its write-back
 # drains after the kernel has ended)
-ENCODE_TRAFFIC_BYTES = {"c3": 102.31e6 + 4.08e6}
-DECODE_TRAFFIC_BYTES = {"c3": 24.61e6 + 44.52e6}
+ENCODE_TRAFFIC_BYTES = {"c3": 102.31e6 + 3.78e6}
+DECODE_TRAFFIC_BYTES = {"c3": 24.67e6 + 44.29e6}
 
 
 def main():
