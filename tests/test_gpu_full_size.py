@@ -61,3 +61,16 @@ def test_c4_sized_down(bucket):
     assert rc == 0
     got = gpu_decode(streams, d, bucket, 4)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_c3_decode_of_eight_workers_as_benchmarked():
+    """The benchmark's decode call: eight distinct ResNet-50-sized gradients, eight streams side by
+    side (the instance of the kernel with the sums in shared memory, 25 warps per SM)."""
+    from paper_1908_06077_b200 import inputs
+    gs = [inputs.c3_input(k) for k in range(1, 9)]
+    d = gs[0].size
+    streams = [gpu_encode(g, 8192, 4, 0, seed=k + 1, offset=0)[0] for k, g in enumerate(gs)]
+    rc, want = O.decode_accumulate(streams, d, 8192, 4)
+    assert rc == 0
+    got = gpu_decode(streams, d, 8192, 4)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
