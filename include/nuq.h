@@ -52,6 +52,9 @@ typedef int nuq_status;
 #define NUQ_ERR_BAD_STREAM (-3)  /* a container failed validation inside nuq_decode_accumulate     */
 #define NUQ_ERR_CUDA (-4)        /* a CUDA runtime call failed (allocation, launch)                */
 #define NUQ_ERR_TIMEOUT (-5)     /* the encoder's cross-tile scan gave up waiting (bounded spin)   */
+#define NUQ_ERR_INTERNAL (-6)    /* an internal capacity check failed (a defect of the library)    */
+#define NUQ_WARN_NONFINITE 1     /* status word only: a bucket with a NaN, infinite or vanishing   *
+                                  * norm was written unquantized (all symbols zero, norm word kept) */
 
 /* norm_kind argument of nuq_encode: bit fields */
 #define NUQ_NORM_L2 0u            /* bits 0-7: Euclidean norm (Sec. 2), the paper's choice        */
@@ -61,6 +64,9 @@ typedef int nuq_status;
 #define NUQ_MODE_ERC (0u << 16)   /* bits 16-23: Elias-recursive token stream (App. A)            */
 #define NUQ_MODE_FIXED (1u << 16) /*             fixed-width fields ("4-bit" variant of Sec. 5)   */
 #define NUQ_TEST_NORMS (1u << 24) /* take bucket norms from nuq_set_test_norms (parity testing)   */
+#define NUQ_TEST_SHORT_PATIENCE (1u << 25) /* test hook: the cross-tile scan gives up after two  *
+                                   * polls instead of tens of milliseconds, so that a test can    *
+                                   * see NUQ_ERR_TIMEOUT without anything being withheld          */
 
 typedef struct nuq_info {
     uint64_t d;

@@ -22,6 +22,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 struct WsEntry {
     Workspace* ptr = nullptr;
     size_t bytes = 0;
+    bool clean = false;      // the scan state is all zero: set by the allocation, kept by every encode kernel
 };
 
 std::mutex g_mu;
@@ -53,7 +54,7 @@ bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geom
     if (d == 0 || d >= (1ull << 40) || !bucket_ok(bucket) || s < 1) return false;
     if (norm_kind > 1 || levelset > 1 || mode > 1) return false;
     if (s > (levelset == kLevelsExp ? 14u : 8u)) return false;
-    if (flags & ~(0x00ffffffu | NUQ_TEST_NORMS)) return false;
+    if (flags & ~(0x00ffffffu | NUQ_TEST_NORMS | NUQ_TEST_SHORT_PATIENCE)) return false;
     G->d = d;
     G->bucket = bucket;
     G->s = s;
@@ -107,9 +108,8 @@ uint32_t token_bits_bound(const Geometry& G, uint32_t elems, uint32_t buckets, b
     return tight < safe ? tight : safe;
 }
 
-// words of shared-memory staging one tile can need
+// words of shared-memory staging the records of one ERC tile can need
 uint32_t stage_words_for(const Geometry& G, bool norms_are_ours) {
-    if (G.mode == kModeFixed) return G.bucket <= kBLK ? G.blocks_per_tile * G.rec_words : kBLK * G.width / 32u;
     uint32_t head = 1u + (G.sb_per_block + 1u) / 2u + 1u;          // norm, lengths, padding
     return G.blocks_per_tile * head + (token_bits_bound(G, kBLK, G.blocks_per_tile, norms_are_ours) + 31u) / 32u;
 }
@@ -151,6 +151,7 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
         if (cudaMemset(p, 0, want) != cudaSuccess) return NUQ_ERR_CUDA;
         e.ptr = static_cast<Workspace*>(p);
         e.bytes = want;
+        e.clean = true;
         if (carried && cudaMemcpy(&e.ptr->status, &carried, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
             return NUQ_ERR_CUDA;
     }
@@ -173,34 +174,28 @@ struct EncodePlan {
     uint32_t want_grid;      // CTAs that give every SM its full share
 };
 
-static EncodePlan plan_encode(EncodeParams& P, int sms, bool norms_are_ours) {
+static EncodePlan plan_encode(EncodeParams& P, int sms, uint32_t flags) {
     const Geometry& G = P.geo;
+    const bool norms_are_ours = (flags & NUQ_TEST_NORMS) == 0;
     EncodePlan pl;
     pl.state_bytes = sizeof(Workspace) + 8 * (G.ntiles + (G.ntiles + 31) / 32);
     pl.norms_bytes = G.bucket > kBLK ? 4 * G.nb : 0;
-    P.stage_words = (stage_words_for(G, norms_are_ours) + 3u) & ~3u;
+    // a look-back wait polls this often (with a pause in between: tens of ms in all) before it gives up
+    P.patience = (flags & NUQ_TEST_SHORT_PATIENCE) ? 2u : 1u << 16;
+    P.window_words = 0;
+    P.stage_words = 0;
     if (G.mode == kModeErc) {
+        P.stage_words = (stage_words_for(G, norms_are_ours) + 3u) & ~3u;
         // a warp's 1024 elements lie in at most this many buckets
         const uint32_t warp_elems = kBLK / kEncWarps;
         // (tiles start at bucket boundaries and a warp's part at a multiple of 1024 elements)
         const uint32_t warp_buckets = G.bucket >= warp_elems ? (G.bucket % warp_elems == 0 ? 1u : 2u)
                                                              : (warp_elems % G.bucket == 0 ? warp_elems / G.bucket : warp_elems / G.bucket + 1u);
         P.window_words = (token_bits_bound(G, warp_elems, warp_buckets, norms_are_ours) + 31u) / 32u + 4u;
-        const uint32_t list_words = G.levelset == kLevelsExp ? kEncChunk / 2u : kEncChunk;   // 16- or 32-bit entries
-        P.warp_smem_words = (P.window_words + list_words + 3u) & ~3u;
-    } else {
-        P.window_words = 0;
-        P.warp_smem_words = 0;
     }
-    // two staged tiles let the writer warp lag one tile behind the workers; a third one, taken when
-    // it costs no resident CTA, lets it lag two
-    P.stages = G.mode == kModeErc ? 2u : 1u;
-    int per_sm = encode_blocks_per_sm(P);
-    if (G.mode == kModeErc) {
-        P.stages = 3;
-        if (encode_blocks_per_sm(P) < per_sm) P.stages = 2;
-    }
-    if (per_sm < 1) per_sm = 1;
+    int best = encode_blocks_per_sm(P);                     // resident CTAs per SM: what shared memory and registers allow
+    if (best > kEncMaxBlocks) best = kEncMaxBlocks;
+    const int per_sm = best < 1 ? 1 : best;
     const uint64_t cap = (uint64_t)sms * (uint64_t)per_sm;
     pl.want_grid = (uint32_t)(G.ntiles < cap ? G.ntiles : cap);
     return pl;
@@ -210,16 +205,21 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, bool norms_are_ours) {
 // enqueues the kernels.  `ws` must hold pl.state_bytes + pl.norms_bytes.
 static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const float* g, uint32_t norm_kind,
                                  uint64_t seed, uint64_t offset, void* out, uint64_t* out_bits, Workspace* ws,
-                                 int dev, cudaStream_t stream) {
+                                 bool* ws_clean, int dev, cudaStream_t stream) {
     Geometry& G = P.geo;
     const bool test_norms = (norm_kind & NUQ_TEST_NORMS) != 0;
     if (!g_lut_ready.count(dev)) {
         if (upload_erc_lut() != cudaSuccess) return NUQ_ERR_CUDA;
         g_lut_ready.insert(dev);
     }
-    if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, pl.state_bytes - kWorkspaceClearFrom,
-                        stream) != cudaSuccess)
-        return NUQ_ERR_CUDA;
+    // The encode kernel leaves its scan state zeroed when it ends, so a clearing pass is needed only where
+    // that cannot be relied on (ws_clean == nullptr: always clear; *ws_clean false: an earlier launch failed).
+    if (ws_clean == nullptr || !*ws_clean) {
+        if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, pl.state_bytes - kWorkspaceClearFrom,
+                            stream) != cudaSuccess)
+            return NUQ_ERR_CUDA;
+        if (ws_clean) *ws_clean = true;
+    }
 
     P.g = g;
     P.norms_in = nullptr;
@@ -239,7 +239,10 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
         P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
     }
-    if (launch_encode(P, stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (launch_encode(P, stream) != cudaSuccess) {
+        if (ws_clean) *ws_clean = false;
+        return NUQ_ERR_CUDA;
+    }
     // remember the mode of the container at this address: a hint for the decoder's choice of kernels,
     // checked against the header on the device
     if (g_container_mode.size() > 4096) g_container_mode.clear();
@@ -281,12 +284,13 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
-    const EncodePlan pl = plan_encode(P, device_sms(dev), (norm_kind & NUQ_TEST_NORMS) == 0);
+    const EncodePlan pl = plan_encode(P, device_sms(dev), norm_kind);
     P.grid = pl.want_grid;
     Workspace* ws = nullptr;
     nuq_status st = get_workspace(stream, pl.state_bytes + pl.norms_bytes, &ws, &dev);
     if (st != NUQ_OK) return st;
-    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, dev, stream);
+    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, &g_ws[std::make_pair(dev, stream)].clean,
+                          dev, stream);
 }
 
 nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind,
@@ -298,7 +302,7 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
     if (!encode_args_ok(g, d, bucket, s, norm_kind, out, out_bits, &G)) return NUQ_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
-    const EncodePlan pl = plan_encode(P, device_sms(dev), (norm_kind & NUQ_TEST_NORMS) == 0);
+    const EncodePlan pl = plan_encode(P, device_sms(dev), norm_kind);
     if (pl.state_bytes + pl.norms_bytes > kStaticScratchBytes) return NUQ_ERR_CAPACITY;   // vector too long for the array
     P.grid = pl.want_grid;
     auto it = g_static_ws.find(dev);
@@ -311,7 +315,8 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
         }
         it = g_static_ws.emplace(dev, static_cast<Workspace*>(p)).first;
     }
-    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, it->second, dev, stream);
+    // the array is shared by every stream of the device: it is cleared before every call
+    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, it->second, nullptr, dev, stream);
 }
 
 nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,

@@ -15,15 +15,15 @@ constexpr uint32_t kMaxK = 64;
 
 constexpr int kEncThreads = 256;          // 8 warps share a tile, 1024 elements each
 constexpr int kEncWarps = kEncThreads / 32;
-constexpr int kEncMinBlocks = 4;          // resident CTAs per SM the encoder is compiled for
-constexpr uint32_t kEncChunk = 256;       // elements a warp quantizes before it generates their tokens
+constexpr int kEncMinBlocks = 4;          // resident CTAs per SM the encoder is compiled for (register cap) ...
+constexpr int kEncMaxBlocks = 4;          // ... and the most it is launched with
 
 enum : uint32_t { kNormL2 = 0, kNormLinf = 1 };
 enum : uint32_t { kLevelsExp = 0, kLevelsUniform = 1 };
 enum : uint32_t { kModeErc = 0, kModeFixed = 1 };
 
-// status latched by kernels (most negative wins)
-enum : int { kOk = 0, kErrBadStream = -3, kErrTimeout = -5 };
+// status latched by kernels (most negative wins; the warning only when nothing else is latched)
+enum : int { kOk = 0, kWarnNonfinite = 1, kErrBadStream = -3, kErrTimeout = -5, kErrInternal = -6 };
 
 // look-back tile states, kept in the two top bits of a 64-bit word
 constexpr uint64_t kTileAggregate = 1ull << 62;
@@ -73,10 +73,9 @@ struct EncodeParams {
     Workspace* ws;
     uint64_t seed, offset;
     uint32_t round_keys[20]; // Philox4x32-10 key schedule of `seed`: (k0, k1) of round 0, 1, ..., 9
-    uint32_t stage_words;    // shared-memory image of a tile's records (multiple of 4)
-    uint32_t stages;         // staged tile images per CTA (ERC: 2 or 3; fixed width: 1)
-    uint32_t window_words;   // shared-memory token string of one warp
-    uint32_t warp_smem_words;// shared memory of one warp (token string, token list)
+    uint32_t stage_words;    // ERC: shared-memory image of a tile's records (multiple of 4); a CTA holds two
+    uint32_t window_words;   // ERC: shared-memory token string of one warp and tile; a warp holds two
+    uint32_t patience;       // polls a look-back wait may take before it gives up
     uint32_t grid;           // CTAs to launch
 };
 
@@ -90,7 +89,10 @@ struct DecodeParams {
     Workspace* ws;
 };
 
-__device__ __forceinline__ void latch_status(Workspace* ws, int code) { atomicMin(&ws->status, code); }
+__device__ __forceinline__ void latch_status(Workspace* ws, int code) {
+    if (code > 0) atomicCAS(&ws->status, 0, code);          // a warning never hides an error
+    else atomicMin(&ws->status, code);
+}
 
 __device__ __forceinline__ uint32_t lane_id() { return threadIdx.x & 31u; }
 

@@ -49,7 +49,6 @@ constexpr uint32_t kStageWords = 12;                    // token words per chain
 constexpr uint32_t kStagedListWords = kWarpWords - 32u * kStageWords;   // what is left for the lists then (48 entries per chain)
 constexpr uint32_t kStageSoftBits = 32u * (kStageWords - 2u);   // a lane stops here when its chain goes on behind the staged words
 constexpr uint32_t kDecMaxWarps = 25;                   // warps per CTA = per SM (they share the table and the stream heads only)
-constexpr uint32_t kMaxGroup = 8;                       // streams decoded side by side
 
 // One Elias-recursive integer from the top of a 64-bit MSB-first window (Algorithm 2,
 // decoding): N = 1; while the next bit is 1, read that bit plus N more as the new N.

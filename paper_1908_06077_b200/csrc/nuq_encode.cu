@@ -1,37 +1,34 @@
 // ENCODE of NUQSGD (App. A) for one gradient vector: bucket norm, stochastic
-// quantization (Definition 1) and Elias-recursive token packing in one kernel
-// that reads the gradient from HBM exactly once.
+// quantization (Definition 1) and Elias-recursive token packing (Algorithm 2) in one
+// kernel that reads the gradient from HBM exactly once.
 //
 // A persistent CTA takes tiles of up to 8192 consecutive elements (whole buckets, or
-// one 8192-element coding block of a wider bucket) by ticket.  Eight worker warps
-// encode the tile; in the ERC mode a ninth warp, the writer, finds the tile's place
-// in the stream and copies it out, so the workers never wait for other CTAs.
-// The tile's bytes are brought into shared memory by one bulk asynchronous copy
-// (TMA, completion on an mbarrier); the copy of the next tile is started as soon
-// as the current tile has been quantized, so HBM latency hides behind the packing
-// of the current tile and behind the other CTAs of the SM.  Per tile:
-//   1. each warp reduces the squares (fp64) of its 1024 elements per sub-block;
-//      after one barrier every warp derives the bucket norms it needs;
-//   2. each warp quantizes its elements 256 at a time (one 128-bit shared-memory
-//      load and one Philox block per lane and 128-element row), compacts the
-//      nonzero symbols with ballots into a dense list, and turns that list into
-//      tokens, 32 per step, appended to the warp's own bit string;
-//   3. after a second barrier every warp runs the same small scan over the 32
-//      sub-block lengths, which gives the layout of the tile's records, and
-//      shifts its strings to their place in one of two staged tile images; the
-//      tile's size is announced to the tiles behind it at once;
-//   4. the writer warp, woken through a named barrier, sums the sizes announced
-//      by the tile's predecessors (two-level decoupled look-back: single tiles
-//      within a group of 32, whole groups before that; bounded waits), copies the
-//      staged image to its place, writes the block offsets and hands the stage
-//      back through a second named barrier.  The workers meet the writer again
-//      only two tiles later, when they need that stage.
-// In the fixed-width mode the fields go straight to their known place and there
-// is no writer warp.  Counters and the container header are written once per CTA,
-// the header by whichever CTA finishes last.
-//
-// The kernel is bound by instruction issue, not by HBM: the quantizer is branch
-// free and all per-symbol work runs on dense lists.
+// one 8192-element coding block of a wider bucket) by ticket.  The tile's bytes are
+// brought into one of two shared-memory buffers by a bulk asynchronous copy (TMA,
+// completion on an mbarrier); the copy of the next tile runs while the current one
+// is encoded.  Eight worker warps own 1024 elements (four 256-element coding
+// sub-blocks) of the tile each.  Per tile a worker
+//   1. adds up the squares (fp64) of its elements per sub-block; whichever warp is
+//      done last turns the partial sums into the tile's bucket norms, once for the
+//      whole CTA, before the only CTA barrier of the tile;
+//   2. per sub-block: quantizes 8 elements per lane (two Philox blocks), compacts the
+//      nonzero symbols into a dense list (one warp scan of per-lane counts; the list
+//      lies over the sub-block's own, already consumed, input bytes) and turns the list
+//      into tokens ERC(gap) sign ERC(index), 32 per step, appended to the warp's own
+//      bit window (two windows per warp, used in turn);
+//   3. (ERC mode) shifts its strings of the PREVIOUS tile to their place in a staged
+//      image of that tile, which has been laid out in the meantime.
+// In the ERC mode a ninth warp, the writer, does everything that concerns a tile as a
+// whole: the scan over its 32 sub-block lengths (the layout of its records), the block
+// heads, the announcement of its size to the tiles behind it and, once the workers have
+// moved their strings, the tile's place in the stream (two-level decoupled look-back
+// over tile and group sizes, every wait bounded), the copy of the image to the stream
+// and the block offsets.  Workers and writer meet through named barriers on which one
+// side only arrives, so the workers never wait for other CTAs.
+// In the fixed-width mode there is no writer: a lane packs the fields of its eight
+// elements, two lanes exchange halves, and every lane stores one finished word.
+// Counters and the container header are written once per CTA, the header by whichever
+// CTA finishes last.
 #include "nuq_common.cuh"
 #include "nuq_launch.h"
 
@@ -92,13 +89,14 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 //   index e + 1 + [u < p].  For y < 1 the same expression is at most 1, and it is 1
 //   only if u < y as well.
 // y < 1 (r in [0, 2^-s]): p = y, and u < y  <=>  float(m) < y 2^24 (both sides exact).
-// With up = [float(m) < y 2^24] (always true for y >= 1) the index is max(hi, 1) if up, else 0.
+// With up = [float(m) < y 2^24] (always true for y >= 1) the index is max(hi, 1) if up, else 0; the
+// maximum is taken on y itself (max(y, 1) has index 1 and no carry), where it is a cheap float operation.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t quantize_exp(float v, float inv, float top, uint32_t word) {
     const float y = fminf(__fmul_rn(fabsf(v), inv), top);
-    const int hi = (int)(__float_as_uint(y) + (0x007FFFFFu - 0x3F000000u) - (word >> 9)) >> 23;
+    const uint32_t hi = (__float_as_uint(fmaxf(y, 1.0f)) + (0x007FFFFFu - 0x3F000000u) - (word >> 9)) >> 23;
     const bool up = __uint2float_rn(word >> 8) < __fmul_rn(y, 16777216.0f);
-    return up ? (uint32_t)max(hi, 1) : 0u;                  // no round-up: y < 1 and the index is 0
+    return up ? hi : 0u;                                    // no round-up: y < 1 and the index is 0
 }
 
 // Uniform levels k / 2^s:  p = y - floor(y).
@@ -123,6 +121,45 @@ __device__ __forceinline__ void or_bits(uint32_t* dst, uint32_t bitpos, uint64_t
     if (w2) atomicOr(dst + w + 2, w2);
 }
 
+// OR `nbits` (0..32) right-aligned bits of `value` into the MSB-first bit string `dst` at `bitpos`.
+// Two words are touched unconditionally (a zero is OR-ed when there is nothing to add).
+__device__ __forceinline__ void or_bits32(uint32_t* dst, uint32_t bitpos, uint32_t value, uint32_t nbits) {
+    const uint32_t a = nbits ? value << (32u - nbits) : 0u;
+    const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
+    atomicOr(dst + w, a >> sh);
+    atomicOr(dst + w + 1, __funnelshift_r(0u, a, sh));
+}
+
+// OR the left-aligned bits of `a` (zero beyond its last bit) into the MSB-first bit string `dst` at
+// `bitpos`.  Two words are touched unconditionally (a zero is OR-ed when there is nothing to add).
+__device__ __forceinline__ void or_bits_left(uint32_t* dst, uint32_t bitpos, uint32_t a) {
+    const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
+    atomicOr(dst + w, a >> sh);
+    atomicOr(dst + w + 1, __funnelshift_r(0u, a, sh));
+}
+
+// 32 bits of the MSB-first bit string `src` starting at bit `sbit` (>= -31); bits before
+// the string read as garbage and must be masked by the caller.
+__device__ __forceinline__ uint32_t bits_at(const uint32_t* src, int sbit) {
+    if (sbit < 0) return src[0] >> (uint32_t)(-sbit);
+    const uint32_t w = (uint32_t)sbit >> 5;
+    return __funnelshift_l(src[w + 1], src[w], (uint32_t)sbit);
+}
+
+// Inclusive warp scan; the shuffle's own range predicate guards the add.
+__device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .u32 t;\n\t"
+            "shfl.sync.up.b32 t|p, %0, %1, 0, 0xffffffff;\n\t"
+            "@p add.u32 %0, %0, t;\n\t}"
+            : "+r"(v)
+            : "r"(o));
+    }
+    return v;
+}
+
 __device__ __forceinline__ uint64_t ld_volatile_u64(const uint64_t* p) {
     return *reinterpret_cast<const volatile uint64_t*>(p);
 }
@@ -130,6 +167,7 @@ __device__ __forceinline__ void st_volatile_u64(uint64_t* p, uint64_t v) {
     *reinterpret_cast<volatile uint64_t*>(p) = v;
 }
 
+// ---------------------------------------------------------------------------
 // Two-level decoupled look-back over tile payload sizes, run by one warp.  Returns the
 // exclusive prefix (words) of `tile`, or sets *failed.  Every wait is bounded.
 //
@@ -142,38 +180,39 @@ __device__ __forceinline__ void st_volatile_u64(uint64_t* p, uint64_t v) {
 //                   the group's last tile
 // A tile sums the sizes of the tiles before it in its own group (one load per lane), then
 // walks back over whole groups, 64 per step, to the nearest one that knows its prefix.
+// A wait that runs out of patience poisons the tile's own words, so that the tiles behind it
+// give up at once instead of spending their own patience one after the other.
+// ---------------------------------------------------------------------------
 constexpr uint32_t kGroupTiles = 32;
 constexpr uint32_t kGroupCountShift = 48;
 constexpr uint64_t kGroupSumMask = (1ull << kGroupCountShift) - 1;
 
-// The workers' side: tile `tile` takes `words` words.
 __device__ __forceinline__ void announce_tile(uint64_t* tile_state, uint64_t* group_state, uint64_t tile, uint32_t words) {
     st_volatile_u64(tile_state + tile, kTileAggregate | words);
     atomicAdd(reinterpret_cast<unsigned long long*>(group_state + tile / kGroupTiles),
               (1ull << kGroupCountShift) | (unsigned long long)words);
 }
 
-// One more poll of a look-back wait; false when the patience is used up (tens of ms).
-__device__ __forceinline__ bool lookback_backoff(Workspace* ws, uint32_t& polls) {
-    if (++polls > (1u << 16)) {
-        if (lane_id() == 0) latch_status(ws, kErrTimeout);
-        return false;
-    }
+// One more poll of a look-back wait; false when the patience is used up.
+__device__ __forceinline__ bool lookback_backoff(uint32_t patience, uint32_t& polls) {
+    if (++polls > patience) return false;
     __nanosleep(polls < 64 ? 250 : 1000);                   // a waiting warp should not eat issue slots
     return true;
 }
 
-__device__ uint64_t tile_lookback(Workspace* ws, const uint64_t* tile_state, uint64_t* group_state, uint64_t tile,
-                                  uint64_t ntiles, uint32_t words, bool* failed) {
+__device__ uint64_t tile_lookback(const EncodeParams& P, uint64_t* tile_state, uint64_t* group_state, uint64_t tile,
+                                  uint32_t words, bool* failed) {
     const uint32_t lane = lane_id();
+    const uint64_t ntiles = P.geo.ntiles;
     const uint64_t grp = tile / kGroupTiles;
     const uint32_t r = (uint32_t)(tile % kGroupTiles);      // tiles of the group before this one
     uint32_t polls = 0;
     uint64_t exclusive = 0;
-    *failed = true;
+    bool ok = true;
     // ---- the tiles before this one in its own group ----
     for (;;) {
         const uint64_t v = lane < r ? ld_volatile_u64(tile_state + grp * kGroupTiles + lane) : kTileAggregate;
+        if (__any_sync(0xffffffffu, (v >> 62) == 3)) { ok = false; break; }             // a predecessor gave up
         const uint32_t missing = __ballot_sync(0xffffffffu, (v >> 62) != 1);
         if (!missing) {
             exclusive = __reduce_add_sync(0xffffffffu, (uint32_t)v);           // a tile has far fewer than 2^27 words
@@ -181,15 +220,16 @@ __device__ uint64_t tile_lookback(Workspace* ws, const uint64_t* tile_state, uin
         }
         // wait for the first missing one alone, then look at all of them again
         const uint64_t* p = tile_state + grp * kGroupTiles + (__ffs(missing) - 1);
-        while ((ld_volatile_u64(p) >> 62) != 1)
-            if (!lookback_backoff(ws, polls)) return 0;
+        while (ok && (ld_volatile_u64(p) >> 62) == 0) ok = lookback_backoff(P.patience, polls);
+        if (!ok) break;
     }
     // ---- whole groups, nearest first: lane l looks at groups base - l and base - 32 - l ----
     int64_t base = (int64_t)grp - 1;
-    while (base >= 0) {
+    while (ok && base >= 0) {
         const int64_t i0 = base - (int64_t)lane, i1 = i0 - 32;
         const uint64_t v0 = i0 >= 0 ? ld_volatile_u64(group_state + i0) : kTilePrefix;    // before group 0: prefix 0
         const uint64_t v1 = i1 >= 0 ? ld_volatile_u64(group_state + i1) : kTilePrefix;
+        if (__any_sync(0xffffffffu, (v0 >> 62) == 3 || (v1 >> 62) == 3)) { ok = false; break; }
         const bool p0 = (v0 >> 62) == 2, p1 = (v1 >> 62) == 2;                    // knows its prefix
         const bool n0 = !p0 && (v0 >> kGroupCountShift) != kGroupTiles;           // still collecting (earlier groups are full ones)
         const bool n1 = !p1 && (v1 >> kGroupCountShift) != kGroupTiles;
@@ -202,8 +242,8 @@ __device__ uint64_t tile_lookback(Workspace* ws, const uint64_t* tile_state, uin
             const uint64_t* p = group_state + (base - (int64_t)first_n);
             for (;;) {
                 const uint64_t v = ld_volatile_u64(p);
-                if ((v >> 62) == 2 || (v >> kGroupCountShift) == kGroupTiles) break;
-                if (!lookback_backoff(ws, polls)) return 0;
+                if ((v >> 62) >= 2 || (v >> kGroupCountShift) == kGroupTiles) break;
+                if (!lookback_backoff(P.patience, polls)) { ok = false; break; }
             }
             continue;
         }
@@ -217,22 +257,27 @@ __device__ uint64_t tile_lookback(Workspace* ws, const uint64_t* tile_state, uin
         base -= 64;
     }
     // ---- whoever places the last tile of a group tells the later groups where it ends ----
-    if (r == kGroupTiles - 1u || tile == ntiles - 1) {
+    const bool closes_group = r == kGroupTiles - 1u || tile == ntiles - 1;
+    if (ok && closes_group) {
         const uint64_t members = tile == ntiles - 1 ? r + 1u : kGroupTiles;
         for (;;) {                                          // every member's size has been added (they were all seen above)
             const uint64_t v = ld_volatile_u64(group_state + grp);
             if ((v >> kGroupCountShift) == members) break;
-            if (!lookback_backoff(ws, polls)) return 0;
+            if (!lookback_backoff(P.patience, polls)) { ok = false; break; }
         }
-        if (lane == 0) st_volatile_u64(group_state + grp, kTilePrefix | (exclusive + words));
+        if (ok && lane == 0) st_volatile_u64(group_state + grp, kTilePrefix | (exclusive + words));
     }
-    *failed = false;
+    if (!ok && lane == 0) {
+        latch_status(P.ws, kErrTimeout);
+        st_volatile_u64(tile_state + tile, kTilePoison);
+        if (closes_group) st_volatile_u64(group_state + grp, kTilePoison);
+    }
+    *failed = !ok;
     return exclusive;
 }
 
 // ---------------------------------------------------------------------------
-// Bulk asynchronous copy (TMA, untiled form) and its mbarrier.  One CTA-local
-// barrier, never a cluster multicast.
+// Bulk asynchronous copy (TMA, untiled form) and its mbarrier.  CTA-local barriers only.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -276,31 +321,14 @@ struct Sym {
     static constexpr uint32_t kMask = (1u << kBits) - 1u;
 };
 
-// OR `nbits` (0..32) right-aligned bits of `value` into the MSB-first bit string `dst` at `bitpos`.
-// Two words are touched unconditionally (a zero is OR-ed when there is nothing to add).
-__device__ __forceinline__ void or_bits32(uint32_t* dst, uint32_t bitpos, uint32_t value, uint32_t nbits) {
-    const uint32_t a = nbits ? value << (32u - nbits) : 0u;
-    const uint32_t w = bitpos >> 5, sh = bitpos & 31u;
-    atomicOr(dst + w, a >> sh);
-    atomicOr(dst + w + 1, __funnelshift_r(0u, a, sh));
-}
-
-// 32 bits of the MSB-first bit string `src` starting at bit `sbit` (>= -31); bits before
-// the string read as garbage and must be masked by the caller.
-__device__ __forceinline__ uint32_t bits_at(const uint32_t* src, int sbit) {
-    if (sbit < 0) return src[0] >> (uint32_t)(-sbit);
-    const uint32_t w = (uint32_t)sbit >> 5;
-    return __funnelshift_l(src[w + 1], src[w], (uint32_t)sbit);
-}
-
 constexpr uint32_t kWarpElems = kBLK / kEncWarps;   // 1024 elements of a tile per warp (4 sub-blocks)
-constexpr uint32_t kChunk = kEncChunk;              // elements quantized before their tokens are generated
-constexpr uint32_t kChunkRows = kChunk / 128;
 
-// Named CTA barriers.  The 8 worker warps meet at kBarWork; the writer warp (ERC mode) and the
-// workers hand the two staged tiles back and forth through kBarStaged + b (workers arrive, the
-// writer waits) and kBarFree + b (the writer arrives, workers wait).
-constexpr uint32_t kBarWork = 1, kBarStaged = 2, kBarFree = 5;     // kBarStaged + b, kBarFree + b for stage b < 3
+// Named CTA barriers.  The 8 worker warps meet at kBarWork once per tile.  In the ERC mode the workers and the writer warp pass
+// a tile k from hand to hand through three barriers with index k & 1:
+//   kBarDone    the workers arrive when their strings of tile k are complete, the writer waits;
+//   kBarLayout  the writer arrives when it has laid the tile out, the workers wait (a tile later);
+//   kBarMerged  the workers arrive when they have moved their strings into the image, the writer waits.
+constexpr uint32_t kBarWork = 1, kBarDone = 2, kBarLayout = 4, kBarMerged = 6;
 constexpr uint32_t kEncAllThreads = kEncThreads + 32;      // ERC mode: workers + the writer warp
 template <uint32_t ID, uint32_t COUNT>
 __device__ __forceinline__ void bar_sync() {
@@ -311,45 +339,65 @@ __device__ __forceinline__ void bar_arrive() {
     __threadfence_block();
     asm volatile("bar.arrive %0, %1;" ::"n"(ID), "n"(COUNT) : "memory");
 }
-// the pair of barriers of stage b (0, 1 or 2); immediate barrier numbers, so that the kernel claims only those it uses
+// the barrier BASE + p of tile parity p; immediate barrier numbers, so that the kernel claims only those it uses
 template <uint32_t BASE>
-__device__ __forceinline__ void stage_sync(uint32_t b) {
-    if (b == 0) bar_sync<BASE, kEncAllThreads>();
-    else if (b == 1) bar_sync<BASE + 1, kEncAllThreads>();
-    else bar_sync<BASE + 2, kEncAllThreads>();
+__device__ __forceinline__ void pair_sync(uint32_t p) {
+    if (p == 0) bar_sync<BASE, kEncAllThreads>();
+    else bar_sync<BASE + 1, kEncAllThreads>();
 }
 template <uint32_t BASE>
-__device__ __forceinline__ void stage_arrive(uint32_t b) {
-    if (b == 0) bar_arrive<BASE, kEncAllThreads>();
-    else if (b == 1) bar_arrive<BASE + 1, kEncAllThreads>();
-    else bar_arrive<BASE + 2, kEncAllThreads>();
+__device__ __forceinline__ void pair_arrive(uint32_t p) {
+    if (p == 0) bar_arrive<BASE, kEncAllThreads>();
+    else bar_arrive<BASE + 1, kEncAllThreads>();
 }
+
+// Geometry of a tile, worked out once by the thread that took its ticket.
+struct TileInfo {
+    unsigned long long tile;                               // >= ntiles: there is no such tile
+    unsigned long long elem0;                              // first element
+    unsigned long long first_block;                        // first coding block (ERC) / bucket (narrow buckets)
+    unsigned long long bucket_idx;                         // wide buckets: the bucket the tile lies in
+    uint32_t tile_len, nsb;                                // elements, sub-blocks
+    uint32_t bib;                                          // wide buckets: which 8192-element block of its bucket
+    uint32_t rec_len;                                      // wide buckets: elements of that bucket
+};
+
+// What the workers and the writer tell one another about a tile (ERC mode).
+struct TileMeta {
+    unsigned long long tile;
+    uint32_t nsb, pad;
+    uint32_t sb_bits[32];                                  // token bits of each sub-block ...
+    uint32_t sb_src[32];                                   // ... and where they start in the owning warp's window
+    uint32_t blk_norm[32];                                 // norm word of each coding block of the tile
+    uint32_t bitoff[32];                                   // written by the writer: where each sub-block's string goes in the image
+    uint32_t wnnz[kEncWarps];                              // nonzero symbols each warp produced
+};
 
 // A tile whose records are staged in shared memory and whose place in the stream is not
 // yet known.
 struct Pending {
     unsigned long long tile;
-    uint32_t words, nblk, code_bits, nnz, valid, pad;
+    uint32_t words, nblk, code_bits, nnz;
     uint32_t blk_wordoff[32];                              // word offset of block bi within the tile
 };
 
-// What a CTA has written so far (shared memory; updated by one thread at a time, CTA barriers in between).
+// What a CTA has written so far (shared memory; updated by one thread at a time).
 struct CtaTotals {
     uint64_t nnz, code_bits;
-    uint32_t tiles, stop;                                  // stop: iterations the workers ran (set when they leave)
+    uint32_t tiles, stop;                                  // stop: tiles the workers encoded (set when they leave)
 };
 
 // Bookkeeping of a CTA that has written all its tiles: counters, and the container header by
-// whichever CTA finishes last.  One thread, after a CTA barrier behind the last write.
+// whichever CTA finishes last (returns true there).  One thread, after a CTA barrier behind the last write.
 template <uint32_t MODE>
-__device__ void finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, uint64_t code_bits) {
+__device__ bool finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, uint64_t code_bits) {
     const Geometry& G = P.geo;
-    if (tiles == 0) return;
+    if (tiles == 0) return false;
     if (nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)nnz);
     if (code_bits) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)code_bits);
     __threadfence();
     const unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), (unsigned long long)tiles);
-    if (prev + tiles != G.ntiles) return;
+    if (prev + tiles != G.ntiles) return false;
     __threadfence();
     uint64_t code_total, words;
     const uint64_t nnz_total = ld_volatile_u64(&P.ws->nnz);
@@ -374,17 +422,63 @@ __device__ void finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, 
     h[12] = (uint32_t)code_total; h[13] = (uint32_t)(code_total >> 32);
     h[14] = (uint32_t)nnz_total; h[15] = (uint32_t)(nnz_total >> 32);
     if (P.out_bits) *P.out_bits = container_bits;
+    return true;
 }
 
-// One warp: find the place of a staged tile (its predecessors announced their sizes an
-// iteration ago, so the walk rarely waits), copy the image to the stream, clear the stage.
-__device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot, uint32_t* stg, const uint64_t* tile_state,
+// The writer warp, first half of its work on a tile: the layout of the tile's records from the 32
+// sub-block lengths (lane = sub-block), the block heads written into the (zeroed) image, the tile's
+// size announced to the tiles behind it, and what the second half needs noted in `pd`.
+__device__ void lay_out_tile(const EncodeParams& P, TileMeta& m, Pending& pd, uint32_t* stg, uint64_t* tile_state,
+                             uint64_t* group_state, uint32_t lane) {
+    const Geometry& G = P.geo;
+    const bool narrow = G.bucket <= kBLK;
+    const uint32_t spb = narrow ? G.sb_per_block : 32u;
+    const uint32_t nsb = m.nsb;
+    const uint32_t v = lane < nsb ? m.sb_bits[lane] : 0u;
+    const uint32_t incl = warp_incl_scan(v);
+    const uint32_t excl = incl - v;
+    const uint32_t bi = lane / spb, sb0 = bi * spb;
+    const uint32_t sb_last = min(sb0 + spb, nsb) - 1u;                  // meaningful when lane < nsb
+    const uint32_t excl0 = __shfl_sync(0xffffffffu, excl, sb0 & 31u);
+    const uint32_t incl_last = __shfl_sync(0xffffffffu, incl, sb_last & 31u);
+    const uint32_t nsb_blk = sb_last - sb0 + 1u;
+    const uint32_t head_words = 1u + (nsb_blk + 1u) / 2u;
+    const bool leader = lane < nsb && lane == sb0;
+    const uint32_t blk_words = leader ? head_words + (incl_last - excl0 + 31u) / 32u : 0u;
+    const uint32_t wincl = warp_incl_scan(blk_words);
+    const uint32_t wexcl = wincl - blk_words;
+    const uint32_t blk_off = __shfl_sync(0xffffffffu, wexcl, sb0 & 31u);                // words before my block
+    m.bitoff[lane] = 32u * (blk_off + head_words) + (excl - excl0);                      // where sub-block `lane` goes
+    const uint32_t tile_words = __shfl_sync(0xffffffffu, wincl, 31);
+    const uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
+    if (lane == 0) announce_tile(tile_state, group_state, m.tile, tile_words);
+    // block heads: the norm word, then the u16 lengths of the block's sub-blocks, two per word
+    if (leader) stg[blk_off] = m.blk_norm[bi];
+    const uint32_t nv = __shfl_down_sync(0xffffffffu, v, 1);
+    if (lane < nsb && ((lane - sb0) & 1u) == 0)
+        stg[blk_off + 1u + (lane - sb0) / 2u] = v | ((lane + 1u <= sb_last ? nv : 0u) << 16);
+    pd.blk_wordoff[lane] = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
+    uint32_t nnz = lane < (uint32_t)kEncWarps ? m.wnnz[lane] : 0u;
+    nnz = __reduce_add_sync(0xffffffffu, nnz);
+    if (lane == 0) {
+        pd.tile = m.tile;
+        pd.words = tile_words;
+        pd.nblk = narrow ? (nsb + spb - 1u) / spb : 1u;
+        pd.code_bits = code_bits;
+        pd.nnz = nnz;
+    }
+    __syncwarp();
+}
+
+// Second half: find the place of the staged tile (its predecessors announced their sizes when they were
+// laid out, so the walk rarely waits), copy the image to the stream, clear the image.
+__device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot, uint32_t* stg, uint64_t* tile_state,
                               uint64_t* group_state, uint64_t* table, uint32_t* payload, uint32_t lane) {
     const Geometry& G = P.geo;
     const uint64_t tile = pd.tile;
     const uint32_t words = pd.words;
     bool failed;
-    const uint64_t off = tile_lookback(P.ws, tile_state, group_state, tile, G.ntiles, words, &failed);
+    const uint64_t off = tile_lookback(P, tile_state, group_state, tile, words, &failed);
     for (uint32_t i = lane; i < words; i += 32) {
         if (!failed) payload[off + i] = stg[i];
         stg[i] = 0;
@@ -399,7 +493,6 @@ __device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot
     }
     __syncwarp();
     if (lane == 0) {
-        pd.valid = 0;
         tot.tiles += 1;
         tot.nnz += pd.nnz;
         tot.code_bits += pd.code_bits;
@@ -408,189 +501,233 @@ __device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot
 }
 
 template <uint32_t LEVELSET, uint32_t MODE>
-__global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(const __grid_constant__ EncodeParams P) {
+__global__ void __launch_bounds__(MODE == kModeErc ? kEncAllThreads : kEncThreads, kEncMinBlocks)
+encode_kernel(const __grid_constant__ EncodeParams P) {
     extern __shared__ __align__(128) uint32_t smem[];
-    __shared__ __align__(8) uint64_t s_bar;                // completes when the tile's bytes have landed
-    __shared__ uint32_t s_lut[256];                        // ERC(N), N = 1..256: code | len << 16
-    __shared__ uint32_t s_lut_signed[256];                 // exponential levels: sign bit + ERC(index), by field
+    __shared__ __align__(8) uint64_t s_full[kEncWarps];    // s_full[w] completes when warp w's part of a tile has landed
+    __shared__ uint32_t s_lut[256];                        // ERC(N), N = 1..256: code left aligned | length
+    __shared__ uint32_t s_lut_signed[256];                 // exponential levels: sign bit + ERC(index) left aligned | length, by field
     __shared__ double s_partial[32];                       // per sub-block (or per warp) sums of squares
     __shared__ uint32_t s_maxbits[32];                     // ... or max |x| bit patterns
-    __shared__ uint32_t s_sb_bits[32];                     // token bits of each sub-block
-    __shared__ uint32_t s_sb_src[32];                      // where they start in the owning warp's window
-    __shared__ uint32_t s_start[32];                       // scratch: first token offset of a sub-block (per warp 4)
-    __shared__ unsigned long long s_tile[2];
-    __shared__ uint32_t s_abort, s_nnz;
-    __shared__ Pending s_pend[3];                          // ERC: the staged tiles (current and up to two earlier ones)
+    __shared__ float s_sb_inv[32], s_sb_norm[32];          // per sub-block of the current tile: 2^s / norm (0: not quantized), norm
+    __shared__ uint32_t s_sb_bi[32];                       // block (within a tile) of each sub-block
+    __shared__ uint32_t s_arrived;                         // warps that have added up their squares (counts on, modulo 8)
+    __shared__ TileInfo s_info[4];                         // tiles of the iterations it, it + 1, it + 2
+    __shared__ TileMeta s_meta[2];
+    __shared__ Pending s_pend[2];
     __shared__ CtaTotals s_tot;
+    __shared__ uint32_t s_nnz;                             // fixed-width mode: nonzero symbols of this CTA
+    __shared__ uint32_t s_last;                            // this CTA finished last
 
     using S = Sym<LEVELSET>;
     const Geometry& G = P.geo;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
-    float* data = reinterpret_cast<float*>(smem);                               // kBLK floats: the tile
-    uint32_t* stage = smem + kBLK;                                              // image of the tile's records
-    uint32_t* wmem = stage + P.stages * P.stage_words + warp * P.warp_smem_words;
-    uint32_t* window = wmem;                                                    // this warp's token string
-    uint32_t* tokens = wmem + P.window_words;               // kChunk entries: position | field << 10 (uniform levels)
-    uint16_t* tokens16 = reinterpret_cast<uint16_t*>(tokens);   //                position | field << 8  (exponential levels)
+    float* const data = reinterpret_cast<float*>(smem);                         // kBLK floats: the tile
+    uint32_t* const images = smem + kBLK;                                       // [2][stage_words]: staged tile records
+    uint32_t* const windows = images + 2u * P.stage_words;                      // [2][kEncWarps][window_words]: token strings
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
     uint64_t* group_state = tile_state + G.ntiles;
     uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
     uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
     const float top = __uint_as_float((127u + G.s) << 23);
     const uint32_t c2 = (uint32_t)P.offset, c3 = (uint32_t)(P.offset >> 32);
-    const uint32_t lt_mask = (1u << lane) - 1u;
+    const bool narrow = G.bucket <= kBLK;
     const bool coarse = G.bucket % kWarpElems == 0;         // a warp's four sub-blocks always share one bucket
-    const uint32_t spb = G.bucket <= kBLK ? G.sb_per_block : 32u;       // sub-blocks per coding block
-    uint32_t bi_q[4];                                       // block (within a tile) of the warp's four sub-blocks
-#pragma unroll
-    for (int q = 0; q < 4; ++q) bi_q[q] = (warp * 4u + q) / spb;
-    const uint32_t bi_lane = lane / spb;                    // block of sub-block `lane`
+    const uint32_t spb = narrow ? G.sb_per_block : 32u;     // sub-blocks per coding block
 
-    // where tile `t` starts and how long it is
-    auto tile_span = [&](uint64_t t, uint64_t& elem0, uint32_t& tile_len) {
-        if (G.bucket <= kBLK) {
-            elem0 = t * G.blocks_per_tile * G.bucket;
-            const uint64_t left = G.d - elem0;
-            tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
+    // thread 0: take a ticket (a CTA's first tile is the one with its own number, the tickets count on
+    // from there) and work out where that tile lies
+    auto take_ticket = [&](uint32_t iter) {
+        TileInfo& ti = s_info[iter & 3u];
+        const unsigned long long t =
+            iter == 0 ? blockIdx.x : gridDim.x + atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        ti.tile = t;
+        if (t >= G.ntiles) return;
+        if (narrow) {
+            ti.first_block = t * G.blocks_per_tile;
+            ti.elem0 = ti.first_block * G.bucket;
+            const uint64_t left = G.d - ti.elem0;
+            ti.tile_len = left < G.tile_elems ? (uint32_t)left : G.tile_elems;
+            ti.bucket_idx = 0;
+            ti.bib = 0;
+            ti.rec_len = 0;
         } else {
-            const uint64_t bucket_idx = t / G.blk_per_bucket;
-            const uint32_t bib = (uint32_t)(t % G.blk_per_bucket);
-            const uint64_t b0 = bucket_idx * G.bucket;
+            ti.bucket_idx = t / G.blk_per_bucket;
+            ti.bib = (uint32_t)(t % G.blk_per_bucket);
+            ti.first_block = t;
+            const uint64_t b0 = ti.bucket_idx * G.bucket;
             const uint64_t blen = G.d - b0 < G.bucket ? G.d - b0 : G.bucket;
-            elem0 = b0 + (uint64_t)bib * kBLK;
-            const uint64_t left = blen - (uint64_t)bib * kBLK;
-            tile_len = left < kBLK ? (uint32_t)left : kBLK;
+            ti.rec_len = (uint32_t)blen;
+            ti.elem0 = b0 + (uint64_t)ti.bib * kBLK;
+            const uint64_t left = blen - (uint64_t)ti.bib * kBLK;
+            ti.tile_len = left < kBLK ? (uint32_t)left : kBLK;
         }
+        ti.nsb = (ti.tile_len + kSB - 1) / kSB;
     };
-    // thread 0: take a ticket ...
-    auto take_ticket = [&]() { return atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull); };
-    // ... and start the copy of that tile into `data` once nobody reads the previous one
-    auto start_copy = [&](uint32_t slot) {
-        const uint64_t t = s_tile[slot];
-        if (t < G.ntiles) {
-            uint64_t elem0;
-            uint32_t tile_len;
-            tile_span(t, elem0, tile_len);
-            const uint32_t bytes = (tile_len * 4u) & ~15u;
-            if (bytes) bulk_load(data, P.g + elem0, bytes, &s_bar);
-        }
+    // A warp's part of a tile: elements [1024 w, 1024 (w + 1)) of it.  Whole 16-byte pieces come by a bulk
+    // copy that the warp starts itself as soon as it is done with its part of the tile before.
+    const uint32_t wbase = warp * kWarpElems;               // first element of the warp within a tile
+    auto bulk_elems_of = [&](const TileInfo& ti) {
+        const uint32_t n = ti.tile_len > wbase ? min(kWarpElems, ti.tile_len - wbase) : 0u;
+        return ti.tile < G.ntiles ? n & ~3u : 0u;
+    };
+    auto start_copy = [&](uint32_t iter) {                  // one lane of the warp
+        const TileInfo& ti = s_info[iter & 3u];
+        const uint32_t n = bulk_elems_of(ti);
+        if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
     if (tid < 256u) {
-        const uint32_t e = c_erc_lut[tid];
-        s_lut[tid] = e;
+        const uint32_t e = c_erc_lut[tid], elen = e >> 16;  // at most 16 bits
+        s_lut[tid] = ((e & 0xffffu) << (32u - elen)) | elen;
         const uint32_t idx = tid & 0x7Fu;                   // field = sign << 7 | index: sign bit, then ERC(index)
         uint32_t v = 0;
         if (idx >= 1) {
             const uint32_t l = c_erc_lut[idx - 1u], len = l >> 16;
-            v = ((tid >> 7) << len) | (l & 0xffffu) | ((len + 1u) << 16);
+            v = ((((tid >> 7) << len) | (l & 0xffffu)) << (31u - len)) | (len + 1u);
         }
         s_lut_signed[tid] = v;
     }
-    for (uint32_t i = tid; i < P.stages * P.stage_words; i += blockDim.x) stage[i] = 0;
-    if (warp < (uint32_t)kEncWarps)
-        for (uint32_t i = lane; i < P.window_words; i += 32) window[i] = 0;
+    if (tid < 32u) s_sb_bi[tid] = tid / spb;
+    if (MODE == kModeErc)
+        for (uint32_t i = tid; i < 2u * P.stage_words + 2u * kEncWarps * P.window_words; i += blockDim.x) images[i] = 0;
     if (tid == 0) {
-        mbar_init(&s_bar, 1);
-        s_abort = 0;
+        for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
         s_nnz = 0;
-        s_pend[0].valid = 0;
-        s_pend[1].valid = 0;
-        s_pend[2].valid = 0;
+        s_arrived = 0;
         s_tot.nnz = 0;
         s_tot.code_bits = 0;
         s_tot.tiles = 0;
         s_tot.stop = 0xFFFFFFFFu;
+        s_last = 0;
+        take_ticket(0);
     }
     __syncthreads();
-    if (tid == 0) {
-        s_tile[0] = take_ticket();
-        start_copy(0);
-    }
-    __syncthreads();
+    if (warp < (uint32_t)kEncWarps && lane == 0) start_copy(0);
+    if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
 
     const bool writer = MODE == kModeErc && warp == (uint32_t)kEncWarps;
     if (writer) {
-        // ---- the writer warp: finds the place of every staged tile (look-back), copies it to the
-        // stream and hands the stage back; the workers never wait for it unless it falls two tiles behind
-        uint32_t b = 0;                                     // stage of tile k: k mod P.stages
+        // ---- the writer warp: lays out every tile the workers have encoded, and a tile later, when they
+        // have moved their strings into the image, finds the tile's place in the stream and copies it out
         for (uint32_t k = 0;; ++k) {
-            stage_sync<kBarStaged>(b);                      // tile k of this CTA is staged
-            if (k >= *reinterpret_cast<volatile uint32_t*>(&s_tot.stop)) break;
-            flush_pending(P, s_pend[b], s_tot, stage + b * P.stage_words, tile_state, group_state, table, payload, lane);
-            stage_arrive<kBarFree>(b);
-            b = b + 1u == P.stages ? 0u : b + 1u;
+            const uint32_t p = k & 1u;
+            pair_sync<kBarDone>(p);                         // the workers' strings of tile k are complete (or there is no tile k)
+            const bool have = k < *reinterpret_cast<volatile uint32_t*>(&s_tot.stop);
+            if (have) {
+                lay_out_tile(P, s_meta[p], s_pend[p], images + p * P.stage_words, tile_state, group_state, lane);
+                pair_arrive<kBarLayout>(p);
+            }
+            if (k >= 1) {
+                pair_sync<kBarMerged>(p ^ 1u);              // the strings of tile k - 1 are in its image
+                flush_pending(P, s_pend[p ^ 1u], s_tot, images + (p ^ 1u) * P.stage_words, tile_state, group_state, table,
+                              payload, lane);
+            }
+            if (!have) break;
         }
     }
 
-    uint32_t parity = 0;
-    uint32_t it = 0, sg = 0;                                // sg: stage of iteration it, it mod P.stages
-    for (; !writer; ++it, sg = sg + 1u == P.stages ? 0u : sg + 1u) {           // the 8 worker warps
-        const uint64_t tile = s_tile[it & 1u];
-        if (tile >= G.ntiles) break;
-
-        // ---- tile geometry ------------------------------------------------------
-        uint64_t elem0, first_block, bucket_idx = 0;
-        uint32_t tile_len, nblk_tile, blk_elems, bib = 0;
-        tile_span(tile, elem0, tile_len);
-        if (G.bucket <= kBLK) {
-            first_block = tile * G.blocks_per_tile;
-            blk_elems = G.bucket;
-            nblk_tile = (tile_len + G.bucket - 1) / G.bucket;
-        } else {
-            bucket_idx = tile / G.blk_per_bucket;
-            bib = (uint32_t)(tile % G.blk_per_bucket);
-            first_block = tile;
-            blk_elems = kBLK;
-            nblk_tile = 1;
+    // ---- ERC: a worker moves its strings of tile k (window set k & 1, `bits` bits) to their place in
+    // the image once the writer has laid the tile out ----
+    auto merge_tile = [&](uint32_t k, uint32_t bits) {
+        const uint32_t p = k & 1u;
+        pair_sync<kBarLayout>(p);
+        const TileMeta& m = s_meta[p];
+        uint32_t* stg = images + p * P.stage_words;
+        uint32_t* win = windows + (p * kEncWarps + warp) * P.window_words;
+#pragma unroll 1
+        for (uint32_t q = 0; q < 4; q += coarse ? 4u : 1u) {
+            // the strings of sub-blocks of one block follow one another in the window and in the
+            // tile alike, so a warp whose four sub-blocks share a block moves them in one piece
+            const uint32_t sbq = warp * 4u + q;
+            if (sbq >= m.nsb) break;
+            const uint32_t len = coarse ? bits : m.sb_bits[sbq], src = coarse ? 0u : m.sb_src[sbq];
+            const uint32_t dst = m.bitoff[sbq];
+            if (len == 0) continue;
+            const uint32_t w_first = dst >> 5, w_last = (dst + len - 1u) >> 5;
+            for (uint32_t w = w_first + lane; w <= w_last; w += 32) {
+                const int sbit = (int)src + (int)(32u * w) - (int)dst;
+                uint32_t val = bits_at(win, sbit);
+                const uint32_t head = 32u * w < dst ? dst - 32u * w : 0u;     // bits of this word before the string
+                const uint32_t tail_end = min(dst + len - 32u * w, 32u);      // bits of this word up to its end
+                uint32_t mask = 0xFFFFFFFFu >> head;
+                if (tail_end < 32u) mask &= ~(0xFFFFFFFFu >> tail_end);
+                val &= mask;
+                if (val) atomicOr(stg + w, val);
+            }
         }
-        const uint32_t nsb_tile = (tile_len + kSB - 1) / kSB;
-        const uint32_t wbase = warp * kWarpElems;           // first element of the warp within the tile
+        __syncwarp();
+        for (uint32_t i = lane; i < (bits + 31u) / 32u + 2u; i += 32) win[i] = 0;   // ready for tile k + 2
+        __syncwarp();
+        pair_arrive<kBarMerged>(p);                        // the writer may take the tile
+    };
 
-        // ---- the tile's bytes: wait for the bulk copy, fetch the ragged end, zero the rest ----
+    uint32_t it = 0;
+    uint32_t cta_nnz = 0;                                   // fixed-width mode: this thread's count
+    uint32_t prev_bits = 0;                                 // ERC: bits of this warp's strings of the previous tile
+    uint32_t parity = 0;                                    // of the next completion of s_full[warp]
+    for (; !writer; ++it) {                                 // the 8 worker warps
+        const TileInfo& ti = s_info[it & 3u];
+        const uint64_t tile = ti.tile;
+        if (tile >= G.ntiles) break;
+        const uint64_t elem0 = ti.elem0;
+        const uint32_t tile_len = ti.tile_len, nsb_tile = ti.nsb;
+
+        // ---- the warp's part of the tile: wait for the bulk copy, fetch the ragged end, zero the rest ----
         {
-            const uint32_t bulk_elems = ((tile_len * 4u) & ~15u) / 4u;
+            const uint32_t bulk_elems = bulk_elems_of(ti);
             if (bulk_elems) {
-                if (!mbar_wait(&s_bar, parity)) {           // never seen in practice; do not hang
-                    if (tid == 0) {
-                        latch_status(P.ws, kErrTimeout);
-                        s_abort = 1;
-                    }
-                }
+                if (!mbar_wait(&s_full[warp], parity) && lane == 0) latch_status(P.ws, kErrTimeout);   // never seen; do not hang
                 parity ^= 1u;
             }
-            if (tile_len < kBLK) {
-                for (uint32_t i = bulk_elems + tid; i < kBLK; i += kEncThreads)
-                    data[i] = i < tile_len ? __ldg(P.g + elem0 + i) : 0.0f;
-                bar_sync<kBarWork, kEncThreads>();
+            if (bulk_elems < kWarpElems) {
+                for (uint32_t i = bulk_elems + lane; i < kWarpElems; i += 32)
+                    data[wbase + i] = wbase + i < tile_len ? __ldg(P.g + elem0 + wbase + i) : 0.0f;
+                __syncwarp();
             }
         }
         const float4* rows = reinterpret_cast<const float4*>(data + wbase) + lane;   // row j at rows[32 * j]
 
-        // ---- bucket norms: fp64 sums of exact squares (or max |x|), one rounding to fp32 ----
+        // ---- bucket norms.  L2: a lane adds the squares of its 8 elements of a sub-block in fp32 (7 roundings
+        // of 2^-24 relative each, of random sign), everything beyond that in fp64: the norm stays within a
+        // few 1e-8 of the exactly rounded one.  Linf: max |x|, exact. ----
         if (P.norms_in == nullptr) {
             double acc = 0.0;
             uint32_t mx = 0;
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const float4 x = rows[32 * (2 * q + h)];
-                    if (G.norm_kind == kNormL2) {
-                        acc = fma((double)x.x, (double)x.x, acc);
-                        acc = fma((double)x.y, (double)x.y, acc);
-                        acc = fma((double)x.z, (double)x.z, acc);
-                        acc = fma((double)x.w, (double)x.w, acc);
-                    } else {                                // on the bit patterns: NaN sorts above inf
-                        mx = max(max(mx, __float_as_uint(fabsf(x.x))), __float_as_uint(fabsf(x.y)));
-                        mx = max(max(mx, __float_as_uint(fabsf(x.z))), __float_as_uint(fabsf(x.w)));
+                const float4 x = rows[32 * (2 * q)], y = rows[32 * (2 * q + 1)];
+                if (G.norm_kind == kNormL2) {
+                    float a = __fmul_rn(x.x, x.x), b = __fmul_rn(x.y, x.y);
+                    a = __fmaf_rn(x.z, x.z, a); b = __fmaf_rn(x.w, x.w, b);
+                    a = __fmaf_rn(y.x, y.x, a); b = __fmaf_rn(y.y, y.y, b);
+                    a = __fmaf_rn(y.z, y.z, a); b = __fmaf_rn(y.w, y.w, b);
+                    const float p8 = a + b;
+                    // squares that leave the fp32 range (tiny or huge coordinates, NaN): the warp adds this
+                    // sub-block up in fp64 instead
+                    const bool out_of_range = !(p8 >= 0x1p-60f && p8 < 0x1p120f);
+                    if (__any_sync(0xffffffffu, out_of_range)) {
+                        double e = 0.0;
+                        e = fma((double)x.x, (double)x.x, e); e = fma((double)x.y, (double)x.y, e);
+                        e = fma((double)x.z, (double)x.z, e); e = fma((double)x.w, (double)x.w, e);
+                        e = fma((double)y.x, (double)y.x, e); e = fma((double)y.y, (double)y.y, e);
+                        e = fma((double)y.z, (double)y.z, e); e = fma((double)y.w, (double)y.w, e);
+                        acc += e;
+                    } else {
+                        acc += (double)p8;
                     }
+                } else {                                    // on the bit patterns: NaN sorts above inf
+                    mx = max(max(mx, __float_as_uint(fabsf(x.x))), __float_as_uint(fabsf(x.y)));
+                    mx = max(max(mx, __float_as_uint(fabsf(x.z))), __float_as_uint(fabsf(x.w)));
+                    mx = max(max(mx, __float_as_uint(fabsf(y.x))), __float_as_uint(fabsf(y.y)));
+                    mx = max(max(mx, __float_as_uint(fabsf(y.z))), __float_as_uint(fabsf(y.w)));
                 }
                 if (!coarse || q == 3) {                    // one partial per sub-block, or one per warp
+                    if (G.norm_kind == kNormL2) {
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        acc += __shfl_xor_sync(0xffffffffu, acc, o);
-                        mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+                    } else {
+                        mx = __reduce_max_sync(0xffffffffu, mx);
                     }
                     if (lane == 0) {
                         s_partial[warp * 4 + q] = acc;
@@ -598,46 +735,40 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
                     }
                     acc = 0.0;
                     mx = 0;
-                } else if (lane == 0) {
-                    s_partial[warp * 4 + q] = 0.0;
-                    s_maxbits[warp * 4 + q] = 0;
                 }
             }
         }
-        bar_sync<kBarWork, kEncThreads>();                    // B1: partials visible
-        // the next ticket is asked for now and stored just before the next barrier: the round trip
-        // of the atomic is over by then
-        unsigned long long next_ticket = 0;
-        if (tid == 0) next_ticket = take_ticket();
-
-        // every warp derives the norms of the buckets its own sub-blocks belong to (same
-        // reduction tree in every warp, so all agree bit for bit)
-        float inv_q[4], norm_q[4];
+        // the draws of the warp's first sub-block do not depend on the norms: they are made before the
+        // barrier, where the warp would otherwise wait for the slowest one
+        const uint64_t ctr_warp = ((elem0 + wbase) >> 2) + lane;               // Philox counter of row 0's block
+        uint4 rn0 = philox4x32_10((uint32_t)ctr_warp, (uint32_t)(ctr_warp >> 32), c2, c3, P.round_keys);
+        uint4 rn1 = philox4x32_10((uint32_t)(ctr_warp + 32u), (uint32_t)((ctr_warp + 32u) >> 32), c2, c3, P.round_keys);
+        // ---- whichever warp gets here last turns the partial sums into norms, once for the whole CTA ----
         {
-            const double my_part = s_partial[lane];
-            const uint32_t my_max = s_maxbits[lane];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                if (q > 0 && (coarse || bi_q[q] == bi_q[q - 1])) {            // same bucket as the previous sub-block
-                    inv_q[q] = inv_q[q - 1];
-                    norm_q[q] = norm_q[q - 1];
-                    continue;
-                }
-                const uint32_t bi = bi_q[q], sb0 = bi * spb;
+            uint32_t last = 0;
+            __syncwarp();
+            if (lane == 0) {
+                __threadfence_block();
+                last = (atomicAdd(&s_arrived, 1u) & (kEncWarps - 1u)) == kEncWarps - 1u;
+            }
+            if (__shfl_sync(0xffffffffu, last, 0)) {
+                __threadfence_block();
+                // lane = sub-block of the tile; the lanes of one bucket all do the same sum, in the same order
+                const uint32_t bi = lane / spb, sb0 = bi * spb;
                 float norm;
                 if (P.norms_in != nullptr) {
-                    const uint64_t nb_idx = G.bucket <= kBLK ? first_block + bi : bucket_idx;
+                    const uint64_t nb_idx = narrow ? ti.first_block + bi : ti.bucket_idx;
                     norm = nb_idx < G.nb ? P.norms_in[nb_idx] : 0.0f;
+                } else if (G.norm_kind == kNormL2) {
+                    double a = 0.0;
+                    if (coarse) for (uint32_t j = sb0 + 3u; j < sb0 + spb; j += 4u) a += s_partial[j];     // one partial per warp
+                    else for (uint32_t j = sb0; j < sb0 + spb; ++j) a += s_partial[j];
+                    norm = (float)sqrt(a);
                 } else {
-                    const bool in = lane >= sb0 && lane < sb0 + spb;
-                    double a = in ? my_part : 0.0;
-                    uint32_t m = in ? my_max : 0u;
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        a += __shfl_xor_sync(0xffffffffu, a, o);
-                        m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-                    }
-                    norm = G.norm_kind == kNormL2 ? (float)sqrt(a) : __uint_as_float(m);
+                    uint32_t mxb = 0;
+                    if (coarse) for (uint32_t j = sb0 + 3u; j < sb0 + spb; j += 4u) mxb = max(mxb, s_maxbits[j]);
+                    else for (uint32_t j = sb0; j < sb0 + spb; ++j) mxb = max(mxb, s_maxbits[j]);
+                    norm = __uint_as_float(mxb);
                 }
                 if (norm != norm) norm = __uint_as_float(0x7fc00000u);     // one NaN pattern in the stream
                 float inv = 0.0f;                                           // 0: the bucket is not quantized
@@ -645,306 +776,287 @@ __global__ void __launch_bounds__(kEncAllThreads, kEncMinBlocks) encode_kernel(c
                     inv = __fdiv_rn(top, norm);                             // one IEEE division per bucket
                     if (!(inv < __uint_as_float(0x7f800000u))) inv = 0.0f;
                 }
-                inv_q[q] = inv;
-                norm_q[q] = norm;
+                // a bucket that cannot be quantized although it is not all zero: tell the caller
+                if (__any_sync(0xffffffffu, inv == 0.0f && norm != 0.0f && lane < nsb_tile) && lane == 0)
+                    latch_status(P.ws, kWarnNonfinite);
+                s_sb_inv[lane] = inv;
+                s_sb_norm[lane] = norm;
+                if (MODE == kModeErc && lane == sb0 && lane < nsb_tile) s_meta[it & 1u].blk_norm[bi] = __float_as_uint(norm);
             }
         }
+        bar_sync<kBarWork, kEncThreads>();                    // the one barrier of a tile: norms visible,
+                                                            // and every warp is done with the previous tile
+        // the ticket of the tile after the next is taken now: its round trip ends long before anyone looks
+        if (tid == 0) take_ticket(it + 2u);
 
-        // ---- quantize (Definition 1) and generate tokens, one chunk of elements at a time ------
+        TileMeta* const meta = &s_meta[it & 1u];
+        uint32_t* const window = windows + ((it & 1u) * kEncWarps + warp) * P.window_words;   // this warp's token string
+        // ---- quantize (Definition 1) and emit, one sub-block (two 128-element rows) at a time ----
         uint32_t bits = 0;                                  // ERC: bits in this warp's window so far
-        uint32_t my_nnz = 0;
-        if (MODE == kModeErc && lane < 4) s_start[warp * 4 + lane] = 0xFFFFFFFFu;
-        // lane q < 4 keeps 2^s / norm and the block of the warp's sub-block q for the loop below
-        const float inv_own = (lane & 3u) == 0 ? inv_q[0] : (lane & 3u) == 1 ? inv_q[1] : (lane & 3u) == 2 ? inv_q[2] : inv_q[3];
-        const uint32_t bi_own = (lane & 3u) == 0 ? bi_q[0] : (lane & 3u) == 1 ? bi_q[1] : (lane & 3u) == 2 ? bi_q[2] : bi_q[3];
+        uint32_t cum = 0;                                   // ERC: nonzero symbols so far (warp uniform)
+        // fixed-width mode: where a sub-block's 8 * width words go and how many of them exist
+        uint32_t* fx_rec = nullptr;
+        uint32_t fx_sb = 0, fx_words = 0;                   // sub-block within its record, valid field words of the record
 #pragma unroll 1
-        for (uint32_t part = 0; part < kWarpElems / kChunk; ++part) {
-            uint32_t ntok = 0;
-#pragma unroll
-            for (uint32_t r = 0; r < kChunkRows; ++r) {
-                const uint32_t j = part * kChunkRows + r;   // row of the warp
-                const float inv = __shfl_sync(0xffffffffu, inv_own, j >> 1);
-                const uint32_t bi_row = __shfl_sync(0xffffffffu, bi_own, j >> 1);   // block of this row's sub-block
-                if (inv == 0.0f) continue;                  // bucket not quantized (warp uniform)
-                const float4 x = rows[32 * j];
-                const uint32_t base = wbase + j * 128u + lane * 4u;             // element within the tile
-                const uint64_t ctr = (elem0 + base) >> 2;
-                const uint4 rnd = philox4x32_10((uint32_t)ctr, (uint32_t)(ctr >> 32), c2, c3, P.round_keys);
-                uint32_t q0, q1, q2, q3;
-                if (LEVELSET == kLevelsExp) {
-                    q0 = quantize_exp(x.x, inv, top, rnd.x);
-                    q1 = quantize_exp(x.y, inv, top, rnd.y);
-                    q2 = quantize_exp(x.z, inv, top, rnd.z);
-                    q3 = quantize_exp(x.w, inv, top, rnd.w);
-                } else {
-                    q0 = quantize_uniform(x.x, inv, top, rnd.x);
-                    q1 = quantize_uniform(x.y, inv, top, rnd.y);
-                    q2 = quantize_uniform(x.z, inv, top, rnd.z);
-                    q3 = quantize_uniform(x.w, inv, top, rnd.w);
+        for (uint32_t q = 0; q < 4; ++q) {
+            const uint32_t sbq = warp * 4u + q;
+            const uint32_t start_bits = bits;
+            if (sbq >= nsb_tile) {
+                if (MODE == kModeErc && lane == 0) {
+                    meta->sb_bits[sbq] = 0;
+                    meta->sb_src[sbq] = bits;
                 }
-                // fields (index | sign << kBits); in the fixed-width mode a zero symbol must carry no sign
-                uint32_t f = 0, f0 = 0, f1 = 0, f2 = 0, f3 = 0;
+                continue;
+            }
+            const float inv = s_sb_inv[sbq];
+
+            uint32_t* fx_dst = nullptr;
+            uint32_t fx_valid = 0;
+            if (MODE == kModeFixed) {
+                if (q == 0 || !coarse) {
+                    const uint32_t bi = s_sb_bi[sbq];
+                    uint32_t rec_len;
+                    if (narrow) {
+                        fx_rec = payload + (ti.first_block + bi) * G.rec_words;
+                        fx_sb = sbq - bi * spb;
+                        rec_len = min(G.bucket, tile_len - bi * G.bucket);
+                    } else {
+                        fx_rec = payload + ti.bucket_idx * G.rec_words;
+                        fx_sb = ti.bib * 32u + sbq;
+                        rec_len = ti.rec_len;
+                    }
+                    fx_words = (rec_len * G.width + 31u) / 32u;
+                } else {
+                    fx_sb += 1u;
+                }
+                const uint32_t sbw = 8u * G.width;          // words of a full sub-block
+                if (fx_sb == 0 && lane == 0) fx_rec[0] = __float_as_uint(s_sb_norm[sbq]);
+                fx_dst = fx_rec + 1u + fx_sb * sbw;
+                fx_valid = min(sbw, fx_words - fx_sb * sbw);
+            }
+
+            if (inv != 0.0f) {
+                const float4 x0 = rows[32 * (2 * q)], x1 = rows[32 * (2 * q + 1)];
+                __syncwarp();                               // the sub-block's bytes are in registers: their place is scratch now
+                const uint4 r0 = rn0, r1 = rn1;
+                uint32_t qa[8];
                 if (LEVELSET == kLevelsExp) {
-                    const uint32_t syms = q0 | (q1 << 8) | (q2 << 16) | (q3 << 24);
+                    qa[0] = quantize_exp(x0.x, inv, top, r0.x); qa[1] = quantize_exp(x0.y, inv, top, r0.y);
+                    qa[2] = quantize_exp(x0.z, inv, top, r0.z); qa[3] = quantize_exp(x0.w, inv, top, r0.w);
+                    qa[4] = quantize_exp(x1.x, inv, top, r1.x); qa[5] = quantize_exp(x1.y, inv, top, r1.y);
+                    qa[6] = quantize_exp(x1.z, inv, top, r1.z); qa[7] = quantize_exp(x1.w, inv, top, r1.w);
+                } else {
+                    qa[0] = quantize_uniform(x0.x, inv, top, r0.x); qa[1] = quantize_uniform(x0.y, inv, top, r0.y);
+                    qa[2] = quantize_uniform(x0.z, inv, top, r0.z); qa[3] = quantize_uniform(x0.w, inv, top, r0.w);
+                    qa[4] = quantize_uniform(x1.x, inv, top, r1.x); qa[5] = quantize_uniform(x1.y, inv, top, r1.y);
+                    qa[6] = quantize_uniform(x1.z, inv, top, r1.z); qa[7] = quantize_uniform(x1.w, inv, top, r1.w);
+                }
+                const uint32_t xb[8] = {__float_as_uint(x0.x), __float_as_uint(x0.y), __float_as_uint(x0.z), __float_as_uint(x0.w),
+                                        __float_as_uint(x1.x), __float_as_uint(x1.y), __float_as_uint(x1.z), __float_as_uint(x1.w)};
+                // Exponential levels: the four symbols of a row as bytes, index | sign << 7.
+                uint32_t f0 = 0, f1 = 0, nz0 = 0, nz1 = 0;
+                if (LEVELSET == kLevelsExp) {
+                    const uint32_t syms0 = qa[0] | (qa[1] << 8) | (qa[2] << 16) | (qa[3] << 24);
+                    const uint32_t syms1 = qa[4] | (qa[5] << 8) | (qa[6] << 16) | (qa[7] << 24);
                     // top bytes of the four inputs: their sign bits at bits 7, 15, 23, 31
-                    uint32_t tops = __byte_perm(__byte_perm(__float_as_uint(x.x), __float_as_uint(x.y), 0x0073),
-                                                __byte_perm(__float_as_uint(x.z), __float_as_uint(x.w), 0x0073), 0x5410);
-                    if (MODE == kModeFixed) tops &= syms + 0x7F7F7F7Fu;        // bit 7 of a byte: symbol != 0
-                    f = syms | (tops & 0x80808080u);
-                    if (MODE == kModeFixed) { f0 = f & 0xFFu; f1 = (f >> 8) & 0xFFu; f2 = (f >> 16) & 0xFFu; f3 = f >> 24; }
-                } else {
-                    f0 = q0 | (q0 ? (__float_as_uint(x.x) >> 16) & 0x8000u : 0u);
-                    f1 = q1 | (q1 ? (__float_as_uint(x.y) >> 16) & 0x8000u : 0u);
-                    f2 = q2 | (q2 ? (__float_as_uint(x.z) >> 16) & 0x8000u : 0u);
-                    f3 = q3 | (q3 ? (__float_as_uint(x.w) >> 16) & 0x8000u : 0u);
+                    const uint32_t tops0 = __byte_perm(__byte_perm(xb[0], xb[1], 0x0073), __byte_perm(xb[2], xb[3], 0x0073), 0x5410);
+                    const uint32_t tops1 = __byte_perm(__byte_perm(xb[4], xb[5], 0x0073), __byte_perm(xb[6], xb[7], 0x0073), 0x5410);
+                    nz0 = (syms0 + 0x7F7F7F7Fu) & 0x80808080u;                  // bit 7 of a byte: symbol != 0
+                    nz1 = (syms1 + 0x7F7F7F7Fu) & 0x80808080u;
+                    f0 = syms0 | (tops0 & nz0);                                 // a zero symbol carries no sign
+                    f1 = syms1 | (tops1 & nz1);
                 }
+
                 if (MODE == kModeErc) {
-                    // keep the nonzero symbols, in element order: rank = nonzeros in lower lanes + own earlier ones
-                    const uint32_t v0 = __ballot_sync(0xffffffffu, q0 != 0), v1 = __ballot_sync(0xffffffffu, q1 != 0);
-                    const uint32_t v2 = __ballot_sync(0xffffffffu, q2 != 0), v3 = __ballot_sync(0xffffffffu, q3 != 0);
-                    uint32_t at = ntok + __popc(v0 & lt_mask) + __popc(v1 & lt_mask) + __popc(v2 & lt_mask) +
-                                  __popc(v3 & lt_mask);
-                    const uint32_t pos = r * 128u + lane * 4u;                  // position within the 512-element chunk
+                    // ---- keep the nonzero symbols, in element order: a lane's rank = nonzeros of row 0 in lower
+                    // lanes (+ all of row 0 and those of row 1 in lower lanes, for its row-1 elements) ----
+                    uint32_t cnt0, cnt1;
+                    if (LEVELSET == kLevelsExp) {
+                        cnt0 = __popc(nz0);
+                        cnt1 = __popc(nz1);
+                    } else {
+                        cnt0 = (qa[0] != 0) + (qa[1] != 0) + (qa[2] != 0) + (qa[3] != 0);
+                        cnt1 = (qa[4] != 0) + (qa[5] != 0) + (qa[6] != 0) + (qa[7] != 0);
+                    }
+                    const uint32_t packed = cnt0 | (cnt1 << 16);
+                    const uint32_t incl = warp_incl_scan(packed);
+                    const uint32_t totals = __shfl_sync(0xffffffffu, incl, 31);
+                    const uint32_t tot0 = totals & 0xffffu;
+                    const uint32_t ntok = tot0 + (totals >> 16);
+                    uint32_t at0 = (incl & 0xffffu) - cnt0, at1 = tot0 + (incl >> 16) - cnt1;
+                    uint32_t* list32 = reinterpret_cast<uint32_t*>(data + wbase + q * kSB);   // over the sub-block's own bytes
+                    uint16_t* list16 = reinterpret_cast<uint16_t*>(list32);
                     if (LEVELSET == kLevelsExp) {
                         // 16-bit entries position | field << 8, two at a time by byte permutation
-                        const uint32_t pb = pos * 0x01010101u + 0x03020100u;    // the four positions, one per byte
-                        const uint32_t e01 = __byte_perm(pb, f, 0x5140), e23 = __byte_perm(pb, f, 0x7362);
-                        if (q0) tokens16[at++] = (uint16_t)e01;
-                        if (q1) tokens16[at++] = (uint16_t)(e01 >> 16);
-                        if (q2) tokens16[at++] = (uint16_t)e23;
-                        if (q3) tokens16[at++] = (uint16_t)(e23 >> 16);
+                        const uint32_t pb0 = (lane * 4u) * 0x01010101u + 0x03020100u;      // the four positions of row 0, one per byte
+                        const uint32_t pb1 = pb0 + 0x80808080u;                            // ... of row 1
+                        const uint32_t a01 = __byte_perm(pb0, f0, 0x5140), a23 = __byte_perm(pb0, f0, 0x7362);
+                        const uint32_t b01 = __byte_perm(pb1, f1, 0x5140), b23 = __byte_perm(pb1, f1, 0x7362);
+                        if (qa[0]) list16[at0++] = (uint16_t)a01;
+                        if (qa[1]) list16[at0++] = (uint16_t)(a01 >> 16);
+                        if (qa[2]) list16[at0++] = (uint16_t)a23;
+                        if (qa[3]) list16[at0++] = (uint16_t)(a23 >> 16);
+                        if (qa[4]) list16[at1++] = (uint16_t)b01;
+                        if (qa[5]) list16[at1++] = (uint16_t)(b01 >> 16);
+                        if (qa[6]) list16[at1++] = (uint16_t)b23;
+                        if (qa[7]) list16[at1++] = (uint16_t)(b23 >> 16);
                     } else {
-                        if (q0) tokens[at++] = pos | (f0 << 10);
-                        if (q1) tokens[at++] = (pos + 1u) | (f1 << 10);
-                        if (q2) tokens[at++] = (pos + 2u) | (f2 << 10);
-                        if (q3) tokens[at++] = (pos + 3u) | (f3 << 10);
+                        // 32-bit entries position | field << 10, field = index | sign << 15
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            if (qa[c]) list32[at0++] = (lane * 4u + c) | ((qa[c] | ((xb[c] >> 16) & 0x8000u)) << 10);
+                        }
+#pragma unroll
+                        for (int c = 4; c < 8; ++c) {
+                            if (qa[c]) list32[at1++] = (128u + lane * 4u + (c - 4)) | ((qa[c] | ((xb[c] >> 16) & 0x8000u)) << 10);
+                        }
                     }
-                    ntok = __shfl_sync(0xffffffffu, at, 31);                     // lane 31 ends behind the last entry
-                } else if (q0 | q1 | q2 | q3) {
-                    // fixed-width fields, MSB first, straight into the staged tile
+                    __syncwarp();
+                    // ---- tokens ERC(gap) sign ERC(index), 32 per step, appended to the warp's window ----
+                    int carry_pos = -1;                         // position of the last nonzero so far: the run starts at t_0 = 0
+                    for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
+                        const bool valid = t0 + lane < ntok;
+                        uint32_t e = 0;
+                        if (valid) e = LEVELSET == kLevelsExp ? (uint32_t)list16[t0 + lane] : list32[t0 + lane];
+                        const int pos = (int)(e & (LEVELSET == kLevelsExp ? 255u : 1023u));
+                        const uint32_t field = e >> (LEVELSET == kLevelsExp ? 8 : 10);
+                        int prev = __shfl_up_sync(0xffffffffu, pos, 1);
+                        if (lane == 0) prev = carry_pos;
+                        uint32_t gl = 0;                        // stays 0 in lanes without a token: no bits, no length
+                        if (valid) gl = s_lut[(pos - prev - 1) & 255];
+                        uint32_t tlen, tokA, lenA, tokB = 0, lenB = 0;
+                        if (LEVELSET == kLevelsExp) {
+                            // both codes left aligned with their length in the low bits: the token is the gap code
+                            // followed by sign and index code, i.e. the second shifted right by the first's length
+                            const uint32_t ll = s_lut_signed[field & 255u];
+                            lenA = (gl & 31u) + (ll & 31u);
+                            tokA = (gl & ~31u) | ((ll & ~31u) >> (gl & 31u));     // <= 16 + 8 bits, left aligned
+                            tlen = lenA;
+                        } else {
+                            const uint32_t ll = s_lut[((field & S::kMask) - 1u) & 255u];
+                            lenA = gl & 31u;
+                            tokA = gl & ~31u;
+                            lenB = valid ? (ll & 31u) + 1u : 0u;                  // sign + ERC(index) <= 17 bits
+                            tokB = valid ? ((field >> S::kBits) << 31) | ((ll & ~31u) >> 1) : 0u;
+                            tlen = lenA + lenB;
+                        }
+                        const uint32_t incl_bits = warp_incl_scan(tlen);
+                        const uint32_t step_bits = __shfl_sync(0xffffffffu, incl_bits, 31);
+                        // the window is sized for the most bits the warp's elements can produce; checked all the same
+                        if (bits + step_bits > 32u * (P.window_words - 2u)) {
+                            if (lane == 0) latch_status(P.ws, kErrInternal);
+                            break;
+                        }
+                        const uint32_t off = bits + incl_bits - tlen;     // bit of the window where my token starts
+                        or_bits_left(window, off, tokA);
+                        if (LEVELSET != kLevelsExp) or_bits_left(window, off + lenA, tokB);
+                        bits += step_bits;
+                        carry_pos = __shfl_sync(0xffffffffu, pos, min(ntok - t0, 32u) - 1u);
+                    }
+                    cum += ntok;
+                    __syncwarp();
+                } else {
+                    // ---- fixed-width fields (sign bit, then the level index), MSB first ----
                     const uint32_t wbits = G.width;
-                    const uint32_t ff[4] = {f0, f1, f2, f3};
-                    uint64_t str = 0;
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        str = (str << wbits) | ((ff[c] & S::kMask) | ((ff[c] >> S::kBits) << (wbits - 1u)));
-                        my_nnz += (ff[c] & S::kMask) != 0;
-                    }
-                    uint32_t cursor;
-                    if (G.bucket <= kBLK) {
-                        const uint32_t bi = bi_row;
-                        cursor = 32u * (bi * G.rec_words + 1u) + (base - bi * blk_elems) * wbits;
+                    if (LEVELSET == kLevelsExp && wbits == 4u) {
+                        // nibbles sign << 3 | index of the four elements of a row, first element on top
+                        auto pack4 = [](uint32_t f) {
+                            const uint32_t t = (f & 0x07070707u) | ((f >> 4) & 0x08080808u);    // one nibble per byte
+                            const uint32_t r = __byte_perm(t, 0u, 0x0213);                       // bytes n0 n2 n1 n3 from the top
+                            return (r | (r >> 12)) & 0xffffu;                                    // n0 n1 n2 n3
+                        };
+                        const uint32_t h0 = pack4(f0), h1 = pack4(f1);
+                        // even lanes finish a word of row 0, odd lanes one of row 1: the halves trade places
+                        const uint32_t got = __shfl_xor_sync(0xffffffffu, (lane & 1u) ? h0 : h1, 1);
+                        const uint32_t word = (lane & 1u) ? (got << 16) | h1 : (h0 << 16) | got;
+                        const uint32_t wi = (lane & 1u) * 16u + (lane >> 1);
+                        if (wi < fx_valid) fx_dst[wi] = word;
+                        cta_nnz += __popc(nz0) + __popc(nz1);
                     } else {
-                        cursor = base * wbits;
+                        uint32_t ff[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            if (LEVELSET == kLevelsExp) ff[c] = ((c < 4 ? f0 : f1) >> (8 * (c & 3))) & 0xffu;
+                            else ff[c] = qa[c] | (qa[c] ? (xb[c] >> 16) & 0x8000u : 0u);
+                            cta_nnz += qa[c] != 0;
+                        }
+                        // the sub-block's fields are put together over its own bytes, then copied out
+                        uint32_t* stg = reinterpret_cast<uint32_t*>(data + wbase + q * kSB);
+                        for (uint32_t i = lane; i < 8u * wbits + 2u; i += 32) stg[i] = 0;
+                        __syncwarp();
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            uint64_t str = 0;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const uint32_t f = ff[4 * h + c];
+                                str = (str << wbits) | ((f & S::kMask) | ((f >> S::kBits) << (wbits - 1u)));
+                            }
+                            if (str) or_bits(stg, (h * 128u + lane * 4u) * wbits, str, 4u * wbits);
+                        }
+                        __syncwarp();
+                        for (uint32_t i = lane; i < fx_valid; i += 32) fx_dst[i] = stg[i];
                     }
-                    or_bits(stage, cursor, str, 4u * wbits);
                 }
+            } else if (MODE == kModeFixed) {
+                for (uint32_t i = lane; i < fx_valid; i += 32) fx_dst[i] = 0;      // a bucket that is not quantized: all fields zero
             }
-
-            if (MODE == kModeErc) {
-                __syncwarp();
-                // ---- tokens ERC(gap) sign ERC(index), 32 per step, appended to the warp's window ----
-                int carry_pos = -1;                         // position (within the chunk) of the last nonzero so far
-                for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
-                    const bool valid = t0 + lane < ntok;
-                    uint32_t e = 0;
-                    if (valid) e = LEVELSET == kLevelsExp ? (uint32_t)tokens16[t0 + lane] : tokens[t0 + lane];
-                    const int pos = (int)(e & (LEVELSET == kLevelsExp ? 255u : 1023u));
-                    const uint32_t field = e >> (LEVELSET == kLevelsExp ? 8 : 10);
-                    int prev = __shfl_up_sync(0xffffffffu, pos, 1);
-                    if (lane == 0) prev = carry_pos;
-                    const bool first_of_sb = (prev >> 8) != (pos >> 8);      // also when there is no predecessor
-                    if (first_of_sb) prev = (pos & ~255) - 1;                  // the run restarts: t_0 = 0
-                    const uint32_t gl = s_lut[(pos - prev - 1) & 255];
-                    uint32_t tlen, tokA, lenA, tokB = 0, lenB;
-                    if (LEVELSET == kLevelsExp) {
-                        const uint32_t ll = s_lut_signed[field & 255u];
-                        lenB = ll >> 16;
-                        tokA = ((gl & 0xffffu) << lenB) | (ll & 0xffffu);     // <= 16 + 8 bits
-                        lenA = valid ? (gl >> 16) + lenB : 0u;
-                        tlen = lenA;
-                    } else {
-                        const uint32_t ll = s_lut[((field & S::kMask) - 1u) & 255u];
-                        tokA = gl & 0xffffu;
-                        lenA = valid ? gl >> 16 : 0u;
-                        lenB = valid ? (ll >> 16) + 1u : 0u;                  // sign + ERC(index) <= 17 bits
-                        tokB = ((field >> S::kBits) << (ll >> 16)) | (ll & 0xffffu);
-                        tlen = lenA + lenB;
-                    }
-                    uint32_t incl = tlen;
-#pragma unroll
-                    for (int o = 1; o < 32; o <<= 1) {
-                        const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                        if (lane >= (uint32_t)o) incl += t;
-                    }
-                    const uint32_t off = bits + incl - tlen;    // bit of the window where my token starts
-                    // the first token of a sub-block marks where that sub-block's string starts
-                    if (valid && first_of_sb) s_start[warp * 4u + part * (kChunk / kSB) + ((uint32_t)pos >> 8)] = off;
-                    or_bits32(window, off, tokA, lenA);
-                    if (LEVELSET != kLevelsExp) or_bits32(window, off + lenA, tokB, lenB);
-                    bits += __shfl_sync(0xffffffffu, incl, 31);
-                    carry_pos = __shfl_sync(0xffffffffu, pos, min(ntok - t0, 32u) - 1u);
-                }
-                my_nnz += ntok;                             // warp uniform: counted once below
-                __syncwarp();
+            if (MODE == kModeErc && lane == 0) {
+                meta->sb_bits[sbq] = bits - start_bits;
+                meta->sb_src[sbq] = start_bits;
+            }
+            if (q < 3u) {                                   // the draws of the next sub-block
+                const uint64_t ctr0 = ctr_warp + 64u * (q + 1u), ctr1 = ctr0 + 32u;
+                rn0 = philox4x32_10((uint32_t)ctr0, (uint32_t)(ctr0 >> 32), c2, c3, P.round_keys);
+                rn1 = philox4x32_10((uint32_t)ctr1, (uint32_t)(ctr1 >> 32), c2, c3, P.round_keys);
             }
         }
-        if (MODE == kModeErc) {
-            // sub-block strings follow one another: an empty one starts where the next one does
-            uint32_t st = lane < 4 ? s_start[warp * 4u + lane] : 0xFFFFFFFFu;
-            uint32_t s3 = __shfl_sync(0xffffffffu, st, 3), s2 = __shfl_sync(0xffffffffu, st, 2);
-            uint32_t s1 = __shfl_sync(0xffffffffu, st, 1), s0 = __shfl_sync(0xffffffffu, st, 0);
-            if (s3 == 0xFFFFFFFFu) s3 = bits;
-            if (s2 == 0xFFFFFFFFu) s2 = s3;
-            if (s1 == 0xFFFFFFFFu) s1 = s2;
-            if (s0 == 0xFFFFFFFFu) s0 = s1;
-            if (lane < 4) {
-                const uint32_t begin = lane == 0 ? s0 : lane == 1 ? s1 : lane == 2 ? s2 : s3;
-                const uint32_t end = lane == 0 ? s1 : lane == 1 ? s2 : lane == 2 ? s3 : bits;
-                s_sb_src[warp * 4u + lane] = begin;
-                s_sb_bits[warp * 4u + lane] = end - begin;
-            }
-            if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
-        } else {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) my_nnz += __shfl_xor_sync(0xffffffffu, my_nnz, o);
-            if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
-        }
-        if (tid == 0) s_tile[(it + 1u) & 1u] = next_ticket;
-        bar_sync<kBarWork, kEncThreads>();                    // B2: the tile's data is no longer read; lengths visible
-        if (tid == 0) start_copy((it + 1u) & 1u);           // the next tile's bytes arrive while this one is packed
 
-        // ---- layout of the tile's records ---------------------------------------------
+        // The warp is done with its part of the tile (and with the lists that lay over it): the bytes of its
+        // part of the next tile are asked for now and arrive while the warp finishes this one.
+        __syncwarp();
+        if (lane == 0) start_copy(it + 1u);
         if (MODE == kModeErc) {
-            uint32_t* stg = stage + sg * P.stage_words;                      // this tile's image; the others are pending
-            // every warp runs the same scan over the 32 sub-block lengths
-            const uint32_t sb = lane;
-            const uint32_t v = sb < nsb_tile ? s_sb_bits[sb] : 0u;
-            uint32_t incl = v;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= (uint32_t)o) incl += t;
-            }
-            const uint32_t excl = incl - v;
-            const uint32_t bi = bi_lane, sb0 = bi * spb;
-            const uint32_t sb_last = min(sb0 + spb, nsb_tile) - 1u;         // meaningful when sb < nsb_tile
-            const uint32_t excl0 = __shfl_sync(0xffffffffu, excl, sb0 & 31u);
-            const uint32_t incl_last = __shfl_sync(0xffffffffu, incl, sb_last & 31u);
-            const uint32_t nsb_blk = sb_last - sb0 + 1u;
-            const uint32_t head_words = 1u + (nsb_blk + 1u) / 2u;
-            const bool leader = sb < nsb_tile && sb == sb0;
-            const uint32_t blk_words = leader ? head_words + (incl_last - excl0 + 31u) / 32u : 0u;
-            uint32_t wincl = blk_words;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t t = __shfl_up_sync(0xffffffffu, wincl, o);
-                if (lane >= (uint32_t)o) wincl += t;
-            }
-            const uint32_t wexcl = wincl - blk_words;
-            const uint32_t blk_off = __shfl_sync(0xffffffffu, wexcl, sb0 & 31u);    // words before my block
-            const uint32_t my_bitoff = 32u * (blk_off + head_words) + (excl - excl0);   // where sub-block `lane` goes
-            const uint32_t tile_words = __shfl_sync(0xffffffffu, wincl, 31);
-            const uint32_t code_bits = __shfl_sync(0xffffffffu, incl, 31);
-            // announce the tile's size to its successors at once; the writer warp looks up its place
-            if (tid == 0) announce_tile(tile_state, group_state, tile, tile_words);
-            // this stage held the tile of P.stages iterations ago: the writer must be done with it
-            if (it >= P.stages) stage_sync<kBarFree>(sg);
-            // header words of the blocks: norm, then the u16 lengths two per word.  Lanes 4w .. 4w+3
-            // of warp w stand for the warp's own sub-blocks, whose norms it holds.
-            if ((lane >> 2) == warp && sb < nsb_tile) {
-                const uint32_t q = lane & 3u;
-                const float nq = q == 0 ? norm_q[0] : q == 1 ? norm_q[1] : q == 2 ? norm_q[2] : norm_q[3];
-                if (leader) stg[blk_off] = __float_as_uint(nq);
-                const uint32_t sbi = sb - sb0;
-                atomicOr(stg + blk_off + 1u + sbi / 2u, v << (16u * (sbi & 1u)));
-            }
-            if (warp == 0) {
-                Pending& pd = s_pend[sg];
-                pd.blk_wordoff[lane] = __shfl_sync(0xffffffffu, wexcl, (lane * spb) & 31u);
-                if (lane == 0) {
-                    pd.tile = tile;
-                    pd.words = tile_words;
-                    pd.nblk = nblk_tile;
-                    pd.code_bits = code_bits;
-                    pd.nnz = s_nnz;
-                    pd.valid = 1;
-                    s_nnz = 0;
-                }
-            }
-
-            // ---- every warp moves its sub-block strings to their place in the staged tile ----
-            __syncwarp();
-#pragma unroll 1
-            for (uint32_t q = 0; q < 4; q += coarse ? 4u : 1u) {
-                // the strings of sub-blocks of one block follow one another in the window and in the
-                // tile alike, so a warp whose four sub-blocks share a block moves them in one piece
-                const uint32_t sbq = warp * 4u + q;
-                if (sbq >= nsb_tile) break;
-                const uint32_t len = coarse ? bits : s_sb_bits[sbq], src = coarse ? 0u : s_sb_src[sbq];
-                const uint32_t dst = __shfl_sync(0xffffffffu, my_bitoff, sbq);
-                if (len == 0) continue;
-                const uint32_t w_first = dst >> 5, w_last = (dst + len - 1u) >> 5;
-                for (uint32_t w = w_first + lane; w <= w_last; w += 32) {
-                    const int sbit = (int)src + (int)(32u * w) - (int)dst;
-                    uint32_t val = bits_at(window, sbit);
-                    const uint32_t head = 32u * w < dst ? dst - 32u * w : 0u;     // bits of this word before the string
-                    const uint32_t tail_end = min(dst + len - 32u * w, 32u);      // bits of this word up to its end
-                    uint32_t mask = 0xFFFFFFFFu >> head;
-                    if (tail_end < 32u) mask &= ~(0xFFFFFFFFu >> tail_end);
-                    val &= mask;
-                    if (val) atomicOr(stg + w, val);
+            if (lane == 0) {
+                meta->wnnz[warp] = cum;
+                if (warp == 0) {
+                    meta->tile = tile;
+                    meta->nsb = nsb_tile;
                 }
             }
             __syncwarp();
-            for (uint32_t i = lane; i < (bits + 31u) / 32u + 2u; i += 32) window[i] = 0;   // ready for the next tile
-            stage_arrive<kBarStaged>(sg);                  // the writer may take the tile
-        } else {
-            uint64_t tile_off;
-            uint32_t tile_words;
-            if (G.bucket <= kBLK) {
-                tile_off = first_block * G.rec_words;
-                tile_words = (nblk_tile - 1u) * G.rec_words + 1u +
-                             ((tile_len - (nblk_tile - 1u) * G.bucket) * G.width + 31u) / 32u;
-                // norm words: lanes 4w .. 4w+3 of warp w stand for the warp's own sub-blocks
-                if ((lane >> 2) == warp && lane < nsb_tile && lane == bi_lane * spb) {
-                    const uint32_t q = lane & 3u;
-                    const float nq = q == 0 ? norm_q[0] : q == 1 ? norm_q[1] : q == 2 ? norm_q[2] : norm_q[3];
-                    stage[bi_lane * G.rec_words] = __float_as_uint(nq);
-                }
-            } else {
-                tile_off = bucket_idx * G.rec_words + 1u + (uint64_t)bib * (kBLK * G.width / 32u);
-                tile_words = (tile_len * G.width + 31u) / 32u;
-                if (bib == 0 && tid == 0) payload[bucket_idx * G.rec_words] = __float_as_uint(norm_q[0]);
-            }
-            bar_sync<kBarWork, kEncThreads>();                // the staged fields are complete
-            for (uint32_t i = tid; i < tile_words; i += kEncThreads) {
-                payload[tile_off + i] = stage[i];
-                stage[i] = 0;
-            }
-            if (tid == 0) {
-                s_tot.nnz += s_nnz;
-                s_tot.tiles += 1;
-                s_nnz = 0;
-            }
+            pair_arrive<kBarDone>(it & 1u);                 // the writer may lay the tile out
+            if (it > 0) merge_tile(it - 1u, prev_bits);     // the tile before it has been laid out long ago
+            prev_bits = bits;
         }
     }
 
     if (MODE == kModeErc && !writer) {
-        // ---- the workers ran `it` iterations (the next one would use stage sg): wait until the writer
-        // has written the last tiles, telling it in between that no further one comes ----
-        if (it >= P.stages) stage_sync<kBarFree>(sg);       // tile it - stages: its barriers are used again below
+        // ---- the workers ran `it` iterations: tell the writer that no further tile comes, and move the
+        // last tile's strings into its image ----
         if (tid == 0) s_tot.stop = it;
-        stage_arrive<kBarStaged>(sg);
-        for (uint32_t back = P.stages - 1u; back >= 1u; --back) {   // tiles it - stages + 1 .. it - 1
-            if (it >= back) {
-                const uint32_t bb = (sg + P.stages - back) % P.stages;
-                stage_sync<kBarFree>(bb);
-            }
-        }
+        pair_arrive<kBarDone>(it & 1u);
+        if (it > 0) merge_tile(it - 1u, prev_bits);
+    }
+    if (MODE == kModeFixed) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) cta_nnz += __shfl_xor_sync(0xffffffffu, cta_nnz, o);
+        if (lane == 0 && cta_nnz) atomicAdd(&s_nnz, cta_nnz);
     }
     __syncthreads();                                        // every write of this CTA lies behind this barrier
-    if (tid == 0) finish_cta<MODE>(P, s_tot.tiles, s_tot.nnz, s_tot.code_bits);
+    if (tid == 0) {
+        const bool last = MODE == kModeErc ? finish_cta<MODE>(P, s_tot.tiles, s_tot.nnz, s_tot.code_bits)
+                                           : finish_cta<MODE>(P, it, s_nnz, 0);
+        if (last) s_last = 1;
+    }
+    __syncthreads();
+    if (s_last) {
+        // Every tile of the call has been written: nobody looks at the call's scan state any more.  The CTA
+        // that finished last leaves it zeroed, so the next call on this workspace starts without a clearing pass.
+        uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
+        const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + G.ntiles + (G.ntiles + 31) / 32;
+        for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -996,9 +1108,11 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
     return cudaGetLastError();
 }
 
-// shared memory of one CTA: the tile, its staged image, and per warp a bit window and a token list
+// shared memory of one CTA: the tile buffers and, in the ERC mode, two staged tile images and two sets of per-warp token windows
 size_t encode_smem_bytes(const EncodeParams& P) {
-    return 4u * ((size_t)kBLK + (size_t)P.stages * P.stage_words + (size_t)kEncWarps * P.warp_smem_words);
+    size_t words = kBLK;
+    if (P.geo.mode == kModeErc) words += 2u * (size_t)P.stage_words + 2u * (size_t)kEncWarps * P.window_words;
+    return 4u * words;
 }
 
 constexpr int kEncMaxDynSmem = 112 * 1024;
@@ -1019,7 +1133,7 @@ static int blocks_per_sm(const EncodeParams& P) {
     const int threads = M == kModeErc ? (int)kEncAllThreads : kEncThreads;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, encode_kernel<L, M>, threads, encode_smem_bytes(P)) != cudaSuccess)
         return 0;
-    return n < kEncMinBlocks ? n : kEncMinBlocks;
+    return n;
 }
 
 int encode_blocks_per_sm(const EncodeParams& P) {

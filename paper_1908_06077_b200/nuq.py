@@ -14,11 +14,13 @@ import torch
 
 from . import build as _build
 
-NUQ_OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BAD_STREAM, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+NUQ_OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BAD_STREAM, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -1, -2, -3, -4, -5, -6
+WARN_NONFINITE = 1
 NORM_L2, NORM_LINF = 0, 1
 LEVELS_EXP, LEVELS_UNIFORM = 0 << 8, 1 << 8
 MODE_ERC, MODE_FIXED = 0 << 16, 1 << 16
 TEST_NORMS = 1 << 24
+TEST_SHORT_PATIENCE = 1 << 25
 HEADER_WORDS = 16
 STATIC_SCRATCH_BYTES = 512 * 1024
 

@@ -74,3 +74,85 @@ def test_c3_decode_of_eight_workers_as_benchmarked():
     assert rc == 0
     got = gpu_decode(streams, d, 8192, 4)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_c2_in_full():
+    """Config C2: the ResNet-18-sized layout with outliers at 50 sigma, four workers: every worker's
+    symbols against the oracle's, then the decode call of the benchmark (four streams side by side)."""
+    from paper_1908_06077_b200 import inputs
+    gs = [inputs.c2_input(k) for k in (1, 2, 3, 4)]
+    d = gs[0].size
+    streams = []
+    for k, g in enumerate(gs):
+        got, _ = gpu_encode(g, 8192, 4, 0, seed=k + 1, offset=0)
+        nbad, rel = compare_symbols(g, 8192, 4, 0, k + 1, 0, got)
+        assert nbad <= 1e-5 * d and rel <= 1e-6
+        streams.append(got)
+    rc, want = O.decode_accumulate(streams, d, 8192, 4)
+    assert rc == 0
+    got = gpu_decode(streams, d, 8192, 4)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_c3_s3_encode_matches_oracle(c3_inputs):
+    g = c3_inputs[2]
+    got, _ = gpu_encode(g, 8192, 3, 0, seed=3, offset=0)
+    nbad, rel = compare_symbols(g, 8192, 3, 0, 3, 0, got)
+    assert nbad <= 1e-5 * g.size and rel <= 1e-6
+    # given the norms the GPU took, the whole container is the oracle's
+    rc, _, _, gnorms = O.decode_symbols(got, g.size, 8192, 3)
+    assert rc == 0
+    want, _ = O.encode(g, 8192, 3, 0, 3, 0, norms=gnorms)
+    if nbad == 0:
+        assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("norm", [O.NORM_L2, O.NORM_LINF])
+def test_c5_decode_of_uniform_level_streams(c3_inputs, norm):
+    """Config C5: the comparison quantizers (uniform levels k/16 with the Euclidean and with the max
+    norm) at the ResNet-50 size: GPU-written containers decoded and summed by the GPU, against the oracle."""
+    flags = O.make_flags(norm, O.LEVELS_UNIFORM)
+    d = c3_inputs[0].size
+    streams = [gpu_encode(g, 8192, 4, flags, seed=k + 1, offset=0)[0] for k, g in enumerate(c3_inputs)]
+    rc, want = O.decode_accumulate(streams, d, 8192, 4)
+    assert rc == 0
+    got = gpu_decode(streams, d, 8192, 4)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+@pytest.fixture(scope="module")
+def c4_inputs():
+    from paper_1908_06077_b200 import inputs
+    return [inputs.c4_input(k) for k in (1, 2)]
+
+
+@pytest.mark.parametrize("bucket", [8192, 512, 65536])
+def test_c4_at_its_stated_length(c4_inputs, bucket):
+    """Config C4 at d = 2^30: table offsets beyond 2^32 bits, 131072 tiles and thousands of look-back
+    groups, two million buckets at bucket 512, the separate norm pass of the wide buckets, and the
+    decoder's instance for two streams.  Worker 1: the norms of all buckets against the oracle's, and
+    the whole container against the oracle's encode given those norms (bit-exact streams for equal
+    norms).  Then the GPU's sum of both workers' containers against the oracle's sum of them."""
+    d = c4_inputs[0].size
+    assert d == 1 << 30
+    streams = [gpu_encode(g, bucket, 4, 0, seed=k + 1, offset=0)[0] for k, g in enumerate(c4_inputs)]
+    g, st = c4_inputs[0], streams[0]
+    assert O.header(st)["container_bits"] == 32 * st.size
+    table_words = 2 * (O.header(st)["nblk"] + 1)
+    gnorms = np.empty((d + bucket - 1) // bucket, np.float32)
+    # the norm word of a bucket is the first word of its first coding block
+    offs = st[16:16 + table_words].view(np.uint64)[:-1]
+    step = max(1, bucket // 8192)
+    gnorms[:] = st[16 + table_words + (offs[::step] >> np.uint64(5)).astype(np.int64)].view(np.float32)
+    norms = O.bucket_norms(g, bucket, O.NORM_L2)
+    rel = np.abs(gnorms.astype(np.float64) - norms) / norms
+    print(f"C4 bucket {bucket}: largest relative norm difference {rel.max():.3g}, "
+          f"{int((gnorms != norms).sum())} of {norms.size} norms differ in the last place")
+    assert rel.max() <= 1e-6
+    want, _ = O.encode(g, bucket, 4, 0, 1, 0, norms=gnorms)
+    assert want.size == st.size and np.array_equal(st, want)
+    del want
+    rc, want = O.decode_accumulate(streams, d, bucket, 4)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, 4)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))

@@ -119,7 +119,7 @@ def test_invalid_arguments_are_refused():
     torch, nuq = require_cuda()
     g = torch.zeros(4096, device="cuda")
     for bucket, s, flags in ((100, 3, 0), (0, 3, 0), (1024, 0, 0), (1024, 15, 0), (1024, 9, nuq.LEVELS_UNIFORM),
-                             (1024, 3, 2), (1024, 3, 1 << 25), (131072, 3, 0), (1024, 3, nuq.TEST_NORMS)):
+                             (1024, 3, 2), (1024, 3, 1 << 26), (131072, 3, 0), (1024, 3, nuq.TEST_NORMS)):
         assert nuq.encode_bound(4096, bucket, s, flags & ~nuq.TEST_NORMS) == 0 or flags & nuq.TEST_NORMS
         with pytest.raises(nuq.NuqError) as e:
             nuq.encode(g, bucket, s, flags, out=torch.empty(65536, dtype=torch.int32, device="cuda"))
@@ -169,8 +169,16 @@ def test_degenerate_buckets():
     g[2048 + 9] = np.inf                       # infinite norm
     g[3072:4096] = 1e-42                       # 2^s / norm overflows
     for flags in (0, O.make_flags(mode=O.MODE_FIXED), O.make_flags(L2, UNI), O.make_flags(LINF, UNI)):
-        want, _ = O.encode(g, bucket, 4, flags, 1, 0)
-        got, _ = gpu_encode(g, bucket, 4, flags, 1, 0)
+        # buckets 1 to 3 cannot be quantized: the encoder says so (bucket 0 is all zero, which is no warning)
+        got, _ = gpu_encode(g, bucket, 4, flags, 1, 0, expect_status=1)
+        # the degenerate buckets' norm words are the oracle's bit for bit, the ordinary bucket's norm agrees
+        # to 1e-6; given the norms the GPU used, the whole container is the oracle's
+        rc, _, _, gnorms = O.decode_symbols(got, d, bucket, 4)
+        assert rc == 0
+        onorms = O.bucket_norms(g, bucket, flags & 0xff)
+        assert np.array_equal(gnorms[:4].view(np.uint32), onorms[:4].view(np.uint32))
+        assert abs(float(gnorms[4]) - float(onorms[4])) <= 1e-6 * float(onorms[4])
+        want, _ = O.encode(g, bucket, 4, flags, 1, 0, norms=gnorms)
         assert np.array_equal(got, want)
         acc = gpu_decode([got], d, bucket, 4)
         assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([want], d, bucket, 4)[1].view(np.uint32))
@@ -265,3 +273,47 @@ def test_more_streams_than_one_group(K):
     assert rc == 0
     got = gpu_decode(streams, d, bucket, s)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_a_scan_wait_that_runs_out_is_reported_and_does_no_harm():
+    """The look-back over tile sizes waits with a limit.  A test flag shortens that limit to two polls, so
+    that on a vector of several thousand tiles some writer warp does give up: the call must come back at
+    once with NUQ_ERR_TIMEOUT latched, write nothing outside its buffer, and leave the library in a state
+    in which the next ordinary call is bit-exact again.  Nothing is withheld and nothing can hang: the
+    flag only makes the wait shorter."""
+    import time
+    torch, nuq = require_cuda()
+    from paper_1908_06077_b200 import inputs
+    g = inputs.c3_input(1)
+    ref, ref_bits = gpu_encode(g, 8192, 4, 0, seed=1, offset=0)
+    seen = []
+    for attempt in range(4):
+        gd = torch.from_numpy(g).cuda()
+        nbytes = nuq.encode_bound(gd.numel(), 8192, 4, 0)
+        out = torch.full((nbytes // 4 + 64,), -1515870811, dtype=torch.int32, device="cuda")
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        nuq.encode(gd, 8192, 4, nuq.TEST_SHORT_PATIENCE, 1, 0, out=out)
+        status = nuq.last_status()
+        dt = time.perf_counter() - t0
+        assert dt < 0.5, dt
+        assert status in (0, nuq.ERR_TIMEOUT), status
+        host = out.cpu().numpy().view(np.uint32)
+        assert (host[nbytes // 4:] == np.uint32(0xA5A5A5A5)).all()
+        seen.append(status)
+        if status == nuq.ERR_TIMEOUT:
+            break
+    assert nuq.ERR_TIMEOUT in seen, seen
+    again, again_bits = gpu_encode(g, 8192, 4, 0, seed=1, offset=0)
+    assert again_bits == ref_bits and np.array_equal(again, ref)
+
+
+def test_nonfinite_norms_raise_a_warning_only():
+    torch, nuq = require_cuda()
+    g = _input(8192, 5)
+    gpu_encode(g, 1024, 3, 0, 1, 0)                                  # ordinary data: no warning
+    g[100] = np.inf
+    got, _ = gpu_encode(g, 1024, 3, 0, 1, 0, expect_status=nuq.WARN_NONFINITE)
+    want, _ = O.encode(g, 1024, 3, 0, 1, 0, norms=O.decode_symbols(got, g.size, 1024, 3)[3])
+    assert np.array_equal(got, want)
+    gpu_encode(np.zeros(4096, np.float32), 1024, 3, 0, 1, 0)         # an all-zero vector is not a warning
