@@ -293,6 +293,89 @@ __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const St
     if (max_sym >= nlev) latch_status(P.ws, kErrBadStream);
 }
 
+// The same for the 4-bit fields of the paper's "4-bit" variant (exponential levels with s = 3 .. 6; a
+// sign bit and a 3-bit level index) and buckets that are multiples of 2048 elements, where almost all
+// the work can be taken out of the inner loop: a CTA takes a tile of up to 8192 elements of one bucket
+// by ticket, builds, per stream, the table of the 16 values a field can stand for (+-norm * level, the
+// same multiplication as everywhere else, so the sums are bit-identical), and then every thread turns 8
+// consecutive elements -- one word of every stream -- into table look-ups and adds, in stream order.
+// Symbols that do not exist are found on whole words (a carry out of the index bits).
+template <uint32_t LEVELSET>
+__device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const StreamHead* heads) {
+    __shared__ float s_tab[kMaxK][16];
+    __shared__ unsigned long long s_ticket;
+    const Geometry& G = P.geo;
+    const uint32_t K = P.K, tid = threadIdx.x;
+    const uint32_t nlev = heads[0].nlev;                    // <= 8
+    const uint32_t rec_words = 1u + G.bucket / 8u;
+    const uint32_t tile_elems = G.bucket < kBLK ? G.bucket : kBLK;
+    const uint32_t tiles_per_bucket = G.bucket / tile_elems;
+    const uint64_t ntiles = G.nb * tiles_per_bucket;
+    const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
+    const uint32_t over = (8u - nlev) * 0x11111111u;        // added to the index bits, a missing symbol carries into bit 3
+    uint32_t bad = 0;
+    for (;;) {
+        __syncthreads();                                    // the tables and the ticket of the previous tile are no longer read
+        if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        __syncthreads();
+        const uint64_t tile = s_ticket;
+        if (tile >= ntiles) break;
+        const uint64_t b = tile / tiles_per_bucket;
+        const uint32_t part = (uint32_t)(tile % tiles_per_bucket);
+        const uint32_t bucket_len = b == G.nb - 1 ? (uint32_t)last_len : G.bucket;
+        const uint32_t first = part * tile_elems;           // first element of the tile within its bucket
+        if (first >= bucket_len) continue;
+        const uint32_t tile_len = bucket_len - first < tile_elems ? bucket_len - first : tile_elems;
+        for (uint32_t t = tid; t < 16u * K; t += blockDim.x) {
+            const uint32_t k = t >> 4, f = t & 15u, sym = f & 7u;
+            const float norm = __uint_as_float(__ldg(heads[k].hdr + kHeaderWords + b * rec_words));
+            const float v = sym && sym < nlev ? level_times_norm(norm, LEVELSET, G.s, sym) : 0.0f;
+            s_tab[k][f] = (f & 8u) ? -v : v;
+        }
+        __syncthreads();
+        float* const dst_tile = P.acc + b * G.bucket + first;
+        const uint64_t word0 = kHeaderWords + b * rec_words + 1u + first / 8u;     // the tile's first field word in a container
+        for (uint32_t el = 8u * tid; el < tile_len; el += 8u * blockDim.x) {
+            float sum[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) sum[i] = 0.0f;
+            for (uint32_t k0 = 0; k0 < K; k0 += 8u) {
+                uint32_t wv[8];
+#pragma unroll
+                for (uint32_t j = 0; j < 8; ++j) wv[j] = k0 + j < K ? __ldg(heads[k0 + j].hdr + word0 + el / 8u) : 0u;
+#pragma unroll
+                for (uint32_t j = 0; j < 8; ++j) {
+                    if (k0 + j < K) {
+                        const uint32_t x = wv[j];
+                        bad |= ((x & 0x77777777u) + over) & 0x88888888u;
+                        // the eight fields times four (byte offsets into the table), four to a register
+                        const uint32_t a = (x >> 2) & 0x3C3C3C3Cu, c = (x << 2) & 0x3C3C3C3Cu;   // elements 0 2 4 6 / 1 3 5 7 from the top byte
+                        const char* tab = reinterpret_cast<const char*>(s_tab[k0 + j]);
+                        sum[0] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4443));
+                        sum[1] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4443));
+                        sum[2] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4442));
+                        sum[3] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4442));
+                        sum[4] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4441));
+                        sum[5] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4441));
+                        sum[6] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4440));
+                        sum[7] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4440));
+                    }
+                }
+            }
+            float* dst = dst_tile + el;
+            if (el + 8u <= tile_len) {
+                *reinterpret_cast<float4*>(dst) = make_float4(sum[0], sum[1], sum[2], sum[3]);
+                *reinterpret_cast<float4*>(dst + 4) = make_float4(sum[4], sum[5], sum[6], sum[7]);
+            } else {
+#pragma unroll
+                for (uint32_t i = 0; i < 8; ++i)
+                    if (el + i < tile_len) dst[i] = sum[i];
+            }
+        }
+    }
+    if (bad) latch_status(P.ws, kErrBadStream);
+}
+
 // The kernel of that path.  It is launched when the library believes that all streams are in the
 // fixed-width mode (it wrote them itself); it checks the headers like the general kernel and, if they
 // say otherwise, leaves everything to the general kernel, which is launched behind it in any case and
@@ -313,7 +396,10 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
     if (heads[0].levelset == kLevelsExp) {                  // s <= 14: at most 16 levels, 5 bits
         switch (s_width) {
             case 3: decode_all_fixed<3, kLevelsExp>(P, heads); break;
-            case 4: decode_all_fixed<4, kLevelsExp>(P, heads); break;
+            case 4:
+                if (P.geo.bucket % 2048u == 0) decode_fixed4_tiles<kLevelsExp>(P, heads);
+                else decode_all_fixed<4, kLevelsExp>(P, heads);
+                break;
             case 5: decode_all_fixed<5, kLevelsExp>(P, heads); break;
             default: break;
         }
