@@ -317,3 +317,50 @@ def test_nonfinite_norms_raise_a_warning_only():
     want, _ = O.encode(g, 1024, 3, 0, 1, 0, norms=O.decode_symbols(got, g.size, 1024, 3)[3])
     assert np.array_equal(got, want)
     gpu_encode(np.zeros(4096, np.float32), 1024, 3, 0, 1, 0)         # an all-zero vector is not a warning
+
+
+@pytest.mark.parametrize("d,bucket,s", [(70001, 1024, 4), (8192 * 3 + 17, 8192, 2), (200000, 65536, 4), (50000, 512, 7),
+                                        (33000, 256, 3), (255, 256, 3)])
+@pytest.mark.parametrize("K", [5, 8, 11])
+def test_five_to_eleven_erc_streams(d, bucket, s, K):
+    """One partly filled group of streams, one full group, and a full group followed by a partly filled one."""
+    streams = [O.encode(_input(d, 500 * k + d + s), bucket, s, 0, seed=k + 1, offset=k)[0] for k in range(K)]
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+@pytest.mark.parametrize("d,bucket,s", [(20000, 256, 4), (50000, 1024, 5), (100000, 8192, 4)])
+def test_eight_streams_of_mixed_density_and_lists_that_run_over(d, bucket, s):
+    """Every coordinate a token in some streams, ordinary density in others: rounds of positions, and
+    rounds that have to be taken again because a list ran over."""
+    rng = np.random.default_rng(d + 1)
+    streams = []
+    for k in range(8):
+        if k % 3 == 0:
+            g = np.where(rng.random(d) < 0.5, -1.0, 1.0).astype(np.float32) * (1.0 + 0.25 * rng.random(d).astype(np.float32))
+        elif k % 3 == 1:
+            g = _input(d, 9000 + k)
+            g[: d // 2] = np.where(rng.random(d // 2) < 0.5, -1.0, 1.0)      # dense front half, sparse back half
+        else:
+            g = _input(d, 9100 + k)
+        streams.append(O.encode(g, bucket, s, 0, seed=k + 1, offset=0)[0])
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_malformed_container_among_six_streams():
+    d, bucket, s = 40000, 1024, 3
+    good = [O.encode(_input(d, 40 + k), bucket, s, 0, k + 1, 0)[0] for k in range(6)]
+    nblk = 40
+    payload0 = 16 + 2 * (nblk + 1)
+    for word, value in [(0, 0), (5, 4), (16 + 2 * 3, 5), (16 + 2 * 3, 0xFFFFFF00), (payload0 + 1, 0xFFFFFFFF),
+                        (payload0 + 4, 0xFFFFFFFF)]:
+        bad = good[2].copy()
+        bad[word] = value
+        gpu_decode(good[:2] + [bad] + good[3:], d, bucket, s, expect_status=-3)
+    want = O.decode_accumulate(good, d, bucket, s)[1]
+    assert np.array_equal(gpu_decode(good, d, bucket, s).view(np.uint32), want.view(np.uint32))
