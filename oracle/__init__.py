@@ -14,7 +14,7 @@ import numpy as np
 from .build import build as _build
 
 NORM_L2, NORM_LINF = 0, 1
-LEVELS_EXP, LEVELS_UNIFORM = 0, 1
+LEVELS_EXP, LEVELS_UNIFORM, LEVELS_TABLE = 0, 1, 2
 MODE_ERC, MODE_FIXED = 0, 1
 SB = 256
 BLK = 32 * SB
@@ -43,6 +43,7 @@ def _sig(name, res, *args):
 _philox = _sig("nuq_oracle_philox4x32_10", None, _u32p, _u32p, _u32p)
 _draw_word = _sig("nuq_oracle_draw_word", C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64)
 _draw_uniform = _sig("nuq_oracle_draw_uniform", C.c_float, C.c_uint64, C.c_uint64, C.c_uint64)
+_set_levels = _sig("nuq_oracle_set_levels", C.c_int, _f32p, C.c_uint32)
 _num_levels = _sig("nuq_oracle_num_levels", C.c_uint32, C.c_uint32, C.c_uint32)
 _level_value = _sig("nuq_oracle_level_value", C.c_double, C.c_uint32, C.c_uint32, C.c_uint32)
 _fixed_width = _sig("nuq_oracle_fixed_width", C.c_uint32, C.c_uint32, C.c_uint32)
@@ -83,6 +84,14 @@ def draw_word(seed, offset, i):
 
 def draw_uniform(seed, offset, i):
     return float(_draw_uniform(seed, offset, i))
+
+
+def set_levels(interior):
+    """the interior levels l_1 < ... < l_s of the level sequence (0, l_1, ..., l_s, 1) that LEVELS_TABLE calls use"""
+    lv = np.ascontiguousarray(interior, np.float32)
+    rc = _set_levels(lv, lv.size)
+    if rc != 0:
+        raise ValueError("not a level sequence")
 
 
 def num_levels(levelset, s):

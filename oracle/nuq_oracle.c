@@ -16,6 +16,8 @@
  *   - aggregate  sum_i g^_i    Algorithm 1, aggregation line (without alpha/K)
  *   - closed-form variance     Lemma 7 / Eq. (genvar)
  *   - uniform level set k/2^s  (QSGD / QSGDinf comparison, Sec. 1 and 3)
+ *   - arbitrary level sequences L = (0, l_1, ..., l_s, 1), e.g. L_p = (0, p^s, ..., p, 1)
+ *                              (Sec. 3.3, "general level sequences"), given as a table
  *
  * Everything the paper leaves open (bucket tail, fp32 arithmetic order, random
  * generator, container layout) is fixed here in the most literal form; the
@@ -30,7 +32,9 @@
  * 24-bit draw, unbiasedness by full enumeration on tiny vectors and by Monte
  * Carlo, Lemma 7 closed form against the Theorem 4 / Theorem 12 worked
  * examples, Theorem 1 and Lemma 10 bounds, round trip, Philox against the
- * cuRAND host generator.
+ * cuRAND host generator; for level tables: the levels of L_p from exact
+ * fractions, rounding probabilities by enumeration against exact rational
+ * arithmetic, unbiasedness by enumeration, Lemma 7 on hand-worked vectors.
  */
 #include <math.h>
 #include <stdint.h>
@@ -49,7 +53,8 @@
 #define ORC_HEADER_WORDS 16u
 
 enum { NORM_L2 = 0, NORM_LINF = 1 };
-enum { LEVELS_EXP = 0, LEVELS_UNIFORM = 1 };
+enum { LEVELS_EXP = 0, LEVELS_UNIFORM = 1, LEVELS_TABLE = 2 };
+#define ORC_MAX_S 14u
 enum { MODE_ERC = 0, MODE_FIXED = 1 };
 
 /* ------------------------------------------------------------------ */
@@ -91,14 +96,38 @@ float nuq_oracle_draw_uniform(uint64_t seed, uint64_t offset, uint64_t i) {
 /* ------------------------------------------------------------------ */
 /* Level sets.                                                          */
 /* ------------------------------------------------------------------ */
+/* The level table of LEVELS_TABLE (Sec. 3.3): l_0 = 0 < l_1 < ... < l_s < l_{s+1} = 1 in fp32, and
+ * 1 / (l_{j+1} - l_j) in fp32 (one IEEE division each), which the quantizer multiplies by.            */
+typedef struct { uint32_t s; float level[ORC_MAX_S + 2]; float inv_width[ORC_MAX_S + 2]; } level_table;
+static level_table g_table;
+
+static int make_table(const float* interior, uint32_t s, level_table* t) {
+    if (s < 1 || s > ORC_MAX_S) return ORC_ERR_ARG;
+    t->s = s;
+    t->level[0] = 0.0f;
+    for (uint32_t j = 1; j <= s; ++j) t->level[j] = interior[j - 1];
+    t->level[s + 1] = 1.0f;
+    for (uint32_t j = 0; j <= s; ++j) {
+        if (!(t->level[j] < t->level[j + 1])) return ORC_ERR_ARG;          /* strictly increasing, no NaN */
+        t->inv_width[j] = 1.0f / (t->level[j + 1] - t->level[j]);
+        if (isinf(t->inv_width[j])) return ORC_ERR_ARG;
+    }
+    t->inv_width[s + 1] = 0.0f;
+    return ORC_OK;
+}
+
+/* the interior levels l_1 .. l_s that LEVELS_TABLE calls use from now on */
+int nuq_oracle_set_levels(const float* interior, uint32_t s) { return make_table(interior, s, &g_table); }
+
 /* number of levels including 0 and 1 */
 uint32_t nuq_oracle_num_levels(uint32_t levelset, uint32_t s) {
-    return levelset == LEVELS_EXP ? s + 2u : (1u << s) + 1u;
+    return levelset == LEVELS_UNIFORM ? (1u << s) + 1u : s + 2u;
 }
 
 /* value of level `sym` as an fp64 number (exact) */
 double nuq_oracle_level_value(uint32_t levelset, uint32_t s, uint32_t sym) {
     if (sym == 0) return 0.0;
+    if (levelset == LEVELS_TABLE) return sym <= g_table.s + 1 ? (double)g_table.level[sym] : 1.0;
     if (levelset == LEVELS_EXP) return ldexp(1.0, (int)sym - 1 - (int)s); /* l_j = 2^(j-1-s) */
     return ldexp((double)sym, -(int)s);                                    /* l_k = k / 2^s   */
 }
@@ -140,10 +169,10 @@ void nuq_oracle_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uint32
     }
 }
 
-/* A bucket is quantized only when 2^s / norm is a finite positive number. */
-static int bucket_is_live(float norm, uint32_t s, float* inv_out) {
+/* A bucket is quantized only when 2^s / norm (for a level table: 1 / norm) is a finite positive number. */
+static int bucket_is_live(float norm, uint32_t s, uint32_t levelset, float* inv_out) {
     if (!(norm > 0.0f) || isinf(norm)) return 0;
-    float inv = ldexpf(1.0f, (int)s) / norm;   /* one IEEE division per bucket */
+    float inv = (levelset == LEVELS_TABLE ? 1.0f : ldexpf(1.0f, (int)s)) / norm;   /* one IEEE division per bucket */
     if (isinf(inv) || inv != inv) return 0;
     *inv_out = inv;
     return 1;
@@ -157,6 +186,17 @@ static int bucket_is_live(float norm, uint32_t s, float* inv_out) {
 /* The coordinate moves to the upper level iff u < p.                    */
 /* ------------------------------------------------------------------ */
 static void split_coordinate(float v, float inv, uint32_t s, uint32_t levelset, uint32_t* low, float* p) {
+    if (levelset == LEVELS_TABLE) {
+        /* general level sequence (Sec. 3.3): r = |v| / norm, l_j <= r < l_{j+1},
+         * p = (r - l_j) / (l_{j+1} - l_j), all in fp32 */
+        float r = fabsf(v) * inv;
+        if (!(r < 1.0f)) r = 1.0f;    /* r > 1 can only come from norm rounding */
+        uint32_t j = 0;
+        while (j <= s && g_table.level[j + 1] <= r) ++j;
+        *low = j;
+        *p = (r - g_table.level[j]) * g_table.inv_width[j];   /* 0 at the top level */
+        return;
+    }
     float top = ldexpf(1.0f, (int)s);
     float y = fabsf(v) * inv;
     if (!(y < top)) y = top;          /* r > 1 can only come from norm rounding */
@@ -189,7 +229,7 @@ static uint32_t quantize_coordinate(float v, float inv, uint32_t s, uint32_t lev
 /* lower level index and probability of moving up, for the pins */
 void nuq_oracle_round_probability(float v, float norm, uint32_t s, uint32_t levelset, uint32_t* low, float* p) {
     float inv;
-    if (!bucket_is_live(norm, s, &inv)) { *low = 0; *p = 0.0f; return; }
+    if (!bucket_is_live(norm, s, levelset, &inv)) { *low = 0; *p = 0.0f; return; }
     split_coordinate(v, inv, s, levelset, low, p);
 }
 
@@ -199,7 +239,7 @@ void nuq_oracle_round_probability(float v, float norm, uint32_t s, uint32_t leve
 void nuq_oracle_quantize_bucket(const float* v, uint64_t n, float norm, uint32_t s, uint32_t levelset,
                                 uint64_t seed, uint64_t offset, uint64_t i0, uint8_t* sign, uint16_t* sym) {
     float inv;
-    if (!bucket_is_live(norm, s, &inv)) {
+    if (!bucket_is_live(norm, s, levelset, &inv)) {
         for (uint64_t i = 0; i < n; ++i) { sign[i] = 0; sym[i] = 0; }
         return;
     }
@@ -215,7 +255,7 @@ void nuq_oracle_quantize_bucket(const float* v, uint64_t n, float norm, uint32_t
 void nuq_oracle_quantize_with_draws(const float* v, uint64_t n, float norm, uint32_t s, uint32_t levelset,
                                     const float* u, uint8_t* sign, uint16_t* sym) {
     float inv;
-    int live = bucket_is_live(norm, s, &inv);
+    int live = bucket_is_live(norm, s, levelset, &inv);
     for (uint64_t i = 0; i < n; ++i) {
         uint32_t q = live ? quantize_coordinate(v[i], inv, s, levelset, u[i]) : 0u;
         sym[i] = (uint16_t)q;
@@ -332,10 +372,16 @@ static uint32_t max_level_code_bits(uint32_t levelset, uint32_t s) {
 }
 
 static int check_args(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint32_t levelset, uint32_t mode) {
-    if (d == 0 || bucket == 0 || s < 1 || s > 14) return ORC_ERR_ARG;
-    if (norm_kind > 1 || levelset > 1 || mode > 1) return ORC_ERR_ARG;
+    if (d == 0 || bucket == 0 || s < 1 || s > ORC_MAX_S) return ORC_ERR_ARG;
+    if (norm_kind > 1 || levelset > 2 || mode > 1) return ORC_ERR_ARG;
     if (levelset == LEVELS_UNIFORM && s > 8) return ORC_ERR_ARG;
     return ORC_OK;
+}
+
+/* A container with a level table carries the s interior levels (fp32 words) behind the 16 header
+ * words, padded with a zero word to an even count so that the offset table stays 8-byte aligned.  */
+static uint32_t header_words(uint32_t levelset, uint32_t s) {
+    return ORC_HEADER_WORDS + (levelset == LEVELS_TABLE ? ((s + 1u) & ~1u) : 0u);
 }
 
 /* bytes that always suffice for the container */
@@ -343,13 +389,14 @@ uint64_t nuq_oracle_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32
     uint32_t levelset = (flags >> 8) & 0xff, mode = (flags >> 16) & 0xff;
     if (check_args(d, bucket, s, flags & 0xff, levelset, mode) != ORC_OK) return 0;
     uint64_t nb = (d + bucket - 1) / bucket;
+    uint64_t hw = header_words(levelset, s);
     if (mode == MODE_FIXED) {
         uint64_t w = nuq_oracle_fixed_width(levelset, s);
-        return 4 * (ORC_HEADER_WORDS + nb * (1 + ((uint64_t)bucket * w + 31) / 32));
+        return 4 * (hw + nb * (1 + ((uint64_t)bucket * w + 31) / 32));
     }
     uint64_t nblk = count_blocks(d, bucket);
     uint64_t token_bits = d * (2 + (uint64_t)max_level_code_bits(levelset, s));
-    return 4 * ORC_HEADER_WORDS + 8 * (nblk + 1) + nblk * (4 + 64 + 4) + (token_bits + 7) / 8;
+    return 4 * hw + 8 * (nblk + 1) + nblk * (4 + 64 + 4) + (token_bits + 7) / 8;
 }
 
 /* ENCODE (App. A) of a whole vector, bucket by bucket.
@@ -361,14 +408,18 @@ int nuq_oracle_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     uint32_t norm_kind = flags & 0xff, levelset = (flags >> 8) & 0xff, mode = (flags >> 16) & 0xff;
     int rc = check_args(d, bucket, s, norm_kind, levelset, mode);
     if (rc != ORC_OK) return rc;
+    if (levelset == LEVELS_TABLE && g_table.s != s) return ORC_ERR_ARG;   /* the table set by nuq_oracle_set_levels */
     if (capacity_bytes < nuq_oracle_encode_bound(d, bucket, s, flags)) return ORC_ERR_CAPACITY;
     memset(out, 0, (size_t)nuq_oracle_encode_bound(d, bucket, s, flags));
 
     uint32_t* words = (uint32_t*)out;
     uint64_t nb = (d + bucket - 1) / bucket;
     uint64_t nblk = mode == MODE_ERC ? count_blocks(d, bucket) : nb;
-    uint64_t* table = (uint64_t*)(words + ORC_HEADER_WORDS);
-    uint32_t* payload = mode == MODE_ERC ? words + ORC_HEADER_WORDS + 2 * (nblk + 1) : words + ORC_HEADER_WORDS;
+    uint32_t hw = header_words(levelset, s);
+    if (levelset == LEVELS_TABLE)
+        for (uint32_t j = 1; j <= s; ++j) words[ORC_HEADER_WORDS + j - 1] = float_bits(g_table.level[j]);
+    uint64_t* table = (uint64_t*)(words + hw);
+    uint32_t* payload = mode == MODE_ERC ? words + hw + 2 * (nblk + 1) : words + hw;
     uint32_t w = nuq_oracle_fixed_width(levelset, s);
 
     uint8_t* sign = (uint8_t*)malloc(bucket);
@@ -459,16 +510,23 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
     uint64_t container_bits = (uint64_t)words[10] | ((uint64_t)words[11] << 32);
     uint32_t nlev = nuq_oracle_num_levels(levelset, s);
     uint32_t w = nuq_oracle_fixed_width(levelset, s);
+    uint32_t hw = header_words(levelset, s);
+    if (levelset == LEVELS_TABLE) {                          /* the levels must be a level sequence */
+        level_table t;
+        float interior[ORC_MAX_S];
+        for (uint32_t j = 0; j < s; ++j) interior[j] = bits_float(words[ORC_HEADER_WORDS + j]);
+        if (make_table(interior, s, &t) != ORC_OK) return ORC_ERR_STREAM;
+    }
     memset(sign, 0, (size_t)d);
     memset(sym, 0, 2 * (size_t)d);
 
     if (mode == MODE_FIXED) {
         if (nblk != nb) return ORC_ERR_STREAM;
         uint64_t last = d - (nb - 1) * (uint64_t)bucket;
-        if (container_bits != 32u * (ORC_HEADER_WORDS + (nb - 1) * (1 + ((uint64_t)bucket * w + 31) / 32) +
+        if (container_bits != 32u * (hw + (nb - 1) * (1 + ((uint64_t)bucket * w + 31) / 32) +
                                      1 + (last * w + 31) / 32))
             return ORC_ERR_STREAM;
-        const uint32_t* payload = words + ORC_HEADER_WORDS;
+        const uint32_t* payload = words + hw;
         for (uint64_t b = 0; b < nb; ++b) {
             uint64_t lo = b * (uint64_t)bucket, n = lo + bucket < d ? bucket : d - lo;
             uint64_t p = b * 32u * (1 + ((uint64_t)bucket * w + 31) / 32);
@@ -487,9 +545,9 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
     }
 
     if (nblk != count_blocks(d, bucket)) return ORC_ERR_STREAM;
-    const uint64_t* table = (const uint64_t*)(words + ORC_HEADER_WORDS);
-    const uint32_t* payload = words + ORC_HEADER_WORDS + 2 * (nblk + 1);
-    if (container_bits != 32u * (ORC_HEADER_WORDS + 2 * (nblk + 1)) + table[nblk]) return ORC_ERR_STREAM;
+    const uint64_t* table = (const uint64_t*)(words + hw);
+    const uint32_t* payload = words + hw + 2 * (nblk + 1);
+    if (container_bits != 32u * (hw + 2 * (nblk + 1)) + table[nblk]) return ORC_ERR_STREAM;
     uint64_t blk = 0;
     for (uint64_t b = 0; b < nb; ++b) {
         uint64_t lo = b * (uint64_t)bucket, n = lo + bucket < d ? bucket : d - lo;
@@ -557,9 +615,20 @@ int nuq_oracle_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     for (uint32_t k = 0; k < K && rc == ORC_OK; ++k) {
         rc = nuq_oracle_decode_symbols(streams[k], d, bucket, s, sign, sym, norms);
         if (rc != ORC_OK) break;
-        uint32_t levelset = (((const uint32_t*)streams[k])[6] >> 8) & 0xff;
-        for (uint64_t i = 0; i < d; ++i)
-            if (sym[i]) acc[i] = acc[i] + nuq_oracle_dequantize(norms[i / bucket], s, levelset, sign[i], sym[i]);
+        const uint32_t* words = (const uint32_t*)streams[k];
+        uint32_t levelset = (words[6] >> 8) & 0xff;
+        for (uint64_t i = 0; i < d; ++i) {
+            if (!sym[i]) continue;
+            float q;
+            if (levelset == LEVELS_TABLE) {                  /* the levels this container carries */
+                float level = sym[i] <= s ? bits_float(words[ORC_HEADER_WORDS + sym[i] - 1]) : 1.0f;
+                q = norms[i / bucket] * level;
+                if (sign[i]) q = -q;
+            } else {
+                q = nuq_oracle_dequantize(norms[i / bucket], s, levelset, sign[i], sym[i]);
+            }
+            acc[i] = acc[i] + q;
+        }
     }
     free(sign); free(sym); free(norms);
     return rc;

@@ -344,3 +344,125 @@ def test_degenerate_buckets():
     v = np.array([-0.0, 0.0, 1.0, -1.0], np.float32)
     sign, sym, _ = O.quantize(v, 4, 3, 0, 0, 1, 0)
     assert list(sym[:2]) == [0, 0] and list(sign[:2]) == [0, 0] and sign[3] == 1 and sign[2] == 0
+
+
+# ---------------------------------------------------------------- general level sequences (Sec. 3.3)
+def _lp_levels(p, s):
+    """interior levels of L_p = (0, p^s, ..., p^2, p, 1) as exact fractions"""
+    return [Fraction(p) ** (s + 1 - j) for j in range(1, s + 1)]
+
+
+def test_level_table_is_the_sequence_it_was_given():
+    for p, s in ((Fraction(1, 3), 3), (Fraction(3, 10), 5), (Fraction(1, 2), 4)):
+        want = _lp_levels(p, s)
+        lv32 = np.array([float(x) for x in want], np.float32)
+        O.set_levels(lv32)
+        assert O.num_levels(O.LEVELS_TABLE, s) == s + 2
+        got = [O.level_value(O.LEVELS_TABLE, s, j) for j in range(s + 2)]
+        assert got[0] == 0.0 and got[-1] == 1.0
+        assert [np.float32(x) for x in got[1:-1]] == list(lv32)
+        assert all(abs(Fraction(float(g)) - w) <= w * Fraction(1, 2 ** 23) for g, w in zip(got[1:-1], want))
+    # p = 1/2 is the paper's own level set
+    O.set_levels(np.array([2.0 ** -(4 - j) for j in range(4)], np.float32))
+    assert [O.level_value(O.LEVELS_TABLE, 4, j) for j in range(6)] == [O.level_value(O.LEVELS_EXP, 4, j) for j in range(6)]
+    for bad in ([0.5, 0.25], [0.0, 0.5], [0.5, 1.0], [0.3, 0.3], [float("nan")]):
+        with pytest.raises(ValueError):
+            O.set_levels(np.array(bad, np.float32))
+
+
+def test_level_table_rounding_probability_against_exact_arithmetic():
+    """p = (r - l_j) / (l_{j+1} - l_j) (Definition 1 for a general sequence, Sec. 3.3) in exact rational
+    arithmetic on the fp32 inputs; the oracle's fp32 value may differ by its few roundings only, and of
+    all 2^24 draws exactly ceil(p 2^24) move the coordinate up."""
+    lv = np.array([0.027, 0.09, 0.3], np.float32)
+    O.set_levels(lv)
+    levels = [Fraction(0)] + [Fraction(float(x)) for x in lv] + [Fraction(1)]
+    norm = np.float32(3.7)
+    draws = (np.arange(1 << 24, dtype=np.float64) / (1 << 24)).astype(np.float32)
+    for v in (0.01, -0.2, 0.5, 1.0, -2.9, 3.6999):
+        v32 = np.float32(v)
+        low, p = O.round_probability(v32, norm, 3, O.LEVELS_TABLE)
+        r = abs(Fraction(float(v32))) / Fraction(float(norm))
+        j = max(k for k in range(5) if levels[k] <= r)
+        assert low == j
+        exact = (r - levels[j]) / (levels[j + 1] - levels[j])
+        assert abs(Fraction(float(p)) - exact) <= Fraction(1, 10 ** 6)
+        sign, sym = O.quantize_with_draws(np.full(1 << 24, v32, np.float32), norm, 3, O.LEVELS_TABLE, draws)
+        ups = int((sym == j + 1).sum())
+        assert ups + int((sym == j).sum()) == 1 << 24
+        assert ups == math.ceil(Fraction(float(p)) * (1 << 24))
+        assert (sign == (1 if v < 0 else 0)).all() or j == 0
+    # r = 1 exactly, and r > 1 from a norm that is too small: the top level, never above it
+    assert O.round_probability(np.float32(4.0), np.float32(4.0), 3, O.LEVELS_TABLE) == (4, np.float32(0.0))
+    assert O.round_probability(np.float32(5.0), norm, 3, O.LEVELS_TABLE) == (4, np.float32(0.0))
+    low, p = O.round_probability(norm, norm, 3, O.LEVELS_TABLE)        # |v| * fl(1 / norm) may fall one place short of 1
+    assert (low, p) == (4, np.float32(0.0)) or (low == 3 and p >= 1.0 - 2.0 ** -22)
+
+
+def test_level_table_unbiased_by_enumeration():
+    """E[Q(v)] = v for any level sequence (Sec. 3.3): all 2^d up/down outcomes of a tiny vector with the
+    oracle's own probabilities."""
+    O.set_levels(np.array([0.05, 0.2, 0.6], np.float32))
+    v = np.array([0.3, -1.1, 0.02, 0.7, -0.45, 2.0], np.float32)
+    norm = O.norm(v)
+    lows, ps = zip(*[O.round_probability(x, norm, 3, O.LEVELS_TABLE) for x in v])
+    mean = np.zeros(v.size)
+    for ups in itertools.product((0, 1), repeat=v.size):
+        prob = np.prod([float(p) if u else 1.0 - float(p) for u, p in zip(ups, ps)])
+        q = [float(O.dequantize(norm, 3, O.LEVELS_TABLE, x < 0, low + u)) for x, low, u in zip(v, lows, ups)]
+        mean += prob * np.array(q)
+    assert np.abs(mean - v).max() <= 1e-6 * float(norm)
+
+
+def test_level_table_variance_closed_form_by_hand_and_by_monte_carlo():
+    """Lemma 7 for sequences other than the paper's (tests/golden/general_levels.txt), then the same
+    closed form against the sample variance of the quantizer itself."""
+    for p, s, d, want in golden_rows("general_levels.txt"):
+        p, s, d, want = Fraction(p), int(s), int(d), Fraction(want)
+        O.set_levels(np.array([float(x) for x in _lp_levels(p, s)], np.float32))
+        v = np.full(d, 0.75, np.float32)
+        norm = O.norm(v)
+        got = O.variance_closed_form(v, norm, s, O.LEVELS_TABLE) / float(norm) ** 2
+        assert abs(got - float(want)) <= 1e-6, (p, s, d, got)
+    O.set_levels(np.array([0.3 ** 3, 0.3 ** 2, 0.3], np.float32))
+    rng = np.random.default_rng(7)
+    v = (rng.standard_normal(512) * 10.0 ** rng.uniform(-2, 0, 512)).astype(np.float32)
+    norm = O.norm(v)
+    cf = O.variance_closed_form(v, norm, 3, O.LEVELS_TABLE)
+    errs = []
+    for seed in range(400):
+        sign, sym = O.quantize_bucket(v, norm, 3, O.LEVELS_TABLE, seed, 0, 0)
+        q = np.array([float(O.dequantize(norm, 3, O.LEVELS_TABLE, a, b)) for a, b in zip(sign, sym)])
+        errs.append(float(((q - v.astype(np.float64)) ** 2).sum()))
+    assert abs(np.mean(errs) - cf) <= 4 * np.std(errs) / math.sqrt(len(errs))
+
+
+def test_level_table_container():
+    """The container of a level-table stream carries the s interior levels behind the header (padded to an
+    even number of words); everything else is laid out as for the paper's levels."""
+    lv = np.array([0.3 ** 3, 0.3 ** 2, 0.3], np.float32)
+    O.set_levels(lv)
+    rng = np.random.default_rng(3)
+    g = (rng.standard_normal(3000) * 10.0 ** rng.uniform(-3, 0, 3000)).astype(np.float32)
+    for mode in (O.MODE_ERC, O.MODE_FIXED):
+        flags = O.make_flags(O.NORM_L2, O.LEVELS_TABLE, mode)
+        st, bits = O.encode(g, 512, 3, flags, 5, 1)
+        assert bits == 32 * st.size and O.header(st)["flags"] == flags
+        assert np.array_equal(st[16:19].view(np.float32), lv) and st[19] == 0           # 3 levels + a pad word
+        rc, sign, sym, norms = O.decode_symbols(st, g.size, 512, 3)
+        assert rc == 0
+        s2, y2, n2 = O.quantize(g, 512, 3, O.NORM_L2, O.LEVELS_TABLE, 5, 1)
+        assert np.array_equal(sign, s2) and np.array_equal(sym, y2) and np.array_equal(norms, n2)
+        rc, acc = O.decode_accumulate([st], g.size, 512, 3)
+        assert rc == 0 and np.array_equal(acc, O.quantize_dequantize(g, 512, 3, O.NORM_L2, O.LEVELS_TABLE, 5, 1))
+        # the decoder takes the levels from the container, not from the table that happens to be set
+        O.set_levels(np.array([0.1, 0.2, 0.4], np.float32))
+        assert np.array_equal(O.decode_accumulate([st], g.size, 512, 3)[1], acc)
+        O.set_levels(lv)
+        bad = st.copy()
+        bad[17] = bad[16]                                                                # not increasing
+        assert O.decode_symbols(bad, g.size, 512, 3)[0] == -3
+    # with the paper's levels in the table every symbol stands for the same value as in the paper's level set
+    O.set_levels(np.array([2.0 ** -3, 2.0 ** -2, 2.0 ** -1], np.float32))
+    for sym in range(5):
+        assert O.dequantize(np.float32(1.7), 3, O.LEVELS_TABLE, 1, sym) == O.dequantize(np.float32(1.7), 3, O.LEVELS_EXP, 1, sym)
