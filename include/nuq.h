@@ -18,14 +18,17 @@
  *     size"), s = number of internal levels (Sec. 3.1).
  *
  * Limits: 1 <= d < 2^40; bucket a multiple of 256 with 256 <= bucket <= 8192,
- * or bucket in {16384, 32768, 65536}; 1 <= s <= 14 (exponential levels) or
- * 1 <= s <= 8 (uniform levels); 1 <= K <= 64.
+ * or bucket in {16384, 32768, 65536}; 1 <= s <= 14 (exponential levels and
+ * level tables) or 1 <= s <= 8 (uniform levels); 1 <= K <= 64.
  *
  * Container written by nuq_encode (all u32 words little endian; bit p of a bit
  * string sits in word p>>5 at bit 31-(p&31)):
  *   words 0..15   header: magic 'NUQ1', version, d (2 words), bucket, s,
  *                 flags (norm | levels<<8 | mode<<16), 256, nblk (2),
  *                 container_bits (2), code_bits (2), nnz (2)
+ *   level table   only in streams with NUQ_LEVELS_TABLE: the s interior
+ *                 levels l_1 .. l_s as fp32 words, then a zero word if s is
+ *                 odd; everything below follows behind it
  *   ERC mode      (nblk+1) u64 bit offsets of the coding blocks, relative to
  *                 the payload that follows the table.  A coding block is up to
  *                 8192 consecutive elements of one bucket: norm (fp32 bits) |
@@ -61,6 +64,8 @@ typedef int nuq_status;
 #define NUQ_NORM_LINF 1u          /*           max-abs norm (QSGDinf comparison, Sec. 1)          */
 #define NUQ_LEVELS_EXP (0u << 8)  /* bits 8-15: levels (0, 2^-s, ..., 1/2, 1)  (Sec. 3.1)         */
 #define NUQ_LEVELS_UNIFORM (1u << 8) /*         levels k / 2^s, k = 0..2^s    (QSGD comparison)   */
+#define NUQ_LEVELS_TABLE (2u << 8) /*           levels (0, l_1, ..., l_s, 1) set by               *
+                                    *           nuq_set_level_table   (Sec. 3.3)                  */
 #define NUQ_MODE_ERC (0u << 16)   /* bits 16-23: Elias-recursive token stream (App. A)            */
 #define NUQ_MODE_FIXED (1u << 16) /*             fixed-width fields ("4-bit" variant of Sec. 5)   */
 #define NUQ_TEST_NORMS (1u << 24) /* take bucket norms from nuq_set_test_norms (parity testing)   */
@@ -150,7 +155,9 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
  *     (different streams, no dependency between them) race on it and produce
  *     garbage: serialise them.
  *   - Kernel-detected errors (NUQ_ERR_TIMEOUT) are latched in the array and are
- *     reported, and cleared, by nuq_last_status on any stream of that device.
+ *     reported, and cleared, by nuq_last_status on that device.  nuq_last_status
+ *     waits only for the stream it is given: pass the stream the static call ran
+ *     on (or synchronise the device first), or a status latched later is missed.
  */
 #define NUQ_STATIC_SCRATCH_BYTES (512u * 1024u)
 nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind,
@@ -159,13 +166,27 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
 /* Bytes that `out` of nuq_encode must hold for these arguments (0 if they are invalid). */
 uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind);
 
+/*
+ * General level sequences (Sec. 3.3, e.g. L_p = (0, p^s, ..., p, 1)): sets the s interior
+ * levels 0 < l_1 < ... < l_s < 1 (HOST array, copied) that nuq_encode uses from now on when
+ * it is called with NUQ_LEVELS_TABLE and this s.  A coordinate with l_j <= r < l_{j+1},
+ * r = |v| / norm, moves to l_{j+1} with probability (r - l_j) / (l_{j+1} - l_j) (fp32: r
+ * is |v| times the rounded 1 / norm, the quotient a product with the rounded inverse
+ * width).  The container carries the levels; nuq_decode_accumulate reads them from there.
+ * Returns NUQ_ERR_INVALID_ARG unless the levels increase strictly inside (0, 1) and
+ * 1 <= s <= 14.
+ */
+nuq_status nuq_set_level_table(const float* interior_levels, uint32_t s);
+
 /* Parity-test hook: device array of ceil(d/bucket) bucket norms that nuq_encode uses in
  * place of its own reduction when NUQ_TEST_NORMS is set; NULL clears it.  The pointer is
  * kept, not copied.                                                                        */
 nuq_status nuq_set_test_norms(const float* norms);
 
 /* Synchronises `stream` and returns, then clears, the status latched by the kernels that
- * ran on it since the last call (NUQ_OK, NUQ_ERR_BAD_STREAM, NUQ_ERR_TIMEOUT).            */
+ * ran on it since the last call: NUQ_OK, an error (NUQ_ERR_BAD_STREAM, NUQ_ERR_TIMEOUT,
+ * NUQ_ERR_INTERNAL; the most negative one wins), or NUQ_WARN_NONFINITE when no error was
+ * latched and some bucket was written unquantized.                                         */
 nuq_status nuq_last_status(void* stream);
 
 /* Copies the header of a container (device) into *host_out; synchronises `stream`.        */

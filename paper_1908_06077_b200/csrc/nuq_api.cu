@@ -25,11 +25,15 @@ struct WsEntry {
     bool clean = false;      // the scan state is all zero: set by the allocation, kept by every encode kernel
 };
 
+// One mutex guards the host-side bookkeeping below (maps, tables); it is held for the microseconds a
+// call spends on the host, never across a wait for the device, except where a workspace has to grow.
 std::mutex g_mu;
 std::map<std::pair<int, cudaStream_t>, WsEntry> g_ws;
 std::map<int, int> g_sms;                 // device -> SM count
 std::set<int> g_lut_ready;                // devices whose constant LUT is uploaded
-const float* g_test_norms = nullptr;
+std::map<int, const float*> g_test_norms;   // device -> bucket norms of nuq_set_test_norms
+float g_levels[kMaxTableS + 2], g_inv_width[kMaxTableS + 2];   // the level table of nuq_set_level_table ...
+uint32_t g_levels_s = 0;                                       // ... and its number of interior levels (0: none set)
 std::map<int, Workspace*> g_static_ws;   // device -> address of g_static_scratch on that device
 uint32_t g_erc_len[256];
 bool g_erc_len_ready = false;
@@ -52,8 +56,8 @@ bool bucket_ok(uint32_t bucket) {
 bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geometry* G) {
     const uint32_t norm_kind = flags & 0xffu, levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
     if (d == 0 || d >= (1ull << 40) || !bucket_ok(bucket) || s < 1) return false;
-    if (norm_kind > 1 || levelset > 1 || mode > 1) return false;
-    if (s > (levelset == kLevelsExp ? 14u : 8u)) return false;
+    if (norm_kind > 1 || levelset > 2 || mode > 1) return false;
+    if (s > (levelset == kLevelsUniform ? 8u : 14u)) return false;
     if (flags & ~(0x00ffffffu | NUQ_TEST_NORMS | NUQ_TEST_SHORT_PATIENCE)) return false;
     G->d = d;
     G->bucket = bucket;
@@ -62,7 +66,9 @@ bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geom
     G->levelset = levelset;
     G->mode = mode;
     G->nb = (d + bucket - 1) / bucket;
-    G->nlev = levelset == kLevelsExp ? s + 2u : (1u << s) + 1u;
+    G->nlev = levelset == kLevelsUniform ? (1u << s) + 1u : s + 2u;
+    G->header_words = kHeaderWords + (levelset == kLevelsTable ? ((s + 1u) & ~1u) : 0u);
+    G->pad = 0;
     uint32_t b = 0;
     while ((1u << b) < G->nlev) ++b;
     G->width = b + 1u;
@@ -101,7 +107,7 @@ uint32_t max_level_code_bits(const Geometry& G) {
 uint32_t token_bits_bound(const Geometry& G, uint32_t elems, uint32_t buckets, bool norms_are_ours) {
     const uint32_t L = max_level_code_bits(G);
     const uint32_t safe = elems * (2u + L);
-    if (!norms_are_ours || G.norm_kind != kNormL2 || G.s > 7u) return safe;
+    if (!norms_are_ours || G.norm_kind != kNormL2 || G.levelset != kLevelsExp || G.s > 7u) return safe;
     const uint64_t high = (uint64_t)buckets * ((1ull << (2u * G.s)) + 8u);      // + slack for the rounding of the norm
     const uint32_t nhigh = high < elems ? (uint32_t)high : elems;
     const uint32_t tight = 3u * elems + nhigh * (L - 1u);
@@ -115,10 +121,10 @@ uint32_t stage_words_for(const Geometry& G, bool norms_are_ours) {
 }
 
 uint64_t bound_bytes(const Geometry& G) {
-    if (G.mode == kModeFixed) return 4ull * (kHeaderWords + G.nb * G.rec_words);
+    if (G.mode == kModeFixed) return 4ull * (G.header_words + G.nb * G.rec_words);
     uint64_t head = 1u + (G.sb_per_block + 1u) / 2u + 1u;
     uint64_t token_words = (G.d * (2ull + max_level_code_bits(G)) + 31) / 32;
-    return 4ull * (kHeaderWords + 2 * (G.nblk + 1) + G.nblk * head + token_words);
+    return 4ull * (G.header_words + 2 * (G.nblk + 1) + G.nblk * head + token_words);
 }
 
 int device_sms(int dev) {
@@ -164,8 +170,10 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
 
 using namespace nuq;
 
-// Mode of the containers this process has encoded, by address (see enqueue_encode).  Guarded by g_mu.
-static std::map<const void*, uint32_t> g_container_mode;
+// Mode of the containers this process has encoded, by device and address (see enqueue_encode): a hint
+// for the decoder's choice of kernels, which check it against the containers' headers on the device.
+// Guarded by g_mu.
+static std::map<std::pair<int, const void*>, uint32_t> g_container_mode;
 
 // What one encode call needs from its workspace and from shared memory.
 struct EncodePlan {
@@ -224,7 +232,7 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     P.g = g;
     P.norms_in = nullptr;
     if (test_norms) {
-        P.norms_in = g_test_norms;
+        P.norms_in = g_test_norms[dev];
     } else if (pl.norms_bytes) {
         float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + pl.state_bytes);
         if (launch_bucket_norms(g, G.d, G.bucket, G.norm_kind, norms, G.nb, stream) != cudaSuccess) return NUQ_ERR_CUDA;
@@ -235,6 +243,10 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     P.ws = ws;
     P.seed = seed;
     P.offset = offset;
+    for (uint32_t j = 0; j < kMaxTableS + 2u; ++j) {
+        P.levels[j] = G.levelset == kLevelsTable ? g_levels[j] : 0.0f;
+        P.inv_width[j] = G.levelset == kLevelsTable ? g_inv_width[j] : 0.0f;
+    }
     for (uint32_t r = 0; r < 10; ++r) {               // Philox key schedule (Weyl sequence)
         P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
@@ -246,7 +258,7 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     // remember the mode of the container at this address: a hint for the decoder's choice of kernels,
     // checked against the header on the device
     if (g_container_mode.size() > 4096) g_container_mode.clear();
-    g_container_mode[out] = G.mode;
+    g_container_mode[std::make_pair(dev, static_cast<const void*>(out))] = G.mode;
     return NUQ_OK;
 }
 
@@ -256,7 +268,11 @@ static bool encode_args_ok(const float* g, uint64_t d, uint32_t bucket, uint32_t
     if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u) ||
         (reinterpret_cast<uintptr_t>(out_bits) & 7u))
         return false;
-    if ((norm_kind & NUQ_TEST_NORMS) && !g_test_norms) return false;
+    if (norm_kind & NUQ_TEST_NORMS) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || !g_test_norms.count(dev) || !g_test_norms[dev]) return false;
+    }
+    if (G->levelset == kLevelsTable && g_levels_s != s) return false;   // no level table of this length has been set
     return true;
 }
 
@@ -269,9 +285,32 @@ uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm
     return (bound_bytes(G) + 15) & ~15ull;
 }
 
+nuq_status nuq_set_level_table(const float* interior_levels, uint32_t s) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!interior_levels || s < 1 || s > kMaxTableS) return NUQ_ERR_INVALID_ARG;
+    float lv[kMaxTableS + 2], iw[kMaxTableS + 2];
+    lv[0] = 0.0f;
+    for (uint32_t j = 1; j <= s; ++j) lv[j] = interior_levels[j - 1];
+    lv[s + 1] = 1.0f;
+    for (uint32_t j = 0; j <= s; ++j) {
+        if (!(lv[j] < lv[j + 1])) return NUQ_ERR_INVALID_ARG;              // strictly increasing inside (0, 1), no NaN
+        iw[j] = 1.0f / (lv[j + 1] - lv[j]);                                 // one IEEE division per level
+        if (!(iw[j] < __builtin_huge_valf())) return NUQ_ERR_INVALID_ARG;
+    }
+    iw[s + 1] = 0.0f;
+    for (uint32_t j = 0; j < kMaxTableS + 2u; ++j) {
+        g_levels[j] = j <= s + 1 ? lv[j] : 1.0f;
+        g_inv_width[j] = j <= s + 1 ? iw[j] : 0.0f;
+    }
+    g_levels_s = s;
+    return NUQ_OK;
+}
+
 nuq_status nuq_set_test_norms(const float* norms) {
     std::lock_guard<std::mutex> lock(g_mu);
-    g_test_norms = norms;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    g_test_norms[dev] = norms;
     return NUQ_OK;
 }
 
@@ -335,14 +374,15 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     for (uint32_t k = K; k < kMaxK; ++k) P.streams[k] = nullptr;
     P.K = K;
     P.group = K >= 8 ? 8u : K >= 3 ? 4u : K;            // 1, 2, 4 or 8 streams side by side
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
     P.after_fixed = 1;                                  // all streams believed to be in the fixed-width mode?
     for (uint32_t k = 0; k < K; ++k) {
-        auto it = g_container_mode.find(streams[k]);
+        auto it = g_container_mode.find(std::make_pair(dev, streams[k]));
         if (it == g_container_mode.end() || it->second != kModeFixed) P.after_fixed = 0;
     }
     P.acc = acc;
     Workspace* ws = nullptr;
-    int dev = 0;
     nuq_status st = get_workspace(stream, sizeof(Workspace), &ws, &dev);
     if (st != NUQ_OK) return st;
     P.ws = ws;

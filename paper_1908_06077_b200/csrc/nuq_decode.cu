@@ -84,10 +84,13 @@ __device__ __forceinline__ uint64_t window64(Fetch word, uint32_t cur, uint32_t 
     return win;
 }
 
-__device__ __forceinline__ float level_times_norm(float norm, uint32_t levelset, uint32_t s, uint32_t sym) {
-    // exponential: l_j = 2^(j-1-s) (exact scaling);  uniform: l_k = k / 2^s
-    float level = levelset == kLevelsExp ? __uint_as_float((126u + sym - s) << 23)
-                                         : (float)sym * __uint_as_float((127u - s) << 23);
+// `hdr`: the container (a level-table stream carries its s interior levels behind the 16 header words)
+__device__ __forceinline__ float level_times_norm(float norm, uint32_t levelset, uint32_t s, uint32_t sym, const uint32_t* hdr) {
+    // exponential: l_j = 2^(j-1-s) (exact scaling);  uniform: l_k = k / 2^s;  table: l_j as stored, l_{s+1} = 1
+    float level;
+    if (levelset == kLevelsExp) level = __uint_as_float((126u + sym - s) << 23);
+    else if (levelset == kLevelsUniform) level = (float)sym * __uint_as_float((127u - s) << 23);
+    else level = sym <= s ? __uint_as_float(__ldg(hdr + kHeaderWords + sym - 1u)) : 1.0f;
     return __fmul_rn(norm, level);
 }
 
@@ -128,7 +131,8 @@ struct Chain {
 struct StreamHead {
     const uint32_t* hdr;
     uint64_t cwords;         // container words the header declares
-    uint32_t ok, mode, levelset, nlev, width, pad;
+    uint32_t ok, mode, levelset, nlev, width;
+    uint32_t hwords;         // header words: 16, plus the level table of a level-table stream
 };
 
 // Where a tile lies in the vector and in the containers.
@@ -151,8 +155,8 @@ __device__ bool describe_chain(const Geometry& G, const TileGeo& T, const Stream
     const uint32_t blk_len = min(T.blk_elems, T.tile_len - min(T.tile_len, bi * T.blk_elems));
     const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
     if (hd.mode == kModeErc) {
-        const uint64_t head = kHeaderWords + 2 * (G.nblk + 1);
-        const uint64_t* table = reinterpret_cast<const uint64_t*>(hd.hdr + kHeaderWords);
+        const uint64_t head = hd.hwords + 2 * (G.nblk + 1);
+        const uint64_t* table = reinterpret_cast<const uint64_t*>(hd.hdr + hd.hwords);
         const uint32_t* payload = hd.hdr + head;
         const uint64_t payload_words = hd.cwords - head;
         const uint64_t off = __ldg(table + T.first_block + bi), end = __ldg(table + T.first_block + bi + 1);
@@ -178,7 +182,7 @@ __device__ bool describe_chain(const Geometry& G, const TileGeo& T, const Stream
     } else {
         const uint32_t rec_words = 1u + (G.bucket * hd.width + 31u) / 32u;
         const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
-        const uint32_t* payload = hd.hdr + kHeaderWords;
+        const uint32_t* payload = hd.hdr + hd.hwords;
         const uint64_t bucket_of_sb = G.bucket <= kBLK ? T.first_block + bi : T.bucket_idx;
         const uint32_t* rec = payload + bucket_of_sb * rec_words;
         const uint64_t bucket_len = bucket_of_sb == G.nb - 1 ? last_len : G.bucket;
@@ -199,22 +203,32 @@ __device__ StreamHead read_head(const Geometry& G, const uint32_t* hdr) {
     const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
     const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
     bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
-              __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 1u && mode <= 1u &&
+              __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 2u && mode <= 1u &&
               (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
-    const uint32_t nlev = levelset == kLevelsExp ? G.s + 2u : (1u << G.s) + 1u;
+    const uint32_t nlev = levelset == kLevelsUniform ? (1u << G.s) + 1u : G.s + 2u;
+    const uint32_t hwords = kHeaderWords + (levelset == kLevelsTable ? ((G.s + 1u) & ~1u) : 0u);
+    if (ok && levelset == kLevelsTable) {                   // the levels must increase strictly inside (0, 1)
+        float below = 0.0f;
+        for (uint32_t j = 0; j < G.s; ++j) {
+            const float l = __uint_as_float(__ldg(hdr + kHeaderWords + j));
+            ok = ok && below < l;
+            below = l;
+        }
+        ok = ok && below < 1.0f;
+    }
     const uint32_t width = 1u + (32u - __clz(nlev - 1u));                   // fixed mode: sign bit + ceil(log2(levels))
     const uint64_t cwords = cbits >> 5;
     if (ok && mode == kModeErc) {
-        ok = hnblk == G.nblk && cwords > kHeaderWords + 2 * (G.nblk + 1);
+        ok = hnblk == G.nblk && cwords > hwords + 2 * (G.nblk + 1);
     } else if (ok) {
         const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
         const uint64_t last_len = G.d - (G.nb - 1) * G.bucket;
         ok = hnblk == G.nb &&
-             cwords == kHeaderWords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
+             cwords == hwords + (G.nb - 1) * (uint64_t)rec_words + 1 + (last_len * width + 31) / 32;
     }
     StreamHead h;
     h.hdr = hdr; h.cwords = cwords; h.ok = ok ? 1u : 0u; h.mode = mode; h.levelset = levelset;
-    h.nlev = nlev; h.width = width; h.pad = 0;
+    h.nlev = nlev; h.width = width; h.hwords = hwords;
     return h;
 }
 
@@ -329,7 +343,7 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
         for (uint32_t t = tid; t < 16u * K; t += blockDim.x) {
             const uint32_t k = t >> 4, f = t & 15u, sym = f & 7u;
             const float norm = __uint_as_float(__ldg(heads[k].hdr + kHeaderWords + b * rec_words));
-            const float v = sym && sym < nlev ? level_times_norm(norm, LEVELSET, G.s, sym) : 0.0f;
+            const float v = sym && sym < nlev ? level_times_norm(norm, LEVELSET, G.s, sym, heads[k].hdr) : 0.0f;
             s_tab[k][f] = (f & 8u) ? -v : v;
         }
         __syncthreads();
@@ -388,7 +402,8 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
     if (threadIdx.x == 0) {
         bool same = true;
         for (uint32_t k = 0; k < P.K; ++k)
-            same = same && heads[k].ok && heads[k].mode == kModeFixed && heads[k].levelset == heads[0].levelset;
+            same = same && heads[k].ok && heads[k].mode == kModeFixed && heads[k].levelset == heads[0].levelset &&
+                   heads[k].levelset != kLevelsTable;       // (streams with a level table take the general kernel)
         s_width = same ? heads[0].width : 0u;
         if (same && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0]) = 1;   // tell the general kernel
     }
@@ -734,7 +749,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                             for (uint32_t i = i0; i < n_c; i += per_chain) {
                                 const uint32_t e = wide ? list[i * 32u + owner]
                                                         : (uint32_t)reinterpret_cast<const uint16_t*>(list)[i * 32u + owner];
-                                const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u);
+                                const float v = level_times_norm(norm_c, sj.levelset, G.s, (e >> 9) + 1u, sj.hdr);
                                 add_to(part0 + (e & 0xffu), (e >> 8) & 1u ? -v : v);
                             }
                         }
@@ -764,7 +779,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                                 if (c < nel && p + c >= fixed_lo && p + c < fixed_hi) {
                                     if (sym >= sj.nlev) field_bad = true;
                                     else if (sym) {
-                                        const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym);
+                                        const float v = level_times_norm(cf.norm, sj.levelset, G.s, sym, sj.hdr);
                                         add_to(grp * 4u + c, (field >> (wd - 1u)) ? -v : v);
                                     }
                                 }

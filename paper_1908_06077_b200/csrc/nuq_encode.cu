@@ -107,6 +107,19 @@ __device__ __forceinline__ uint32_t quantize_uniform(float v, float inv, float t
     return (uint32_t)fl + ((__uint2float_rn(word >> 8) < p * 16777216.0f) ? 1u : 0u);
 }
 
+// A general level sequence (0, l_1, ..., l_s, 1) given as a table (Sec. 3.3): r = |v| / norm clamped
+// to 1, l_j <= r < l_{j+1}, p = (r - l_j) / (l_{j+1} - l_j) computed as a product with the inverse
+// width; the draw is compared as u = m 2^-24.  `lv`, `iw`: the tables in shared memory.
+__device__ __forceinline__ uint32_t quantize_table(float v, float inv, uint32_t s, uint32_t word, const float* lv,
+                                                   const float* iw) {
+    const float r = fminf(__fmul_rn(fabsf(v), inv), 1.0f);
+    uint32_t j = 0;
+    for (uint32_t k = 1; k <= s + 1u; ++k) j += r >= lv[k] ? 1u : 0u;    // the levels increase: j = index of the last one <= r
+    const float p = __fmul_rn(__fsub_rn(r, lv[j]), iw[j]);
+    const float u = __fmul_rn(__uint2float_rn(word >> 8), 0x1p-24f);
+    return j + (u < p ? 1u : 0u);
+}
+
 // OR `nbits` (1..64) right-aligned bits of `value` into the MSB-first bit string `dst` at
 // `bitpos`.  Up to three words are touched; dst[bitpos/32 + 2] must exist.
 __device__ __forceinline__ void or_bits(uint32_t* dst, uint32_t bitpos, uint64_t value, uint32_t nbits) {
@@ -317,7 +330,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
 // Symbols travel as small fields: level index in the low bits, sign above it.
 template <uint32_t LEVELSET>
 struct Sym {
-    static constexpr uint32_t kBits = LEVELSET == kLevelsExp ? 7u : 15u;     // index <= 15 resp. <= 256
+    static constexpr uint32_t kBits = LEVELSET != kLevelsUniform ? 7u : 15u;  // index <= 15 resp. <= 256
     static constexpr uint32_t kMask = (1u << kBits) - 1u;
 };
 
@@ -404,11 +417,11 @@ __device__ bool finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, 
     const uint64_t nrec = MODE == kModeErc ? G.nblk : G.nb;
     if (MODE == kModeErc) {
         code_total = ld_volatile_u64(&P.ws->code_bits);
-        words = kHeaderWords + 2 * (G.nblk + 1) + ld_volatile_u64(&P.ws->total_words);
+        words = G.header_words + 2 * (G.nblk + 1) + ld_volatile_u64(&P.ws->total_words);
     } else {
         code_total = G.d * G.width;
         const uint64_t last = G.d - (G.nb - 1) * G.bucket;
-        words = kHeaderWords + (G.nb - 1) * G.rec_words + 1 + (last * G.width + 31) / 32;
+        words = G.header_words + (G.nb - 1) * G.rec_words + 1 + (last * G.width + 31) / 32;
     }
     const uint64_t container_bits = 32 * words;
     uint32_t* h = P.out;
@@ -421,6 +434,8 @@ __device__ bool finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, 
     h[10] = (uint32_t)container_bits; h[11] = (uint32_t)(container_bits >> 32);
     h[12] = (uint32_t)code_total; h[13] = (uint32_t)(code_total >> 32);
     h[14] = (uint32_t)nnz_total; h[15] = (uint32_t)(nnz_total >> 32);
+    if (G.levelset == kLevelsTable)                         // the interior levels, then zero padding
+        for (uint32_t j = 0; j < G.header_words - kHeaderWords; ++j) h[kHeaderWords + j] = j < G.s ? __float_as_uint(P.levels[j + 1]) : 0u;
     if (P.out_bits) *P.out_bits = container_bits;
     return true;
 }
@@ -511,6 +526,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     __shared__ uint32_t s_maxbits[32];                     // ... or max |x| bit patterns
     __shared__ float s_sb_inv[32], s_sb_norm[32];          // per sub-block of the current tile: 2^s / norm (0: not quantized), norm
     __shared__ uint32_t s_sb_bi[32];                       // block (within a tile) of each sub-block
+    __shared__ float s_levels[kMaxTableS + 2], s_invw[kMaxTableS + 2];   // level table (level-table streams)
     __shared__ uint32_t s_arrived;                         // warps that have added up their squares (counts on, modulo 8)
     __shared__ TileInfo s_info[4];                         // tiles of the iterations it, it + 1, it + 2
     __shared__ TileMeta s_meta[2];
@@ -527,9 +543,10 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     uint32_t* const windows = images + 2u * P.stage_words;                      // [2][kEncWarps][window_words]: token strings
     uint64_t* tile_state = reinterpret_cast<uint64_t*>(P.ws + 1);
     uint64_t* group_state = tile_state + G.ntiles;
-    uint64_t* table = reinterpret_cast<uint64_t*>(P.out + kHeaderWords);
-    uint32_t* payload = MODE == kModeErc ? P.out + kHeaderWords + 2 * (G.nblk + 1) : P.out + kHeaderWords;
-    const float top = __uint_as_float((127u + G.s) << 23);
+    uint64_t* table = reinterpret_cast<uint64_t*>(P.out + G.header_words);
+    uint32_t* payload = MODE == kModeErc ? P.out + G.header_words + 2 * (G.nblk + 1) : P.out + G.header_words;
+    constexpr bool kSmall = LEVELSET != kLevelsUniform;     // level index <= 15: symbols travel as bytes
+    const float top = LEVELSET == kLevelsTable ? 1.0f : __uint_as_float((127u + G.s) << 23);   // the norm is divided into this
     const uint32_t c2 = (uint32_t)P.offset, c3 = (uint32_t)(P.offset >> 32);
     const bool narrow = G.bucket <= kBLK;
     const bool coarse = G.bucket % kWarpElems == 0;         // a warp's four sub-blocks always share one bucket
@@ -589,6 +606,10 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         s_lut_signed[tid] = v;
     }
     if (tid < 32u) s_sb_bi[tid] = tid / spb;
+    if (tid < kMaxTableS + 2u) {
+        s_levels[tid] = P.levels[tid];
+        s_invw[tid] = P.inv_width[tid];
+    }
     if (MODE == kModeErc)
         for (uint32_t i = tid; i < 2u * P.stage_words + 2u * kEncWarps * P.window_words; i += blockDim.x) images[i] = 0;
     if (tid == 0) {
@@ -840,7 +861,12 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                 __syncwarp();                               // the sub-block's bytes are in registers: their place is scratch now
                 const uint4 r0 = rn0, r1 = rn1;
                 uint32_t qa[8];
-                if (LEVELSET == kLevelsExp) {
+                if (LEVELSET == kLevelsTable) {
+                    qa[0] = quantize_table(x0.x, inv, G.s, r0.x, s_levels, s_invw); qa[1] = quantize_table(x0.y, inv, G.s, r0.y, s_levels, s_invw);
+                    qa[2] = quantize_table(x0.z, inv, G.s, r0.z, s_levels, s_invw); qa[3] = quantize_table(x0.w, inv, G.s, r0.w, s_levels, s_invw);
+                    qa[4] = quantize_table(x1.x, inv, G.s, r1.x, s_levels, s_invw); qa[5] = quantize_table(x1.y, inv, G.s, r1.y, s_levels, s_invw);
+                    qa[6] = quantize_table(x1.z, inv, G.s, r1.z, s_levels, s_invw); qa[7] = quantize_table(x1.w, inv, G.s, r1.w, s_levels, s_invw);
+                } else if (LEVELSET == kLevelsExp) {
                     qa[0] = quantize_exp(x0.x, inv, top, r0.x); qa[1] = quantize_exp(x0.y, inv, top, r0.y);
                     qa[2] = quantize_exp(x0.z, inv, top, r0.z); qa[3] = quantize_exp(x0.w, inv, top, r0.w);
                     qa[4] = quantize_exp(x1.x, inv, top, r1.x); qa[5] = quantize_exp(x1.y, inv, top, r1.y);
@@ -855,7 +881,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                                         __float_as_uint(x1.x), __float_as_uint(x1.y), __float_as_uint(x1.z), __float_as_uint(x1.w)};
                 // Exponential levels: the four symbols of a row as bytes, index | sign << 7.
                 uint32_t f0 = 0, f1 = 0, nz0 = 0, nz1 = 0;
-                if (LEVELSET == kLevelsExp) {
+                if (kSmall) {
                     const uint32_t syms0 = qa[0] | (qa[1] << 8) | (qa[2] << 16) | (qa[3] << 24);
                     const uint32_t syms1 = qa[4] | (qa[5] << 8) | (qa[6] << 16) | (qa[7] << 24);
                     // top bytes of the four inputs: their sign bits at bits 7, 15, 23, 31
@@ -871,7 +897,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                     // ---- keep the nonzero symbols, in element order: a lane's rank = nonzeros of row 0 in lower
                     // lanes (+ all of row 0 and those of row 1 in lower lanes, for its row-1 elements) ----
                     uint32_t cnt0, cnt1;
-                    if (LEVELSET == kLevelsExp) {
+                    if (kSmall) {
                         cnt0 = __popc(nz0);
                         cnt1 = __popc(nz1);
                     } else {
@@ -886,7 +912,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                     uint32_t at0 = (incl & 0xffffu) - cnt0, at1 = tot0 + (incl >> 16) - cnt1;
                     uint32_t* list32 = reinterpret_cast<uint32_t*>(data + wbase + q * kSB);   // over the sub-block's own bytes
                     uint16_t* list16 = reinterpret_cast<uint16_t*>(list32);
-                    if (LEVELSET == kLevelsExp) {
+                    if (kSmall) {
                         // 16-bit entries position | field << 8, two at a time by byte permutation
                         const uint32_t pb0 = (lane * 4u) * 0x01010101u + 0x03020100u;      // the four positions of row 0, one per byte
                         const uint32_t pb1 = pb0 + 0x80808080u;                            // ... of row 1
@@ -917,15 +943,15 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                     for (uint32_t t0 = 0; t0 < ntok; t0 += 32) {
                         const bool valid = t0 + lane < ntok;
                         uint32_t e = 0;
-                        if (valid) e = LEVELSET == kLevelsExp ? (uint32_t)list16[t0 + lane] : list32[t0 + lane];
-                        const int pos = (int)(e & (LEVELSET == kLevelsExp ? 255u : 1023u));
-                        const uint32_t field = e >> (LEVELSET == kLevelsExp ? 8 : 10);
+                        if (valid) e = kSmall ? (uint32_t)list16[t0 + lane] : list32[t0 + lane];
+                        const int pos = (int)(e & (kSmall ? 255u : 1023u));
+                        const uint32_t field = e >> (kSmall ? 8 : 10);
                         int prev = __shfl_up_sync(0xffffffffu, pos, 1);
                         if (lane == 0) prev = carry_pos;
                         uint32_t gl = 0;                        // stays 0 in lanes without a token: no bits, no length
                         if (valid) gl = s_lut[(pos - prev - 1) & 255];
                         uint32_t tlen, tokA, lenA, tokB = 0, lenB = 0;
-                        if (LEVELSET == kLevelsExp) {
+                        if (kSmall) {
                             // both codes left aligned with their length in the low bits: the token is the gap code
                             // followed by sign and index code, i.e. the second shifted right by the first's length
                             const uint32_t ll = s_lut_signed[field & 255u];
@@ -949,7 +975,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                         }
                         const uint32_t off = bits + incl_bits - tlen;     // bit of the window where my token starts
                         or_bits_left(window, off, tokA);
-                        if (LEVELSET != kLevelsExp) or_bits_left(window, off + lenA, tokB);
+                        if (!kSmall) or_bits_left(window, off + lenA, tokB);
                         bits += step_bits;
                         carry_pos = __shfl_sync(0xffffffffu, pos, min(ntok - t0, 32u) - 1u);
                     }
@@ -958,7 +984,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                 } else {
                     // ---- fixed-width fields (sign bit, then the level index), MSB first ----
                     const uint32_t wbits = G.width;
-                    if (LEVELSET == kLevelsExp && wbits == 4u) {
+                    if (kSmall && wbits == 4u) {
                         // nibbles sign << 3 | index of the four elements of a row, first element on top
                         auto pack4 = [](uint32_t f) {
                             const uint32_t t = (f & 0x07070707u) | ((f >> 4) & 0x08080808u);    // one nibble per byte
@@ -976,7 +1002,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                         uint32_t ff[8];
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
-                            if (LEVELSET == kLevelsExp) ff[c] = ((c < 4 ? f0 : f1) >> (8 * (c & 3))) & 0xffu;
+                            if (kSmall) ff[c] = ((c < 4 ? f0 : f1) >> (8 * (c & 3))) & 0xffu;
                             else ff[c] = qa[c] | (qa[c] ? (xb[c] >> 16) & 0x8000u : 0u);
                             cta_nnz += qa[c] != 0;
                         }
@@ -1139,6 +1165,7 @@ static int blocks_per_sm(const EncodeParams& P) {
 int encode_blocks_per_sm(const EncodeParams& P) {
     const bool uni = P.geo.levelset == kLevelsUniform, fixed = P.geo.mode == kModeFixed;
     if (encode_smem_bytes(P) > (size_t)kEncMaxDynSmem) return 0;
+    if (P.geo.levelset == kLevelsTable) return fixed ? blocks_per_sm<kLevelsTable, kModeFixed>(P) : blocks_per_sm<kLevelsTable, kModeErc>(P);
     if (!uni && !fixed) return blocks_per_sm<kLevelsExp, kModeErc>(P);
     if (!uni && fixed) return blocks_per_sm<kLevelsExp, kModeFixed>(P);
     if (uni && !fixed) return blocks_per_sm<kLevelsUniform, kModeErc>(P);
@@ -1157,6 +1184,7 @@ static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
 
 cudaError_t launch_encode(const EncodeParams& P, cudaStream_t stream) {
     const bool uni = P.geo.levelset == kLevelsUniform, fixed = P.geo.mode == kModeFixed;
+    if (P.geo.levelset == kLevelsTable) return fixed ? launch_one<kLevelsTable, kModeFixed>(P, stream) : launch_one<kLevelsTable, kModeErc>(P, stream);
     if (!uni && !fixed) return launch_one<kLevelsExp, kModeErc>(P, stream);
     if (!uni && fixed) return launch_one<kLevelsExp, kModeFixed>(P, stream);
     if (uni && !fixed) return launch_one<kLevelsUniform, kModeErc>(P, stream);

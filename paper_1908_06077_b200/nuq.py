@@ -17,7 +17,7 @@ from . import build as _build
 NUQ_OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BAD_STREAM, ERR_CUDA, ERR_TIMEOUT, ERR_INTERNAL = 0, -1, -2, -3, -4, -5, -6
 WARN_NONFINITE = 1
 NORM_L2, NORM_LINF = 0, 1
-LEVELS_EXP, LEVELS_UNIFORM = 0 << 8, 1 << 8
+LEVELS_EXP, LEVELS_UNIFORM, LEVELS_TABLE = 0 << 8, 1 << 8, 2 << 8
 MODE_ERC, MODE_FIXED = 0 << 16, 1 << 16
 TEST_NORMS = 1 << 24
 TEST_SHORT_PATIENCE = 1 << 25
@@ -52,6 +52,8 @@ def _load():
                                           C.c_void_p, C.c_void_p]
     lib.nuq_encode_bound.restype = C.c_uint64
     lib.nuq_encode_bound.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
+    lib.nuq_set_level_table.restype = C.c_int
+    lib.nuq_set_level_table.argtypes = [C.POINTER(C.c_float), C.c_uint32]
     lib.nuq_set_test_norms.restype = C.c_int
     lib.nuq_set_test_norms.argtypes = [C.c_void_p]
     lib.nuq_last_status.restype = C.c_int
@@ -83,6 +85,15 @@ def version() -> str:
 
 def encode_bound(d, bucket, s, norm_kind=0) -> int:
     return int(_lib.nuq_encode_bound(d, bucket, s, norm_kind))
+
+
+def set_level_table(interior_levels):
+    """interior levels l_1 < ... < l_s of the level sequence (0, l_1, ..., l_s, 1) used with LEVELS_TABLE"""
+    vals = [float(x) for x in interior_levels]
+    arr = (C.c_float * len(vals))(*vals)
+    rc = _lib.nuq_set_level_table(arr, len(vals))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_set_level_table", rc)
 
 
 def set_test_norms(norms: torch.Tensor | None):

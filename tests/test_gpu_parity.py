@@ -364,3 +364,67 @@ def test_malformed_container_among_six_streams():
         gpu_decode(good[:2] + [bad] + good[3:], d, bucket, s, expect_status=-3)
     want = O.decode_accumulate(good, d, bucket, s)[1]
     assert np.array_equal(gpu_decode(good, d, bucket, s).view(np.uint32), want.view(np.uint32))
+
+
+# ---------------------------------------------------------------- general level sequences (Sec. 3.3)
+def _lp(p, s):
+    return np.array([p ** (s + 1 - j) for j in range(1, s + 1)], np.float32)
+
+
+TABLE_CASES = [
+    (70001, 1024, _lp(0.3, 3)),
+    (3 * 8192 + 5, 8192, _lp(0.5, 4)),                     # the paper's own levels, as a table
+    (20000, 512, _lp(0.7, 6)),
+    (150001, 16384, _lp(0.25, 2)),
+    (40000, 2048, np.array([0.01, 0.02, 0.05, 0.1, 0.15, 0.2, 0.3, 0.4, 0.5, 0.6, 0.7, 0.8, 0.9, 0.95], np.float32)),
+    (257, 256, np.array([0.5], np.float32)),
+]
+
+
+@pytest.mark.parametrize("d,bucket,levels", TABLE_CASES)
+@pytest.mark.parametrize("mode", [O.MODE_ERC, O.MODE_FIXED])
+def test_level_table_streams_match_the_oracle(d, bucket, levels, mode):
+    """Level sequences given as a table: with the oracle's norms the container is the oracle's bit for bit
+    (level words behind the header included); free running, norms and symbols agree by the usual rule;
+    the decoded vector is the oracle's."""
+    torch, nuq = require_cuda()
+    s = levels.size
+    O.set_levels(levels)
+    nuq.set_level_table(levels)
+    flags = O.make_flags(O.NORM_L2, O.LEVELS_TABLE, mode)
+    g = _input(d, 31 * d + s)
+    norms = O.bucket_norms(g, bucket, O.NORM_L2)
+    want, want_bits = O.encode(g, bucket, s, flags, seed=11, offset=3, norms=norms)
+    got, got_bits = gpu_encode(g, bucket, s, flags, seed=11, offset=3, norms=norms)
+    assert got_bits == want_bits and np.array_equal(got, want)
+    free, _ = gpu_encode(g, bucket, s, flags, seed=5, offset=0)
+    compare_symbols(g, bucket, s, flags, 5, 0, free)
+    acc = gpu_decode([free], d, bucket, s)
+    assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([free], d, bucket, s)[1].view(np.uint32))
+
+
+def test_level_table_streams_sum_with_others_and_bad_tables_are_refused():
+    torch, nuq = require_cuda()
+    d, bucket, s = 50000, 1024, 4
+    O.set_levels(_lp(0.35, s))
+    streams = []
+    for k in range(6):                                       # tables of two kinds, the paper's levels, fixed width
+        ls = O.LEVELS_TABLE if k % 2 == 0 else O.LEVELS_EXP
+        if k == 4:
+            O.set_levels(_lp(0.6, s))
+        mode = O.MODE_FIXED if k in (2, 3) else O.MODE_ERC
+        streams.append(O.encode(_input(d, 77 + k), bucket, s, O.make_flags(O.NORM_L2, ls, mode), k + 1, 0)[0])
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    bad = streams[0].copy()
+    bad[17] = bad[16]                                        # levels that do not increase
+    gpu_decode([bad], d, bucket, s, expect_status=-3)
+    for levels in ([0.5, 0.25], [0.0, 0.5], [0.5, 1.0], [float("nan")], [0.1] * 15):
+        with pytest.raises(nuq.NuqError):
+            nuq.set_level_table(levels)
+    nuq.set_level_table([0.25, 0.5])
+    g = torch.zeros(4096, device="cuda")
+    with pytest.raises(nuq.NuqError):                        # the table has two levels, the call asks for three
+        nuq.encode(g, 1024, 3, nuq.LEVELS_TABLE)
