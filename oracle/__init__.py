@@ -15,7 +15,8 @@ from .build import build as _build
 
 NORM_L2, NORM_LINF = 0, 1
 LEVELS_EXP, LEVELS_UNIFORM, LEVELS_TABLE = 0, 1, 2
-MODE_ERC, MODE_FIXED = 0, 1
+MODE_ERC, MODE_FIXED, MODE_CODED = 0, 1, 2
+MAX_CODED_S = 7
 SB = 256
 BLK = 32 * SB
 HEADER_WORDS = 16
@@ -44,6 +45,10 @@ _philox = _sig("nuq_oracle_philox4x32_10", None, _u32p, _u32p, _u32p)
 _draw_word = _sig("nuq_oracle_draw_word", C.c_uint32, C.c_uint64, C.c_uint64, C.c_uint64)
 _draw_uniform = _sig("nuq_oracle_draw_uniform", C.c_float, C.c_uint64, C.c_uint64, C.c_uint64)
 _set_levels = _sig("nuq_oracle_set_levels", C.c_int, _f32p, C.c_uint32)
+_huff = _sig("nuq_oracle_huffman_lengths", C.c_int, np.ctypeslib.ndpointer(np.uint64, flags="C_CONTIGUOUS"),
+             C.c_uint32, _u8p)
+_set_code = _sig("nuq_oracle_set_level_code", C.c_int, _u8p, C.c_uint32)
+_level_code = _sig("nuq_oracle_level_code", C.c_uint32, C.c_uint32, _u8p)
 _num_levels = _sig("nuq_oracle_num_levels", C.c_uint32, C.c_uint32, C.c_uint32)
 _level_value = _sig("nuq_oracle_level_value", C.c_double, C.c_uint32, C.c_uint32, C.c_uint32)
 _fixed_width = _sig("nuq_oracle_fixed_width", C.c_uint32, C.c_uint32, C.c_uint32)
@@ -92,6 +97,34 @@ def set_levels(interior):
     rc = _set_levels(lv, lv.size)
     if rc != 0:
         raise ValueError("not a level sequence")
+
+
+def huffman_lengths(weights):
+    """code lengths of a Huffman tree over the given weights (2 to 8 of them), ties as the C file states"""
+    w = np.ascontiguousarray(weights, np.uint64)
+    out = np.zeros(w.size, np.uint8)
+    if _huff(w, w.size, out) != 0:
+        raise ValueError("2 to 8 weights")
+    return out
+
+
+def set_level_code(lengths):
+    """code lengths of the level indices 1..s+1 that MODE_CODED calls use (canonical code words)"""
+    ln = np.ascontiguousarray(lengths, np.uint8)
+    if _set_code(ln, ln.size - 1) != 0:
+        raise ValueError("not the lengths of a prefix code of at most 7 bits")
+
+
+def level_code(j):
+    """bits of the code word of level index j under the code last set"""
+    bits = np.zeros(8, np.uint8)
+    n = _level_code(j, bits)
+    return bits[:n].copy()
+
+
+def level_histogram(sym, s):
+    """how often each level index 0..s+1 occurs (the sample a code is fitted on)"""
+    return np.bincount(np.asarray(sym).ravel(), minlength=s + 2).astype(np.uint64)
 
 
 def num_levels(levelset, s):

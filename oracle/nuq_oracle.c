@@ -18,6 +18,9 @@
  *   - uniform level set k/2^s  (QSGD / QSGDinf comparison, Sec. 1 and 3)
  *   - arbitrary level sequences L = (0, l_1, ..., l_s, 1), e.g. L_p = (0, p^s, ..., p, 1)
  *                              (Sec. 3.3, "general level sequences"), given as a table
+ *   - coded level indices      the level index of a token written with a Huffman code fitted on
+ *                              a histogram of level indices and then kept (Sec. 5, "efficient
+ *                              encoding": the variant the paper calls encoded NUQSGD)
  *
  * Everything the paper leaves open (bucket tail, fp32 arithmetic order, random
  * generator, container layout) is fixed here in the most literal form; the
@@ -34,7 +37,10 @@
  * examples, Theorem 1 and Lemma 10 bounds, round trip, Philox against the
  * cuRAND host generator; for level tables: the levels of L_p from exact
  * fractions, rounding probabilities by enumeration against exact rational
- * arithmetic, unbiasedness by enumeration, Lemma 7 on hand-worked vectors.
+ * arithmetic, unbiasedness by enumeration, Lemma 7 on hand-worked vectors;
+ * for coded level indices: code lengths of hand-worked trees, least cost among
+ * all prefix codes by brute force, the Kraft sum, canonical code words listed
+ * by hand, a hand-assembled container, the same symbols as the ERC mode.
  */
 #include <math.h>
 #include <stdint.h>
@@ -55,7 +61,8 @@
 enum { NORM_L2 = 0, NORM_LINF = 1 };
 enum { LEVELS_EXP = 0, LEVELS_UNIFORM = 1, LEVELS_TABLE = 2 };
 #define ORC_MAX_S 14u
-enum { MODE_ERC = 0, MODE_FIXED = 1 };
+enum { MODE_ERC = 0, MODE_FIXED = 1, MODE_CODED = 2 };
+#define ORC_MAX_CODED_S 7u         /* coded level indices: at most 8 symbols, code words of at most 7 bits */
 
 /* ------------------------------------------------------------------ */
 /* Philox4x32-10 (Salmon, Moraes, Dror, Shaw 2011).                    */
@@ -118,6 +125,80 @@ static int make_table(const float* interior, uint32_t s, level_table* t) {
 
 /* the interior levels l_1 .. l_s that LEVELS_TABLE calls use from now on */
 int nuq_oracle_set_levels(const float* interior, uint32_t s) { return make_table(interior, s, &g_table); }
+
+/* ------------------------------------------------------------------ */
+/* Coded level indices (Sec. 5, "efficient encoding").  The paper says only that a Huffman code
+ * is fitted on an initial sample and then kept.  Fixed here: the symbols are the level indices
+ * 1..s+1 of the nonzero coordinates; the tree is built by joining, n - 1 times, the two nodes
+ * of least weight, where among nodes of equal weight a leaf goes before a joined node, leaves
+ * go by index and joined nodes by age; only the code lengths are taken from the tree, and the
+ * code words are the canonical ones for those lengths (symbols ordered by length, then index;
+ * the first word is all zeros, each next word is the previous plus one, extended with zeros). */
+typedef struct { uint32_t n; uint8_t len[ORC_MAX_CODED_S + 1]; uint32_t word[ORC_MAX_CODED_S + 1]; } level_code;
+static level_code g_code;
+
+int nuq_oracle_huffman_lengths(const uint64_t* weight, uint32_t n, uint8_t* len) {
+    if (n < 2 || n > ORC_MAX_CODED_S + 1) return ORC_ERR_ARG;
+    uint64_t w[2 * (ORC_MAX_CODED_S + 1)];
+    int parent[2 * (ORC_MAX_CODED_S + 1)], open[2 * (ORC_MAX_CODED_S + 1)];
+    uint32_t nodes = n;
+    for (uint32_t i = 0; i < n; ++i) { w[i] = weight[i]; parent[i] = -1; open[i] = 1; }
+    for (uint32_t join = 0; join + 1 < n; ++join) {
+        int pick[2];
+        for (int k = 0; k < 2; ++k) {                        /* least weight; the lowest node number among equals */
+            int best = -1;
+            for (uint32_t i = 0; i < nodes; ++i)
+                if (open[i] && (best < 0 || w[i] < w[best])) best = (int)i;
+            open[best] = 0;
+            pick[k] = best;
+        }
+        w[nodes] = w[pick[0]] + w[pick[1]];
+        parent[nodes] = -1; open[nodes] = 1;
+        parent[pick[0]] = parent[pick[1]] = (int)nodes;
+        ++nodes;
+    }
+    for (uint32_t i = 0; i < n; ++i) {
+        uint32_t depth = 0;
+        for (int at = (int)i; parent[at] >= 0; at = parent[at]) ++depth;
+        len[i] = (uint8_t)depth;
+    }
+    return ORC_OK;
+}
+
+static int make_code(const uint8_t* len, uint32_t n, level_code* c) {
+    if (n < 2 || n > ORC_MAX_CODED_S + 1) return ORC_ERR_ARG;
+    uint32_t kraft = 0;                                      /* in units of 2^-7 */
+    for (uint32_t i = 0; i < n; ++i) {
+        if (len[i] < 1 || len[i] > ORC_MAX_CODED_S) return ORC_ERR_ARG;
+        kraft += 1u << (ORC_MAX_CODED_S - len[i]);
+    }
+    if (kraft > (1u << ORC_MAX_CODED_S)) return ORC_ERR_ARG; /* no prefix code has these lengths */
+    c->n = n;
+    uint32_t next = 0, prev_len = 0;
+    for (uint32_t l = 1; l <= ORC_MAX_CODED_S; ++l)
+        for (uint32_t i = 0; i < n; ++i) {
+            if (len[i] != l) continue;
+            next <<= (l - prev_len);
+            prev_len = l;
+            c->len[i] = (uint8_t)l;
+            c->word[i] = next++;
+        }
+    return ORC_OK;
+}
+
+/* lengths[j-1] = code length of level index j, j = 1..s+1 */
+int nuq_oracle_set_level_code(const uint8_t* lengths, uint32_t s) {
+    if (s < 1 || s > ORC_MAX_CODED_S) return ORC_ERR_ARG;
+    return make_code(lengths, s + 1, &g_code);
+}
+
+/* the code word of level index j under the code last set, one bit per byte; returns its length */
+uint32_t nuq_oracle_level_code(uint32_t j, uint8_t* bits) {
+    if (j < 1 || j > g_code.n) return 0;
+    uint32_t l = g_code.len[j - 1];
+    for (uint32_t k = 0; k < l; ++k) bits[k] = (uint8_t)((g_code.word[j - 1] >> (l - 1 - k)) & 1u);
+    return l;
+}
 
 /* number of levels including 0 and 1 */
 uint32_t nuq_oracle_num_levels(uint32_t levelset, uint32_t s) {
@@ -364,8 +445,9 @@ static uint64_t count_blocks(uint64_t d, uint32_t bucket) {
 }
 
 /* longest ERC code of a level index, for the capacity bound */
-static uint32_t max_level_code_bits(uint32_t levelset, uint32_t s) {
+static uint32_t max_level_code_bits(uint32_t levelset, uint32_t s, uint32_t mode) {
     uint8_t tmp[160];
+    if (mode == MODE_CODED) return ORC_MAX_CODED_S;
     uint32_t nlev = nuq_oracle_num_levels(levelset, s), best = 0;
     for (uint32_t j = 1; j < nlev; ++j) { uint32_t l = nuq_oracle_erc_encode(j, tmp); if (l > best) best = l; }
     return best;
@@ -373,15 +455,18 @@ static uint32_t max_level_code_bits(uint32_t levelset, uint32_t s) {
 
 static int check_args(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint32_t levelset, uint32_t mode) {
     if (d == 0 || bucket == 0 || s < 1 || s > ORC_MAX_S) return ORC_ERR_ARG;
-    if (norm_kind > 1 || levelset > 2 || mode > 1) return ORC_ERR_ARG;
+    if (norm_kind > 1 || levelset > 2 || mode > 2) return ORC_ERR_ARG;
     if (levelset == LEVELS_UNIFORM && s > 8) return ORC_ERR_ARG;
+    if (mode == MODE_CODED && (levelset == LEVELS_UNIFORM || s > ORC_MAX_CODED_S)) return ORC_ERR_ARG;
     return ORC_OK;
 }
 
 /* A container with a level table carries the s interior levels (fp32 words) behind the 16 header
  * words, padded with a zero word to an even count so that the offset table stays 8-byte aligned.  */
-static uint32_t header_words(uint32_t levelset, uint32_t s) {
-    return ORC_HEADER_WORDS + (levelset == LEVELS_TABLE ? ((s + 1u) & ~1u) : 0u);
+/* A container with coded level indices carries, behind that, the s + 1 code lengths as the bytes of
+ * two words (byte j - 1 in memory = length of index j, the rest zero).                               */
+static uint32_t header_words(uint32_t levelset, uint32_t s, uint32_t mode) {
+    return ORC_HEADER_WORDS + (levelset == LEVELS_TABLE ? ((s + 1u) & ~1u) : 0u) + (mode == MODE_CODED ? 2u : 0u);
 }
 
 /* bytes that always suffice for the container */
@@ -389,13 +474,13 @@ uint64_t nuq_oracle_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32
     uint32_t levelset = (flags >> 8) & 0xff, mode = (flags >> 16) & 0xff;
     if (check_args(d, bucket, s, flags & 0xff, levelset, mode) != ORC_OK) return 0;
     uint64_t nb = (d + bucket - 1) / bucket;
-    uint64_t hw = header_words(levelset, s);
+    uint64_t hw = header_words(levelset, s, mode);
     if (mode == MODE_FIXED) {
         uint64_t w = nuq_oracle_fixed_width(levelset, s);
         return 4 * (hw + nb * (1 + ((uint64_t)bucket * w + 31) / 32));
     }
     uint64_t nblk = count_blocks(d, bucket);
-    uint64_t token_bits = d * (2 + (uint64_t)max_level_code_bits(levelset, s));
+    uint64_t token_bits = d * (2 + (uint64_t)max_level_code_bits(levelset, s, mode));
     return 4 * hw + 8 * (nblk + 1) + nblk * (4 + 64 + 4) + (token_bits + 7) / 8;
 }
 
@@ -409,17 +494,20 @@ int nuq_oracle_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     int rc = check_args(d, bucket, s, norm_kind, levelset, mode);
     if (rc != ORC_OK) return rc;
     if (levelset == LEVELS_TABLE && g_table.s != s) return ORC_ERR_ARG;   /* the table set by nuq_oracle_set_levels */
+    if (mode == MODE_CODED && g_code.n != s + 1) return ORC_ERR_ARG;      /* the code set by nuq_oracle_set_level_code */
     if (capacity_bytes < nuq_oracle_encode_bound(d, bucket, s, flags)) return ORC_ERR_CAPACITY;
     memset(out, 0, (size_t)nuq_oracle_encode_bound(d, bucket, s, flags));
 
     uint32_t* words = (uint32_t*)out;
     uint64_t nb = (d + bucket - 1) / bucket;
-    uint64_t nblk = mode == MODE_ERC ? count_blocks(d, bucket) : nb;
-    uint32_t hw = header_words(levelset, s);
+    uint64_t nblk = mode != MODE_FIXED ? count_blocks(d, bucket) : nb;
+    uint32_t hw = header_words(levelset, s, mode);
     if (levelset == LEVELS_TABLE)
         for (uint32_t j = 1; j <= s; ++j) words[ORC_HEADER_WORDS + j - 1] = float_bits(g_table.level[j]);
+    if (mode == MODE_CODED)
+        for (uint32_t j = 1; j <= s + 1; ++j) ((uint8_t*)(words + hw - 2))[j - 1] = g_code.len[j - 1];
     uint64_t* table = (uint64_t*)(words + hw);
-    uint32_t* payload = mode == MODE_ERC ? words + hw + 2 * (nblk + 1) : words + hw;
+    uint32_t* payload = mode != MODE_FIXED ? words + hw + 2 * (nblk + 1) : words + hw;
     uint32_t w = nuq_oracle_fixed_width(levelset, s);
 
     uint8_t* sign = (uint8_t*)malloc(bucket);
@@ -467,7 +555,8 @@ int nuq_oracle_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
                     uint32_t l = nuq_oracle_erc_encode(t - t_prev, code);           /* ERC(gap)   */
                     for (uint32_t k = 0; k < l; ++k) put_bit(payload, pbits++, code[k]);
                     put_bit(payload, pbits++, sign[slo + i]);                       /* sign bit   */
-                    l = nuq_oracle_erc_encode(sym[slo + i], code);                  /* ERC(level) */
+                    if (mode == MODE_CODED) l = nuq_oracle_level_code(sym[slo + i], code);   /* its code word */
+                    else l = nuq_oracle_erc_encode(sym[slo + i], code);             /* ERC(level) */
                     for (uint32_t k = 0; k < l; ++k) put_bit(payload, pbits++, code[k]);
                     t_prev = t;
                     ++nnz;
@@ -480,7 +569,7 @@ int nuq_oracle_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
             pbits = (pbits + 31) & ~(uint64_t)31;
         }
     }
-    if (mode == MODE_ERC) table[nblk] = pbits;
+    if (mode != MODE_FIXED) table[nblk] = pbits;
 
     uint64_t container_bits = 32u * (uint64_t)(payload - words) + pbits;
     words[0] = ORC_MAGIC; words[1] = ORC_VERSION;
@@ -510,7 +599,9 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
     uint64_t container_bits = (uint64_t)words[10] | ((uint64_t)words[11] << 32);
     uint32_t nlev = nuq_oracle_num_levels(levelset, s);
     uint32_t w = nuq_oracle_fixed_width(levelset, s);
-    uint32_t hw = header_words(levelset, s);
+    uint32_t hw = header_words(levelset, s, mode);
+    level_code lc;
+    if (mode == MODE_CODED && make_code((const uint8_t*)(words + hw - 2), s + 1, &lc) != ORC_OK) return ORC_ERR_STREAM;
     if (levelset == LEVELS_TABLE) {                          /* the levels must be a level sequence */
         level_table t;
         float interior[ORC_MAX_S];
@@ -581,15 +672,25 @@ int nuq_oracle_decode_symbols(const void* stream, uint64_t d, uint32_t bucket, u
                     t += N;
                     if (t > sn || p >= end) return ORC_ERR_STREAM;
                     uint32_t sg = get_bit(payload, p++);     /* the sign bit */
-                    /* ERC^-1: the level index */
                     N = 1;
-                    for (;;) {
-                        if (p >= end) return ORC_ERR_STREAM;
-                        if (get_bit(payload, p) == 0) { ++p; break; }
-                        if (N + 1 > 32 || p + N + 1 > end) return ORC_ERR_STREAM;
-                        uint64_t v = 0;
-                        for (uint64_t i = 0; i <= N; ++i) v = (v << 1) | get_bit(payload, p + i);
-                        p += N + 1; N = v;
+                    if (mode == MODE_CODED) {                /* the level index: bits until they spell a code word */
+                        uint32_t v = 0, l = 0, found = 0;
+                        while (!found) {
+                            if (p >= end || l == ORC_MAX_CODED_S) return ORC_ERR_STREAM;
+                            v = (v << 1) | get_bit(payload, p++);
+                            ++l;
+                            for (uint32_t j = 0; j < lc.n; ++j)
+                                if (lc.len[j] == l && lc.word[j] == v) { N = j + 1; found = 1; }
+                        }
+                    } else {                                 /* ERC^-1: the level index */
+                        for (;;) {
+                            if (p >= end) return ORC_ERR_STREAM;
+                            if (get_bit(payload, p) == 0) { ++p; break; }
+                            if (N + 1 > 32 || p + N + 1 > end) return ORC_ERR_STREAM;
+                            uint64_t v = 0;
+                            for (uint64_t i = 0; i <= N; ++i) v = (v << 1) | get_bit(payload, p + i);
+                            p += N + 1; N = v;
+                        }
                     }
                     if (N >= nlev) return ORC_ERR_STREAM;
                     sym[slo + t - 1] = (uint16_t)N;

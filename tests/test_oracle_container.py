@@ -153,3 +153,81 @@ def test_c1_reference_statistics():
     rc, acc = O.decode_accumulate([st], g.size, 1024, 3)
     rel = float(((acc - g) ** 2).sum() / (g ** 2).sum())
     assert rc == 0 and 1.5 < rel < 3.125                # below Theorem 1's bound for (1024, 3)
+
+
+# ---- coded level indices (Sec. 5, "efficient encoding") -------------------------------------------
+
+CODED = O.make_flags(mode=O.MODE_CODED)
+
+
+def _erc_len(n):
+    return len(O.erc_encode(n))
+
+
+def test_coded_stream_built_by_hand():
+    """Lengths (2, 2, 1) for the indices 1, 2, 3 give the words 10, 11, 0.  Tokens ERC(gap) | sign | word:
+    pos 2 -> 100|0|11, pos 5 -> 110|1|10, pos 6 -> 0|0|0  (15 bits: 1000 1111 0110 000)."""
+    v, norms = _hand_vector()
+    O.set_level_code([2, 2, 1])
+    st, bits = O.encode(v, 7, 2, CODED, seed=3, offset=0, norms=norms)
+    h = O.header(st)
+    assert (h["nblk"], h["code_bits"], h["nnz"], h["flags"]) == (1, 15, 3, 2 << 16)
+    assert [hex(x) for x in st[16:18]] == ["0x10202", "0x0"]           # the lengths, one byte each
+    assert list(st[18:22].view(np.uint64)) == [0, 96]
+    assert [hex(x) for x in st[22:25]] == ["0x3f800000", "0xf", "0x8f600000"]
+    assert bits == h["container_bits"] == 32 * 25 and st.size == 25
+    rc, sign, sym, nrm = O.decode_symbols(st, 7, 7, 2)
+    assert rc == 0 and list(sym) == [0, 2, 0, 0, 1, 3, 0] and list(sign) == [0, 0, 0, 0, 1, 0, 0]
+    O.set_level_code([1, 2, 2])                              # the decoder reads the code from the container
+    rc, acc = O.decode_accumulate([st, st], 7, 7, 2)
+    assert rc == 0 and list(acc) == [0.0, 1.0, 0.0, 0.0, -0.5, 2.0, 0.0]
+
+
+@pytest.mark.parametrize("s, levelset", [(4, O.LEVELS_EXP), (2, O.LEVELS_EXP), (7, O.LEVELS_EXP), (3, O.LEVELS_TABLE)])
+def test_coded_mode_sends_the_same_symbols_and_saves_what_the_histogram_says(s, levelset):
+    rng = np.random.default_rng(s)
+    d, bucket = 20_000, 2048
+    g = (rng.standard_t(3, d) * 10.0 ** rng.uniform(-3, 0, d)).astype(np.float32)
+    if levelset == O.LEVELS_TABLE:
+        O.set_levels(np.array([0.3 ** 3, 0.3 ** 2, 0.3], np.float32))
+    erc = O.make_flags(O.NORM_L2, levelset, O.MODE_ERC)
+    coded = O.make_flags(O.NORM_L2, levelset, O.MODE_CODED)
+    sign, sym, norms = O.quantize(g, bucket, s, O.NORM_L2, levelset, 9, 2)
+    hist = O.level_histogram(sym, s)
+    assert hist.sum() == d and hist.size == s + 2
+    lengths = O.huffman_lengths(hist[1:])
+    O.set_level_code(lengths)
+    a, abits = O.encode(g, bucket, s, erc, 9, 2)
+    b, bbits = O.encode(g, bucket, s, coded, 9, 2)
+    rc, sign_b, sym_b, norms_b = O.decode_symbols(b, d, bucket, s)
+    assert rc == 0 and np.array_equal(sign_b, sign) and np.array_equal(sym_b, sym) and np.array_equal(norms_b, norms)
+    ha, hb = O.header(a), O.header(b)
+    saved = sum(int(hist[j]) * (_erc_len(j) - int(lengths[j - 1])) for j in range(1, s + 2))
+    assert ha["nnz"] == hb["nnz"] and ha["code_bits"] - hb["code_bits"] == saved
+    assert saved >= 0                                        # ERC is a prefix code too, and Huffman's is the cheapest
+    assert np.array_equal(O.decode_accumulate([a], d, bucket, s)[1], O.decode_accumulate([b], d, bucket, s)[1])
+    assert np.array_equal(O.decode_accumulate([a, b], d, bucket, s)[1], O.decode_accumulate([b, a], d, bucket, s)[1])
+    # any other code the lengths allow works as well: here every index gets a word of the same length
+    worse = np.full(s + 1, int(np.ceil(np.log2(s + 1))), np.uint8)
+    O.set_level_code(worse)
+    c, _ = O.encode(g, bucket, s, coded, 9, 2)
+    assert O.header(c)["code_bits"] - ha["code_bits"] == sum(int(hist[j]) * (int(worse[j - 1]) - _erc_len(j)) for j in range(1, s + 2))
+    assert np.array_equal(O.decode_symbols(c, d, bucket, s)[2], sym)
+
+
+def test_malformed_coded_streams_are_rejected():
+    rng = np.random.default_rng(2)
+    g = rng.standard_normal(3000).astype(np.float32)
+    O.set_level_code([1, 2, 3, 3])
+    st, _ = O.encode(g, 512, 3, CODED, 1, 0)
+    assert O.decode_symbols(st, 3000, 512, 3)[0] == 0
+    bad = st.copy(); bad[16] = 0x01010101                    # Kraft sum 2: no prefix code
+    assert O.decode_symbols(bad, 3000, 512, 3)[0] == -3
+    bad = st.copy(); bad[16] = 0x03030200                    # a zero length
+    assert O.decode_symbols(bad, 3000, 512, 3)[0] == -3
+    bad = st.copy(); bad[16] = 0x04040403                    # an incomplete code: chains that run into an unused word
+    assert O.decode_symbols(bad, 3000, 512, 3)[0] == -3
+    assert O.encode_bound(3000, 512, 8, CODED) == 0          # more than 8 level indices
+    assert O.encode_bound(3000, 512, 4, O.make_flags(O.NORM_L2, O.LEVELS_UNIFORM, O.MODE_CODED)) == 0
+    with pytest.raises(Exception):
+        O.encode(g, 512, 4, CODED, 1, 0)                     # the code set has 4 words, s = 4 needs 5

@@ -466,3 +466,44 @@ def test_level_table_container():
     O.set_levels(np.array([2.0 ** -3, 2.0 ** -2, 2.0 ** -1], np.float32))
     for sym in range(5):
         assert O.dequantize(np.float32(1.7), 3, O.LEVELS_TABLE, 1, sym) == O.dequantize(np.float32(1.7), 3, O.LEVELS_EXP, 1, sym)
+
+
+# ---- coded level indices (Sec. 5, "efficient encoding") -------------------------------------------
+
+def test_huffman_lengths_and_code_words_of_hand_worked_trees():
+    for row in golden_rows("level_codes.txt"):
+        n = int(row[0])
+        weights = [int(x) for x in row[1:1 + n]]
+        lengths = [int(x) for x in row[1 + n:1 + 2 * n]]
+        words = row[1 + 2 * n:1 + 3 * n]
+        assert list(O.huffman_lengths(weights)) == lengths, weights
+        O.set_level_code(lengths)
+        assert ["".join(str(b) for b in O.level_code(j)) for j in range(1, n + 1)] == words, weights
+        assert len(O.level_code(0)) == 0 and len(O.level_code(n + 1)) == 0
+
+
+def test_huffman_cost_is_the_least_of_any_prefix_code():
+    """A prefix code with lengths l_i exists iff sum 2^-l_i <= 1 (Kraft); the Huffman lengths reach the
+    least sum w_i l_i over all of them, and fill the Kraft sum exactly."""
+    rng = np.random.default_rng(11)
+    for n in (2, 3, 4, 5, 6):
+        grids = np.stack(np.meshgrid(*[np.arange(1, 8)] * n, indexing="ij"), -1).reshape(-1, n)
+        feasible = grids[(2.0 ** -grids).sum(1) <= 1.0]
+        for trial in range(6):
+            w = rng.integers(0, 5 if trial % 2 else 1000, n).astype(np.uint64)
+            ln = O.huffman_lengths(w).astype(np.int64)
+            assert sum(Fraction(1, 2 ** int(l)) for l in ln) == 1
+            assert int((w.astype(np.int64) * ln).sum()) == int((feasible * w.astype(np.int64)).sum(1).min()), (w, ln)
+
+
+def test_level_code_words_are_prefix_free_and_bad_lengths_are_refused():
+    for lengths in ([1, 2, 3, 3], [2, 2, 2, 3, 4, 4], [3, 3, 3, 3, 3, 3, 3, 3], [1, 7], [2, 3, 1]):
+        O.set_level_code(lengths)                            # Kraft sum <= 1: incomplete codes are codes too
+        words = ["".join(str(b) for b in O.level_code(j)) for j in range(1, len(lengths) + 1)]
+        assert [len(w) for w in words] == lengths
+        for a in range(len(words)):
+            for b in range(len(words)):
+                assert a == b or not words[b].startswith(words[a])
+    for lengths in ([1, 1, 2], [0, 1], [1, 8], [2], [1] * 9, [1, 2, 3, 3, 3]):
+        with pytest.raises(ValueError):
+            O.set_level_code(lengths)
