@@ -19,7 +19,8 @@
  *
  * Limits: 1 <= d < 2^40; bucket a multiple of 256 with 256 <= bucket <= 8192,
  * or bucket in {16384, 32768, 65536}; 1 <= s <= 14 (exponential levels and
- * level tables) or 1 <= s <= 8 (uniform levels); 1 <= K <= 64.
+ * level tables) or 1 <= s <= 8 (uniform levels) or 1 <= s <= 7 (coded level
+ * indices); 1 <= K <= 64.
  *
  * Container written by nuq_encode (all u32 words little endian; bit p of a bit
  * string sits in word p>>5 at bit 31-(p&31)):
@@ -29,6 +30,9 @@
  *   level table   only in streams with NUQ_LEVELS_TABLE: the s interior
  *                 levels l_1 .. l_s as fp32 words, then a zero word if s is
  *                 odd; everything below follows behind it
+ *   code lengths  only in streams with NUQ_MODE_CODED: two words whose bytes (in
+ *                 memory order) are the code lengths of the level indices
+ *                 1 .. s+1, the remaining bytes zero; behind the level table
  *   ERC mode      (nblk+1) u64 bit offsets of the coding blocks, relative to
  *                 the payload that follows the table.  A coding block is up to
  *                 8192 consecutive elements of one bucket: norm (fp32 bits) |
@@ -36,6 +40,11 @@
  *                 a word) | the sub-blocks' token strings back to back | zero
  *                 padding to a word.  A token is ERC(gap) sign ERC(level
  *                 index); the gap is counted from the start of the sub-block.
+ *   coded mode    as the ERC mode, but the level index of a token is written
+ *                 with the canonical prefix code of the lengths above (Sec. 5,
+ *                 "efficient encoding": Huffman-coded levels): level indices
+ *                 ordered by (length, index), the first word all zeros, each
+ *                 next word the previous plus one, extended with zeros.
  *   fixed mode    per bucket: norm word | fields of w bits (sign, level index)
  *                 MSB first | zero padding to a word; no table.
  */
@@ -68,6 +77,9 @@ typedef int nuq_status;
                                     *           nuq_set_level_table   (Sec. 3.3)                  */
 #define NUQ_MODE_ERC (0u << 16)   /* bits 16-23: Elias-recursive token stream (App. A)            */
 #define NUQ_MODE_FIXED (1u << 16) /*             fixed-width fields ("4-bit" variant of Sec. 5)   */
+#define NUQ_MODE_CODED (2u << 16) /*             as NUQ_MODE_ERC with the level indices written   *
+                                   *             in the code of nuq_set_level_code ("encoded       *
+                                   *             NUQSGD", Sec. 5); not with uniform levels; s <= 7 */
 #define NUQ_TEST_NORMS (1u << 24) /* take bucket norms from nuq_set_test_norms (parity testing)   */
 #define NUQ_TEST_SHORT_PATIENCE (1u << 25) /* test hook: the cross-tile scan gives up after two  *
                                    * polls instead of tens of milliseconds, so that a test can    *
@@ -177,6 +189,33 @@ uint64_t nuq_encode_bound(uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm
  * 1 <= s <= 14.
  */
 nuq_status nuq_set_level_table(const float* interior_levels, uint32_t s);
+
+/*
+ * Coded level indices (Sec. 5, "efficient encoding": a Huffman code is fitted on an initial
+ * sample of gradients and then kept; the paper calls the variant encoded NUQSGD).  Three steps:
+ *
+ * nuq_level_histogram  quantizes g exactly as nuq_encode would (same arguments, same draws;
+ *            norm_kind without a mode, not NUQ_LEVELS_UNIFORM) and counts how often each level
+ *            index 0 .. s+1 comes out.  hist: DEVICE array of s + 2 u64 counters, 8-byte
+ *            aligned, overwritten in stream order.  Bucket norms are taken in a pass of
+ *            their own (fp64 sums), so a coordinate within rounding of a decision threshold
+ *            may be counted one level off what nuq_encode sends.
+ * nuq_fit_level_code   HOST arrays: from hist[1 .. s+1] (hist[0], the zeros, is not coded)
+ *            builds a Huffman tree and returns the s + 1 code lengths, lengths[j-1] for level
+ *            index j.  The tree joins, s times, the two nodes of least weight; among equal
+ *            weights a leaf goes before a joined node, leaves by index, joined nodes by age.
+ *            A level index that never occurred still gets a word.  1 <= s <= 7, so no word is
+ *            longer than 7 bits.
+ * nuq_set_level_code   HOST array of s + 1 lengths (1 .. 7 each, Kraft sum at most 1; those
+ *            of nuq_fit_level_code or any others): the code nuq_encode uses from now on when
+ *            called with NUQ_MODE_CODED and this s.  The container carries the lengths;
+ *            nuq_decode_accumulate reads them from there.
+ * Each returns NUQ_ERR_INVALID_ARG for arguments outside these ranges.
+ */
+nuq_status nuq_level_histogram(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
+                               uint64_t offset, uint64_t* hist, void* stream);
+nuq_status nuq_fit_level_code(const uint64_t* hist, uint32_t s, uint8_t* lengths);
+nuq_status nuq_set_level_code(const uint8_t* lengths, uint32_t s);
 
 /* Parity-test hook: device array of ceil(d/bucket) bucket norms that nuq_encode uses in
  * place of its own reduction when NUQ_TEST_NORMS is set; NULL clears it.  The pointer is

@@ -22,7 +22,10 @@ static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBy
 struct WsEntry {
     Workspace* ptr = nullptr;
     size_t bytes = 0;
-    bool clean = false;      // the scan state is all zero: set by the allocation, kept by every encode kernel
+    // Bytes from the start that may hold something else than zeros where an encode call keeps its scan state
+    // (0: none).  The allocation is zeroed and every encode kernel leaves its scan state zeroed, but the bucket
+    // norms of a wide-bucket call or of a histogram call stay behind, at a place that depends on that call's size.
+    size_t dirty_to = 0;
 };
 
 // One mutex guards the host-side bookkeeping below (maps, tables); it is held for the microseconds a
@@ -34,6 +37,8 @@ std::set<int> g_lut_ready;                // devices whose constant LUT is uploa
 std::map<int, const float*> g_test_norms;   // device -> bucket norms of nuq_set_test_norms
 float g_levels[kMaxTableS + 2], g_inv_width[kMaxTableS + 2];   // the level table of nuq_set_level_table ...
 uint32_t g_levels_s = 0;                                       // ... and its number of interior levels (0: none set)
+uint32_t g_level_code[kMaxCodedS + 1];                         // the code of nuq_set_level_code: word | length << 16 ...
+uint32_t g_level_code_n = 0;                                   // ... and how many level indices it covers (0: none set)
 std::map<int, Workspace*> g_static_ws;   // device -> address of g_static_scratch on that device
 uint32_t g_erc_len[256];
 bool g_erc_len_ready = false;
@@ -56,7 +61,8 @@ bool bucket_ok(uint32_t bucket) {
 bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geometry* G) {
     const uint32_t norm_kind = flags & 0xffu, levelset = (flags >> 8) & 0xffu, mode = (flags >> 16) & 0xffu;
     if (d == 0 || d >= (1ull << 40) || !bucket_ok(bucket) || s < 1) return false;
-    if (norm_kind > 1 || levelset > 2 || mode > 1) return false;
+    if (norm_kind > 1 || levelset > 2 || mode > 2) return false;
+    if (mode == kModeCoded && (levelset == kLevelsUniform || s > kMaxCodedS)) return false;
     if (s > (levelset == kLevelsUniform ? 8u : 14u)) return false;
     if (flags & ~(0x00ffffffu | NUQ_TEST_NORMS | NUQ_TEST_SHORT_PATIENCE)) return false;
     G->d = d;
@@ -67,7 +73,7 @@ bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geom
     G->mode = mode;
     G->nb = (d + bucket - 1) / bucket;
     G->nlev = levelset == kLevelsUniform ? (1u << s) + 1u : s + 2u;
-    G->header_words = kHeaderWords + (levelset == kLevelsTable ? ((s + 1u) & ~1u) : 0u);
+    G->header_words = kHeaderWords + (levelset == kLevelsTable ? ((s + 1u) & ~1u) : 0u) + (mode == kModeCoded ? 2u : 0u);
     G->pad = 0;
     uint32_t b = 0;
     while ((1u << b) < G->nlev) ++b;
@@ -93,6 +99,7 @@ bool make_geometry(uint64_t d, uint32_t bucket, uint32_t s, uint32_t flags, Geom
 }
 
 uint32_t max_level_code_bits(const Geometry& G) {
+    if (G.mode == kModeCoded) return kMaxCodedS;            // whatever code is set
     uint32_t best = 0;
     for (uint32_t sym = 1; sym < G.nlev; ++sym) best = erc_len(sym) > best ? erc_len(sym) : best;
     return best;
@@ -104,13 +111,25 @@ uint32_t max_level_code_bits(const Geometry& G) {
 // itself a much smaller bound holds: a symbol above the lowest level needs r > 2^-s, and at most
 // 4^s coordinates of a bucket can have that (the counting step of the paper's sparsity lemma,
 // Lemma 10); all others cost at most |ERC(1)| + 1 + |ERC(1)| = 3 bits per consumed position.
+// In the coded mode the same holds with the lengths of the code in use: a lowest-level token costs
+// at most 2 + len(1) bits per consumed position (|ERC(gap)| + 1 + len(1) <= gap (2 + len(1))), the
+// others at most the longest of the remaining words more.
 uint32_t token_bits_bound(const Geometry& G, uint32_t elems, uint32_t buckets, bool norms_are_ours) {
-    const uint32_t L = max_level_code_bits(G);
+    uint32_t L = max_level_code_bits(G), low = 1u, rest = L;    // longest code, code of index 1, longest of the others
+    if (G.mode == kModeCoded) {
+        L = rest = 0;
+        low = g_level_code[0] >> 16;
+        for (uint32_t j = 0; j <= G.s; ++j) {
+            const uint32_t len = g_level_code[j] >> 16;
+            L = len > L ? len : L;
+            if (j >= 1) rest = len > rest ? len : rest;
+        }
+    }
     const uint32_t safe = elems * (2u + L);
     if (!norms_are_ours || G.norm_kind != kNormL2 || G.levelset != kLevelsExp || G.s > 7u) return safe;
     const uint64_t high = (uint64_t)buckets * ((1ull << (2u * G.s)) + 8u);      // + slack for the rounding of the norm
     const uint32_t nhigh = high < elems ? (uint32_t)high : elems;
-    const uint32_t tight = 3u * elems + nhigh * (L - 1u);
+    const uint32_t tight = (2u + low) * elems + nhigh * (rest > low ? rest - low : 0u);
     return tight < safe ? tight : safe;
 }
 
@@ -157,7 +176,7 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
         if (cudaMemset(p, 0, want) != cudaSuccess) return NUQ_ERR_CUDA;
         e.ptr = static_cast<Workspace*>(p);
         e.bytes = want;
-        e.clean = true;
+        e.dirty_to = 0;
         if (carried && cudaMemcpy(&e.ptr->status, &carried, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
             return NUQ_ERR_CUDA;
     }
@@ -192,7 +211,7 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, uint32_t flags) {
     P.patience = (flags & NUQ_TEST_SHORT_PATIENCE) ? 2u : 1u << 16;
     P.window_words = 0;
     P.stage_words = 0;
-    if (G.mode == kModeErc) {
+    if (G.mode != kModeFixed) {
         P.stage_words = (stage_words_for(G, norms_are_ours) + 3u) & ~3u;
         // a warp's 1024 elements lie in at most this many buckets
         const uint32_t warp_elems = kBLK / kEncWarps;
@@ -213,7 +232,7 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, uint32_t flags) {
 // enqueues the kernels.  `ws` must hold pl.state_bytes + pl.norms_bytes.
 static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const float* g, uint32_t norm_kind,
                                  uint64_t seed, uint64_t offset, void* out, uint64_t* out_bits, Workspace* ws,
-                                 bool* ws_clean, int dev, cudaStream_t stream) {
+                                 WsEntry* entry, int dev, cudaStream_t stream) {
     Geometry& G = P.geo;
     const bool test_norms = (norm_kind & NUQ_TEST_NORMS) != 0;
     if (!g_lut_ready.count(dev)) {
@@ -221,12 +240,16 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
         g_lut_ready.insert(dev);
     }
     // The encode kernel leaves its scan state zeroed when it ends, so a clearing pass is needed only where
-    // that cannot be relied on (ws_clean == nullptr: always clear; *ws_clean false: an earlier launch failed).
-    if (ws_clean == nullptr || !*ws_clean) {
-        if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, pl.state_bytes - kWorkspaceClearFrom,
-                            stream) != cudaSuccess)
+    // that cannot be relied on: entry == nullptr (the shared static array: always), or something was left
+    // behind in the workspace (then all of that is cleared, not only what this call will use: a later, longer
+    // call keeps scan state further up).
+    if (entry == nullptr || entry->dirty_to > kWorkspaceClearFrom) {
+        size_t upto = pl.state_bytes;
+        if (entry && entry->dirty_to > upto) upto = entry->dirty_to < entry->bytes ? entry->dirty_to : entry->bytes;
+        if (cudaMemsetAsync(reinterpret_cast<char*>(ws) + kWorkspaceClearFrom, 0, upto - kWorkspaceClearFrom, stream) !=
+            cudaSuccess)
             return NUQ_ERR_CUDA;
-        if (ws_clean) *ws_clean = true;
+        if (entry) entry->dirty_to = 0;
     }
 
     P.g = g;
@@ -247,12 +270,16 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
         P.levels[j] = G.levelset == kLevelsTable ? g_levels[j] : 0.0f;
         P.inv_width[j] = G.levelset == kLevelsTable ? g_inv_width[j] : 0.0f;
     }
+    for (uint32_t j = 0; j <= kMaxCodedS; ++j) P.level_code[j] = G.mode == kModeCoded ? g_level_code[j] : 0u;
     for (uint32_t r = 0; r < 10; ++r) {               // Philox key schedule (Weyl sequence)
         P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
     }
+    // the bucket norms of a wide-bucket call lie behind its scan state, where a later call with more tiles
+    // keeps scan state: the next call has to clear first
+    if (pl.norms_bytes && entry && !test_norms) entry->dirty_to = pl.state_bytes + pl.norms_bytes;
     if (launch_encode(P, stream) != cudaSuccess) {
-        if (ws_clean) *ws_clean = false;
+        if (entry) entry->dirty_to = entry->bytes;          // whatever state the failed launch left
         return NUQ_ERR_CUDA;
     }
     // remember the mode of the container at this address: a hint for the decoder's choice of kernels,
@@ -273,6 +300,7 @@ static bool encode_args_ok(const float* g, uint64_t d, uint32_t bucket, uint32_t
         if (cudaGetDevice(&dev) != cudaSuccess || !g_test_norms.count(dev) || !g_test_norms[dev]) return false;
     }
     if (G->levelset == kLevelsTable && g_levels_s != s) return false;   // no level table of this length has been set
+    if (G->mode == kModeCoded && g_level_code_n != s + 1) return false; // no code for s + 1 level indices has been set
     return true;
 }
 
@@ -306,6 +334,115 @@ nuq_status nuq_set_level_table(const float* interior_levels, uint32_t s) {
     return NUQ_OK;
 }
 
+// Canonical code words for the given lengths: level indices ordered by (length, index); the first
+// word is all zeros, each next one is the previous plus one, extended with zeros to its length.
+static bool canonical_code(const uint8_t* lengths, uint32_t n, uint32_t* code) {
+    uint32_t kraft = 0;                                      // in units of 2^-7
+    for (uint32_t j = 0; j < n; ++j) {
+        if (lengths[j] < 1 || lengths[j] > kMaxCodedS) return false;
+        kraft += 1u << (kMaxCodedS - lengths[j]);
+    }
+    if (kraft > (1u << kMaxCodedS)) return false;           // no prefix code has these lengths
+    uint32_t word = 0, have = 0;
+    for (uint32_t len = 1; len <= kMaxCodedS; ++len) {
+        word <<= 1;
+        for (uint32_t j = 0; j < n; ++j)
+            if (lengths[j] == len) { code[j] = word | (len << 16); ++word; ++have; }
+    }
+    return have == n;
+}
+
+nuq_status nuq_set_level_code(const uint8_t* lengths, uint32_t s) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    if (!lengths || s < 1 || s > kMaxCodedS) return NUQ_ERR_INVALID_ARG;
+    uint32_t code[kMaxCodedS + 1] = {0};
+    if (!canonical_code(lengths, s + 1, code)) return NUQ_ERR_INVALID_ARG;
+    for (uint32_t j = 0; j <= kMaxCodedS; ++j) g_level_code[j] = j <= s ? code[j] : 0u;
+    g_level_code_n = s + 1;
+    return NUQ_OK;
+}
+
+nuq_status nuq_fit_level_code(const uint64_t* hist, uint32_t s, uint8_t* lengths) {
+    if (!hist || !lengths || s < 1 || s > kMaxCodedS) return NUQ_ERR_INVALID_ARG;
+    // Huffman's construction with two queues: the leaves sorted by (count, index) and the joined nodes in
+    // the order they were made (their weights never decrease).  The lighter front is taken, a leaf
+    // before a joined node of the same weight.
+    const uint32_t n = s + 1;
+    uint32_t order[kMaxCodedS + 1];
+    for (uint32_t i = 0; i < n; ++i) order[i] = i;
+    for (uint32_t i = 1; i < n; ++i)                        // insertion sort, stable: equal counts stay in index order
+        for (uint32_t k = i; k > 0 && hist[1 + order[k]] < hist[1 + order[k - 1]]; --k) {
+            const uint32_t t = order[k]; order[k] = order[k - 1]; order[k - 1] = t;
+        }
+    uint64_t weight[2 * (kMaxCodedS + 1)];
+    int parent[2 * (kMaxCodedS + 1)];
+    for (uint32_t i = 0; i < n; ++i) { weight[i] = hist[1 + i]; parent[i] = -1; }
+    uint32_t leaf = 0, joined = n, made = n;                // fronts of the two queues, next node to make
+    for (uint32_t step = 0; step + 1 < n; ++step) {
+        int pick[2];
+        for (int k = 0; k < 2; ++k) {
+            const bool leaf_left = leaf < n, joined_left = joined < made;
+            if (leaf_left && (!joined_left || weight[order[leaf]] <= weight[joined])) pick[k] = (int)order[leaf++];
+            else pick[k] = (int)joined++;
+        }
+        weight[made] = weight[pick[0]] + weight[pick[1]];
+        parent[made] = -1;
+        parent[pick[0]] = parent[pick[1]] = (int)made;
+        ++made;
+    }
+    for (uint32_t i = 0; i < n; ++i) {
+        uint32_t depth = 0;
+        for (int at = (int)i; parent[at] >= 0; at = parent[at]) ++depth;
+        lengths[i] = (uint8_t)depth;
+    }
+    return NUQ_OK;
+}
+
+nuq_status nuq_level_histogram(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
+                               uint64_t offset, uint64_t* hist, void* stream_) {
+    std::lock_guard<std::mutex> lock(g_mu);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    EncodeParams P;
+    Geometry& G = P.geo;
+    if (!g || !hist || (reinterpret_cast<uintptr_t>(hist) & 7u) || (reinterpret_cast<uintptr_t>(g) & 15u)) return NUQ_ERR_INVALID_ARG;
+    if ((norm_kind >> 16) & 0xffu) return NUQ_ERR_INVALID_ARG;                      // no mode: nothing is coded here
+    if (!make_geometry(d, bucket, s, norm_kind, &G) || G.levelset == kLevelsUniform) return NUQ_ERR_INVALID_ARG;
+    if (G.levelset == kLevelsTable && g_levels_s != s) return NUQ_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    P.g = g;
+    P.norms_in = nullptr;
+    if (norm_kind & NUQ_TEST_NORMS) {
+        if (!g_test_norms.count(dev) || !g_test_norms[dev]) return NUQ_ERR_INVALID_ARG;
+        P.norms_in = g_test_norms[dev];
+    } else {
+        Workspace* ws = nullptr;
+        nuq_status st = get_workspace(stream, sizeof(Workspace) + 4 * G.nb, &ws, &dev);
+        if (st != NUQ_OK) return st;
+        WsEntry& e = g_ws[std::make_pair(dev, stream)];     // the norms lie where an encode call keeps its scan state
+        if (e.dirty_to < sizeof(Workspace) + 4 * G.nb) e.dirty_to = sizeof(Workspace) + 4 * G.nb;
+        float* norms = reinterpret_cast<float*>(reinterpret_cast<char*>(ws) + sizeof(Workspace));
+        if (launch_bucket_norms(g, G.d, G.bucket, G.norm_kind, norms, G.nb, stream) != cudaSuccess) return NUQ_ERR_CUDA;
+        P.norms_in = norms;
+    }
+    P.out = nullptr; P.out_bits = nullptr; P.ws = nullptr;
+    P.seed = seed;
+    P.offset = offset;
+    for (uint32_t j = 0; j < kMaxTableS + 2u; ++j) {
+        P.levels[j] = G.levelset == kLevelsTable ? g_levels[j] : 0.0f;
+        P.inv_width[j] = G.levelset == kLevelsTable ? g_inv_width[j] : 0.0f;
+    }
+    for (uint32_t j = 0; j <= kMaxCodedS; ++j) P.level_code[j] = 0;
+    for (uint32_t r = 0; r < 10; ++r) {
+        P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
+        P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
+    }
+    P.stage_words = P.window_words = P.patience = P.grid = 0;
+    if (cudaMemsetAsync(hist, 0, 8 * (s + 2), stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    if (launch_level_histogram(P, hist, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
+    return NUQ_OK;
+}
+
 nuq_status nuq_set_test_norms(const float* norms) {
     std::lock_guard<std::mutex> lock(g_mu);
     int dev = 0;
@@ -328,7 +465,7 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     Workspace* ws = nullptr;
     nuq_status st = get_workspace(stream, pl.state_bytes + pl.norms_bytes, &ws, &dev);
     if (st != NUQ_OK) return st;
-    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, &g_ws[std::make_pair(dev, stream)].clean,
+    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, &g_ws[std::make_pair(dev, stream)],
                           dev, stream);
 }
 

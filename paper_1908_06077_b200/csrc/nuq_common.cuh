@@ -21,7 +21,8 @@ constexpr int kEncMaxBlocks = 4;          // ... and the most it is launched wit
 enum : uint32_t { kNormL2 = 0, kNormLinf = 1 };
 enum : uint32_t { kLevelsExp = 0, kLevelsUniform = 1, kLevelsTable = 2 };
 constexpr uint32_t kMaxTableS = 14;       // interior levels of a level table
-enum : uint32_t { kModeErc = 0, kModeFixed = 1 };
+enum : uint32_t { kModeErc = 0, kModeFixed = 1, kModeCoded = 2 };   // coded: as ERC, the level index written with a fitted prefix code
+constexpr uint32_t kMaxCodedS = 7;        // coded level indices: at most 8 of them, code words of at most 7 bits
 
 // status latched by kernels (most negative wins; the warning only when nothing else is latched)
 enum : int { kOk = 0, kWarnNonfinite = 1, kErrBadStream = -3, kErrTimeout = -5, kErrInternal = -6 };
@@ -63,7 +64,8 @@ struct Geometry {
     uint32_t nlev;           // number of levels including zero
     uint32_t width;          // fixed-mode bits per element
     uint32_t rec_words;      // fixed mode: words per full bucket record
-    uint32_t header_words;   // 16, plus the level table (padded to an even count) of a level-table stream
+    uint32_t header_words;   // 16, plus the level table (padded to an even count) of a level-table stream,
+                             // plus two words of code lengths in the coded mode (the last two)
     uint32_t pad;
 };
 
@@ -78,6 +80,7 @@ struct EncodeParams {
     uint32_t round_keys[20]; // Philox4x32-10 key schedule of `seed`: (k0, k1) of round 0, 1, ..., 9
     float levels[kMaxTableS + 2];    // level table: l_0 = 0, l_1 .. l_s, l_{s+1} = 1 ...
     float inv_width[kMaxTableS + 2]; // ... and 1 / (l_{j+1} - l_j), 0 for the last
+    uint32_t level_code[kMaxCodedS + 1];   // coded mode: word | length << 16 of level index j at [j - 1]
     uint32_t stage_words;    // ERC: shared-memory image of a tile's records (multiple of 4); a CTA holds two
     uint32_t window_words;   // ERC: shared-memory token string of one warp and tile; a warp holds two
     uint32_t patience;       // polls a look-back wait may take before it gives up

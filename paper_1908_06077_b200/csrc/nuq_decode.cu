@@ -154,7 +154,7 @@ __device__ bool describe_chain(const Geometry& G, const TileGeo& T, const Stream
     const uint32_t bi = sb / T.spb, sb0 = bi * T.spb, sbi = sb - sb0;
     const uint32_t blk_len = min(T.blk_elems, T.tile_len - min(T.tile_len, bi * T.blk_elems));
     const uint32_t nsb_blk = (blk_len + kSB - 1) / kSB;
-    if (hd.mode == kModeErc) {
+    if (hd.mode != kModeFixed) {
         const uint64_t head = hd.hwords + 2 * (G.nblk + 1);
         const uint64_t* table = reinterpret_cast<const uint64_t*>(hd.hdr + hd.hwords);
         const uint32_t* payload = hd.hdr + head;
@@ -203,10 +203,20 @@ __device__ StreamHead read_head(const Geometry& G, const uint32_t* hdr) {
     const uint64_t hnblk = (uint64_t)__ldg(hdr + 8) | ((uint64_t)__ldg(hdr + 9) << 32);
     const uint64_t cbits = (uint64_t)__ldg(hdr + 10) | ((uint64_t)__ldg(hdr + 11) << 32);
     bool ok = __ldg(hdr) == kMagic && __ldg(hdr + 1) == kVersion && hd == G.d && __ldg(hdr + 4) == G.bucket &&
-              __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 2u && mode <= 1u &&
+              __ldg(hdr + 5) == G.s && __ldg(hdr + 7) == kSB && levelset <= 2u && mode <= 2u &&
               (flags & 0xffu) <= 1u && !(levelset == kLevelsUniform && G.s > 8u) && (cbits & 31u) == 0;
     const uint32_t nlev = levelset == kLevelsUniform ? (1u << G.s) + 1u : G.s + 2u;
-    const uint32_t hwords = kHeaderWords + (levelset == kLevelsTable ? ((G.s + 1u) & ~1u) : 0u);
+    const uint32_t hwords = kHeaderWords + (levelset == kLevelsTable ? ((G.s + 1u) & ~1u) : 0u) + (mode == kModeCoded ? 2u : 0u);
+    if (ok && mode == kModeCoded) {                         // the lengths must be those of a prefix code of at most 7 bits
+        ok = levelset != kLevelsUniform && G.s <= kMaxCodedS;
+        uint32_t kraft = 0;
+        for (uint32_t j = 0; ok && j <= G.s; ++j) {
+            const uint32_t len = (__ldg(hdr + hwords - 2u + (j >> 2)) >> (8u * (j & 3u))) & 0xffu;
+            ok = len >= 1u && len <= kMaxCodedS;
+            kraft += ok ? 1u << (kMaxCodedS - len) : 0u;
+        }
+        ok = ok && kraft <= (1u << kMaxCodedS);
+    }
     if (ok && levelset == kLevelsTable) {                   // the levels must increase strictly inside (0, 1)
         float below = 0.0f;
         for (uint32_t j = 0; j < G.s; ++j) {
@@ -218,7 +228,7 @@ __device__ StreamHead read_head(const Geometry& G, const uint32_t* hdr) {
     }
     const uint32_t width = 1u + (32u - __clz(nlev - 1u));                   // fixed mode: sign bit + ceil(log2(levels))
     const uint64_t cwords = cbits >> 5;
-    if (ok && mode == kModeErc) {
+    if (ok && mode != kModeFixed) {
         ok = hnblk == G.nblk && cwords > hwords + 2 * (G.nblk + 1);
     } else if (ok) {
         const uint32_t rec_words = 1u + (G.bucket * width + 31u) / 32u;
@@ -433,10 +443,33 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
     }
 }
 
-// shared memory: the two ERC^-1 tables, the stream heads, then per warp the running sums of its S sub-blocks
+// A stream with coded level indices brings its own code: per stream a table over the next 7 bits,
+// (index - 1) | length << 3, or 0 where no code word starts (possible only with an incomplete code).
+constexpr uint32_t kCodedEntries = 1u << kMaxCodedS;
+__device__ __forceinline__ void build_coded_table(const StreamHead& hd, uint8_t* tab, uint32_t s, uint32_t tid, uint32_t nthreads) {
+    const uint32_t w0 = __ldg(hd.hdr + hd.hwords - 2u), w1 = __ldg(hd.hdr + hd.hwords - 1u);   // the lengths, one byte each
+    auto len_of = [&](uint32_t j) { return ((j < 4u ? w0 : w1) >> (8u * (j & 3u))) & 0xffu; };
+    for (uint32_t i = tid; i < kCodedEntries; i += nthreads) {
+        uint32_t e = 0;
+        for (uint32_t j = 0; j <= s; ++j) {
+            // canonical words: level indices by (length, index), the first word all zeros, each next one the
+            // previous plus one; so the word of j counts, in units of its own length, the words before it
+            const uint32_t lj = len_of(j);
+            uint32_t word = 0;
+            for (uint32_t k = 0; k <= s; ++k) {
+                const uint32_t lk = len_of(k);
+                if (lk < lj || (lk == lj && k < j)) word += 1u << (lj - lk);
+            }
+            if ((i >> (kMaxCodedS - lj)) == word) e = j | (lj << 3);
+        }
+        tab[i] = (uint8_t)e;
+    }
+}
+
+// shared memory: the two ERC^-1 tables, the stream heads, the streams' own code tables, then per warp the running sums of its S sub-blocks
 // and kWarpWords for lists and staged tokens
 __host__ __device__ inline size_t decode_warp_offset(uint32_t K) {
-    return (2u * ((1u << kLutBits) + (1u << kSignedBits)) + (size_t)K * sizeof(StreamHead) + 15u) & ~(size_t)15u;
+    return (2u * ((1u << kLutBits) + (1u << kSignedBits)) + (size_t)K * (sizeof(StreamHead) + kCodedEntries) + 15u) & ~(size_t)15u;
 }
 // `sums_in_l2`: the running sums of a unit live in the output vector itself (see decode_kernel)
 __host__ __device__ inline size_t decode_warp_bytes(uint32_t group, bool sums_in_l2) {
@@ -460,6 +493,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     uint16_t* lut = reinterpret_cast<uint16_t*>(dsm);                             // ERC^-1 of 12-bit prefixes
     uint16_t* lut2 = lut + (1u << kLutBits);                                      // sign + ERC^-1 of 7-bit prefixes
     StreamHead* heads = reinterpret_cast<StreamHead*>(lut2 + (1u << kSignedBits));   // [K]
+    uint8_t* coded_tabs = reinterpret_cast<uint8_t*>(heads + P.K);                   // [K][128], filled for streams with coded level indices
     float* accw = reinterpret_cast<float*>(dsm + decode_warp_offset(P.K) + warp * decode_warp_bytes(NG, SUMS_IN_L2));   // S * 256 running sums
     uint32_t* list = reinterpret_cast<uint32_t*>(accw + (SUMS_IN_L2 ? 0u : S * kSB));
 
@@ -474,7 +508,17 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
         for (uint32_t i = lane * 4u; i < S * kSB; i += 128u)
             *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
 
-    __syncthreads();                                        // table and headers are ready; from here on warps run alone
+    __syncthreads();                                        // tables and headers are ready
+    {
+        bool any = false;
+        for (uint32_t k = 0; k < P.K; ++k) {
+            if (!(heads[k].ok && heads[k].mode == kModeCoded)) continue;
+            build_coded_table(heads[k], coded_tabs + k * kCodedEntries, G.s, threadIdx.x, blockDim.x);
+            any = true;
+        }
+        if (any) __syncthreads();                           // (the same streams in every thread)
+    }
+    // from here on warps run alone
 
     // Work is handed out one warp-sized unit at a time (S sub-blocks of one tile, all streams).  The
     // ticket of the next unit is asked for while the current one is decoded, except near the end: a
@@ -557,7 +601,11 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             Chain ch;                                       // each lane describes the chain it walks
             const bool chain_ok = describe_chain(G, T, si, mine && si.ok ? my_sb : 32u, &ch);
             if (__any_sync(0xffffffffu, !chain_ok) && lane == 0) latch_status(P.ws, kErrBadStream);
-            const bool has_chain = mine && si.ok && chain_ok && si.mode == kModeErc && my_sn > 0 && ch.cur < ch.end;
+            const bool has_chain = mine && si.ok && chain_ok && si.mode != kModeFixed && my_sn > 0 && ch.cur < ch.end;
+            // level indices written with the stream's own code (Sec. 5, "efficient encoding")
+            constexpr uint32_t kNoTab = 0xFFFFFFFFu;          // my_tab: where my stream's table starts in coded_tabs
+            const uint32_t my_tab = mine && si.ok && si.mode == kModeCoded ? (g0 + lj) * kCodedEntries : kNoTab;
+            const bool any_coded = __any_sync(0xffffffffu, my_tab != kNoTab);
 
             // A round decodes, for all 32 chains at once, the tokens whose position lies below a limit,
             // and then adds them stream after stream; every element still receives its terms in ascending
@@ -612,6 +660,14 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                         hi = ((t >> 31) << 8) | (((e2 & 0xffu) - 1u) << 9);
                         good = e1 != 0 && e2 != 0;
                     }
+                    if (any_coded) {                        // warp uniform
+                        if (my_tab != kNoTab) {             // sign bit, then a word of the stream's own code
+                            const uint32_t c = coded_tabs[my_tab + ((t << 1) >> (32u - kMaxCodedS))];
+                            used = (e1 >> 8) + 1u + (c >> 3);
+                            hi = ((t >> 31) << 8) | ((c & 7u) << 9);
+                            good = e1 != 0 && c != 0;
+                        }
+                    }
                     if (__any_sync(0xffffffffu, running && !good)) {
                         if (running && !good) {             // a code longer than the table's prefix: Algorithm 2 as a loop
                             uint64_t win64 = window64(word, rcur, rlast);
@@ -621,7 +677,14 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                             const uint32_t negative = (uint32_t)(win64 >> 63);
                             win64 <<= 1;
                             used += 1;
-                            good = good && erc_read(win64, used, sym);
+                            if (my_tab != kNoTab) {
+                                const uint32_t c = coded_tabs[my_tab + (uint32_t)(win64 >> (64u - kMaxCodedS))];
+                                good = good && c != 0;
+                                used += c >> 3;
+                                sym = (c & 7u) + 1u;
+                            } else {
+                                good = good && erc_read(win64, used, sym);
+                            }
                             hi = (negative << 8) | ((min(sym, 0x10000u) - 1u) << 9);
                             if (!good) {                    // not a code at all: the chain is malformed
                                 bad = true;
@@ -712,7 +775,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                     const uint32_t n_c = __shfl_sync(0xffffffffu, n, owner);
                     const float norm_c = __shfl_sync(0xffffffffu, ch.norm, owner);
                     if (!sj.ok) continue;
-                    if (sj.mode == kModeErc) {
+                    if (sj.mode != kModeFixed) {
                         const uint32_t part0 = c * kSB;      // first element of chain c's sub-block within the unit
                         if (!wide && sj.levelset == kLevelsExp) {
                             // value = +-norm * 2^(index - 1 - s): the exponent field is built from the entry

@@ -435,7 +435,16 @@ __device__ bool finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, 
     h[12] = (uint32_t)code_total; h[13] = (uint32_t)(code_total >> 32);
     h[14] = (uint32_t)nnz_total; h[15] = (uint32_t)(nnz_total >> 32);
     if (G.levelset == kLevelsTable)                         // the interior levels, then zero padding
-        for (uint32_t j = 0; j < G.header_words - kHeaderWords; ++j) h[kHeaderWords + j] = j < G.s ? __float_as_uint(P.levels[j + 1]) : 0u;
+        for (uint32_t j = 0; j < ((G.s + 1u) & ~1u); ++j) h[kHeaderWords + j] = j < G.s ? __float_as_uint(P.levels[j + 1]) : 0u;
+    if (G.mode == kModeCoded) {                             // the code lengths, one byte per level index
+        uint32_t w0 = 0, w1 = 0;
+        for (uint32_t j = 0; j <= G.s; ++j) {
+            const uint32_t len = P.level_code[j] >> 16;
+            if (j < 4u) w0 |= len << (8u * j); else w1 |= len << (8u * (j - 4u));
+        }
+        h[G.header_words - 2u] = w0;
+        h[G.header_words - 1u] = w1;
+    }
     if (P.out_bits) *P.out_bits = container_bits;
     return true;
 }
@@ -600,7 +609,9 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         const uint32_t idx = tid & 0x7Fu;                   // field = sign << 7 | index: sign bit, then ERC(index)
         uint32_t v = 0;
         if (idx >= 1) {
-            const uint32_t l = c_erc_lut[idx - 1u], len = l >> 16;
+            // the index's code word: ERC(index), or in the coded mode the word of the fitted code
+            const bool coded = G.mode == kModeCoded;
+            const uint32_t l = coded ? (idx <= kMaxCodedS + 1u ? P.level_code[idx - 1u] : 0u) : c_erc_lut[idx - 1u], len = l >> 16;
             v = ((((tid >> 7) << len) | (l & 0xffffu)) << (31u - len)) | (len + 1u);
         }
         s_lut_signed[tid] = v;
@@ -1134,10 +1145,71 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// Level histogram: how often each level index 0..s+1 comes out of the quantizer (Definition 1) for the
+// given vector, seed and offset: the sample on which a code for the level indices is fitted (Sec. 5,
+// "efficient encoding").  The quantizer and the draws are the encoder's; the bucket norms are given.
+// Not part of the per-step path: a plain grid-stride loop, four elements (one Philox block) per thread.
+// ---------------------------------------------------------------------------
+template <uint32_t LEVELSET>
+__global__ void __launch_bounds__(256) level_histogram_kernel(const __grid_constant__ EncodeParams P,
+                                                              unsigned long long* __restrict__ hist) {
+    __shared__ unsigned int s_hist[kMaxTableS + 2];
+    __shared__ float s_levels[kMaxTableS + 2], s_invw[kMaxTableS + 2];
+    const Geometry& G = P.geo;
+    const uint32_t tid = threadIdx.x;
+    if (tid < kMaxTableS + 2u) {
+        s_hist[tid] = 0;
+        s_levels[tid] = P.levels[tid];
+        s_invw[tid] = P.inv_width[tid];
+    }
+    __syncthreads();
+    const float top = LEVELSET == kLevelsTable ? 1.0f : __uint_as_float((127u + G.s) << 23);
+    const float inf = __uint_as_float(0x7f800000u);
+    const uint64_t nquads = (G.d + 3) / 4;
+    uint32_t zeros = 0;
+    for (uint64_t q = blockIdx.x * 256ull + tid; q < nquads; q += gridDim.x * 256ull) {
+        const uint64_t i0 = 4 * q;                          // a bucket is a multiple of 4 elements: one norm
+        const float norm = __ldg(P.norms_in + i0 / G.bucket);
+        float inv = 0.0f;                                   // 0: the bucket is not quantized
+        if (norm > 0.0f && norm < inf) {
+            inv = __fdiv_rn(top, norm);
+            if (!(inv < inf)) inv = 0.0f;
+        }
+        const uint4 r = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), (uint32_t)P.offset, (uint32_t)(P.offset >> 32),
+                                      P.round_keys);
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (i0 + c >= G.d) break;
+            const float v = __ldg(P.g + i0 + c);
+            const uint32_t sym = LEVELSET == kLevelsTable ? quantize_table(v, inv, G.s, w[c], s_levels, s_invw)
+                                                          : quantize_exp(v, inv, top, w[c]);
+            if (sym) atomicAdd(&s_hist[sym], 1u);
+            else ++zeros;
+        }
+    }
+    zeros = __reduce_add_sync(0xffffffffu, zeros);
+    if ((tid & 31u) == 0 && zeros) atomicAdd(&s_hist[0], zeros);
+    __syncthreads();
+    if (tid < G.s + 2u && s_hist[tid]) atomicAdd(hist + tid, (unsigned long long)s_hist[tid]);
+}
+
+cudaError_t launch_level_histogram(const EncodeParams& P, uint64_t* hist, int sms, cudaStream_t stream) {
+    const uint64_t nquads = (P.geo.d + 3) / 4;
+    const uint64_t want = (nquads + 255) / 256, cap = (uint64_t)sms * 8u;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    if (P.geo.levelset == kLevelsTable)
+        level_histogram_kernel<kLevelsTable><<<grid, 256, 0, stream>>>(P, reinterpret_cast<unsigned long long*>(hist));
+    else
+        level_histogram_kernel<kLevelsExp><<<grid, 256, 0, stream>>>(P, reinterpret_cast<unsigned long long*>(hist));
+    return cudaGetLastError();
+}
+
 // shared memory of one CTA: the tile buffers and, in the ERC mode, two staged tile images and two sets of per-warp token windows
 size_t encode_smem_bytes(const EncodeParams& P) {
     size_t words = kBLK;
-    if (P.geo.mode == kModeErc) words += 2u * (size_t)P.stage_words + 2u * (size_t)kEncWarps * P.window_words;
+    if (P.geo.mode != kModeFixed) words += 2u * (size_t)P.stage_words + 2u * (size_t)kEncWarps * P.window_words;
     return 4u * words;
 }
 

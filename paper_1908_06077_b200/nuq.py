@@ -18,7 +18,7 @@ NUQ_OK, ERR_INVALID_ARG, ERR_CAPACITY, ERR_BAD_STREAM, ERR_CUDA, ERR_TIMEOUT, ER
 WARN_NONFINITE = 1
 NORM_L2, NORM_LINF = 0, 1
 LEVELS_EXP, LEVELS_UNIFORM, LEVELS_TABLE = 0 << 8, 1 << 8, 2 << 8
-MODE_ERC, MODE_FIXED = 0 << 16, 1 << 16
+MODE_ERC, MODE_FIXED, MODE_CODED = 0 << 16, 1 << 16, 2 << 16
 TEST_NORMS = 1 << 24
 TEST_SHORT_PATIENCE = 1 << 25
 HEADER_WORDS = 16
@@ -54,6 +54,13 @@ def _load():
     lib.nuq_encode_bound.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
     lib.nuq_set_level_table.restype = C.c_int
     lib.nuq_set_level_table.argtypes = [C.POINTER(C.c_float), C.c_uint32]
+    lib.nuq_level_histogram.restype = C.c_int
+    lib.nuq_level_histogram.argtypes = [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64,
+                                        C.c_uint64, C.c_void_p, C.c_void_p]
+    lib.nuq_fit_level_code.restype = C.c_int
+    lib.nuq_fit_level_code.argtypes = [C.POINTER(C.c_uint64), C.c_uint32, C.POINTER(C.c_uint8)]
+    lib.nuq_set_level_code.restype = C.c_int
+    lib.nuq_set_level_code.argtypes = [C.POINTER(C.c_uint8), C.c_uint32]
     lib.nuq_set_test_norms.restype = C.c_int
     lib.nuq_set_test_norms.argtypes = [C.c_void_p]
     lib.nuq_last_status.restype = C.c_int
@@ -94,6 +101,39 @@ def set_level_table(interior_levels):
     rc = _lib.nuq_set_level_table(arr, len(vals))
     if rc != NUQ_OK:
         raise NuqError("nuq_set_level_table", rc)
+
+
+def level_histogram(g: torch.Tensor, bucket, s, norm_kind=0, seed=0, offset=0, hist=None, stream=None):
+    """how often each level index 0..s+1 comes out of the quantizer for g: int64 CUDA tensor of s + 2 counters"""
+    assert g.is_cuda and g.dtype == torch.float32 and g.is_contiguous()
+    if hist is None:
+        hist = torch.empty(s + 2, dtype=torch.int64, device=g.device)
+    rc = _lib.nuq_level_histogram(C.c_void_p(g.data_ptr()), g.numel(), bucket, s, norm_kind, seed, offset,
+                                  C.c_void_p(hist.data_ptr()), _stream(stream))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_level_histogram", rc)
+    return hist
+
+
+def fit_level_code(hist, s):
+    """code lengths of the level indices 1..s+1 (Huffman) from the s + 2 counts of level_histogram (host values)"""
+    vals = [int(x) for x in hist]
+    assert len(vals) == s + 2
+    arr = (C.c_uint64 * len(vals))(*vals)
+    out = (C.c_uint8 * (s + 1))()
+    rc = _lib.nuq_fit_level_code(arr, s, out)
+    if rc != NUQ_OK:
+        raise NuqError("nuq_fit_level_code", rc)
+    return list(out)
+
+
+def set_level_code(lengths):
+    """code lengths of the level indices 1..s+1 that MODE_CODED calls use from now on"""
+    vals = [int(x) for x in lengths]
+    arr = (C.c_uint8 * len(vals))(*vals)
+    rc = _lib.nuq_set_level_code(arr, len(vals) - 1)
+    if rc != NUQ_OK:
+        raise NuqError("nuq_set_level_code", rc)
 
 
 def set_test_norms(norms: torch.Tensor | None):

@@ -95,3 +95,22 @@ def compare_symbols(g, bucket, s, flags, seed, offset, gpu_stream):
     print(f"symbol mismatches={int(bad.size)} of d={d} (all within 1e-6 of the rounding threshold), "
           f"largest relative norm difference {worst:.3g}")
     return int(bad.size), worst
+
+
+def gpu_level_histogram(g, bucket, s, flags, seed, offset, norms=None):
+    """counts of the level indices 0..s+1 from nuq_level_histogram (uint64 numpy)"""
+    torch, nuq = require_cuda()
+    gd = torch.from_numpy(np.ascontiguousarray(g, np.float32)).cuda()
+    buf = torch.full((s + 2 + 2,), -1, dtype=torch.int64, device="cuda")     # a guard word on either side
+    if norms is not None:
+        nd = torch.from_numpy(np.ascontiguousarray(norms, np.float32)).cuda()
+        nuq.set_test_norms(nd)
+        flags |= nuq.TEST_NORMS
+    nuq.level_histogram(gd, bucket, s, flags, seed, offset, hist=buf[1:s + 3])
+    status = nuq.last_status()
+    if norms is not None:
+        nuq.set_test_norms(None)
+    assert status == 0, status
+    host = buf.cpu().numpy()
+    assert host[0] == -1 and host[-1] == -1, "histogram wrote outside its counters"
+    return host[1:-1].astype(np.uint64)

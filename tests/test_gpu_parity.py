@@ -105,6 +105,28 @@ def test_encode_is_deterministic_and_ignores_stale_output():
     assert not np.array_equal(a, c)
 
 
+def test_scan_state_is_clean_after_a_call_with_wide_buckets():
+    """A call with buckets wider than a tile keeps its bucket norms behind its scan state in the stream's
+    workspace.  A later call with more tiles keeps scan state at that place and must find it cleared."""
+    gpu_encode(_input(2_000_000, 5), 8192, 4, 0, 1, 0)       # the workspace grows once, here
+    for (d_wide, b_wide, d_next) in ((100_000, 16384, 300_001), (40_000, 32768, 8192 * 12 + 7), (200_000, 65536, 8192 * 40),
+                                     # the next call's group word (a sum that is added to) lies where the norms were
+                                     (200_000, 65536, 8192 * 25 + 100), (100_000, 16384, 8192 * 13 + 50), (40_000, 32768, 8192 * 5 + 9)):
+        for rep in range(3):
+            gpu_encode(_input(d_wide, d_wide + rep), b_wide, 4, 0, 3, rep)
+            if rep == 1:                                      # a short call in between clears only what it uses itself
+                gpu_encode(_input(1000, 1), 256, 3, 0, 1, 0)
+            if rep == 2:                                      # the histogram's norms lie at the front of the workspace
+                from gpu_util import gpu_level_histogram
+                gpu_level_histogram(_input(d_wide, 9), 512, 4, 0, 1, 0)
+                gpu_encode(_input(1000, 1), 256, 3, 0, 1, 0)
+            g = _input(d_next, d_next + rep)
+            norms = O.bucket_norms(g, 8192, L2)
+            want, want_bits = O.encode(g, 8192, 4, 0, seed=5, offset=rep, norms=norms)
+            got, got_bits = gpu_encode(g, 8192, 4, 0, seed=5, offset=rep, norms=norms)
+            assert got_bits == want_bits and np.array_equal(got, want)
+
+
 def test_stream_info_and_status():
     torch, nuq = require_cuda()
     g = torch.from_numpy(_input(50000, 2)).cuda()
@@ -428,3 +450,123 @@ def test_level_table_streams_sum_with_others_and_bad_tables_are_refused():
     g = torch.zeros(4096, device="cuda")
     with pytest.raises(nuq.NuqError):                        # the table has two levels, the call asks for three
         nuq.encode(g, 1024, 3, nuq.LEVELS_TABLE)
+
+
+# ---- coded level indices (Sec. 5, "efficient encoding") -------------------------------------------
+
+CODED_CASES = [
+    (100037, 8192, 4, O.LEVELS_EXP),
+    (70000, 768, 3, O.LEVELS_EXP),
+    (3 * 8192 + 5, 256, 2, O.LEVELS_EXP),
+    (200000, 65536, 7, O.LEVELS_EXP),
+    (40000, 2048, 1, O.LEVELS_EXP),
+    (60000, 4096, 5, O.LEVELS_TABLE),
+    (257, 256, 3, O.LEVELS_EXP),
+]
+
+
+@pytest.mark.parametrize("d,bucket,s,ls", CODED_CASES)
+def test_coded_streams_match_the_oracle(d, bucket, s, ls):
+    """The whole of the coded variant: the level histogram equals the oracle's (given its norms; free running
+    it moves by a few counts), the lengths fitted on it are the oracle's, the container written with that
+    code is the oracle's bit for bit, and the decoded vector is the oracle's."""
+    from gpu_util import gpu_level_histogram
+    torch, nuq = require_cuda()
+    if ls == O.LEVELS_TABLE:
+        levels = _lp(0.4, s)
+        O.set_levels(levels)
+        nuq.set_level_table(levels)
+    g = _input(d, 17 * d + s)
+    norms = O.bucket_norms(g, bucket, O.NORM_L2)
+    sign, sym, _ = O.quantize(g, bucket, s, O.NORM_L2, ls, 11, 3, norms=norms)
+    want_hist = O.level_histogram(sym, s)
+    hist = gpu_level_histogram(g, bucket, s, O.make_flags(O.NORM_L2, ls, 0), 11, 3, norms=norms)
+    assert np.array_equal(hist, want_hist)
+    free_hist = gpu_level_histogram(g, bucket, s, O.make_flags(O.NORM_L2, ls, 0), 11, 3)
+    assert free_hist.sum() == d and np.abs(free_hist.astype(np.int64) - want_hist.astype(np.int64)).sum() <= 2 + 2e-5 * d
+    lengths = nuq.fit_level_code(hist, s)
+    assert lengths == list(O.huffman_lengths(want_hist[1:]))
+    O.set_level_code(lengths)
+    nuq.set_level_code(lengths)
+    flags = O.make_flags(O.NORM_L2, ls, O.MODE_CODED)
+    want, want_bits = O.encode(g, bucket, s, flags, seed=11, offset=3, norms=norms)
+    got, got_bits = gpu_encode(g, bucket, s, flags, seed=11, offset=3, norms=norms)
+    assert got_bits == want_bits and np.array_equal(got, want)
+    free, _ = gpu_encode(g, bucket, s, flags, seed=5, offset=0)
+    compare_symbols(g, bucket, s, flags, 5, 0, free)
+    acc = gpu_decode([free], d, bucket, s)
+    assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([free], d, bucket, s)[1].view(np.uint32))
+    # the code is kept: another vector, the same words
+    g2 = _input(d, 17 * d + s + 1)
+    norms2 = O.bucket_norms(g2, bucket, O.NORM_L2)
+    want2, _ = O.encode(g2, bucket, s, flags, seed=12, offset=4, norms=norms2)
+    got2, _ = gpu_encode(g2, bucket, s, flags, seed=12, offset=4, norms=norms2)
+    assert np.array_equal(got2, want2)
+
+
+@pytest.mark.parametrize("K", [1, 2, 4, 8, 11])
+def test_coded_streams_sum_with_streams_of_the_other_modes(K):
+    """Each stream brings its own code; streams of all three modes are summed in stream order."""
+    torch, nuq = require_cuda()
+    d, bucket, s = 90000, 2048, 4
+    codes = ([1, 2, 3, 4, 4], [3, 3, 2, 2, 2], [2, 2, 2, 3, 3], [4, 4, 3, 2, 1], [3, 3, 3, 3, 3])
+    streams = []
+    for k in range(K):
+        O.set_level_code(codes[k % len(codes)])
+        mode = (O.MODE_CODED, O.MODE_CODED, O.MODE_ERC, O.MODE_CODED, O.MODE_FIXED)[k % 5] if K > 1 else O.MODE_CODED
+        g = _input(d, 5 + k) * (30.0 if k % 3 == 1 else 1.0)
+        streams.append(O.encode(g, bucket, s, O.make_flags(O.NORM_L2, O.LEVELS_EXP, mode), k + 1, k)[0])
+    rc, want = O.decode_accumulate(streams, d, bucket, s)
+    assert rc == 0
+    got = gpu_decode(streams, d, bucket, s)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_coded_streams_with_dense_symbols_and_long_words_stay_inside_the_staging_buffers():
+    """A code that gives the commonest level index the longest word, on inputs where most coordinates are
+    nonzero: the token strings are as long as they can get."""
+    torch, nuq = require_cuda()
+    for (d, bucket, s, lengths, scale) in ((50000, 256, 7, [7, 7, 6, 5, 4, 3, 2, 1], 1.0),
+                                           (50000, 8192, 2, [2, 2, 2], 1.0),
+                                           (30000, 512, 3, [3, 3, 3, 3], 1.0)):
+        rng = np.random.default_rng(d + s)
+        g = (rng.uniform(0.5, 1.0, d) * rng.choice([-1.0, 1.0], d)).astype(np.float32)      # every coordinate large
+        O.set_level_code(lengths)
+        nuq.set_level_code(lengths)
+        flags = O.make_flags(O.NORM_L2, O.LEVELS_EXP, O.MODE_CODED)
+        norms = O.bucket_norms(g, bucket, O.NORM_L2)
+        want, want_bits = O.encode(g, bucket, s, flags, seed=2, offset=1, norms=norms)
+        got, got_bits = gpu_encode(g, bucket, s, flags, seed=2, offset=1, norms=norms)
+        assert got_bits == want_bits and np.array_equal(got, want)
+        free, _ = gpu_encode(g, bucket, s, flags, seed=2, offset=1)
+        compare_symbols(g, bucket, s, flags, 2, 1, free)
+        got_acc = gpu_decode([free, want], d, bucket, s)
+        assert np.array_equal(got_acc.view(np.uint32), O.decode_accumulate([free, want], d, bucket, s)[1].view(np.uint32))
+
+
+def test_malformed_coded_containers_and_bad_codes_are_refused():
+    torch, nuq = require_cuda()
+    d, bucket, s = 30000, 1024, 3
+    O.set_level_code([1, 2, 3, 3])
+    st, _ = O.encode(_input(d, 3), bucket, s, O.make_flags(O.NORM_L2, O.LEVELS_EXP, O.MODE_CODED), 1, 0)
+    gpu_decode([st], d, bucket, s)
+    for word in (0x01010101, 0x03030200, 0x08030201):        # Kraft sum above one, a zero length, a length above 7
+        bad = st.copy()
+        bad[16] = word
+        gpu_decode([bad], d, bucket, s, expect_status=-3)
+    bad = st.copy()
+    bad[16] = 0x04040403                                     # an incomplete code: chains run into bits that spell no word
+    gpu_decode([bad], d, bucket, s, expect_status=-3)
+    other = O.encode(_input(d, 4), bucket, s, 0, 2, 0)[0]
+    gpu_decode([other, bad, other], d, bucket, s, expect_status=-3)
+    for lengths in ([1, 1, 2], [0, 1], [1, 8], [1, 2, 3, 3, 3]):
+        with pytest.raises(nuq.NuqError):
+            nuq.set_level_code(lengths)
+    nuq.set_level_code([1, 2, 2])
+    g = torch.zeros(4096, device="cuda")
+    with pytest.raises(nuq.NuqError):                        # the code has three words, s = 3 needs four
+        nuq.encode(g, 1024, 3, nuq.MODE_CODED)
+    with pytest.raises(nuq.NuqError):                        # no coded level indices with uniform levels
+        nuq.encode(g, 1024, 2, nuq.MODE_CODED | nuq.LEVELS_UNIFORM)
+    with pytest.raises(nuq.NuqError):
+        nuq.level_histogram(g, 1024, 2, nuq.LEVELS_UNIFORM)
