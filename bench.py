@@ -45,6 +45,8 @@ WORKLOADS = {
     "c3-s2": ("C3 ResNet-50-sized, s=2, ERC, K=8", 25_557_032, 8192, 2, 0, 8),
     "c3-s3": ("C3 ResNet-50-sized, s=3, ERC, K=8", 25_557_032, 8192, 3, 0, 8),
     "c3-fixed": ("C3 ResNet-50-sized, s=4, fixed 4-bit, K=8", 25_557_032, 8192, 4, 1 << 16, 8),
+    "c3-coded": ("C3 ResNet-50-sized, s=4, level indices in a Huffman code fitted on worker 1's gradient, K=8",
+                 25_557_032, 8192, 4, 2 << 16, 8),
     "c4-512": ("C4 flat Laplace d=2^30, bucket 512, s=4, ERC, K=2", 1 << 30, 512, 4, 0, 2),
     "c4-8192": ("C4 flat Laplace d=2^30, bucket 8192, s=4, ERC, K=2", 1 << 30, 8192, 4, 0, 2),
     "c4-65536": ("C4 flat Laplace d=2^30, bucket 65536, s=4, ERC, K=2", 1 << 30, 65536, 4, 0, 2),
@@ -52,7 +54,7 @@ WORKLOADS = {
     "c5-qsgdinf": ("C5 ResNet-50-sized, uniform levels k/16, Linf norm, ERC, K=8", 25_557_032, 8192, 4, (1 << 8) | 1, 8),
 }
 # timed briefly behind the headline workload when that is the default one
-SIDE_WORKLOADS = ["c3-fixed", "c3-s2", "c3-s3", "c5-qsgd", "c5-qsgdinf", "c2", "c1"]
+SIDE_WORKLOADS = ["c3-fixed", "c3-coded", "c3-s2", "c3-s3", "c5-qsgd", "c5-qsgdinf", "c2", "c1"]
 
 _input_cache = {}
 
@@ -161,6 +163,18 @@ def _oracle_encode_job(job):
     return O.encode(g, bucket, s, flags, k + 1, 0)[0]
 
 
+def _oracle_fit_code(workload, n, bucket, s, flags):
+    """coded level indices: the oracle fits its own code on worker 1's gradient (as the GPU leg does with its own)"""
+    import oracle as O
+    if (flags >> 16) & 0xff != O.MODE_CODED:
+        return None
+    g = worker_input(workload, 1, n)[:n]
+    _, sym, _ = O.quantize(g, bucket, s, flags & 0xff, (flags >> 8) & 0xff, 1, 0)
+    lengths = O.huffman_lengths(O.level_histogram(sym, s)[1:])
+    O.set_level_code(lengths)
+    return [int(x) for x in lengths]
+
+
 def oracle_step(workload, steps, warmup, all_cores=False):
     """the CPU oracle on the same workload: K encodes + one decode_accumulate per step; on one core, or
     with the K encodes spread over a process pool (the oracle's C code itself is single threaded)"""
@@ -168,6 +182,7 @@ def oracle_step(workload, steps, warmup, all_cores=False):
     desc, d, bucket, s, flags, K = WORKLOADS[workload]
     n = min(d, 1 << 22) if workload.startswith("c4") else d          # bounded sample for the 2^30 case
     gs = [worker_input(workload, k + 1, n)[:n] for k in range(K)]
+    _oracle_fit_code(workload, n, bucket, s, flags)         # before the pool forks: its processes inherit the code
     pool, cores = None, 1
     if all_cores and K > 1:
         import multiprocessing as mp
@@ -267,6 +282,14 @@ class Workload:
         self.outs = [torch.empty(nbytes // 4, dtype=torch.int32, device="cuda") for _ in range(self.K)]
         self.bits = [torch.zeros(1, dtype=torch.int64, device="cuda") for _ in range(self.K)]
         self.acc = torch.empty(self.d, dtype=torch.float32, device="cuda")
+        self.level_code = None
+        if (self.flags >> 16) & 0xff == 2:
+            # coded level indices: the code is fitted once on worker 1's gradient (the paper's "initial
+            # sample"), outside the timed region, and kept for every step and every worker
+            hist = nuq.level_histogram(self.gs[0], self.bucket, self.s, self.flags & 0xffff, seed=1, offset=0)
+            self.level_histogram = [int(x) for x in hist.cpu().tolist()]
+            self.level_code = nuq.fit_level_code(self.level_histogram, self.s)
+            nuq.set_level_code(self.level_code)
 
     def step(self, flush):
         torch, nuq = self.torch, self.nuq
@@ -325,7 +348,7 @@ class Workload:
         # come first), one decode kernel (two when all streams are fixed-width: that path's own kernel,
         # then the general one, which returns at once)
         wide = self.bucket > 8192
-        return self.K * (2 if wide else 1) + (2 if (self.flags >> 16) & 0xff else 1)
+        return self.K * (2 if wide else 1) + (2 if (self.flags >> 16) & 0xff == 1 else 1)
 
 
 def summarize(ms):
@@ -350,6 +373,9 @@ def side_report(w, steps, flush, peak):
            "encode_frac": (4.0 * w.d + sum(cb) / w.K) / (statistics.median(enc_call) / 1e3) / 1e9 / peak,
            "decode_frac": (sum(cb) + 4.0 * w.d) / (statistics.median(dec) / 1e3) / 1e9 / peak}
     rep.update(stats)
+    if w.level_code is not None:
+        rep["level_code_lengths"] = w.level_code
+        rep["level_histogram"] = w.level_histogram
     rep["variance_single_draw"] = w.single_draw_variance()
     rep["variance_bound"] = variance_bounds(w.bucket, w.s, w.flags)
     if w.d <= 30_000_000:                                   # the ResNet-sized and tiny configurations: L2 left warm
@@ -459,6 +485,9 @@ def run_gpu(args):
             "clocks": clocks,
         }
         line.update(stats)
+        if w.level_code is not None:
+            line["level_code_lengths"] = w.level_code
+            line["level_histogram"] = w.level_histogram
         line["variance_single_draw"] = w.single_draw_variance()
         line["variance_bound"] = variance_bounds(bucket, s, flags)
         if e2e is not None:

@@ -35,7 +35,10 @@
 // they share only the tables and the validated stream headers.  Nothing spins.
 //
 // Calls whose streams are all in the fixed-width mode have no chains to walk; they are
-// served by a kernel of their own (decode_fixed_kernel below).
+// served by a kernel of their own (decode_fixed_kernel below).  A stream whose level indices
+// are written in a fitted prefix code (Sec. 5, "efficient encoding") brings the code lengths
+// in its header; the CTA builds a small table from them and the stream's lanes look their
+// level indices up there instead of in the ERC^-1 table, in the same loop.
 #include <type_traits>
 
 #include "nuq_common.cuh"
@@ -443,10 +446,11 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
     }
 }
 
-// A stream with coded level indices brings its own code: per stream a table over the next 7 bits,
-// (index - 1) | length << 3, or 0 where no code word starts (possible only with an incomplete code).
+// A stream with coded level indices brings its own code: per stream a table over the next 7 bits in the
+// format of the ERC^-1 table, index | length << 8, or 0 where no code word starts (possible only with
+// an incomplete code).  A lane of such a stream looks its level index up there instead.
 constexpr uint32_t kCodedEntries = 1u << kMaxCodedS;
-__device__ __forceinline__ void build_coded_table(const StreamHead& hd, uint8_t* tab, uint32_t s, uint32_t tid, uint32_t nthreads) {
+__device__ __forceinline__ void build_coded_table(const StreamHead& hd, uint16_t* tab, uint32_t s, uint32_t tid, uint32_t nthreads) {
     const uint32_t w0 = __ldg(hd.hdr + hd.hwords - 2u), w1 = __ldg(hd.hdr + hd.hwords - 1u);   // the lengths, one byte each
     auto len_of = [&](uint32_t j) { return ((j < 4u ? w0 : w1) >> (8u * (j & 3u))) & 0xffu; };
     for (uint32_t i = tid; i < kCodedEntries; i += nthreads) {
@@ -460,16 +464,16 @@ __device__ __forceinline__ void build_coded_table(const StreamHead& hd, uint8_t*
                 const uint32_t lk = len_of(k);
                 if (lk < lj || (lk == lj && k < j)) word += 1u << (lj - lk);
             }
-            if ((i >> (kMaxCodedS - lj)) == word) e = j | (lj << 3);
+            if ((i >> (kMaxCodedS - lj)) == word) e = (j + 1u) | (lj << 8);
         }
-        tab[i] = (uint8_t)e;
+        tab[i] = (uint16_t)e;
     }
 }
 
 // shared memory: the two ERC^-1 tables, the stream heads, the streams' own code tables, then per warp the running sums of its S sub-blocks
 // and kWarpWords for lists and staged tokens
 __host__ __device__ inline size_t decode_warp_offset(uint32_t K) {
-    return (2u * ((1u << kLutBits) + (1u << kSignedBits)) + (size_t)K * (sizeof(StreamHead) + kCodedEntries) + 15u) & ~(size_t)15u;
+    return (2u * ((1u << kLutBits) + (1u << kSignedBits)) + (size_t)K * (sizeof(StreamHead) + 2u * kCodedEntries) + 15u) & ~(size_t)15u;
 }
 // `sums_in_l2`: the running sums of a unit live in the output vector itself (see decode_kernel)
 __host__ __device__ inline size_t decode_warp_bytes(uint32_t group, bool sums_in_l2) {
@@ -493,7 +497,7 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     uint16_t* lut = reinterpret_cast<uint16_t*>(dsm);                             // ERC^-1 of 12-bit prefixes
     uint16_t* lut2 = lut + (1u << kLutBits);                                      // sign + ERC^-1 of 7-bit prefixes
     StreamHead* heads = reinterpret_cast<StreamHead*>(lut2 + (1u << kSignedBits));   // [K]
-    uint8_t* coded_tabs = reinterpret_cast<uint8_t*>(heads + P.K);                   // [K][128], filled for streams with coded level indices
+    uint16_t* coded_tabs = reinterpret_cast<uint16_t*>(heads + P.K);                 // [K][128], filled for streams with coded level indices
     float* accw = reinterpret_cast<float*>(dsm + decode_warp_offset(P.K) + warp * decode_warp_bytes(NG, SUMS_IN_L2));   // S * 256 running sums
     uint32_t* list = reinterpret_cast<uint32_t*>(accw + (SUMS_IN_L2 ? 0u : S * kSB));
 
@@ -602,10 +606,13 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
             const bool chain_ok = describe_chain(G, T, si, mine && si.ok ? my_sb : 32u, &ch);
             if (__any_sync(0xffffffffu, !chain_ok) && lane == 0) latch_status(P.ws, kErrBadStream);
             const bool has_chain = mine && si.ok && chain_ok && si.mode != kModeFixed && my_sn > 0 && ch.cur < ch.end;
-            // level indices written with the stream's own code (Sec. 5, "efficient encoding")
-            constexpr uint32_t kNoTab = 0xFFFFFFFFu;          // my_tab: where my stream's table starts in coded_tabs
-            const uint32_t my_tab = mine && si.ok && si.mode == kModeCoded ? (g0 + lj) * kCodedEntries : kNoTab;
-            const bool any_coded = __any_sync(0xffffffffu, my_tab != kNoTab);
+            // Level indices written with the stream's own code (Sec. 5, "efficient encoding"): such a lane
+            // looks the index up in its stream's table (7-bit prefixes) instead of the ERC^-1 table (12-bit).
+            // tab2: where the table starts, in entries from `lut`; sh2: 32 - its prefix bits.
+            const bool my_coded = mine && si.ok && si.mode == kModeCoded;
+            const uint32_t tab2 = my_coded ? (uint32_t)(coded_tabs - lut) + (g0 + lj) * kCodedEntries : 0u;
+            const uint32_t sh2 = my_coded ? 32u - kMaxCodedS : 32u - kLutBits;
+            small_index = small_index && !__any_sync(0xffffffffu, my_coded);
 
             // A round decodes, for all 32 chains at once, the tokens whose position lies below a limit,
             // and then adds them stream after stream; every element still receives its terms in ascending
@@ -655,18 +662,10 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                         hi = e2 & 0xff00u;
                         good = e1 != 0 && e2 != 0;
                     } else {
-                        const uint32_t e2 = lut[(t << 1) >> (32u - kLutBits)];
+                        const uint32_t e2 = lut[tab2 + ((t << 1) >> sh2)];   // the ERC^-1 table, or the stream's own
                         used = (e1 >> 8) + 1u + (e2 >> 8);
                         hi = ((t >> 31) << 8) | (((e2 & 0xffu) - 1u) << 9);
                         good = e1 != 0 && e2 != 0;
-                    }
-                    if (any_coded) {                        // warp uniform
-                        if (my_tab != kNoTab) {             // sign bit, then a word of the stream's own code
-                            const uint32_t c = coded_tabs[my_tab + ((t << 1) >> (32u - kMaxCodedS))];
-                            used = (e1 >> 8) + 1u + (c >> 3);
-                            hi = ((t >> 31) << 8) | ((c & 7u) << 9);
-                            good = e1 != 0 && c != 0;
-                        }
                     }
                     if (__any_sync(0xffffffffu, running && !good)) {
                         if (running && !good) {             // a code longer than the table's prefix: Algorithm 2 as a loop
@@ -677,11 +676,11 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
                             const uint32_t negative = (uint32_t)(win64 >> 63);
                             win64 <<= 1;
                             used += 1;
-                            if (my_tab != kNoTab) {
-                                const uint32_t c = coded_tabs[my_tab + (uint32_t)(win64 >> (64u - kMaxCodedS))];
+                            if (sh2 != 32u - kLutBits) {  // a stream with its own code: every word is in its table
+                                const uint32_t c = lut[tab2 + (uint32_t)(win64 >> (64u - kMaxCodedS))];
                                 good = good && c != 0;
-                                used += c >> 3;
-                                sym = (c & 7u) + 1u;
+                                used += c >> 8;
+                                sym = c & 0xffu;
                             } else {
                                 good = good && erc_read(win64, used, sym);
                             }

@@ -4,13 +4,14 @@
 //
 // A persistent CTA takes tiles of up to 8192 consecutive elements (whole buckets, or
 // one 8192-element coding block of a wider bucket) by ticket.  The tile's bytes are
-// brought into one of two shared-memory buffers by a bulk asynchronous copy (TMA,
-// completion on an mbarrier); the copy of the next tile runs while the current one
-// is encoded.  Eight worker warps own 1024 elements (four 256-element coding
-// sub-blocks) of the tile each.  Per tile a worker
-//   1. adds up the squares (fp64) of its elements per sub-block; whichever warp is
-//      done last turns the partial sums into the tile's bucket norms, once for the
-//      whole CTA, before the only CTA barrier of the tile;
+// brought into shared memory by bulk asynchronous copies (TMA, completion on an
+// mbarrier), one per warp: eight worker warps own 1024 elements (four 256-element
+// coding sub-blocks) of the tile each, and a warp starts the copy of its part of the
+// next tile as soon as it is done with its part of this one.  Per tile a worker
+//   1. adds up the squares of its elements per sub-block (eight per lane in fp32,
+//      everything beyond that in fp64); whichever warp is done last turns the partial
+//      sums into the tile's bucket norms, once for the whole CTA, before the only CTA
+//      barrier of the tile;
 //   2. per sub-block: quantizes 8 elements per lane (two Philox blocks), compacts the
 //      nonzero symbols into a dense list (one warp scan of per-lane counts; the list
 //      lies over the sub-block's own, already consumed, input bytes) and turns the list
