@@ -528,9 +528,11 @@ def run_gpu(args):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures
-# summarised under profiles/ (null until the captures of the present kernels are in)
-ENCODE_TRAFFIC_BYTES = {}
-DECODE_TRAFFIC_BYTES = {}
+# summarised under profiles/.  Reads equal the algorithmic reads; the writes counted are those that
+# had left the 126 MB L2 when the kernel ended (a container or the sums of C3 fit in it), so the
+# totals of the decoders and of the fixed-width encoder lie below the algorithmic bytes.
+ENCODE_TRAFFIC_BYTES = {"c3": 102_302_208 + 3_524_608, "c3-fixed": 102_291_968 + 4_743_936}
+DECODE_TRAFFIC_BYTES = {"c3": 24_614_144 + 44_172_800, "c3-fixed": 102_397_952 + 59_644_928}
 
 
 def main():

@@ -914,6 +914,11 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
             warps = w;
         }
     }
+    const uint64_t want = (units + warps - 1) / warps;
+    const uint64_t grid = want < (uint64_t)sms ? want : (uint64_t)sms;
+    // a CTA of a small call still gets 8 warps: they share the work of building the tables (4096 entries),
+    // which one or two warps alone would spend longer on than on decoding; warps without a unit leave at once
+    if (warps < 8u && wmax >= 8u) warps = 8u;
     const size_t smem = decode_smem_bytes(P.group, P.K, warps, sums_in_l2);
     if (smem > kSmemMaxCta) return cudaErrorInvalidValue;
     if (cudaMemsetAsync(&P.ws->dec_ticket, 0, 2 * sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;   // ticket and the flag behind it
@@ -922,8 +927,6 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
         decode_fixed_kernel<<<(unsigned)(want_fixed < cap_fixed ? want_fixed : cap_fixed), 256, 0, stream>>>(P);
         if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
     }
-    const uint64_t want = (units + warps - 1) / warps;
-    const uint64_t grid = want < (uint64_t)sms ? want : (uint64_t)sms;
     if (sums_in_l2) decode_kernel<true><<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
     else decode_kernel<false><<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
     return cudaGetLastError();

@@ -156,3 +156,53 @@ def test_c4_at_its_stated_length(c4_inputs, bucket):
     assert rc == 0
     got = gpu_decode(streams, d, bucket, 4)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_c3_coded_level_indices_as_benchmarked(c3_inputs):
+    """The coded workload of the benchmark: the code is fitted on worker 1's gradient from the GPU's own
+    histogram and kept; the histogram, the lengths, the symbols of two workers and the decoded sum of two
+    coded streams and one ERC stream are the oracle's."""
+    from gpu_util import gpu_level_histogram, require_cuda
+    torch, nuq = require_cuda()
+    d = c3_inputs[0].size
+    hist = gpu_level_histogram(c3_inputs[0], 8192, 4, 0, 1, 0)
+    _, sym, _ = O.quantize(c3_inputs[0], 8192, 4, O.NORM_L2, O.LEVELS_EXP, 1, 0)
+    want_hist = O.level_histogram(sym, 4)
+    assert hist.sum() == d and np.abs(hist.astype(np.int64) - want_hist.astype(np.int64)).sum() <= 2e-5 * d
+    lengths = nuq.fit_level_code(hist, 4)
+    assert lengths == list(O.huffman_lengths(want_hist[1:]))
+    nuq.set_level_code(lengths)
+    O.set_level_code(lengths)
+    coded = O.make_flags(mode=O.MODE_CODED)
+    streams = []
+    for k in (0, 1):
+        got, _ = gpu_encode(c3_inputs[k], 8192, 4, coded, seed=k + 1, offset=0)
+        nbad, rel = compare_symbols(c3_inputs[k], 8192, 4, coded, k + 1, 0, got)
+        assert nbad <= 1e-5 * d and rel <= 1e-6
+        streams.append(got)
+    streams.append(gpu_encode(c3_inputs[2], 8192, 4, 0, seed=3, offset=0)[0])
+    rc, want = O.decode_accumulate(streams, d, 8192, 4)
+    assert rc == 0
+    got = gpu_decode(streams, d, 8192, 4)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_c3_with_a_level_table(c3_inputs):
+    """General level sequences at the benchmark's size: L_p with p = 0.4, s = 4, in both modes."""
+    from gpu_util import require_cuda
+    torch, nuq = require_cuda()
+    levels = np.array([0.4 ** 4, 0.4 ** 3, 0.4 ** 2, 0.4], np.float32)
+    O.set_levels(levels)
+    nuq.set_level_table(levels)
+    g, d = c3_inputs[1], c3_inputs[1].size
+    streams = []
+    for mode in (O.MODE_ERC, O.MODE_FIXED):
+        flags = O.make_flags(O.NORM_L2, O.LEVELS_TABLE, mode)
+        got, _ = gpu_encode(g, 8192, 4, flags, seed=2, offset=0)
+        nbad, rel = compare_symbols(g, 8192, 4, flags, 2, 0, got)
+        assert nbad <= 1e-5 * d and rel <= 1e-6
+        streams.append(got)
+    rc, want = O.decode_accumulate(streams, d, 8192, 4)
+    assert rc == 0
+    got = gpu_decode(streams, d, 8192, 4)
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
