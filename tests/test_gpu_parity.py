@@ -570,3 +570,80 @@ def test_malformed_coded_containers_and_bad_codes_are_refused():
         nuq.encode(g, 1024, 2, nuq.MODE_CODED | nuq.LEVELS_UNIFORM)
     with pytest.raises(nuq.NuqError):
         nuq.level_histogram(g, 1024, 2, nuq.LEVELS_UNIFORM)
+
+
+def test_a_long_sequence_of_calls_of_many_shapes_on_one_stream():
+    """Every call on a stream uses the same workspace (scan state, tickets, bucket norms of wide buckets,
+    histogram norms, the decoder's ticket).  A seeded sequence of encode, histogram and decode calls of
+    unrelated shapes and modes must give, call after call, the container the oracle writes when it is
+    given the norms the GPU took (bit for bit), and the oracle's sums."""
+    from gpu_util import gpu_level_histogram
+    torch, nuq = require_cuda()
+    rng = np.random.default_rng(2024)
+    buckets = [256, 512, 768, 1024, 2048, 4096, 8192, 16384, 32768, 65536]
+    O.set_level_code([1, 2, 3, 4, 4])
+    nuq.set_level_code([1, 2, 3, 4, 4])
+    checked = 0
+    for it in range(160):
+        d = int(rng.choice([rng.integers(1, 3000), rng.integers(3000, 120_000), rng.integers(120_000, 600_000)]))
+        bucket = int(rng.choice(buckets))
+        mode = int(rng.choice([O.MODE_ERC, O.MODE_ERC, O.MODE_FIXED, O.MODE_CODED]))
+        ls = O.LEVELS_EXP if mode == O.MODE_CODED or rng.random() < 0.7 else O.LEVELS_UNIFORM
+        s = 4 if mode == O.MODE_CODED else int(rng.integers(1, 8))
+        nk = int(rng.integers(0, 2)) if ls == O.LEVELS_UNIFORM else O.NORM_L2
+        flags = O.make_flags(nk, ls, mode)
+        g = _input(d, 1000 + it)
+        seed, offset = int(rng.integers(0, 2 ** 40)), int(rng.integers(0, 2 ** 20))
+        got, bits = gpu_encode(g, bucket, s, flags, seed, offset)
+        rc, sign, sym, norms = O.decode_symbols(got, d, bucket, s)
+        assert rc == 0, (it, d, bucket, s, flags)
+        want, want_bits = O.encode(g, bucket, s, flags, seed, offset, norms=norms)
+        assert bits == want_bits and np.array_equal(got, want), (it, d, bucket, s, flags)
+        ref_norms = O.bucket_norms(g, bucket, nk)
+        live = np.isfinite(ref_norms) & (ref_norms > 0)
+        assert np.all(np.abs(norms[live].astype(np.float64) - ref_norms[live]) <= 1e-6 * ref_norms[live])
+        if it % 5 == 2:                                      # a histogram call leaves its norms in the workspace
+            hist = gpu_level_histogram(g, min(bucket, 8192), 4, 0, seed, offset)
+            assert hist.sum() == d
+        if it % 4 == 1:                                      # the decoder uses the same workspace
+            acc = gpu_decode([got, got], d, bucket, s)
+            assert np.array_equal(acc.view(np.uint32), O.decode_accumulate([got, got], d, bucket, s)[1].view(np.uint32))
+        checked += 1
+    assert checked == 160
+
+
+def test_two_streams_work_side_by_side_and_the_library_starts_over_after_shutdown():
+    """Every (device, stream) pair has a workspace of its own: calls enqueued alternately on two streams,
+    whose kernels may overlap, give the oracle's containers and sums; after nuq_shutdown the next call
+    allocates again and is bit-exact as before; a status is reported on the stream that latched it."""
+    torch, nuq = require_cuda()
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    shapes = [(300_001, 8192, 4, 0), (200_000, 65536, 3, 0), (150_000, 1024, 4, O.make_flags(mode=O.MODE_FIXED)),
+              (90_000, 512, 2, O.make_flags(O.NORM_LINF, O.LEVELS_UNIFORM))]
+    for round_ in range(2):
+        jobs = []
+        for i, (d, bucket, s, flags) in enumerate(shapes * 2):
+            st = sa if i % 2 == 0 else sb
+            g = _input(d, 500 + i)
+            with torch.cuda.stream(st):
+                gd = torch.from_numpy(g).cuda()
+                out, bits = nuq.encode(gd, bucket, s, flags, seed=i + 1, offset=round_, stream=st)
+                acc = nuq.decode_accumulate([out, out], d, bucket, s, stream=st)
+            jobs.append((g, d, bucket, s, flags, i, gd, out, bits, acc))
+        torch.cuda.synchronize()
+        assert nuq.last_status(sa) == 0 and nuq.last_status(sb) == 0
+        for (g, d, bucket, s, flags, i, gd, out, bits, acc) in jobs:
+            got = out.cpu().numpy().view(np.uint32)[: int(bits.item()) // 32].copy()
+            rc, sign, sym, norms = O.decode_symbols(got, d, bucket, s)
+            assert rc == 0
+            want, _ = O.encode(g, bucket, s, flags, i + 1, round_, norms=norms)
+            assert np.array_equal(got, want), (round_, i)
+            ref = O.decode_accumulate([got, got], d, bucket, s)[1]
+            assert np.array_equal(acc.cpu().numpy().view(np.uint32), ref.view(np.uint32)), (round_, i)
+        nuq.shutdown()                                       # the second round starts from nothing
+    # a malformed container on one stream is reported there and not on the other
+    bad = torch.zeros(4096, dtype=torch.int32, device="cuda")
+    with torch.cuda.stream(sa):
+        nuq.decode_accumulate([bad], 1000, 256, 3, stream=sa)
+    torch.cuda.synchronize()
+    assert nuq.last_status(sb) == 0 and nuq.last_status(sa) == nuq.ERR_BAD_STREAM and nuq.last_status(sa) == 0
