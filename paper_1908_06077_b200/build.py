@@ -5,8 +5,8 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnuq.so")
-SOURCES = ["nuq_api.cu", "nuq_encode.cu", "nuq_decode.cu"]
-HEADERS = ["nuq_common.cuh", "nuq_launch.h", os.path.join("..", "..", "include", "nuq.h")]
+SOURCES = ["nuq_api.cu", "nuq_encode.cu", "nuq_encode_fixed4.cu", "nuq_decode.cu"]
+HEADERS = ["nuq_common.cuh", "nuq_encode_common.cuh", "nuq_launch.h", os.path.join("..", "..", "include", "nuq.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--fmad=false", "-Xcompiler", "-fPIC", "-shared"]
 

@@ -14,6 +14,9 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
 size_t encode_smem_bytes(const EncodeParams& P);      // dynamic shared memory of one encoder CTA
 int encode_blocks_per_sm(const EncodeParams& P);      // encoder CTAs one SM holds at once (0 on error)
 cudaError_t launch_encode(const EncodeParams& P, cudaStream_t stream);
+bool fixed4_applies(const Geometry& G);               // the call is served by the 4-bit fixed-width encoder
+int fixed4_blocks_per_sm(const EncodeParams& P);
+cudaError_t launch_encode_fixed4(const EncodeParams& P, cudaStream_t stream);
 cudaError_t launch_level_histogram(const EncodeParams& P, uint64_t* hist, int sms, cudaStream_t stream);   // hist: s + 2 zeroed counters
 cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream);
 
