@@ -225,6 +225,23 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, uint32_t flags) {
     const int per_sm = best < 1 ? 1 : best;
     const uint64_t cap = (uint64_t)sms * (uint64_t)per_sm;
     pl.want_grid = (uint32_t)(G.ntiles < cap ? G.ntiles : cap);
+    // A bucket wider than a tile: a thread-block cluster of as many CTAs as the bucket has tiles encodes it and adds
+    // up its norm through distributed shared memory, so there is no separate pass over the gradient for the norms.
+    // (Not with norms supplied by the caller, and not in the 4-bit fixed-width encoder.)
+    P.cluster = 0;
+    P.pad = 0;
+    if (G.bucket > kBLK && norms_are_ours && !fixed4_applies(G)) {
+        P.cluster = G.blk_per_bucket;
+        int clusters = encode_max_clusters(P);
+        const int cap_clusters = sms * per_sm / (int)P.cluster;
+        if (clusters > cap_clusters) clusters = cap_clusters;
+        if (clusters >= 1) {
+            pl.norms_bytes = 0;
+            pl.want_grid = (uint32_t)(G.nb < (uint64_t)clusters ? G.nb : (uint64_t)clusters) * P.cluster;
+        } else {
+            P.cluster = 0;                                  // no room for a cluster: the separate norm pass
+        }
+    }
     return pl;
 }
 
@@ -437,7 +454,7 @@ nuq_status nuq_level_histogram(const float* g, uint64_t d, uint32_t bucket, uint
         P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
     }
-    P.stage_words = P.window_words = P.patience = P.grid = 0;
+    P.stage_words = P.window_words = P.patience = P.grid = P.cluster = P.pad = 0;
     if (cudaMemsetAsync(hist, 0, 8 * (s + 2), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     if (launch_level_histogram(P, hist, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;

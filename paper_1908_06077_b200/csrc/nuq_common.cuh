@@ -85,6 +85,8 @@ struct EncodeParams {
     uint32_t window_words;   // ERC: shared-memory token string of one warp and tile; a warp holds two
     uint32_t patience;       // polls a look-back wait may take before it gives up
     uint32_t grid;           // CTAs to launch
+    uint32_t cluster;        // CTAs per thread-block cluster: the blocks of one wide bucket (0: no clusters)
+    uint32_t pad;
 };
 
 struct DecodeParams {

@@ -396,6 +396,10 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     __shared__ CtaTotals s_tot;
     __shared__ uint32_t s_nnz;                             // fixed-width mode: nonzero symbols of this CTA
     __shared__ uint32_t s_last;                            // this CTA finished last
+    // clusters (buckets wider than a tile): what the CTAs of a cluster tell one another
+    __shared__ __align__(8) uint64_t s_xbar[2];            // s_xbar[p] completes when every CTA's part of the bucket's norm (iteration parity p) is here
+    __shared__ uint64_t s_xchg[2][8];                      // s_xchg[p][r]: CTA r's sum of squares (bits of a double) or max |x| bits
+    __shared__ unsigned long long s_bucket[4];             // buckets of the iterations to come, handed out by the cluster's first CTA
 
     using S = Sym<LEVELSET>;
     const Geometry& G = P.geo;
@@ -414,12 +418,30 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     const bool coarse = G.bucket % kWarpElems == 0;         // a warp's four sub-blocks always share one bucket
     const uint32_t spb = narrow ? G.sb_per_block : 32u;     // sub-blocks per coding block
 
+    // Clusters: a bucket wider than a tile is encoded by a cluster of as many CTAs as it has tiles, CTA r
+    // taking tile r of the bucket; they add up the bucket's norm among themselves through distributed shared
+    // memory, so the gradient is read from HBM once.  The cluster's first CTA takes the tickets (they count
+    // buckets then) and writes them into every CTA's s_bucket.
+    const uint32_t cl = P.cluster > 1u ? P.cluster : 1u;
+    const uint32_t crank = cl > 1u ? cluster_rank() : 0u;
+    const unsigned long long nclusters = gridDim.x / cl;
+    auto hand_out_bucket = [&](uint32_t iter) {             // thread 0 of the cluster's first CTA
+        const unsigned long long b = nclusters + atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        for (uint32_t r = 0; r < cl; ++r) st_cluster_u64(cluster_addr(&s_bucket[iter & 3u], r), b);
+        asm volatile("fence.acq_rel.cluster;" ::: "memory");
+    };
     // thread 0: take a ticket (a CTA's first tile is the one with its own number, the tickets count on
     // from there) and work out where that tile lies
     auto take_ticket = [&](uint32_t iter) {
         TileInfo& ti = s_info[iter & 3u];
-        const unsigned long long t =
-            iter == 0 ? blockIdx.x : gridDim.x + atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        unsigned long long t;
+        if (cl > 1u) {
+            const unsigned long long b = iter == 0 ? blockIdx.x / cl : *reinterpret_cast<volatile unsigned long long*>(&s_bucket[iter & 3u]);
+            t = b >= G.nb ? G.ntiles : b * cl + crank;
+            if (b < G.nb && t >= G.ntiles) t = G.ntiles + 1u;    // the last bucket is short and has no tile for this CTA
+        } else {
+            t = iter == 0 ? blockIdx.x : gridDim.x + atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        }
         describe_tile(G, t, &ti);
     };
     // A warp's part of a tile: elements [1024 w, 1024 (w + 1)) of it.  Whole 16-byte pieces come by a bulk
@@ -464,9 +486,21 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         s_tot.tiles = 0;
         s_tot.stop = 0xFFFFFFFFu;
         s_last = 0;
+        if (cl > 1u) {
+            mbar_init(&s_xbar[0], cl);
+            mbar_init(&s_xbar[1], cl);
+        }
         take_ticket(0);
     }
     __syncthreads();
+    if (cl > 1u) {
+        cluster_sync_all();                                 // every CTA's barriers exist before anyone arrives at them
+        if (tid == 0 && crank == 0) {
+            hand_out_bucket(1);
+            hand_out_bucket(2);
+        }
+        cluster_sync_all();                                 // the buckets of the next two iterations are known everywhere
+    }
     if (warp < (uint32_t)kEncWarps && lane == 0) start_copy(0);
     if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
 
@@ -533,7 +567,14 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     for (; !writer; ++it) {                                 // the 8 worker warps
         const TileInfo& ti = s_info[it & 3u];
         const uint64_t tile = ti.tile;
-        if (tile >= G.ntiles) break;
+        if (tile >= G.ntiles) {
+            // a CTA without a tile in the cluster's last, short bucket adds nothing to its norm, but says so
+            if (cl > 1u && tile == G.ntiles + 1u && warp == 0 && lane < cl) {
+                st_cluster_u64(cluster_addr(&s_xchg[it & 1u][crank], lane), 0ull);
+                mbar_arrive_cluster(cluster_addr(&s_xbar[it & 1u], lane));
+            }
+            break;
+        }
         const uint64_t elem0 = ti.elem0;
         const uint32_t tile_len = ti.tile_len, nsb_tile = ti.nsb;
 
@@ -623,6 +664,34 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                 if (P.norms_in != nullptr) {
                     const uint64_t nb_idx = narrow ? ti.first_block + bi : ti.bucket_idx;
                     norm = nb_idx < G.nb ? P.norms_in[nb_idx] : 0.0f;
+                } else if (cl > 1u) {
+                    // this CTA's tile is one part of its bucket: every CTA of the cluster sends its sum (or
+                    // maximum) to all of them, and all add the parts up in the same order
+                    double a = 0.0;
+                    uint32_t mxb = 0;
+                    for (uint32_t j = 3u; j < 32u; j += 4u) {       // one partial per warp
+                        a += s_partial[j];
+                        mxb = max(mxb, s_maxbits[j]);
+                    }
+                    const uint32_t xp = it & 1u;
+                    if (lane < cl) {
+                        st_cluster_u64(cluster_addr(&s_xchg[xp][crank], lane),
+                                       G.norm_kind == kNormL2 ? (uint64_t)__double_as_longlong(a) : (uint64_t)mxb);
+                        mbar_arrive_cluster(cluster_addr(&s_xbar[xp], lane));
+                    }
+                    __syncwarp();
+                    norm = 0.0f;
+                    if (!mbar_wait_cluster(&s_xbar[xp], (it >> 1) & 1u)) {
+                        if (lane == 0) latch_status(P.ws, kErrTimeout);   // never seen; do not hang
+                    } else if (G.norm_kind == kNormL2) {
+                        a = 0.0;
+                        for (uint32_t r = 0; r < cl; ++r) a += __longlong_as_double((long long)s_xchg[xp][r]);
+                        norm = (float)sqrt(a);
+                    } else {
+                        mxb = 0;
+                        for (uint32_t r = 0; r < cl; ++r) mxb = max(mxb, (uint32_t)s_xchg[xp][r]);
+                        norm = __uint_as_float(mxb);
+                    }
                 } else if (G.norm_kind == kNormL2) {
                     double a = 0.0;
                     if (coarse) for (uint32_t j = sb0 + 3u; j < sb0 + spb; j += 4u) a += s_partial[j];     // one partial per warp
@@ -652,6 +721,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
                                                             // and every warp is done with the previous tile
         // the ticket of the tile after the next is taken now: its round trip ends long before anyone looks
         if (tid == 0) take_ticket(it + 2u);
+        if (cl > 1u && tid == 0 && crank == 0) hand_out_bucket(it + 3u);   // seen by the others after the next exchange of norms
 
         TileMeta* const meta = &s_meta[it & 1u];
         uint32_t* const window = windows + ((it & 1u) * kEncWarps + warp) * P.window_words;   // this warp's token string
@@ -926,6 +996,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + G.ntiles + (G.ntiles + 31) / 32;
         for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;
     }
+    if (cl > 1u) cluster_sync_all();                        // nobody leaves while another CTA may still write into its shared memory
 }
 
 // ---------------------------------------------------------------------------
@@ -1078,14 +1149,62 @@ int encode_blocks_per_sm(const EncodeParams& P) {
     return blocks_per_sm<kLevelsUniform, kModeFixed>(P);
 }
 
+// launch configuration of a call, with the cluster shape when it has one
+struct EncodeLaunch {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+};
+template <uint32_t M>
+static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, cudaStream_t stream) {
+    L->cfg = cudaLaunchConfig_t{};
+    L->cfg.gridDim = dim3(grid);
+    L->cfg.blockDim = dim3(M == kModeErc ? kEncAllThreads : (uint32_t)kEncThreads);
+    L->cfg.dynamicSmemBytes = encode_smem_bytes(P);
+    L->cfg.stream = stream;
+    L->cfg.attrs = L->attr;
+    L->cfg.numAttrs = 0;
+    if (P.cluster > 1u) {
+        L->attr[0].id = cudaLaunchAttributeClusterDimension;
+        L->attr[0].val.clusterDim.x = P.cluster;
+        L->attr[0].val.clusterDim.y = 1;
+        L->attr[0].val.clusterDim.z = 1;
+        L->cfg.numAttrs = 1;
+    }
+}
+
 template <uint32_t L, uint32_t M>
 static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
     const size_t smem = encode_smem_bytes(P);
     cudaError_t e = prepare_kernel<L, M>();
     if (e != cudaSuccess) return e;
-    if (smem > (size_t)kEncMaxDynSmem || P.grid == 0) return cudaErrorInvalidValue;
-    encode_kernel<L, M><<<P.grid, M == kModeErc ? kEncAllThreads : (uint32_t)kEncThreads, smem, stream>>>(P);
-    return cudaGetLastError();
+    if (smem > (size_t)kEncMaxDynSmem || P.grid == 0 || (P.cluster > 1u && P.grid % P.cluster != 0)) return cudaErrorInvalidValue;
+    EncodeLaunch cfg;
+    fill_launch<M>(&cfg, P, P.grid, stream);
+    return cudaLaunchKernelEx(&cfg.cfg, encode_kernel<L, M>, P);
+}
+
+// clusters of P.cluster CTAs the device holds at once (0 on error)
+template <uint32_t L, uint32_t M>
+static int max_clusters(const EncodeParams& P) {
+    if (prepare_kernel<L, M>() != cudaSuccess) return 0;
+    EncodeLaunch cfg;
+    fill_launch<M>(&cfg, P, P.cluster, nullptr);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, encode_kernel<L, M>, &cfg.cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    return n;
+}
+
+int encode_max_clusters(const EncodeParams& P) {
+    const bool uni = P.geo.levelset == kLevelsUniform, fixed = P.geo.mode == kModeFixed;
+    if (encode_smem_bytes(P) > (size_t)kEncMaxDynSmem) return 0;
+    if (P.geo.levelset == kLevelsTable) return fixed ? max_clusters<kLevelsTable, kModeFixed>(P) : max_clusters<kLevelsTable, kModeErc>(P);
+    if (!uni && !fixed) return max_clusters<kLevelsExp, kModeErc>(P);
+    if (!uni && fixed) return max_clusters<kLevelsExp, kModeFixed>(P);
+    if (uni && !fixed) return max_clusters<kLevelsUniform, kModeErc>(P);
+    return max_clusters<kLevelsUniform, kModeFixed>(P);
 }
 
 cudaError_t launch_encode(const EncodeParams& P, cudaStream_t stream) {

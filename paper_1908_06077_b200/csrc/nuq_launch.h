@@ -13,6 +13,7 @@ cudaError_t launch_bucket_norms(const float* g, uint64_t d, uint32_t bucket, uin
                                 uint64_t nb, cudaStream_t stream);
 size_t encode_smem_bytes(const EncodeParams& P);      // dynamic shared memory of one encoder CTA
 int encode_blocks_per_sm(const EncodeParams& P);      // encoder CTAs one SM holds at once (0 on error)
+int encode_max_clusters(const EncodeParams& P);       // clusters of P.cluster encoder CTAs the device holds at once (0 on error)
 cudaError_t launch_encode(const EncodeParams& P, cudaStream_t stream);
 bool fixed4_applies(const Geometry& G);               // the call is served by the 4-bit fixed-width encoder
 int fixed4_blocks_per_sm(const EncodeParams& P);
