@@ -362,41 +362,59 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
         __syncthreads();
         float* const dst_tile = P.acc + b * G.bucket + first;
         const uint64_t word0 = kHeaderWords + b * rec_words + 1u + first / 8u;     // the tile's first field word in a container
-        for (uint32_t el = 8u * tid; el < tile_len; el += 8u * blockDim.x) {
-            float sum[8];
+        // Two groups of eight elements per thread and step (el and el + 8 * blockDim.x): the words of both are
+        // asked for before either is used, which keeps twice as many loads in flight.
+        const uint32_t stride = 8u * blockDim.x;
+        for (uint32_t el = 8u * tid; el < tile_len; el += 2u * stride) {
+            const bool second = el + stride < tile_len;
+            float sum[2][8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) sum[i] = 0.0f;
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int i = 0; i < 8; ++i) sum[h][i] = 0.0f;
             for (uint32_t k0 = 0; k0 < K; k0 += 8u) {
-                uint32_t wv[8];
+                uint32_t wv[2][8];
 #pragma unroll
-                for (uint32_t j = 0; j < 8; ++j) wv[j] = k0 + j < K ? __ldg(heads[k0 + j].hdr + word0 + el / 8u) : 0u;
+                for (uint32_t j = 0; j < 8; ++j) {
+                    const uint32_t* w = heads[k0 + j < K ? k0 + j : 0u].hdr + word0 + el / 8u;
+                    wv[0][j] = k0 + j < K ? __ldg(w) : 0u;
+                    wv[1][j] = k0 + j < K && second ? __ldg(w + blockDim.x) : 0u;
+                }
 #pragma unroll
                 for (uint32_t j = 0; j < 8; ++j) {
                     if (k0 + j < K) {
-                        const uint32_t x = wv[j];
-                        bad |= ((x & 0x77777777u) + over) & 0x88888888u;
-                        // the eight fields times four (byte offsets into the table), four to a register
-                        const uint32_t a = (x >> 2) & 0x3C3C3C3Cu, c = (x << 2) & 0x3C3C3C3Cu;   // elements 0 2 4 6 / 1 3 5 7 from the top byte
                         const char* tab = reinterpret_cast<const char*>(s_tab[k0 + j]);
-                        sum[0] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4443));
-                        sum[1] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4443));
-                        sum[2] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4442));
-                        sum[3] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4442));
-                        sum[4] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4441));
-                        sum[5] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4441));
-                        sum[6] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4440));
-                        sum[7] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4440));
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t x = wv[h][j];
+                            bad |= ((x & 0x77777777u) + over) & 0x88888888u;
+                            // the eight fields times four (byte offsets into the table), four to a register
+                            const uint32_t a = (x >> 2) & 0x3C3C3C3Cu, c = (x << 2) & 0x3C3C3C3Cu;   // elements 0 2 4 6 / 1 3 5 7 from the top byte
+                            sum[h][0] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4443));
+                            sum[h][1] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4443));
+                            sum[h][2] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4442));
+                            sum[h][3] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4442));
+                            sum[h][4] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4441));
+                            sum[h][5] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4441));
+                            sum[h][6] += *reinterpret_cast<const float*>(tab + __byte_perm(a, 0u, 0x4440));
+                            sum[h][7] += *reinterpret_cast<const float*>(tab + __byte_perm(c, 0u, 0x4440));
+                        }
                     }
                 }
             }
-            float* dst = dst_tile + el;
-            if (el + 8u <= tile_len) {
-                *reinterpret_cast<float4*>(dst) = make_float4(sum[0], sum[1], sum[2], sum[3]);
-                *reinterpret_cast<float4*>(dst + 4) = make_float4(sum[4], sum[5], sum[6], sum[7]);
-            } else {
 #pragma unroll
-                for (uint32_t i = 0; i < 8; ++i)
-                    if (el + i < tile_len) dst[i] = sum[i];
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t e0 = el + h * stride;
+                if (h == 1 && !second) break;
+                float* dst = dst_tile + e0;
+                if (e0 + 8u <= tile_len) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(sum[h][0], sum[h][1], sum[h][2], sum[h][3]);
+                    *reinterpret_cast<float4*>(dst + 4) = make_float4(sum[h][4], sum[h][5], sum[h][6], sum[h][7]);
+                } else {
+#pragma unroll
+                    for (uint32_t i = 0; i < 8; ++i)
+                        if (e0 + i < tile_len) dst[i] = sum[h][i];
+                }
             }
         }
     }
