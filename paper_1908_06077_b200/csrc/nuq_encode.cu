@@ -377,7 +377,8 @@ __device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot
     __syncwarp();
 }
 
-template <uint32_t LEVELSET, uint32_t MODE>
+// CLUSTERS: the call's buckets are wider than a tile and each is encoded by a thread-block cluster (see below).
+template <uint32_t LEVELSET, uint32_t MODE, bool CLUSTERS>
 __global__ void __launch_bounds__(MODE == kModeErc ? kEncAllThreads : kEncThreads, kEncMinBlocks)
 encode_kernel(const __grid_constant__ EncodeParams P) {
     extern __shared__ __align__(128) uint32_t smem[];
@@ -422,7 +423,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     // taking tile r of the bucket; they add up the bucket's norm among themselves through distributed shared
     // memory, so the gradient is read from HBM once.  The cluster's first CTA takes the tickets (they count
     // buckets then) and writes them into every CTA's s_bucket.
-    const uint32_t cl = P.cluster > 1u ? P.cluster : 1u;
+    const uint32_t cl = CLUSTERS ? P.cluster : 1u;
     const uint32_t crank = cl > 1u ? cluster_rank() : 0u;
     const unsigned long long nclusters = gridDim.x / cl;
     auto hand_out_bucket = [&](uint32_t iter) {             // thread 0 of the cluster's first CTA
@@ -1123,7 +1124,9 @@ template <uint32_t L, uint32_t M>
 static cudaError_t prepare_kernel() {
     static bool attr_set = false;
     if (attr_set) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M>, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncMaxDynSmem);
+    cudaError_t e = cudaFuncSetAttribute(encode_kernel<L, M, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncMaxDynSmem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(encode_kernel<L, M, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kEncMaxDynSmem);
     if (e == cudaSuccess) attr_set = true;
     return e;
 }
@@ -1133,7 +1136,7 @@ static int blocks_per_sm(const EncodeParams& P) {
     if (prepare_kernel<L, M>() != cudaSuccess) return 0;
     int n = 0;
     const int threads = M == kModeErc ? (int)kEncAllThreads : kEncThreads;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, encode_kernel<L, M>, threads, encode_smem_bytes(P)) != cudaSuccess)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, encode_kernel<L, M, false>, threads, encode_smem_bytes(P)) != cudaSuccess)
         return 0;
     return n;
 }
@@ -1180,7 +1183,8 @@ static cudaError_t launch_one(const EncodeParams& P, cudaStream_t stream) {
     if (smem > (size_t)kEncMaxDynSmem || P.grid == 0 || (P.cluster > 1u && P.grid % P.cluster != 0)) return cudaErrorInvalidValue;
     EncodeLaunch cfg;
     fill_launch<M>(&cfg, P, P.grid, stream);
-    return cudaLaunchKernelEx(&cfg.cfg, encode_kernel<L, M>, P);
+    if (P.cluster > 1u) return cudaLaunchKernelEx(&cfg.cfg, encode_kernel<L, M, true>, P);
+    return cudaLaunchKernelEx(&cfg.cfg, encode_kernel<L, M, false>, P);
 }
 
 // clusters of P.cluster CTAs the device holds at once (0 on error)
@@ -1190,7 +1194,7 @@ static int max_clusters(const EncodeParams& P) {
     EncodeLaunch cfg;
     fill_launch<M>(&cfg, P, P.cluster, nullptr);
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, encode_kernel<L, M>, &cfg.cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, encode_kernel<L, M, true>, &cfg.cfg) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
