@@ -26,6 +26,7 @@ struct WsEntry {
     // (0: none).  The allocation is zeroed and every encode kernel leaves its scan state zeroed, but the bucket
     // norms of a wide-bucket call or of a histogram call stay behind, at a place that depends on that call's size.
     size_t dirty_to = 0;
+    uint32_t dec_epoch = 0;  // decode calls made on this workspace (see DecodeParams::epoch)
 };
 
 // One mutex guards the host-side bookkeeping below (maps, tables); it is held for the microseconds a
@@ -540,6 +541,12 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     nuq_status st = get_workspace(stream, sizeof(Workspace), &ws, &dev);
     if (st != NUQ_OK) return st;
     P.ws = ws;
+    // The ticket counter a decode call uses has been zeroed by the call before it (or by the allocation, or by an
+    // encode call, which leaves both zeroed): calls take the two counters in turn and each zeroes the other one.
+    WsEntry& entry = g_ws[std::make_pair(dev, stream)];
+    if (++entry.dec_epoch == 0) entry.dec_epoch = 2;        // never 0, parity kept
+    P.epoch = entry.dec_epoch;
+    P.pad = 0;
     if (launch_decode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;
 }

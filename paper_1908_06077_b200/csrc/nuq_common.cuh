@@ -36,15 +36,14 @@ constexpr uint64_t kTileValueMask = (1ull << 62) - 1;
 // per-stream scratch owned by the library
 struct Workspace {
     int status;             // latched kernel status; survives calls until nuq_last_status reads it
-    int pad;
+    uint32_t dec_done_epoch; // decoder: the call (DecodeParams::epoch) whose fixed-width kernel did all the work
     // everything below is cleared at the start of every encode call
     uint64_t ticket;        // next tile to hand out
     uint64_t done;          // tiles finished
     uint64_t code_bits;     // token bits of the whole call
     uint64_t nnz;           // nonzero symbols of the whole call
     uint64_t total_words;   // payload words of the whole call
-    uint64_t dec_ticket;    // decoder: next tile to hand out (cleared before each decode launch)
-    uint64_t reserved[1];
+    uint64_t dec_ticket[2]; // decoder: next unit to hand out; a call uses the counter of its epoch's parity and zeroes the other one
     // followed by: uint64_t tile_state[ntiles], group_state[ceil(ntiles / 32)], then float norms[nb] for wide buckets
 };
 constexpr size_t kWorkspaceClearFrom = 8;
@@ -95,6 +94,8 @@ struct DecodeParams {
     uint32_t K;
     uint32_t group;          // streams decoded side by side (1, 2, 4 or 8)
     uint32_t after_fixed;    // the fixed-width kernel runs first; the general kernel returns if it did the work
+    uint32_t epoch;          // number of this decode call on its workspace (never 0)
+    uint32_t pad;
     float* acc;
     Workspace* ws;
 };

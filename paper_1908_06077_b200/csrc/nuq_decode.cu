@@ -343,7 +343,7 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
     uint32_t bad = 0;
     for (;;) {
         __syncthreads();                                    // the tables and the ticket of the previous tile are no longer read
-        if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        if (tid == 0) s_ticket = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket[P.epoch & 1u]), 1ull);
         __syncthreads();
         const uint64_t tile = s_ticket;
         if (tile >= ntiles) break;
@@ -436,7 +436,8 @@ __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant
             same = same && heads[k].ok && heads[k].mode == kModeFixed && heads[k].levelset == heads[0].levelset &&
                    heads[k].levelset != kLevelsTable;       // (streams with a level table take the general kernel)
         s_width = same ? heads[0].width : 0u;
-        if (same && blockIdx.x == 0) *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0]) = 1;   // tell the general kernel
+        if (same && blockIdx.x == 0) *reinterpret_cast<volatile uint32_t*>(&P.ws->dec_done_epoch) = P.epoch;   // tell the general kernel
+        if (blockIdx.x == 0) P.ws->dec_ticket[(P.epoch & 1u) ^ 1u] = 0;     // the next call's counter (nobody uses it during this call)
     }
     __syncthreads();
     if (heads[0].levelset == kLevelsExp) {                  // s <= 14: at most 16 levels, 5 bits
@@ -507,7 +508,8 @@ __host__ __device__ inline size_t decode_warp_bytes(uint32_t group, bool sums_in
 template <bool SUMS_IN_L2>
 __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
-    if (P.after_fixed && *reinterpret_cast<volatile uint64_t*>(&P.ws->reserved[0])) return;   // the fixed-width kernel did it all
+    if (P.after_fixed && *reinterpret_cast<volatile uint32_t*>(&P.ws->dec_done_epoch) == P.epoch) return;   // the fixed-width kernel did it all
+    if (blockIdx.x == 0 && threadIdx.x == 0) P.ws->dec_ticket[(P.epoch & 1u) ^ 1u] = 0;   // the next call's counter (nobody uses it during this call)
     const Geometry& G = P.geo;
     const uint32_t NG = P.group;                            // streams decoded side by side (1, 2, 4 or 8)
     const uint32_t S = 32u / NG;                            // sub-blocks per warp
@@ -551,13 +553,13 @@ __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_
     unsigned long long next_unit = 0;
     bool have_next = false;
     for (;;) {
-        if (!have_next && lane == 0) next_unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        if (!have_next && lane == 0) next_unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket[P.epoch & 1u]), 1ull);
         const unsigned long long unit = __shfl_sync(0xffffffffu, next_unit, 0);
         if (unit >= nunits) break;
         const uint64_t tile = unit / NG;
         const uint32_t part = (uint32_t)(unit % NG);        // which S sub-blocks of the tile
         have_next = unit < reserve_until;
-        if (have_next && lane == 0) next_unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket), 1ull);
+        if (have_next && lane == 0) next_unit = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->dec_ticket[P.epoch & 1u]), 1ull);
         // ---- tile geometry (same tiling as the encoder) ---------------------------
         TileGeo T;
         T.bucket_idx = 0;
@@ -939,7 +941,6 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     if (warps < 8u && wmax >= 8u) warps = 8u;
     const size_t smem = decode_smem_bytes(P.group, P.K, warps, sums_in_l2);
     if (smem > kSmemMaxCta) return cudaErrorInvalidValue;
-    if (cudaMemsetAsync(&P.ws->dec_ticket, 0, 2 * sizeof(uint64_t), stream) != cudaSuccess) return cudaErrorUnknown;   // ticket and the flag behind it
     if (P.after_fixed) {
         const uint64_t groups = (P.geo.d + 31) / 32, want_fixed = (groups + 255) / 256, cap_fixed = (uint64_t)sms * 4u;
         decode_fixed_kernel<<<(unsigned)(want_fixed < cap_fixed ? want_fixed : cap_fixed), 256, 0, stream>>>(P);
