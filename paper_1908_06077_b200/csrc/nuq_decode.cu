@@ -508,6 +508,9 @@ __host__ __device__ inline size_t decode_warp_bytes(uint32_t group, bool sums_in
 template <bool SUMS_IN_L2>
 __global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
+    // Behind the fixed-width kernel this one is launched with programmatic stream serialization: its launch is
+    // worked off while that kernel still runs, and it waits here until that kernel's writes are visible.
+    if (P.after_fixed) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (P.after_fixed && *reinterpret_cast<volatile uint32_t*>(&P.ws->dec_done_epoch) == P.epoch) return;   // the fixed-width kernel did it all
     if (blockIdx.x == 0 && threadIdx.x == 0) P.ws->dec_ticket[(P.epoch & 1u) ^ 1u] = 0;   // the next call's counter (nobody uses it during this call)
     const Geometry& G = P.geo;
@@ -946,9 +949,21 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
         decode_fixed_kernel<<<(unsigned)(want_fixed < cap_fixed ? want_fixed : cap_fixed), 256, 0, stream>>>(P);
         if (cudaGetLastError() != cudaSuccess) return cudaErrorUnknown;
     }
-    if (sums_in_l2) decode_kernel<true><<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
-    else decode_kernel<false><<<(unsigned)grid, 32u * warps, smem, stream>>>(P);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(32u * warps);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 0;
+    if (P.after_fixed) {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 1;
+    }
+    if (sums_in_l2) return cudaLaunchKernelEx(&cfg, decode_kernel<true>, P);
+    return cudaLaunchKernelEx(&cfg, decode_kernel<false>, P);
 }
 
 }  // namespace nuq
