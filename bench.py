@@ -344,11 +344,13 @@ class Workload:
         return float(num / (g[finite] ** 2).sum())
 
     def launches_per_step(self):
-        # my kernels only: one encode kernel per worker (two for buckets wider than a tile: the norms
-        # come first), one decode kernel (two when all streams are fixed-width: that path's own kernel,
-        # then the general one, which returns at once)
+        # my kernels only: one encode kernel per worker (two for buckets wider than a tile in the 4-bit
+        # fixed-width mode: the norms come first; otherwise a cluster adds the norm up inside the encode
+        # kernel), one decode kernel (two when all streams are fixed-width: that path's own kernel, then
+        # the general one, which returns at once)
+        fixed = (self.flags >> 16) & 0xff == 1
         wide = self.bucket > 8192
-        return self.K * (2 if wide else 1) + (2 if (self.flags >> 16) & 0xff == 1 else 1)
+        return self.K * (2 if wide and fixed else 1) + (2 if fixed else 1)
 
 
 def summarize(ms):
@@ -477,9 +479,9 @@ def run_gpu(args):
             "encode_ms_per_call": enc_launch_ms, "decode_ms_per_call": t_dec,
             "encode_us_per_call": {k: 1e3 * v for k, v in summarize([e / K for e in enc_ms]).items()},
             "decode_us_per_call": {k: 1e3 * v for k, v in summarize(dec_ms).items()},
-            "roofline": roofline_entry("encode_kernel", enc_bytes, enc_launch_ms, peak, peak_kind,
+            "roofline": roofline_entry(ENCODE_KERNEL.get(args.workload, "encode_kernel"), enc_bytes, enc_launch_ms, peak, peak_kind,
                                        ENCODE_TRAFFIC_BYTES.get(args.workload) if full else None),
-            "roofline_decode": roofline_entry("decode_kernel", dec_bytes, t_dec, peak, peak_kind,
+            "roofline_decode": roofline_entry(DECODE_KERNEL.get(args.workload, "decode_kernel"), dec_bytes, t_dec, peak, peak_kind,
                                               DECODE_TRAFFIC_BYTES.get(args.workload) if full else None),
             "gpu_launches": steps * w.launches_per_step(),
             "clocks": clocks,
@@ -531,8 +533,11 @@ def run_gpu(args):
 # summarised under profiles/.  Reads equal the algorithmic reads; the writes counted are those that
 # had left the 126 MB L2 when the kernel ended (a container or the sums of C3 fit in it), so the
 # totals of the decoders and of the fixed-width encoder lie below the algorithmic bytes.
-ENCODE_TRAFFIC_BYTES = {"c3": 102_302_208 + 3_524_608, "c3-fixed": 102_291_968 + 4_743_936}
-DECODE_TRAFFIC_BYTES = {"c3": 24_614_144 + 44_172_800, "c3-fixed": 102_397_952 + 59_644_928}
+ENCODE_TRAFFIC_BYTES = {"c3": 102_302_208 + 3_524_608, "c3-fixed": 102_289_152 + 5_162_496}
+DECODE_TRAFFIC_BYTES = {"c3": 24_614_144 + 44_172_800, "c3-fixed": 102_405_888 + 56_554_240}
+# the kernel that does the work of a call, where it is not the general one
+ENCODE_KERNEL = {"c3-fixed": "encode_fixed4_kernel"}
+DECODE_KERNEL = {"c3-fixed": "decode_fixed_kernel"}
 
 
 def main():

@@ -113,7 +113,8 @@ def test_scan_state_is_clean_after_a_call_with_wide_buckets():
                                      # the next call's group word (a sum that is added to) lies where the norms were
                                      (200_000, 65536, 8192 * 25 + 100), (100_000, 16384, 8192 * 13 + 50), (40_000, 32768, 8192 * 5 + 9)):
         for rep in range(3):
-            gpu_encode(_input(d_wide, d_wide + rep), b_wide, 4, 0, 3, rep)
+            # (4-bit fixed-width calls take their norms from the workspace; ERC calls add them up in clusters)
+            gpu_encode(_input(d_wide, d_wide + rep), b_wide, 4, O.make_flags(mode=O.MODE_FIXED) if rep % 2 == 0 else 0, 3, rep)
             if rep == 1:                                      # a short call in between clears only what it uses itself
                 gpu_encode(_input(1000, 1), 256, 3, 0, 1, 0)
             if rep == 2:                                      # the histogram's norms lie at the front of the workspace
@@ -125,6 +126,28 @@ def test_scan_state_is_clean_after_a_call_with_wide_buckets():
             want, want_bits = O.encode(g, 8192, 4, 0, seed=5, offset=rep, norms=norms)
             got, got_bits = gpu_encode(g, 8192, 4, 0, seed=5, offset=rep, norms=norms)
             assert got_bits == want_bits and np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("d,bucket,nk,ls", [(6_000_001, 16384, L2, EXP), (6_000_001, 32768, LINF, EXP),
+                                            (5_000_000 + 8192 * 3 + 11, 65536, L2, UNI), (65536 * 3 + 8192 * 2 + 1, 65536, L2, EXP)])
+def test_wide_buckets_encoded_by_clusters(d, bucket, nk, ls):
+    """Buckets wider than a tile: a cluster of 2, 4 or 8 CTAs encodes a bucket and adds up its norm among
+    themselves.  More buckets than resident clusters (so that buckets are handed out by ticket), a last
+    bucket with fewer tiles than the cluster has CTAs, both norms; the decoded sum of two such streams."""
+    flags = O.make_flags(nk, ls, O.MODE_ERC)
+    gs = [_input(d, 31 * d + k) for k in range(2)]
+    streams = []
+    for k, g in enumerate(gs):
+        got, _ = gpu_encode(g, bucket, 4, flags, seed=7 + k, offset=k)
+        compare_symbols(g, bucket, 4, flags, 7 + k, k, got)
+        # given the norms the clusters agreed on, the whole container is the oracle's
+        rc, _, _, gnorms = O.decode_symbols(got, d, bucket, 4)
+        assert rc == 0
+        want, _ = O.encode(g, bucket, 4, flags, 7 + k, k, norms=gnorms)
+        assert np.array_equal(got, want)
+        streams.append(got)
+    acc = gpu_decode(streams, d, bucket, 4)
+    assert np.array_equal(acc.view(np.uint32), O.decode_accumulate(streams, d, bucket, 4)[1].view(np.uint32))
 
 
 def test_stream_info_and_status():
