@@ -506,7 +506,7 @@ __host__ __device__ inline size_t decode_warp_bytes(uint32_t group, bool sums_in
 // would fit an SM, too few to hide the latency of the walk.  The order of the adds is the same.
 // (Taken for one or two streams side by side; with four, 17 warps fit and shared memory is faster.)
 template <bool SUMS_IN_L2>
-__global__ void __launch_bounds__(32 * kDecMaxWarps) decode_kernel(const __grid_constant__ DecodeParams P) {
+__global__ void __launch_bounds__(32 * (SUMS_IN_L2 ? kDecMaxWarps - 1 : kDecMaxWarps)) decode_kernel(const __grid_constant__ DecodeParams P) {
     extern __shared__ __align__(16) unsigned char dsm[];
     // Behind the fixed-width kernel this one is launched with programmatic stream serialization: its launch is
     // worked off while that kernel still runs, and it waits here until that kernel's writes are visible.
@@ -920,7 +920,7 @@ cudaError_t launch_decode(const DecodeParams& P, int sms, cudaStream_t stream) {
     // the largest unless a smaller one saves 6 % or more.
     const bool sums_in_l2 = P.group < 4u;                  // 1 or 2 streams side by side
     const size_t fixed = decode_warp_offset(P.K) + 1024u, per_warp = decode_warp_bytes(P.group, sums_in_l2);
-    uint32_t wmax = kDecMaxWarps;
+    uint32_t wmax = sums_in_l2 ? kDecMaxWarps - 1u : kDecMaxWarps;   // (the instance with the sums in the L2 needs a few registers more)
     while (wmax > 1 && fixed + wmax * per_warp > kSmemPerSm) --wmax;
     const uint64_t units = P.geo.ntiles * P.group;                          // warp-sized units of work
     uint32_t warps = wmax;
