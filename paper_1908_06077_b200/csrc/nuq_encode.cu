@@ -27,9 +27,13 @@
 // and the block offsets.  Workers and writer meet through named barriers on which one
 // side only arrives, so the workers never wait for other CTAs.
 // In the fixed-width mode there is no writer: a lane packs the fields of its eight
-// elements, two lanes exchange halves, and every lane stores one finished word.
+// elements, two lanes exchange halves, and every lane stores one finished word (4-bit
+// fields of the exponential level set have a leaner kernel of their own, nuq_encode_fixed4.cu).
 // Counters and the container header are written once per CTA, the header by whichever
 // CTA finishes last.
+// A bucket wider than a tile is encoded by a thread-block cluster, one CTA per tile of the
+// bucket: the CTAs send one another their tiles' sums of squares through distributed shared
+// memory and agree on the bucket's norm, so the gradient is still read only once.
 #include "nuq_encode_common.cuh"
 #include "nuq_launch.h"
 
