@@ -155,7 +155,8 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
  * nuq_encode.  Differences:
  *   - Size limit: with T = ceil(d / tile) tiles (a tile is 8192 elements, or
  *     floor(8192 / bucket) buckets) the scan state needs 64 + 8 * (T + ceil(T / 32))
- *     bytes, plus 4 bytes per bucket when bucket > 8192.  If that exceeds
+ *     bytes, plus 4 bytes per bucket when bucket > 8192 and the bucket norms
+ *     come from a pass of their own (4-bit fixed-width fields).  If that exceeds
  *     NUQ_STATIC_SCRATCH_BYTES the call returns NUQ_ERR_CAPACITY and enqueues
  *     nothing (d up to about 5.2e8 with bucket = 8192).
  *   - The first call on each device looks up the array's device address (the

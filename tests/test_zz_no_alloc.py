@@ -36,7 +36,8 @@ def _container(torch, out, bits):
 @pytest.mark.parametrize("d,bucket,s,flags", [
     (300001, 8192, 4, 0),                 # ERC, several tiles and a ragged tail
     (70000, 512, 3, 0),                   # many buckets per tile
-    (200000, 65536, 4, 0),                # wide bucket: norms also live in the static scratch
+    (200000, 65536, 4, 0),                # wide bucket: encoded by clusters of eight CTAs
+    (200000, 65536, 4, 1 << 16),          # wide bucket, fixed-width: norms also live in the static scratch
     (100000, 8192, 4, 1 << 16),           # fixed-width mode
 ])
 def test_static_scratch_encode_equals_allocating_encode_twice(d, bucket, s, flags):
