@@ -1005,8 +1005,8 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         // Every tile of the call has been written: nobody looks at the call's scan state any more.  The CTA
         // that finished last leaves it zeroed, so the next call on this workspace starts without a clearing pass.
         uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
-        const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + G.ntiles + (G.ntiles + 31) / 32;
-        for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;
+        const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + (MODE == kModeErc ? G.ntiles + (G.ntiles + 31) / 32 : 0);
+        for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;    // (only the ERC mode keeps state per tile)
     }
     if (cl > 1u) cluster_sync_all();                        // nobody leaves while another CTA may still write into its shared memory
 }

@@ -284,10 +284,10 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
     if (tid == 0 && finish_cta<kModeFixed>(P, it, s_nnz, 0)) s_last = 1;
     __syncthreads();
     if (s_last) {
-        // Every tile of the call has been written.  The CTA that finished last leaves the call's state zeroed,
-        // so the next call on this workspace starts without a clearing pass.
+        // Every tile of the call has been written.  The CTA that finished last leaves the call's counters zeroed,
+        // so the next call on this workspace starts without a clearing pass (this kernel keeps no state per tile).
         uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
-        const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + G.ntiles + (G.ntiles + 31) / 32;
+        const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8;
         for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;
     }
 }
