@@ -75,6 +75,9 @@ _decode_sym = _sig("nuq_oracle_decode_symbols", C.c_int, C.c_void_p, C.c_uint64,
 _decode_acc = _sig("nuq_oracle_decode_accumulate", C.c_int, C.POINTER(C.c_void_p), C.c_uint32, C.c_uint64,
                    C.c_uint32, C.c_uint32, _f32p)
 _chain_bits = _sig("nuq_oracle_single_chain_bits", C.c_uint64, _u16p, C.c_uint64)
+_f64p = np.ctypeslib.ndpointer(np.float64, flags="C_CONTIGUOUS")
+_momentum = _sig("nuq_oracle_momentum_step", None, _f64p, _f64p, _f32p, C.c_uint64, C.c_double, C.c_uint32,
+                 C.c_double, C.c_double)
 
 
 def philox4x32_10(ctr, key):
@@ -252,6 +255,15 @@ def decode_accumulate(streams, d, bucket, s):
     acc = np.zeros(d, np.float32)
     rc = _decode_acc(ptrs, len(streams), d, bucket, s, acc)
     return rc, acc
+
+
+def momentum_step(w, yl, total, alpha, K, mu=0.0, l=0.0):
+    """(w_next, yl_next) of the aggregation step with momentum, in fp64; `total` = sum of the K decoded gradients"""
+    w = np.array(w, np.float64)
+    yl = np.array(yl, np.float64)
+    total = np.ascontiguousarray(total, np.float32)
+    _momentum(w, yl, total, total.size, float(alpha), int(K), float(mu), float(l))
+    return w, yl
 
 
 def single_chain_bits(sym):

@@ -14,6 +14,8 @@
  *   - Elias recursive coding   Algorithm 2 (App. A)
  *   - ENCODE / DECODE          App. A, applied per bucket (Sec. 5)
  *   - aggregate  sum_i g^_i    Algorithm 1, aggregation line (without alpha/K)
+ *   - the aggregation step     w <- w - (alpha/K) sum_i g^_i  (Algorithm 1, aggregation line, Omega = R^d)
+ *                              and its momentum form (Sec. 4, "NUQSGD with momentum", the rule y, y^l, w)
  *   - closed-form variance     Lemma 7 / Eq. (genvar)
  *   - uniform level set k/2^s  (QSGD / QSGDinf comparison, Sec. 1 and 3)
  *   - arbitrary level sequences L = (0, l_1, ..., l_s, 1), e.g. L_p = (0, p^s, ..., p, 1)
@@ -40,7 +42,9 @@
  * arithmetic, unbiasedness by enumeration, Lemma 7 on hand-worked vectors;
  * for coded level indices: code lengths of hand-worked trees, least cost among
  * all prefix codes by brute force, the Kraft sum, canonical code words listed
- * by hand, a hand-assembled container, the same symbols as the ERC mode.
+ * by hand, a hand-assembled container, the same symbols as the ERC mode;
+ * for the aggregation step: steps worked by hand, heavy-ball and Nesterov
+ * iterations written in their velocity forms, a fixed point.
  */
 #include <math.h>
 #include <stdint.h>
@@ -733,6 +737,24 @@ int nuq_oracle_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     }
     free(sign); free(sym); free(norms);
     return rc;
+}
+
+/* The aggregation step of Algorithm 1 with the momentum rule of Sec. 4 ("NUQSGD with momentum"), where the
+ * gradient is the average g = (1/K) sum_i g^_i of the decoded gradients (`sum` holds sum_i g^_i):
+ *     y      = w - alpha g
+ *     y^l    = w - l alpha g
+ *     w_next = y + mu (y^l - y^l_prev)
+ * l = 0 is the heavy-ball method, l = 1 Nesterov's; mu = 0 is Algorithm 1's own line w - (alpha/K) sum_i g^_i
+ * (no projection: Omega = R^d).  fp64; w and yl (y^l_prev on entry, y^l on return) are updated in place.   */
+void nuq_oracle_momentum_step(double* w, double* yl, const float* sum, uint64_t d, double alpha, uint32_t K,
+                              double mu, double l) {
+    for (uint64_t i = 0; i < d; ++i) {
+        double g = (double)sum[i] / (double)K;
+        double y = w[i] - alpha * g;
+        double yl_next = w[i] - l * alpha * g;
+        w[i] = y + mu * (yl_next - yl[i]);
+        yl[i] = yl_next;
+    }
 }
 
 /* Code length of the paper's own framing (one run per bucket, no sub-block

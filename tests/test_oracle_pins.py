@@ -507,3 +507,47 @@ def test_level_code_words_are_prefix_free_and_bad_lengths_are_refused():
     for lengths in ([1, 1, 2], [0, 1], [1, 8], [2], [1] * 9, [1, 2, 3, 3, 3]):
         with pytest.raises(ValueError):
             O.set_level_code(lengths)
+
+
+def test_momentum_step_worked_by_hand():
+    """The aggregation step of Algorithm 1 and its momentum form (tests/golden/momentum_steps.txt)."""
+    for w, yl, total, alpha, K, mu, l, w_next, yl_next in golden_rows("momentum_steps.txt"):
+        got_w, got_yl = O.momentum_step([float(w)], [float(yl)], [float(total)], float(alpha), int(K), float(mu), float(l))
+        assert got_w[0] == float(w_next) and got_yl[0] == float(yl_next), (w, yl, total)
+
+
+def test_momentum_step_is_heavy_ball_and_nesterov_in_their_velocity_forms():
+    """Sec. 4: l = 0 gives the heavy-ball method, l = 1 Nesterov's.  Both are iterated here in their
+    velocity forms (v <- mu v - alpha grad, w <- w + v; for Nesterov the gradient at the look-ahead point
+    theta + mu v, whose sequence is the rule's w) on a quadratic, K workers sending the same gradient."""
+    rng = np.random.default_rng(5)
+    n, K, alpha, mu = 6, 4, 0.05, 0.8                     # (K a power of two: K times a gradient is exact in fp32)
+    m = rng.standard_normal((n, n))
+    a = m @ m.T / n + 0.5 * np.eye(n)                       # gradient of w' A w / 2 is A w
+    w0 = rng.standard_normal(n)
+    for l in (0.0, 1.0):
+        w, yl = w0.copy(), w0.copy()                        # the rule starts from y^l_0 = w_0, i.e. from rest
+        theta, v = w0.copy(), np.zeros(n)
+        for step in range(60):
+            grad = (a @ w).astype(np.float32)               # what the K workers send, exactly representable sums
+            w, yl = O.momentum_step(w, yl, K * grad.astype(np.float64), alpha, K, mu, l)
+            if l == 0.0:
+                v = mu * v - alpha * grad.astype(np.float64)
+                theta = theta + v
+                want = theta
+            else:
+                v = mu * v - alpha * grad.astype(np.float64)    # grad was taken at theta + mu v (= w, see below)
+                theta = theta + v
+                want = theta + mu * v
+            assert np.allclose(w, want, rtol=0, atol=1e-12 * (1 + np.abs(want).max())), (l, step)
+        assert np.linalg.norm(w) < 0.5 * np.linalg.norm(w0)        # and it does descend
+
+
+def test_momentum_step_fixed_point_and_plain_sgd():
+    w = np.array([1.5, -2.0, 0.0]); zero = np.zeros(3, np.float32)
+    for mu, l in ((0.0, 0.0), (0.9, 0.0), (0.9, 1.0), (0.5, 0.3)):
+        got_w, got_yl = O.momentum_step(w, w, zero, 0.1, 4, mu, l)
+        assert np.array_equal(got_w, w) and np.array_equal(got_yl, w)     # no gradient, at rest: nothing moves
+    total = np.array([8.0, -4.0, 2.0], np.float32)
+    got_w, _ = O.momentum_step(w, w, total, 0.25, 8, 0.0, 0.0)
+    assert np.array_equal(got_w, np.array([1.5 - 0.25, -2.0 + 0.125, -0.0625]))   # w - (alpha / K) sum
