@@ -343,6 +343,44 @@ class Workload:
         num = ((self.acc.double() - g)[finite] ** 2).sum()
         return float(num / (g[finite] ** 2).sum())
 
+    def fused_update(self, flush, reps=5):
+        """The aggregation step of Algorithm 1 fused into the decoder (nuq_decode_update, Nesterov momentum):
+        time per call beside the unfused pair it replaces (the decode call, then an optimizer step made
+        of torch's elementwise kernels, for context)."""
+        torch, nuq = self.torch, self.nuq
+        w = torch.zeros(self.d, device="cuda")
+        yl = torch.zeros(self.d, device="cuda")
+        alpha, mu, l = 0.1, 0.9, 1.0
+        acc = self.acc if self.K < 3 else None              # with one or two streams the library adds up in acc
+        fused, pair = [], []
+        for it in range(reps + 2):
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            flush.fill_(3)
+            ev[0].record()
+            nuq.decode_update(self.outs, self.d, self.bucket, self.s, w, yl, alpha, mu, l, acc=acc)
+            ev[1].record()
+            flush.fill_(4)
+            ev[2].record()
+            nuq.decode_accumulate(self.outs, self.d, self.bucket, self.s, acc=self.acc)
+            c = alpha / self.K                              # y = w - c G; y^l = w - l c G; w = y + mu (y^l - y^l_prev)
+            yl_next = torch.add(w, self.acc, alpha=-l * c)
+            w.add_(self.acc, alpha=-c).add_(yl_next - yl, alpha=mu)
+            yl.copy_(yl_next)
+            ev[3].record()
+            torch.cuda.synchronize()
+            if it >= 2:
+                fused.append(ev[0].elapsed_time(ev[1]))
+                pair.append(ev[2].elapsed_time(ev[3]))
+        assert nuq.last_status() == 0
+        d4 = 4.0 * self.d
+        containers = sum(self.stream_stats()["container_bytes"])
+        ms = statistics.median(fused)
+        return {"what": "w, y^l <- momentum step (mu 0.9, l 1) on the decoded sum, one call",
+                "decode_update_us_per_call": 1e3 * ms,
+                "decode_then_torch_step_us": 1e3 * statistics.median(pair),
+                "algorithmic_bytes": containers + 4 * d4 + (d4 if acc is not None else 0.0),
+                "achieved_gbs": (containers + 4 * d4 + (d4 if acc is not None else 0.0)) / (ms / 1e3) / 1e9}
+
     def launches_per_step(self):
         # my kernels only: one encode kernel per worker (two for buckets wider than a tile in the 4-bit
         # fixed-width mode: the norms come first; otherwise a cluster adds the norm up inside the encode
@@ -431,6 +469,7 @@ def run_gpu(args):
     t_step = t_enc + t_dec
     stats = w.stream_stats()
     container_bytes = stats.pop("container_bytes")
+    fused_update = w.fused_update(flush) if rank == 0 else None
 
     # ---- end to end: pinned host gradients in, summed gradient out ------------------------
     e2e = None
@@ -487,6 +526,7 @@ def run_gpu(args):
             "clocks": clocks,
         }
         line.update(stats)
+        line["fused_update"] = fused_update
         if w.level_code is not None:
             line["level_code_lengths"] = w.level_code
             line["level_histogram"] = w.level_histogram

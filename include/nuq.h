@@ -137,6 +137,32 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
                                  float* acc, void* stream);
 
 /*
+ * The aggregation line of Algorithm 1 fused into DECODE:
+ *     w <- w - (alpha / K) sum_k DECODE(c_k)
+ * and, with mu != 0, the momentum rule of Sec. 4 ("NUQSGD with momentum") in its place:
+ *     y = w - (alpha / K) G,   y^l = w - l (alpha / K) G,   w <- y + mu (y^l - y^l_prev)
+ * with G = sum_k DECODE(c_k); l = 0 is the heavy-ball method, l = 1 Nesterov's.  The
+ * sum is applied where the decoder finishes it, so it is not written out and read
+ * again by an optimizer kernel.  No projection (Omega = R^d).
+ *
+ *   streams, K, d, bucket, s   as for nuq_decode_accumulate
+ *   acc      device, d floats, 16-byte aligned, or NULL.  If given it receives
+ *            the sum as from nuq_decode_accumulate.  With K <= 2 it is REQUIRED
+ *            (the library adds the streams up in it).
+ *   w        device, d floats, 16-byte aligned: the parameters, updated in place
+ *   yl       device, d floats, 16-byte aligned: y^l of the previous step on
+ *            entry (the parameters themselves before the first step), y^l of
+ *            this step on return; may be NULL when mu == 0 (it is not touched)
+ *   alpha    learning rate; mu in [0, 1) momentum; l in [0, 1]
+ * Arithmetic: fp32; alpha / K and l alpha / K are formed on the host in double
+ * and rounded once, each of the three lines is one fused multiply-add.
+ * Errors as for nuq_decode_accumulate; after NUQ_ERR_BAD_STREAM the affected
+ * coordinates of w and yl are unspecified.
+ */
+nuq_status nuq_decode_update(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
+                             float* acc, float* w, float* yl, float alpha, float mu, float l, void* stream);
+
+/*
  * nuq_encode for callers that must not allocate device memory.  (The paper has
  * no counterpart; this entry point exists for deployment reasons only.)
  *

@@ -513,13 +513,20 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
     return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, it->second, nullptr, dev, stream);
 }
 
-nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
-                                 float* acc, void* stream_) {
+// Shared by the two decode entry points.  `w` == nullptr: the sums only.
+static nuq_status enqueue_decode(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s, float* acc,
+                                 float* w, float* yl, float alpha, float mu, float l, void* stream_) {
     std::lock_guard<std::mutex> lock(g_mu);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     DecodeParams P;
-    if (!streams || !acc || K < 1 || K > kMaxK) return NUQ_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(acc) & 15u) return NUQ_ERR_INVALID_ARG;
+    if (!streams || K < 1 || K > kMaxK) return NUQ_ERR_INVALID_ARG;
+    // with one or two streams the sums are added up in acc itself, so it is needed even when only w is wanted
+    if (!acc && (!w || K < 3)) return NUQ_ERR_INVALID_ARG;
+    if (w && mu != 0.0f && !yl) return NUQ_ERR_INVALID_ARG;
+    if (w && !(alpha == alpha && mu >= 0.0f && mu < 1.0f && l >= 0.0f && l <= 1.0f)) return NUQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(acc) & 15u) || (reinterpret_cast<uintptr_t>(w) & 15u) ||
+        (reinterpret_cast<uintptr_t>(yl) & 15u))
+        return NUQ_ERR_INVALID_ARG;
     // the level set and mode come from each container's header; geometry only needs (d, bucket, s)
     if (!make_geometry(d, bucket, s, 0, &P.geo)) return NUQ_ERR_INVALID_ARG;
     for (uint32_t k = 0; k < K; ++k) {
@@ -537,6 +544,12 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
         if (it == g_container_mode.end() || it->second != kModeFixed) P.after_fixed = 0;
     }
     P.acc = acc;
+    P.w = w;
+    P.yl = w && mu != 0.0f ? yl : nullptr;
+    P.step_c = w ? (float)((double)alpha / (double)K) : 0.0f;          // one rounding each
+    P.step_lc = w ? (float)((double)l * (double)alpha / (double)K) : 0.0f;
+    P.mu = w ? mu : 0.0f;
+    P.pad2 = 0;
     Workspace* ws = nullptr;
     nuq_status st = get_workspace(stream, sizeof(Workspace), &ws, &dev);
     if (st != NUQ_OK) return st;
@@ -549,6 +562,18 @@ nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_
     P.pad = 0;
     if (launch_decode(P, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;
+}
+
+nuq_status nuq_decode_accumulate(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s,
+                                 float* acc, void* stream) {
+    if (!acc) return NUQ_ERR_INVALID_ARG;
+    return enqueue_decode(streams, K, d, bucket, s, acc, nullptr, nullptr, 0.0f, 0.0f, 0.0f, stream);
+}
+
+nuq_status nuq_decode_update(const void* const* streams, uint32_t K, uint64_t d, uint32_t bucket, uint32_t s, float* acc,
+                             float* w, float* yl, float alpha, float mu, float l, void* stream) {
+    if (!w) return NUQ_ERR_INVALID_ARG;
+    return enqueue_decode(streams, K, d, bucket, s, acc, w, yl, alpha, mu, l, stream);
 }
 
 nuq_status nuq_last_status(void* stream_) {

@@ -96,6 +96,12 @@ struct DecodeParams {
     uint32_t after_fixed;    // the fixed-width kernel runs first; the general kernel returns if it did the work
     uint32_t epoch;          // number of this decode call on its workspace (never 0)
     uint32_t pad;
+    // the aggregation step fused into the decoder (w == nullptr: none): see step_value in nuq_decode.cu
+    float* w;                // parameters, updated in place
+    float* yl;               // the momentum rule's y^l, updated in place (not touched when mu == 0)
+    float step_c, step_lc;   // alpha / K and l alpha / K
+    float mu;
+    uint32_t pad2;
     float* acc;
     Workspace* ws;
 };

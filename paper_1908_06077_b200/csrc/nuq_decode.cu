@@ -97,6 +97,46 @@ __device__ __forceinline__ float level_times_norm(float norm, uint32_t levelset,
     return __fmul_rn(norm, level);
 }
 
+// ---------------------------------------------------------------------------
+// What happens to the finished sum G = sum_k DECODE(c_k) of an element: it is stored to acc (if there is
+// one) and, when the call carries the aggregation step of Algorithm 1, applied to the parameters at once,
+// so that the sum is not written out and read again by an optimizer kernel:
+//     y = w - (alpha / K) G,   y^l = w - l (alpha / K) G,   w <- y + mu (y^l - y^l_prev)
+// (Sec. 4, "NUQSGD with momentum"; mu = 0 is Algorithm 1's own line and leaves y^l alone).  fp32, each line
+// one fused multiply-add.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float step_value(const DecodeParams& P, float w, float G, float* yl) {
+    const float y = __fmaf_rn(-P.step_c, G, w);
+    if (P.mu == 0.0f) return y;
+    const float yl_next = __fmaf_rn(-P.step_lc, G, w);
+    const float w_next = __fmaf_rn(P.mu, __fsub_rn(yl_next, *yl), y);
+    *yl = yl_next;
+    return w_next;
+}
+// element e (a multiple of 4) and the three behind it
+__device__ __forceinline__ void finish4(const DecodeParams& P, uint64_t e, float4 G, bool store_sum = true) {
+    if (store_sum && P.acc) *reinterpret_cast<float4*>(P.acc + e) = G;
+    if (P.w) {
+        float4 w = *reinterpret_cast<const float4*>(P.w + e);
+        float4 yl = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (P.mu != 0.0f) yl = *reinterpret_cast<const float4*>(P.yl + e);
+        w.x = step_value(P, w.x, G.x, &yl.x);
+        w.y = step_value(P, w.y, G.y, &yl.y);
+        w.z = step_value(P, w.z, G.z, &yl.z);
+        w.w = step_value(P, w.w, G.w, &yl.w);
+        *reinterpret_cast<float4*>(P.w + e) = w;
+        if (P.mu != 0.0f) *reinterpret_cast<float4*>(P.yl + e) = yl;
+    }
+}
+__device__ __forceinline__ void finish1(const DecodeParams& P, uint64_t e, float G, bool store_sum = true) {
+    if (store_sum && P.acc) P.acc[e] = G;
+    if (P.w) {
+        float yl = P.mu != 0.0f ? P.yl[e] : 0.0f;
+        P.w[e] = step_value(P, P.w[e], G, &yl);
+        if (P.mu != 0.0f) P.yl[e] = yl;
+    }
+}
+
 // ERC^-1 of an nbits-bit prefix: value | length << 8, or 0 when the code is longer than the prefix
 // (or is not a code).  Obtained by running Algorithm 2's decoder on the prefix.
 __device__ __forceinline__ uint32_t erc_prefix_entry(uint32_t idx, uint32_t nbits) {
@@ -266,7 +306,6 @@ __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const St
         const uint32_t nel = G.d - e0 < 32 ? (uint32_t)(G.d - e0) : 32u;
         const uint32_t bucket_len = b == G.nb - 1 ? (uint32_t)last_len : G.bucket;
         const uint32_t avail = (bucket_len * W + 31u) / 32u - (eb / 32u) * W;      // field words of the record from here on
-        float* dst = P.acc + e0;
         // branch free: a zero symbol adds +0 (the sums never are -0, so that changes nothing), the
         // largest symbol seen is checked once at the end; `whole`: all 32 elements exist
         auto body = [&](auto whole) {
@@ -306,11 +345,11 @@ __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const St
                 if (decltype(whole)::value) {
 #pragma unroll
                     for (int i = 0; i < 16; i += 4)
-                        *reinterpret_cast<float4*>(dst + 16 * half + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
+                        finish4(P, e0 + 16u * half + i, make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]));
                 } else {
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        if (16u * half + (uint32_t)i < nel) dst[16 * half + i] = acc[i];
+                        if (16u * half + (uint32_t)i < nel) finish1(P, e0 + 16u * half + i, acc[i]);
                 }
             }
         };
@@ -360,7 +399,7 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
             s_tab[k][f] = (f & 8u) ? -v : v;
         }
         __syncthreads();
-        float* const dst_tile = P.acc + b * G.bucket + first;
+        const uint64_t tile_elem0 = b * G.bucket + first;      // the tile's first element
         const uint64_t word0 = kHeaderWords + b * rec_words + 1u + first / 8u;     // the tile's first field word in a container
         // Two groups of eight elements per thread and step (el and el + 8 * blockDim.x): the words of both are
         // asked for before either is used, which keeps twice as many loads in flight.
@@ -406,14 +445,13 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
             for (int h = 0; h < 2; ++h) {
                 const uint32_t e0 = el + h * stride;
                 if (h == 1 && !second) break;
-                float* dst = dst_tile + e0;
                 if (e0 + 8u <= tile_len) {
-                    *reinterpret_cast<float4*>(dst) = make_float4(sum[h][0], sum[h][1], sum[h][2], sum[h][3]);
-                    *reinterpret_cast<float4*>(dst + 4) = make_float4(sum[h][4], sum[h][5], sum[h][6], sum[h][7]);
+                    finish4(P, tile_elem0 + e0, make_float4(sum[h][0], sum[h][1], sum[h][2], sum[h][3]));
+                    finish4(P, tile_elem0 + e0 + 4u, make_float4(sum[h][4], sum[h][5], sum[h][6], sum[h][7]));
                 } else {
 #pragma unroll
                     for (uint32_t i = 0; i < 8; ++i)
-                        if (e0 + i < tile_len) dst[i] = sum[h][i];
+                        if (e0 + i < tile_len) finish1(P, tile_elem0 + e0 + i, sum[h][i]);
                 }
             }
         }
@@ -885,14 +923,23 @@ __global__ void __launch_bounds__(32 * (SUMS_IN_L2 ? kDecMaxWarps - 1 : kDecMaxW
         __syncwarp();
         if (!SUMS_IN_L2) {
             const uint32_t first = part * S * kSB;
-            float* dst = P.acc + elem0 + first;
             for (uint32_t i = lane * 4u; i < S * kSB; i += 128u) {
                 if (first + i + 4u <= tile_len) {
-                    *reinterpret_cast<float4*>(dst + i) = *reinterpret_cast<const float4*>(accw + i);
+                    finish4(P, elem0 + first + i, *reinterpret_cast<const float4*>(accw + i));
                 } else {
-                    for (uint32_t e = i; e < i + 4u && first + e < tile_len; ++e) dst[e] = accw[e];
+                    for (uint32_t e = i; e < i + 4u && first + e < tile_len; ++e) finish1(P, elem0 + first + e, accw[e]);
                 }
                 *reinterpret_cast<float4*>(accw + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        } else if (P.w) {
+            // the unit's sums are complete in acc (this instance adds there): apply them to the parameters
+            for (uint32_t i = lane * 4u; i < unit_len; i += 128u) {
+                const uint64_t e = elem0 + part * S * kSB + i;
+                if (i + 4u <= unit_len) {
+                    finish4(P, e, __ldcg(reinterpret_cast<const float4*>(gsum + i)), false);
+                } else {
+                    for (uint32_t k = i; k < unit_len; ++k) finish1(P, e + (k - i), __ldcg(gsum + k), false);
+                }
             }
         }
         __syncwarp();

@@ -50,6 +50,9 @@ def _load():
     lib.nuq_decode_accumulate.restype = C.c_int
     lib.nuq_decode_accumulate.argtypes = [C.POINTER(C.c_void_p), C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32,
                                           C.c_void_p, C.c_void_p]
+    lib.nuq_decode_update.restype = C.c_int
+    lib.nuq_decode_update.argtypes = [C.POINTER(C.c_void_p), C.c_uint32, C.c_uint64, C.c_uint32, C.c_uint32,
+                                      C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_float, C.c_void_p]
     lib.nuq_encode_bound.restype = C.c_uint64
     lib.nuq_encode_bound.argtypes = [C.c_uint64, C.c_uint32, C.c_uint32, C.c_uint32]
     lib.nuq_set_level_table.restype = C.c_int
@@ -185,6 +188,17 @@ def decode_accumulate(streams, d, bucket, s, acc=None, stream=None):
     if rc != NUQ_OK:
         raise NuqError("nuq_decode_accumulate", rc)
     return acc
+
+
+def decode_update(streams, d, bucket, s, w, yl=None, alpha=1.0, mu=0.0, l=0.0, acc=None, stream=None):
+    """w <- w - (alpha / K) sum_k DECODE(streams[k]), or the momentum rule with yl when mu != 0; in place."""
+    ptrs = (C.c_void_p * len(streams))(*[C.c_void_p(t.data_ptr()) for t in streams])
+    rc = _lib.nuq_decode_update(ptrs, len(streams), d, bucket, s, C.c_void_p(acc.data_ptr() if acc is not None else None),
+                                C.c_void_p(w.data_ptr()), C.c_void_p(yl.data_ptr() if yl is not None else None),
+                                C.c_float(alpha), C.c_float(mu), C.c_float(l), _stream(stream))
+    if rc != NUQ_OK:
+        raise NuqError("nuq_decode_update", rc)
+    return w
 
 
 def last_status(stream=None) -> int:
