@@ -538,7 +538,7 @@ static nuq_status enqueue_decode(const void* const* streams, uint32_t K, uint64_
     P.group = K >= 8 ? 8u : K >= 3 ? 4u : K;            // 1, 2, 4 or 8 streams side by side
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
-    P.after_fixed = 1;                                  // all streams believed to be in the fixed-width mode?
+    P.after_fixed = w ? 0u : 1u;                        // all streams believed to be in the fixed-width mode? (sums only)
     for (uint32_t k = 0; k < K; ++k) {
         auto it = g_container_mode.find(std::make_pair(dev, streams[k]));
         if (it == g_container_mode.end() || it->second != kModeFixed) P.after_fixed = 0;

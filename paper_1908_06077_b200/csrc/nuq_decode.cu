@@ -306,6 +306,7 @@ __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const St
         const uint32_t nel = G.d - e0 < 32 ? (uint32_t)(G.d - e0) : 32u;
         const uint32_t bucket_len = b == G.nb - 1 ? (uint32_t)last_len : G.bucket;
         const uint32_t avail = (bucket_len * W + 31u) / 32u - (eb / 32u) * W;      // field words of the record from here on
+        float* dst = P.acc + e0;
         // branch free: a zero symbol adds +0 (the sums never are -0, so that changes nothing), the
         // largest symbol seen is checked once at the end; `whole`: all 32 elements exist
         auto body = [&](auto whole) {
@@ -345,11 +346,11 @@ __device__ __forceinline__ void decode_all_fixed(const DecodeParams& P, const St
                 if (decltype(whole)::value) {
 #pragma unroll
                     for (int i = 0; i < 16; i += 4)
-                        finish4(P, e0 + 16u * half + i, make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]));
+                        *reinterpret_cast<float4*>(dst + 16 * half + i) = make_float4(acc[i], acc[i + 1], acc[i + 2], acc[i + 3]);
                 } else {
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        if (16u * half + (uint32_t)i < nel) finish1(P, e0 + 16u * half + i, acc[i]);
+                        if (16u * half + (uint32_t)i < nel) dst[16 * half + i] = acc[i];
                 }
             }
         };
@@ -399,7 +400,7 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
             s_tab[k][f] = (f & 8u) ? -v : v;
         }
         __syncthreads();
-        const uint64_t tile_elem0 = b * G.bucket + first;      // the tile's first element
+        float* const dst_tile = P.acc + b * G.bucket + first;
         const uint64_t word0 = kHeaderWords + b * rec_words + 1u + first / 8u;     // the tile's first field word in a container
         // Two groups of eight elements per thread and step (el and el + 8 * blockDim.x): the words of both are
         // asked for before either is used, which keeps twice as many loads in flight.
@@ -445,13 +446,14 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
             for (int h = 0; h < 2; ++h) {
                 const uint32_t e0 = el + h * stride;
                 if (h == 1 && !second) break;
+                float* dst = dst_tile + e0;
                 if (e0 + 8u <= tile_len) {
-                    finish4(P, tile_elem0 + e0, make_float4(sum[h][0], sum[h][1], sum[h][2], sum[h][3]));
-                    finish4(P, tile_elem0 + e0 + 4u, make_float4(sum[h][4], sum[h][5], sum[h][6], sum[h][7]));
+                    *reinterpret_cast<float4*>(dst) = make_float4(sum[h][0], sum[h][1], sum[h][2], sum[h][3]);
+                    *reinterpret_cast<float4*>(dst + 4) = make_float4(sum[h][4], sum[h][5], sum[h][6], sum[h][7]);
                 } else {
 #pragma unroll
                     for (uint32_t i = 0; i < 8; ++i)
-                        if (e0 + i < tile_len) finish1(P, tile_elem0 + e0 + i, sum[h][i]);
+                        if (e0 + i < tile_len) dst[i] = sum[h][i];
                 }
             }
         }
@@ -460,7 +462,8 @@ __device__ __forceinline__ void decode_fixed4_tiles(const DecodeParams& P, const
 }
 
 // The kernel of that path.  It is launched when the library believes that all streams are in the
-// fixed-width mode (it wrote them itself); it checks the headers like the general kernel and, if they
+// fixed-width mode (it wrote them itself) and the call wants the sums only (a call that carries the
+// aggregation step takes the general kernel, which applies it); it checks the headers like the general kernel and, if they
 // say otherwise, leaves everything to the general kernel, which is launched behind it in any case and
 // returns at once when this one has done the work.
 __global__ void __launch_bounds__(256) decode_fixed_kernel(const __grid_constant__ DecodeParams P) {
