@@ -538,6 +538,10 @@ static nuq_status enqueue_decode(const void* const* streams, uint32_t K, uint64_
     P.group = K >= 8 ? 8u : K >= 3 ? 4u : K;            // 1, 2, 4 or 8 streams side by side
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
+    // A small call with the widest units (32 / group sub-blocks per warp) gives only a few warps of the whole
+    // GPU something to do, and a warp's walk is a chain of dependent steps: narrower units (lanes left idle)
+    // put more warps to work.
+    while (P.group < 8u && 2u * P.geo.ntiles * P.group <= 8u * (uint64_t)device_sms(dev)) P.group *= 2u;
     P.after_fixed = w ? 0u : 1u;                        // all streams believed to be in the fixed-width mode? (sums only)
     for (uint32_t k = 0; k < K; ++k) {
         auto it = g_container_mode.find(std::make_pair(dev, streams[k]));

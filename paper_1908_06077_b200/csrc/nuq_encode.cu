@@ -462,16 +462,6 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
-    // The first tile's bytes are asked for before anything else is set up: they arrive while the tables are built.
-    if (tid == 0) {
-        for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
-        take_ticket(0);
-        const TileInfo& ti = s_info[0];
-        for (uint32_t w = 0; w < (uint32_t)kEncWarps; ++w) {
-            const uint32_t n = ti.tile < G.ntiles && ti.tile_len > w * kWarpElems ? min(kWarpElems, ti.tile_len - w * kWarpElems) & ~3u : 0u;
-            if (n) bulk_load(data + w * kWarpElems, P.g + ti.elem0 + w * kWarpElems, 4u * n, &s_full[w]);
-        }
-    }
     if (tid < 256u) {
         const uint32_t e = c_erc_lut[tid], elen = e >> 16;  // at most 16 bits
         s_lut[tid] = ((e & 0xffffu) << (32u - elen)) | elen;
@@ -493,6 +483,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     if (MODE == kModeErc)
         for (uint32_t i = tid; i < 2u * P.stage_words + 2u * kEncWarps * P.window_words; i += blockDim.x) images[i] = 0;
     if (tid == 0) {
+        for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
         s_nnz = 0;
         s_arrived = 0;
         s_tot.nnz = 0;
@@ -504,6 +495,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
             mbar_init(&s_xbar[0], cl);
             mbar_init(&s_xbar[1], cl);
         }
+        take_ticket(0);
     }
     __syncthreads();
     if (cl > 1u) {
@@ -514,6 +506,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         }
         cluster_sync_all();                                 // the buckets of the next two iterations are known everywhere
     }
+    if (warp < (uint32_t)kEncWarps && lane == 0) start_copy(0);
     if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
 
     const bool writer = MODE == kModeErc && warp == (uint32_t)kEncWarps;
