@@ -491,6 +491,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         s_tot.tiles = 0;
         s_tot.stop = 0xFFFFFFFFu;
         s_last = 0;
+        encode_call_begin(P);
         if (cl > 1u) {
             mbar_init(&s_xbar[0], cl);
             mbar_init(&s_xbar[1], cl);
@@ -1000,6 +1001,8 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
         const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + (MODE == kModeErc ? G.ntiles + (G.ntiles + 31) / 32 : 0);
         for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;    // (only the ERC mode keeps state per tile)
+        __syncthreads();
+        if (tid == 0) encode_call_end(P);
     }
     if (cl > 1u) cluster_sync_all();                        // nobody leaves while another CTA may still write into its shared memory
 }
@@ -1159,7 +1162,7 @@ int encode_blocks_per_sm(const EncodeParams& P) {
 // launch configuration of a call, with the cluster shape when it has one
 struct EncodeLaunch {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
 };
 template <uint32_t M>
 static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, cudaStream_t stream) {
@@ -1171,11 +1174,16 @@ static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, c
     L->cfg.attrs = L->attr;
     L->cfg.numAttrs = 0;
     if (P.cluster > 1u) {
-        L->attr[0].id = cudaLaunchAttributeClusterDimension;
-        L->attr[0].val.clusterDim.x = P.cluster;
-        L->attr[0].val.clusterDim.y = 1;
-        L->attr[0].val.clusterDim.z = 1;
-        L->cfg.numAttrs = 1;
+        cudaLaunchAttribute& a = L->attr[L->cfg.numAttrs++];
+        a.id = cudaLaunchAttributeClusterDimension;
+        a.val.clusterDim.x = P.cluster;
+        a.val.clusterDim.y = 1;
+        a.val.clusterDim.z = 1;
+    }
+    if (P.overlap) {                                        // may start while the kernel before it in the stream ends
+        cudaLaunchAttribute& a = L->attr[L->cfg.numAttrs++];
+        a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        a.val.programmaticStreamSerializationAllowed = 1;
     }
 }
 

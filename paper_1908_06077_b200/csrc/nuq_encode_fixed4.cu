@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         s_nnz = 0;
         s_arrived = 0;
         s_last = 0;
+        encode_call_begin(P);
         take_ticket(0);
     }
     __syncthreads();
@@ -289,6 +290,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
         const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8;
         for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;
+        __syncthreads();
+        if (tid == 0) encode_call_end(P);
     }
 }
 
@@ -302,9 +305,20 @@ int fixed4_blocks_per_sm(const EncodeParams& P) {
 
 cudaError_t launch_encode_fixed4(const EncodeParams& P, cudaStream_t stream) {
     if (P.grid == 0) return cudaErrorInvalidValue;
-    if (P.geo.bucket % kFx4WarpElems == 0) encode_fixed4_kernel<true><<<P.grid, kEncThreads, 0, stream>>>(P);
-    else encode_fixed4_kernel<false><<<P.grid, kEncThreads, 0, stream>>>(P);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(P.grid);
+    cfg.blockDim = dim3(kEncThreads);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 0;
+    if (P.overlap) {                                        // may start while the kernel before it in the stream ends
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 1;
+    }
+    if (P.geo.bucket % kFx4WarpElems == 0) return cudaLaunchKernelEx(&cfg, encode_fixed4_kernel<true>, P);
+    return cudaLaunchKernelEx(&cfg, encode_fixed4_kernel<false>, P);
 }
 
 }  // namespace nuq
