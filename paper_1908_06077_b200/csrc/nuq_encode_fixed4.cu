@@ -84,11 +84,11 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         s_nnz = 0;
         s_arrived = 0;
         s_last = 0;
-        encode_call_begin(P);
         take_ticket(0);
     }
     __syncthreads();
     if (lane == 0) start_copy(0);
+    if (tid == 0) encode_call_begin(P);                     // before the workspace is touched; runs while the first bytes arrive
     if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
 
     uint32_t it = 0;
