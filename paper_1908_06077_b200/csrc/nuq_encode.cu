@@ -462,6 +462,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
+    const uint64_t seen_finished = tid == 0 ? encode_call_peek(P) : 0;
     if (tid < 256u) {
         const uint32_t e = c_erc_lut[tid], elen = e >> 16;  // at most 16 bits
         s_lut[tid] = ((e & 0xffffu) << (32u - elen)) | elen;
@@ -491,7 +492,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         s_tot.tiles = 0;
         s_tot.stop = 0xFFFFFFFFu;
         s_last = 0;
-        encode_call_begin(P);
+        encode_call_begin(P, seen_finished);
         if (cl > 1u) {
             mbar_init(&s_xbar[0], cl);
             mbar_init(&s_xbar[1], cl);

@@ -179,18 +179,25 @@ __device__ __forceinline__ void describe_tile(const Geometry& G, unsigned long l
 // on their last tiles.  A call two back used the same workspace as this one: it has long ended, but that is
 // checked (the CTA that finished it last left its number in the workspace), with a bounded wait.
 // Thread 0 of a CTA, before it touches the workspace.
-__device__ __forceinline__ void encode_call_begin(const EncodeParams& P) {
+__device__ __forceinline__ void encode_call_begin(const EncodeParams& P, uint64_t seen) {
     if (!P.overlap) return;
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the call after this one may start as CTAs of this one leave
     const volatile uint64_t* fin = &P.ws->enc_finished;
-    for (uint32_t polls = 0; *fin != P.expect_finished; ++polls) {
+    for (uint32_t polls = 0; seen != P.expect_finished; ++polls) {
         if (polls > (1u << 20)) {                           // never seen; do not hang
             latch_status(P.ws, kErrTimeout);
             break;
         }
         __nanosleep(200);
+        seen = *fin;
     }
     __threadfence();
+}
+// The first look at that number, taken when the CTA starts (its round trip runs under the CTA's set-up), and
+// the signal that the call after this one may start as CTAs of this one leave.  Thread 0.
+__device__ __forceinline__ uint64_t encode_call_peek(const EncodeParams& P) {
+    if (!P.overlap) return 0;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    return *reinterpret_cast<const volatile uint64_t*>(&P.ws->enc_finished);
 }
 // Thread 0 of the CTA that finished the call last, behind a CTA barrier after its last write to the workspace.
 __device__ __forceinline__ void encode_call_end(const EncodeParams& P) {

@@ -79,6 +79,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
+    const uint64_t seen_finished = tid == 0 ? encode_call_peek(P) : 0;
     if (tid == 0) {
         for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
         s_nnz = 0;
@@ -88,7 +89,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
     }
     __syncthreads();
     if (lane == 0) start_copy(0);
-    if (tid == 0) encode_call_begin(P);                     // before the workspace is touched; runs while the first bytes arrive
+    if (tid == 0) encode_call_begin(P, seen_finished);      // before the workspace is touched
     if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
 
     uint32_t it = 0;
