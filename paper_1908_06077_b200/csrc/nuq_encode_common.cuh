@@ -201,6 +201,9 @@ __device__ __forceinline__ uint64_t encode_call_peek(const EncodeParams& P) {
 }
 // Thread 0 of the CTA that finished the call last, behind a CTA barrier after its last write to the workspace.
 __device__ __forceinline__ void encode_call_end(const EncodeParams& P) {
+    // A call that started early must not end before the call it followed has ended (and its writes are
+    // visible): whatever is enqueued behind this call in the ordinary way waits for this call only.
+    if (P.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
     __threadfence();
     *reinterpret_cast<volatile uint64_t*>(&P.ws->enc_finished) = P.epoch;
 }
