@@ -27,15 +27,12 @@ struct WsEntry {
     // norms of a wide-bucket call or of a histogram call stay behind, at a place that depends on that call's size.
     size_t dirty_to = 0;
     uint32_t dec_epoch = 0;  // decode calls made on this workspace (see DecodeParams::epoch)
-    uint64_t enc_calls = 0;  // encode calls made on this (device, stream): they take the two workspaces in turn
-    uint64_t enc_launched = 0;   // number of the last encode call launched on this workspace (0: none since it was allocated)
 };
 
 // One mutex guards the host-side bookkeeping below (maps, tables); it is held for the microseconds a
 // call spends on the host, never across a wait for the device, except where a workspace has to grow.
 std::mutex g_mu;
 std::map<std::pair<int, cudaStream_t>, WsEntry> g_ws;
-std::map<std::pair<int, cudaStream_t>, WsEntry> g_ws_alt;   // the second workspace of a stream: every other encode call runs there
 std::map<int, int> g_sms;                 // device -> SM count
 std::set<int> g_lut_ready;                // devices whose constant LUT is uploaded
 std::map<int, const float*> g_test_norms;   // device -> bucket norms of nuq_set_test_norms
@@ -159,12 +156,12 @@ int device_sms(int dev) {
     return sms;
 }
 
-// Workspace of (current device, stream), grown to `bytes`; `alt`: the stream's second one.  Growing synchronises the stream.
-nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int* dev_out, bool alt = false) {
+// Workspace of (current device, stream), grown to `bytes`.  Growing synchronises the stream.
+nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int* dev_out) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
     *dev_out = dev;
-    WsEntry& e = (alt ? g_ws_alt : g_ws)[std::make_pair(dev, stream)];
+    WsEntry& e = g_ws[std::make_pair(dev, stream)];
     if (e.bytes < bytes) {
         int carried = 0;
         if (e.ptr) {
@@ -181,7 +178,6 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
         e.ptr = static_cast<Workspace*>(p);
         e.bytes = want;
         e.dirty_to = 0;
-        e.enc_launched = 0;
         if (carried && cudaMemcpy(&e.ptr->status, &carried, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
             return NUQ_ERR_CUDA;
     }
@@ -234,6 +230,7 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, uint32_t flags) {
     // up its norm through distributed shared memory, so there is no separate pass over the gradient for the norms.
     // (Not with norms supplied by the caller, and not in the 4-bit fixed-width encoder.)
     P.cluster = 0;
+    P.pad = 0;
     if (G.bucket > kBLK && norms_are_ours && !fixed4_applies(G)) {
         P.cluster = G.blk_per_bucket;
         int clusters = encode_max_clusters(P);
@@ -285,11 +282,6 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     P.out = static_cast<uint32_t*>(out);
     P.out_bits = out_bits;
     P.ws = ws;
-    // (P.epoch is set by the caller) the call that used this workspace last must have ended before this one
-    // touches it; calls on the static array do not overlap
-    // (a call that does not fill the GPU is launched in the ordinary way: there the check costs more than the overlap gains)
-    P.overlap = entry && P.grid >= 2u * (uint32_t)device_sms(dev) ? 1u : 0u;
-    P.expect_finished = entry ? entry->enc_launched : 0;
     P.seed = seed;
     P.offset = offset;
     for (uint32_t j = 0; j < kMaxTableS + 2u; ++j) {
@@ -308,7 +300,6 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
         if (entry) entry->dirty_to = entry->bytes;          // whatever state the failed launch left
         return NUQ_ERR_CUDA;
     }
-    if (entry) entry->enc_launched = P.epoch;
     // remember the mode of the container at this address: a hint for the decoder's choice of kernels,
     // checked against the header on the device
     if (g_container_mode.size() > 4096) g_container_mode.clear();
@@ -464,8 +455,7 @@ nuq_status nuq_level_histogram(const float* g, uint64_t d, uint32_t bucket, uint
         P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
     }
-    P.stage_words = P.window_words = P.patience = P.grid = P.cluster = P.overlap = 0;
-    P.epoch = P.expect_finished = 0;
+    P.stage_words = P.window_words = P.patience = P.grid = P.cluster = P.pad = 0;
     if (cudaMemsetAsync(hist, 0, 8 * (s + 2), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     if (launch_level_histogram(P, hist, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;
@@ -490,15 +480,11 @@ nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, u
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
     const EncodePlan pl = plan_encode(P, device_sms(dev), norm_kind);
     P.grid = pl.want_grid;
-    // Consecutive calls on a stream take the stream's two workspaces in turn: a call is launched so that it may
-    // start while the call before it ends, and must not share scan state with it.
-    P.epoch = ++g_ws[std::make_pair(dev, stream)].enc_calls;
-    const bool alt = (P.epoch & 1u) == 0;
     Workspace* ws = nullptr;
-    nuq_status st = get_workspace(stream, pl.state_bytes + pl.norms_bytes, &ws, &dev, alt);
+    nuq_status st = get_workspace(stream, pl.state_bytes + pl.norms_bytes, &ws, &dev);
     if (st != NUQ_OK) return st;
-    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws,
-                          &(alt ? g_ws_alt : g_ws)[std::make_pair(dev, stream)], dev, stream);
+    return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, ws, &g_ws[std::make_pair(dev, stream)],
+                          dev, stream);
 }
 
 nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind,
@@ -524,7 +510,6 @@ nuq_status nuq_encode_static(const float* g, uint64_t d, uint32_t bucket, uint32
         it = g_static_ws.emplace(dev, static_cast<Workspace*>(p)).first;
     }
     // the array is shared by every stream of the device: it is cleared before every call
-    P.epoch = 1;
     return enqueue_encode(P, pl, g, norm_kind, seed, offset, out, out_bits, it->second, nullptr, dev, stream);
 }
 
@@ -602,20 +587,17 @@ nuq_status nuq_last_status(void* stream_) {
     if (cudaGetDevice(&dev) != cudaSuccess) return NUQ_ERR_CUDA;
     if (cudaStreamSynchronize(stream) != cudaSuccess) return NUQ_ERR_CUDA;
     int status = 0;
-    for (auto* ws_map : {&g_ws, &g_ws_alt}) {             // an error outranks the warning, the most negative error wins
-        auto it = ws_map->find(std::make_pair(dev, stream));
-        if (it == ws_map->end() || !it->second.ptr) continue;
-        int s1 = 0;
-        if (cudaMemcpy(&s1, &it->second.ptr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
-        if (s1 != 0 && cudaMemset(&it->second.ptr->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
-        if ((s1 < 0 && s1 < status) || (status == 0 && s1 > 0)) status = s1;
+    auto it = g_ws.find(std::make_pair(dev, stream));
+    if (it != g_ws.end() && it->second.ptr) {
+        if (cudaMemcpy(&status, &it->second.ptr->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
+        if (status != 0 && cudaMemset(&it->second.ptr->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
     }
     auto st = g_static_ws.find(dev);               // kernels of nuq_encode_static latch into the static scratch
     if (st != g_static_ws.end()) {
         int s2 = 0;
         if (cudaMemcpy(&s2, &st->second->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return NUQ_ERR_CUDA;
         if (s2 != 0 && cudaMemset(&st->second->status, 0, sizeof(int)) != cudaSuccess) return NUQ_ERR_CUDA;
-        if ((s2 < 0 && s2 < status) || (status == 0 && s2 > 0)) status = s2;
+        if (s2 < status) status = s2;
     }
     return status;
 }
@@ -644,15 +626,13 @@ void nuq_shutdown(void) {
     std::lock_guard<std::mutex> lock(g_mu);
     int cur = 0;
     cudaGetDevice(&cur);
-    for (auto* ws_map : {&g_ws, &g_ws_alt}) {
-        for (auto& kv : *ws_map) {
-            if (kv.second.ptr) {
-                cudaSetDevice(kv.first.first);
-                cudaFree(kv.second.ptr);
-            }
+    for (auto& kv : g_ws) {
+        if (kv.second.ptr) {
+            cudaSetDevice(kv.first.first);
+            cudaFree(kv.second.ptr);
         }
-        ws_map->clear();
     }
+    g_ws.clear();
     cudaSetDevice(cur);
 }
 

@@ -37,7 +37,6 @@ constexpr uint64_t kTileValueMask = (1ull << 62) - 1;
 struct Workspace {
     int status;             // latched kernel status; survives calls until nuq_last_status reads it
     uint32_t dec_done_epoch; // decoder: the call (DecodeParams::epoch) whose fixed-width kernel did all the work
-    uint64_t enc_finished;   // encoder: number (EncodeParams::epoch) of the last call on this workspace that has ended
     // everything below is cleared at the start of every encode call
     uint64_t ticket;        // next tile to hand out
     uint64_t done;          // tiles finished
@@ -47,7 +46,7 @@ struct Workspace {
     uint64_t dec_ticket[2]; // decoder: next unit to hand out; a call uses the counter of its epoch's parity and zeroes the other one
     // followed by: uint64_t tile_state[ntiles], group_state[ceil(ntiles / 32)], then float norms[nb] for wide buckets
 };
-constexpr size_t kWorkspaceClearFrom = 16;
+constexpr size_t kWorkspaceClearFrom = 8;
 
 struct Geometry {
     uint64_t d;
@@ -86,9 +85,7 @@ struct EncodeParams {
     uint32_t patience;       // polls a look-back wait may take before it gives up
     uint32_t grid;           // CTAs to launch
     uint32_t cluster;        // CTAs per thread-block cluster: the blocks of one wide bucket (0: no clusters)
-    uint32_t overlap;        // launched with programmatic stream serialization: may start while the call before it ends
-    uint64_t epoch;          // number of this call on its workspace (never 0) ...
-    uint64_t expect_finished;// ... and of the call before it there, which must have ended before this one touches the workspace
+    uint32_t pad;
 };
 
 struct DecodeParams {

@@ -429,23 +429,24 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     // buckets then) and writes them into every CTA's s_bucket.
     const uint32_t cl = CLUSTERS ? P.cluster : 1u;
     const uint32_t crank = cl > 1u ? cluster_rank() : 0u;
-    const unsigned long long nclusters = gridDim.x / cl;
     auto hand_out_bucket = [&](uint32_t iter) {             // thread 0 of the cluster's first CTA
-        const unsigned long long b = nclusters + atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+        const unsigned long long b = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
         for (uint32_t r = 0; r < cl; ++r) st_cluster_u64(cluster_addr(&s_bucket[iter & 3u], r), b);
         asm volatile("fence.acq_rel.cluster;" ::: "memory");
     };
-    // thread 0: take a ticket (a CTA's first tile is the one with its own number, the tickets count on
-    // from there) and work out where that tile lies
+    // thread 0: take a ticket and work out where that tile lies.  Every tile is handed out by ticket, a CTA's
+    // first one too: a tile waits (look-back) for the tiles before it, and those must belong to CTAs that are
+    // running -- the CTAs of a call need not all be resident at once (another stream's kernel may hold SM
+    // slots), and a CTA that is not running must not own a tile that the running ones wait for.
     auto take_ticket = [&](uint32_t iter) {
         TileInfo& ti = s_info[iter & 3u];
         unsigned long long t;
         if (cl > 1u) {
-            const unsigned long long b = iter == 0 ? blockIdx.x / cl : *reinterpret_cast<volatile unsigned long long*>(&s_bucket[iter & 3u]);
+            const unsigned long long b = *reinterpret_cast<volatile unsigned long long*>(&s_bucket[iter & 3u]);
             t = b >= G.nb ? G.ntiles : b * cl + crank;
             if (b < G.nb && t >= G.ntiles) t = G.ntiles + 1u;    // the last bucket is short and has no tile for this CTA
         } else {
-            t = iter == 0 ? blockIdx.x : gridDim.x + atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
+            t = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->ticket), 1ull);
         }
         describe_tile(G, t, &ti);
     };
@@ -462,7 +463,6 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
-    const uint64_t seen_finished = tid == 0 ? encode_call_peek(P) : 0;
     if (tid < 256u) {
         const uint32_t e = c_erc_lut[tid], elen = e >> 16;  // at most 16 bits
         s_lut[tid] = ((e & 0xffffu) << (32u - elen)) | elen;
@@ -492,21 +492,23 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         s_tot.tiles = 0;
         s_tot.stop = 0xFFFFFFFFu;
         s_last = 0;
-        encode_call_begin(P, seen_finished);
         if (cl > 1u) {
             mbar_init(&s_xbar[0], cl);
             mbar_init(&s_xbar[1], cl);
         }
-        take_ticket(0);
+        if (cl == 1u) take_ticket(0);
     }
     __syncthreads();
     if (cl > 1u) {
         cluster_sync_all();                                 // every CTA's barriers exist before anyone arrives at them
-        if (tid == 0 && crank == 0) {
+        if (tid == 0 && crank == 0) {                       // (the first bucket comes by ticket too, like a CTA's first tile)
+            hand_out_bucket(0);
             hand_out_bucket(1);
             hand_out_bucket(2);
         }
-        cluster_sync_all();                                 // the buckets of the next two iterations are known everywhere
+        cluster_sync_all();                                 // the buckets of the first three iterations are known everywhere
+        if (tid == 0) take_ticket(0);
+        __syncthreads();
     }
     if (warp < (uint32_t)kEncWarps && lane == 0) start_copy(0);
     if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
@@ -1002,8 +1004,6 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
         const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8 + (MODE == kModeErc ? G.ntiles + (G.ntiles + 31) / 32 : 0);
         for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;    // (only the ERC mode keeps state per tile)
-        __syncthreads();
-        if (tid == 0) encode_call_end(P);
     }
     if (cl > 1u) cluster_sync_all();                        // nobody leaves while another CTA may still write into its shared memory
 }
@@ -1163,7 +1163,7 @@ int encode_blocks_per_sm(const EncodeParams& P) {
 // launch configuration of a call, with the cluster shape when it has one
 struct EncodeLaunch {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
 };
 template <uint32_t M>
 static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, cudaStream_t stream) {
@@ -1175,16 +1175,11 @@ static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, c
     L->cfg.attrs = L->attr;
     L->cfg.numAttrs = 0;
     if (P.cluster > 1u) {
-        cudaLaunchAttribute& a = L->attr[L->cfg.numAttrs++];
-        a.id = cudaLaunchAttributeClusterDimension;
-        a.val.clusterDim.x = P.cluster;
-        a.val.clusterDim.y = 1;
-        a.val.clusterDim.z = 1;
-    }
-    if (P.overlap) {                                        // may start while the kernel before it in the stream ends
-        cudaLaunchAttribute& a = L->attr[L->cfg.numAttrs++];
-        a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        a.val.programmaticStreamSerializationAllowed = 1;
+        L->attr[0].id = cudaLaunchAttributeClusterDimension;
+        L->attr[0].val.clusterDim.x = P.cluster;
+        L->attr[0].val.clusterDim.y = 1;
+        L->attr[0].val.clusterDim.z = 1;
+        L->cfg.numAttrs = 1;
     }
 }
 

@@ -174,40 +174,6 @@ __device__ __forceinline__ void describe_tile(const Geometry& G, unsigned long l
     ti.nsb = (ti.tile_len + kSB - 1) / kSB;
 }
 
-// Consecutive encode calls on a stream are launched with programmatic stream serialization and take two
-// workspaces in turn, so that the CTAs of a call start while the last CTAs of the call before it still work
-// on their last tiles.  A call two back used the same workspace as this one: it has long ended, but that is
-// checked (the CTA that finished it last left its number in the workspace), with a bounded wait.
-// Thread 0 of a CTA, before it touches the workspace.
-__device__ __forceinline__ void encode_call_begin(const EncodeParams& P, uint64_t seen) {
-    if (!P.overlap) return;
-    const volatile uint64_t* fin = &P.ws->enc_finished;
-    for (uint32_t polls = 0; seen != P.expect_finished; ++polls) {
-        if (polls > (1u << 20)) {                           // never seen; do not hang
-            latch_status(P.ws, kErrTimeout);
-            break;
-        }
-        __nanosleep(200);
-        seen = *fin;
-    }
-    __threadfence();
-}
-// The first look at that number, taken when the CTA starts (its round trip runs under the CTA's set-up), and
-// the signal that the call after this one may start as CTAs of this one leave.  Thread 0.
-__device__ __forceinline__ uint64_t encode_call_peek(const EncodeParams& P) {
-    if (!P.overlap) return 0;
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    return *reinterpret_cast<const volatile uint64_t*>(&P.ws->enc_finished);
-}
-// Thread 0 of the CTA that finished the call last, behind a CTA barrier after its last write to the workspace.
-__device__ __forceinline__ void encode_call_end(const EncodeParams& P) {
-    // A call that started early must not end before the call it followed has ended (and its writes are
-    // visible): whatever is enqueued behind this call in the ordinary way waits for this call only.
-    if (P.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
-    __threadfence();
-    *reinterpret_cast<volatile uint64_t*>(&P.ws->enc_finished) = P.epoch;
-}
-
 // Bookkeeping of a CTA that has written all its tiles: counters, and the container header by
 // whichever CTA finishes last (returns true there).  One thread, after a CTA barrier behind the last write.
 template <uint32_t MODE>

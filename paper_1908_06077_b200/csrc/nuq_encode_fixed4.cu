@@ -79,7 +79,6 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
-    const uint64_t seen_finished = tid == 0 ? encode_call_peek(P) : 0;
     if (tid == 0) {
         for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
         s_nnz = 0;
@@ -89,7 +88,6 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
     }
     __syncthreads();
     if (lane == 0) start_copy(0);
-    if (tid == 0) encode_call_begin(P, seen_finished);      // before the workspace is touched
     if (tid == 0) take_ticket(1);                           // its round trip runs while the first bytes arrive
 
     uint32_t it = 0;
@@ -291,8 +289,6 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         uint64_t* state = reinterpret_cast<uint64_t*>(reinterpret_cast<char*>(P.ws) + kWorkspaceClearFrom);
         const uint64_t n = (sizeof(Workspace) - kWorkspaceClearFrom) / 8;
         for (uint64_t i = tid; i < n; i += blockDim.x) state[i] = 0;
-        __syncthreads();
-        if (tid == 0) encode_call_end(P);
     }
 }
 
@@ -306,20 +302,9 @@ int fixed4_blocks_per_sm(const EncodeParams& P) {
 
 cudaError_t launch_encode_fixed4(const EncodeParams& P, cudaStream_t stream) {
     if (P.grid == 0) return cudaErrorInvalidValue;
-    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
-    cudaLaunchAttribute attr[1];
-    cfg.gridDim = dim3(P.grid);
-    cfg.blockDim = dim3(kEncThreads);
-    cfg.stream = stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 0;
-    if (P.overlap) {                                        // may start while the kernel before it in the stream ends
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.numAttrs = 1;
-    }
-    if (P.geo.bucket % kFx4WarpElems == 0) return cudaLaunchKernelEx(&cfg, encode_fixed4_kernel<true>, P);
-    return cudaLaunchKernelEx(&cfg, encode_fixed4_kernel<false>, P);
+    if (P.geo.bucket % kFx4WarpElems == 0) encode_fixed4_kernel<true><<<P.grid, kEncThreads, 0, stream>>>(P);
+    else encode_fixed4_kernel<false><<<P.grid, kEncThreads, 0, stream>>>(P);
+    return cudaGetLastError();
 }
 
 }  // namespace nuq
