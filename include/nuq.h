@@ -113,14 +113,9 @@ typedef struct nuq_info {
  *   out_bits  device u64 (may be NULL): receives container_bits
  *   returns   NUQ_ERR_INVALID_ARG for bad arguments, NUQ_ERR_CUDA if the
  *             per-stream workspace cannot be allocated or a launch fails.
- * The call may allocate (and then synchronise the device) when a per-stream
- * workspace has to grow; otherwise it is asynchronous.  Consecutive calls on one
- * stream that fill the GPU are launched so that a call's thread blocks may start
- * while the last blocks of the call before it still run (programmatic stream
- * serialization; the calls take two workspaces in turn).  Work that the caller
- * enqueues behind a call in the ordinary way starts, as always, when the call is
- * complete; only a kernel that the caller itself launches with programmatic
- * stream serialization could see a container before it is finished.
+ * The call may allocate (and then synchronise the device) when the per-stream
+ * workspace has to grow; otherwise it is asynchronous.  Calls on different
+ * streams may run at the same time (each stream has its own workspace).
  */
 nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
                       uint64_t offset, void* out, uint64_t* out_bits, void* stream);
@@ -186,7 +181,7 @@ nuq_status nuq_decode_update(const void* const* streams, uint32_t K, uint64_t d,
  * Arguments, container, random draws and results are exactly those of
  * nuq_encode.  Differences:
  *   - Size limit: with T = ceil(d / tile) tiles (a tile is 8192 elements, or
- *     floor(8192 / bucket) buckets) the scan state needs 72 + 8 * (T + ceil(T / 32))
+ *     floor(8192 / bucket) buckets) the scan state needs 64 + 8 * (T + ceil(T / 32))
  *     bytes, plus 4 bytes per bucket when bucket > 8192 and the bucket norms
  *     come from a pass of their own (4-bit fixed-width fields).  If that exceeds
  *     NUQ_STATIC_SCRATCH_BYTES the call returns NUQ_ERR_CAPACITY and enqueues

@@ -206,3 +206,36 @@ def test_c3_with_a_level_table(c3_inputs):
     assert rc == 0
     got = gpu_decode(streams, d, 8192, 4)
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
+def test_two_streams_encode_at_the_same_time(c3_inputs):
+    """Two streams, each with several ResNet-50-sized encode calls in flight: neither call has all its CTAs
+    resident, so a tile may only ever belong to a CTA that is running (every tile is handed out by ticket).
+    The containers are those of the same calls made alone, and no wait runs out."""
+    import torch
+    from gpu_util import require_cuda
+    torch, nuq = require_cuda()
+    gs = [torch.from_numpy(g).cuda() for g in c3_inputs[:2]]
+    d = gs[0].numel()
+    nbytes = nuq.encode_bound(d, 8192, 4, 0)
+    alone = []
+    for k, g in enumerate(gs):
+        out = torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda")
+        _, bits = nuq.encode(g, 8192, 4, 0, seed=k + 1, offset=0, out=out)
+        assert nuq.last_status() == 0
+        alone.append(out.cpu().numpy().view(np.uint32)[: int(bits.item()) // 32].copy())
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda") for _ in range(4)] for _ in range(2)]
+    bits = [[torch.zeros(1, dtype=torch.int64, device="cuda") for _ in range(4)] for _ in range(2)]
+    torch.cuda.synchronize()
+    for rep in range(4):
+        for k in range(2):
+            with torch.cuda.stream(streams[k]):
+                nuq.encode(gs[k], 8192, 4, 0, seed=k + 1, offset=0, out=outs[k][rep], out_bits=bits[k][rep], stream=streams[k])
+    torch.cuda.synchronize()
+    for k in range(2):
+        assert nuq.last_status(streams[k]) == 0
+        for rep in range(4):
+            n = int(bits[k][rep].item())
+            assert n == 32 * alone[k].size
+            assert np.array_equal(outs[k][rep].cpu().numpy().view(np.uint32)[: n // 32], alone[k])
