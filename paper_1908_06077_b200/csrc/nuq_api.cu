@@ -174,11 +174,14 @@ nuq_status get_workspace(cudaStream_t stream, size_t bytes, Workspace** out, int
         size_t want = bytes + bytes / 2;
         void* p = nullptr;
         if (cudaMalloc(&p, want) != cudaSuccess) { cudaGetLastError(); return NUQ_ERR_CUDA; }
-        if (cudaMemset(p, 0, want) != cudaSuccess) return NUQ_ERR_CUDA;
+        // (in the call's own stream: a clearing pass on the default stream is not ordered before kernels of a
+        // non-blocking stream, which would then run on a workspace that is still being cleared)
+        if (cudaMemsetAsync(p, 0, want, stream) != cudaSuccess) return NUQ_ERR_CUDA;
         e.ptr = static_cast<Workspace*>(p);
         e.bytes = want;
         e.dirty_to = 0;
-        if (carried && cudaMemcpy(&e.ptr->status, &carried, sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess)
+        if (carried && (cudaMemcpyAsync(&e.ptr->status, &carried, sizeof(int), cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+                        cudaStreamSynchronize(stream) != cudaSuccess))
             return NUQ_ERR_CUDA;
     }
     *out = e.ptr;
