@@ -39,7 +39,7 @@ struct Workspace {
     uint32_t dec_done_epoch; // decoder: the call (DecodeParams::epoch) whose fixed-width kernel did all the work
     // everything below is cleared at the start of every encode call
     uint64_t ticket;        // next tile to hand out
-    uint64_t done;          // tiles finished
+    uint64_t done;          // CTAs that have finished (they take no further ticket)
     uint64_t code_bits;     // token bits of the whole call
     uint64_t nnz;           // nonzero symbols of the whole call
     uint64_t total_words;   // payload words of the whole call

@@ -303,7 +303,7 @@ struct Pending {
 // What a CTA has written so far (shared memory; updated by one thread at a time).
 struct CtaTotals {
     uint64_t nnz, code_bits;
-    uint32_t tiles, stop;                                  // stop: tiles the workers encoded (set when they leave)
+    uint32_t stop, pad;                                    // stop: tiles the workers encoded (set when they leave)
 };
 
 // The writer warp, first half of its work on a tile: the layout of the tile's records from the 32
@@ -374,7 +374,6 @@ __device__ void flush_pending(const EncodeParams& P, Pending& pd, CtaTotals& tot
     }
     __syncwarp();
     if (lane == 0) {
-        tot.tiles += 1;
         tot.nnz += pd.nnz;
         tot.code_bits += pd.code_bits;
     }
@@ -489,7 +488,6 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         s_arrived = 0;
         s_tot.nnz = 0;
         s_tot.code_bits = 0;
-        s_tot.tiles = 0;
         s_tot.stop = 0xFFFFFFFFu;
         s_last = 0;
         if (cl > 1u) {
@@ -993,8 +991,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     }
     __syncthreads();                                        // every write of this CTA lies behind this barrier
     if (tid == 0) {
-        const bool last = MODE == kModeErc ? finish_cta<MODE>(P, s_tot.tiles, s_tot.nnz, s_tot.code_bits)
-                                           : finish_cta<MODE>(P, it, s_nnz, 0);
+        const bool last = MODE == kModeErc ? finish_cta<MODE>(P, s_tot.nnz, s_tot.code_bits) : finish_cta<MODE>(P, s_nnz, 0);
         if (last) s_last = 1;
     }
     __syncthreads();

@@ -174,17 +174,19 @@ __device__ __forceinline__ void describe_tile(const Geometry& G, unsigned long l
     ti.nsb = (ti.tile_len + kSB - 1) / kSB;
 }
 
-// Bookkeeping of a CTA that has written all its tiles: counters, and the container header by
-// whichever CTA finishes last (returns true there).  One thread, after a CTA barrier behind the last write.
+// Bookkeeping of a CTA that has written all its tiles and takes no further ticket: counters, and the
+// container header by whichever CTA finishes last (returns true there; that CTA then zeroes the call's
+// state).  One thread, after a CTA barrier behind the last write.  CTAs are counted, not tiles: a CTA
+// that started late and found no tile left has taken tickets all the same, and the ticket counter must
+// not be zeroed before it has (the next call would start counting above zero and skip its first tiles).
 template <uint32_t MODE>
-__device__ bool finish_cta(const EncodeParams& P, uint32_t tiles, uint64_t nnz, uint64_t code_bits) {
+__device__ bool finish_cta(const EncodeParams& P, uint64_t nnz, uint64_t code_bits) {
     const Geometry& G = P.geo;
-    if (tiles == 0) return false;
     if (nnz) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->nnz), (unsigned long long)nnz);
     if (code_bits) atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->code_bits), (unsigned long long)code_bits);
     __threadfence();
-    const unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), (unsigned long long)tiles);
-    if (prev + tiles != G.ntiles) return false;
+    const unsigned long long prev = atomicAdd(reinterpret_cast<unsigned long long*>(&P.ws->done), 1ull);
+    if (prev + 1ull != (unsigned long long)gridDim.x) return false;
     __threadfence();
     uint64_t code_total, words;
     const uint64_t nnz_total = ld_volatile_u64(&P.ws->nnz);

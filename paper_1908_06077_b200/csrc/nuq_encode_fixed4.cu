@@ -281,7 +281,7 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
     for (int o = 16; o > 0; o >>= 1) my_nnz += __shfl_xor_sync(0xffffffffu, my_nnz, o);
     if (lane == 0 && my_nnz) atomicAdd(&s_nnz, my_nnz);
     __syncthreads();                                        // every write of this CTA lies behind this barrier
-    if (tid == 0 && finish_cta<kModeFixed>(P, it, s_nnz, 0)) s_last = 1;
+    if (tid == 0 && finish_cta<kModeFixed>(P, s_nnz, 0)) s_last = 1;
     __syncthreads();
     if (s_last) {
         // Every tile of the call has been written.  The CTA that finished last leaves the call's counters zeroed,

@@ -208,34 +208,48 @@ def test_c3_with_a_level_table(c3_inputs):
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
 
 
-def test_two_streams_encode_at_the_same_time(c3_inputs):
+@pytest.mark.parametrize("bucket,mode", [(8192, O.MODE_ERC), (65536, O.MODE_ERC), (32768, O.MODE_ERC), (8192, O.MODE_FIXED),
+                                         (65536, O.MODE_FIXED)])
+def test_two_streams_encode_at_the_same_time(c3_inputs, bucket, mode):
     """Two streams, each with several ResNet-50-sized encode calls in flight: neither call has all its CTAs
-    resident, so a tile may only ever belong to a CTA that is running (every tile is handed out by ticket).
-    The containers are those of the same calls made alone, and no wait runs out."""
+    resident, so a tile may only ever belong to a CTA that is running (every tile is handed out by ticket),
+    and a CTA that starts when no tile is left still takes tickets, so the call's counters may be zeroed
+    only when every CTA has finished (else the next call on the stream starts counting above zero and never
+    encodes its first tiles).  Buckets wider than a tile are encoded by clusters, which take a ticket per
+    bucket.  The containers are those of the same calls made alone, and no wait runs out."""
     import torch
     from gpu_util import require_cuda
     torch, nuq = require_cuda()
+    flags = O.make_flags(mode=mode)
     gs = [torch.from_numpy(g).cuda() for g in c3_inputs[:2]]
     d = gs[0].numel()
-    nbytes = nuq.encode_bound(d, 8192, 4, 0)
+    nbytes = nuq.encode_bound(d, bucket, 4, flags)
     alone = []
     for k, g in enumerate(gs):
         out = torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda")
-        _, bits = nuq.encode(g, 8192, 4, 0, seed=k + 1, offset=0, out=out)
+        _, bits = nuq.encode(g, bucket, 4, flags, seed=k + 1, offset=0, out=out)
         assert nuq.last_status() == 0
         alone.append(out.cpu().numpy().view(np.uint32)[: int(bits.item()) // 32].copy())
     streams = [torch.cuda.Stream(), torch.cuda.Stream()]
     outs = [[torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda") for _ in range(4)] for _ in range(2)]
     bits = [[torch.zeros(1, dtype=torch.int64, device="cuda") for _ in range(4)] for _ in range(2)]
-    torch.cuda.synchronize()
-    for rep in range(4):
+    for attempt in range(3):
         for k in range(2):
-            with torch.cuda.stream(streams[k]):
-                nuq.encode(gs[k], 8192, 4, 0, seed=k + 1, offset=0, out=outs[k][rep], out_bits=bits[k][rep], stream=streams[k])
-    torch.cuda.synchronize()
-    for k in range(2):
-        assert nuq.last_status(streams[k]) == 0
+            for rep in range(4):
+                outs[k][rep].zero_()
+                bits[k][rep].zero_()
+        torch.cuda.synchronize()
         for rep in range(4):
-            n = int(bits[k][rep].item())
-            assert n == 32 * alone[k].size
-            assert np.array_equal(outs[k][rep].cpu().numpy().view(np.uint32)[: n // 32], alone[k])
+            for k in range(2):
+                with torch.cuda.stream(streams[k]):
+                    nuq.encode(gs[k], bucket, 4, flags, seed=k + 1, offset=0, out=outs[k][rep], out_bits=bits[k][rep],
+                               stream=streams[k])
+            if attempt == 1 and rep == 0:
+                torch.cuda.synchronize()                     # the later calls start at another moment of the other stream's
+        torch.cuda.synchronize()
+        for k in range(2):
+            assert nuq.last_status(streams[k]) == 0
+            for rep in range(4):
+                n = int(bits[k][rep].item())
+                assert n == 32 * alone[k].size
+                assert np.array_equal(outs[k][rep].cpu().numpy().view(np.uint32)[: n // 32], alone[k])
