@@ -233,7 +233,7 @@ static EncodePlan plan_encode(EncodeParams& P, int sms, uint32_t flags) {
     // up its norm through distributed shared memory, so there is no separate pass over the gradient for the norms.
     // (Not with norms supplied by the caller, and not in the 4-bit fixed-width encoder.)
     P.cluster = 0;
-    P.pad = 0;
+    P.overlap = 0;
     if (G.bucket > kBLK && norms_are_ours && !fixed4_applies(G)) {
         P.cluster = G.blk_per_bucket;
         int clusters = encode_max_clusters(P);
@@ -285,6 +285,10 @@ static nuq_status enqueue_encode(EncodeParams& P, const EncodePlan& pl, const fl
     P.out = static_cast<uint32_t*>(out);
     P.out_bits = out_bits;
     P.ws = ws;
+    // The kernel may be set up (its CTAs started, their tables built) while the kernel before it in the stream
+    // ends; it touches global memory only when that kernel has ended.  Not on the static array, which is
+    // cleared before every call.
+    P.overlap = entry ? 1u : 0u;
     P.seed = seed;
     P.offset = offset;
     for (uint32_t j = 0; j < kMaxTableS + 2u; ++j) {
@@ -458,7 +462,7 @@ nuq_status nuq_level_histogram(const float* g, uint64_t d, uint32_t bucket, uint
         P.round_keys[2 * r] = (uint32_t)seed + r * 0x9E3779B9u;
         P.round_keys[2 * r + 1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
     }
-    P.stage_words = P.window_words = P.patience = P.grid = P.cluster = P.pad = 0;
+    P.stage_words = P.window_words = P.patience = P.grid = P.cluster = P.overlap = 0;
     if (cudaMemsetAsync(hist, 0, 8 * (s + 2), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     if (launch_level_histogram(P, hist, device_sms(dev), stream) != cudaSuccess) return NUQ_ERR_CUDA;
     return NUQ_OK;

@@ -85,7 +85,7 @@ struct EncodeParams {
     uint32_t patience;       // polls a look-back wait may take before it gives up
     uint32_t grid;           // CTAs to launch
     uint32_t cluster;        // CTAs per thread-block cluster: the blocks of one wide bucket (0: no clusters)
-    uint32_t pad;
+    uint32_t overlap;        // launched so that its CTAs are set up while the kernel before it in the stream ends
 };
 
 struct DecodeParams {

@@ -462,6 +462,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
+    let_next_kernel_start(P);
     if (tid < 256u) {
         const uint32_t e = c_erc_lut[tid], elen = e >> 16;  // at most 16 bits
         s_lut[tid] = ((e & 0xffffu) << (32u - elen)) | elen;
@@ -482,6 +483,7 @@ encode_kernel(const __grid_constant__ EncodeParams P) {
     }
     if (MODE == kModeErc)
         for (uint32_t i = tid; i < 2u * P.stage_words + 2u * kEncWarps * P.window_words; i += blockDim.x) images[i] = 0;
+    wait_for_previous_kernel(P);                            // nothing above reads or writes global memory
     if (tid == 0) {
         for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
         s_nnz = 0;
@@ -1160,7 +1162,7 @@ int encode_blocks_per_sm(const EncodeParams& P) {
 // launch configuration of a call, with the cluster shape when it has one
 struct EncodeLaunch {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
 };
 template <uint32_t M>
 static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, cudaStream_t stream) {
@@ -1172,11 +1174,16 @@ static void fill_launch(EncodeLaunch* L, const EncodeParams& P, unsigned grid, c
     L->cfg.attrs = L->attr;
     L->cfg.numAttrs = 0;
     if (P.cluster > 1u) {
-        L->attr[0].id = cudaLaunchAttributeClusterDimension;
-        L->attr[0].val.clusterDim.x = P.cluster;
-        L->attr[0].val.clusterDim.y = 1;
-        L->attr[0].val.clusterDim.z = 1;
-        L->cfg.numAttrs = 1;
+        cudaLaunchAttribute& a = L->attr[L->cfg.numAttrs++];
+        a.id = cudaLaunchAttributeClusterDimension;
+        a.val.clusterDim.x = P.cluster;
+        a.val.clusterDim.y = 1;
+        a.val.clusterDim.z = 1;
+    }
+    if (P.overlap) {                                        // may be set up while the kernel before it in the stream ends
+        cudaLaunchAttribute& a = L->attr[L->cfg.numAttrs++];
+        a.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        a.val.programmaticStreamSerializationAllowed = 1;
     }
 }
 

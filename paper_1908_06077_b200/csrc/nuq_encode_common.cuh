@@ -174,6 +174,19 @@ __device__ __forceinline__ void describe_tile(const Geometry& G, unsigned long l
     ti.nsb = (ti.tile_len + kSB - 1) / kSB;
 }
 
+// Kernels that follow one another in a stream (programmatic dependent launch).  An encode kernel says at once,
+// as each CTA starts, that the kernel behind it may be launched: that kernel's CTAs then take the SM slots as
+// this one's leave them and do their set-up (tables in shared memory, barriers) while the last CTAs here still
+// work.  A kernel launched that way must not touch global memory before the kernel in front of it has ended
+// and its writes are visible: every thread waits for that ahead of its first access (the input may have been
+// written by that very kernel).  Without the launch attribute both instructions do nothing.
+__device__ __forceinline__ void let_next_kernel_start(const EncodeParams& P) {
+    if (P.overlap) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void wait_for_previous_kernel(const EncodeParams& P) {
+    if (P.overlap) asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Bookkeeping of a CTA that has written all its tiles and takes no further ticket: counters, and the
 // container header by whichever CTA finishes last (returns true there; that CTA then zeroes the call's
 // state).  One thread, after a CTA barrier behind the last write.  CTAs are counted, not tiles: a CTA

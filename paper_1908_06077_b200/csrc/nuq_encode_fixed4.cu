@@ -79,6 +79,8 @@ __global__ void __launch_bounds__(kEncThreads, kEncMinBlocks) encode_fixed4_kern
         if (n) bulk_load(data + wbase, P.g + ti.elem0 + wbase, 4u * n, &s_full[warp]);
     };
 
+    let_next_kernel_start(P);
+    wait_for_previous_kernel(P);                            // (this kernel has next to no set-up to do meanwhile)
     if (tid == 0) {
         for (int w = 0; w < kEncWarps; ++w) mbar_init(&s_full[w], 1);
         s_nnz = 0;
@@ -302,9 +304,20 @@ int fixed4_blocks_per_sm(const EncodeParams& P) {
 
 cudaError_t launch_encode_fixed4(const EncodeParams& P, cudaStream_t stream) {
     if (P.grid == 0) return cudaErrorInvalidValue;
-    if (P.geo.bucket % kFx4WarpElems == 0) encode_fixed4_kernel<true><<<P.grid, kEncThreads, 0, stream>>>(P);
-    else encode_fixed4_kernel<false><<<P.grid, kEncThreads, 0, stream>>>(P);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
+    cudaLaunchAttribute attr[1];
+    cfg.gridDim = dim3(P.grid);
+    cfg.blockDim = dim3(kEncThreads);
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 0;
+    if (P.overlap) {                                        // may be set up while the kernel before it in the stream ends
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.numAttrs = 1;
+    }
+    if (P.geo.bucket % kFx4WarpElems == 0) return cudaLaunchKernelEx(&cfg, encode_fixed4_kernel<true>, P);
+    return cudaLaunchKernelEx(&cfg, encode_fixed4_kernel<false>, P);
 }
 
 }  // namespace nuq

@@ -253,3 +253,43 @@ def test_two_streams_encode_at_the_same_time(c3_inputs, bucket, mode):
                 n = int(bits[k][rep].item())
                 assert n == 32 * alone[k].size
                 assert np.array_equal(outs[k][rep].cpu().numpy().view(np.uint32)[: n // 32], alone[k])
+
+
+@pytest.mark.parametrize("bucket,mode", [(8192, O.MODE_ERC), (8192, O.MODE_FIXED), (65536, O.MODE_ERC), (65536, O.MODE_FIXED)])
+def test_encode_calls_keep_the_order_of_their_stream(c3_inputs, bucket, mode):
+    """An encode kernel is set up while the kernel before it in the stream ends, but touches memory only when
+    that kernel has ended: a gradient written by the kernel just before the call is the one that is encoded, a
+    kernel that overwrites the gradient after the call does not reach into it, and of two calls into the same
+    buffer the second one's container stays."""
+    from gpu_util import require_cuda
+    torch, nuq = require_cuda()
+    flags = O.make_flags(mode=mode)
+    src = [torch.from_numpy(g).cuda() for g in c3_inputs]
+    d = src[0].numel()
+    nbytes = nuq.encode_bound(d, bucket, 4, flags)
+    alone = []
+    for k, g in enumerate(src):
+        out = torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda")
+        _, bits = nuq.encode(g, bucket, 4, flags, seed=7, offset=k, out=out)
+        assert nuq.last_status() == 0
+        alone.append(out.cpu().numpy().view(np.uint32)[: int(bits.item()) // 32].copy())
+    g = torch.zeros(d, dtype=torch.float32, device="cuda")
+    outs = [torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda") for _ in range(6)]
+    bits = [torch.zeros(1, dtype=torch.int64, device="cuda") for _ in range(6)]
+    same = torch.zeros(nbytes // 4, dtype=torch.int32, device="cuda")
+    same_bits = torch.zeros(1, dtype=torch.int64, device="cuda")
+    torch.cuda.synchronize()
+    for i in range(6):                                       # copy kernel, encode, copy kernel, encode, ... nothing waits
+        g.copy_(src[i % 3])
+        nuq.encode(g, bucket, 4, flags, seed=7, offset=i % 3, out=outs[i], out_bits=bits[i])
+    for i in range(3):                                       # three calls in a row into one buffer
+        nuq.encode(src[i], bucket, 4, flags, seed=7, offset=i, out=same, out_bits=same_bits)
+    torch.cuda.synchronize()
+    assert nuq.last_status() == 0
+    for i in range(6):
+        n = int(bits[i].item())
+        assert n == 32 * alone[i % 3].size
+        assert np.array_equal(outs[i].cpu().numpy().view(np.uint32)[: n // 32], alone[i % 3])
+    n = int(same_bits.item())
+    assert n == 32 * alone[2].size
+    assert np.array_equal(same.cpu().numpy().view(np.uint32)[: n // 32], alone[2])
