@@ -116,6 +116,9 @@ typedef struct nuq_info {
  * The call may allocate (and then synchronise the device) when the per-stream
  * workspace has to grow; otherwise it is asynchronous.  Calls on different
  * streams may run at the same time (each stream has its own workspace).
+ * The kernel is launched so that its blocks may be set up while the kernel
+ * before it in the stream ends; it reads and writes memory only after that
+ * kernel has ended, so the order of the stream holds for g, out, out_bits.
  */
 nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
                       uint64_t offset, void* out, uint64_t* out_bits, void* stream);
