@@ -119,6 +119,11 @@ typedef struct nuq_info {
  * The kernel is launched so that its blocks may be set up while the kernel
  * before it in the stream ends; it reads and writes memory only after that
  * kernel has ended, so the order of the stream holds for g, out, out_bits.
+ * Once the stream's workspace exists (after a first call of at least this
+ * size on the stream), encode calls may be captured into a CUDA graph and
+ * replayed: the kernels leave the workspace as they found it.  Decode calls
+ * may not: their hand-out counter alternates with the number of the call,
+ * which a replay does not advance.
  */
 nuq_status nuq_encode(const float* g, uint64_t d, uint32_t bucket, uint32_t s, uint32_t norm_kind, uint64_t seed,
                       uint64_t offset, void* out, uint64_t* out_bits, void* stream);

@@ -293,3 +293,44 @@ def test_encode_calls_keep_the_order_of_their_stream(c3_inputs, bucket, mode):
     n = int(same_bits.item())
     assert n == 32 * alone[2].size
     assert np.array_equal(same.cpu().numpy().view(np.uint32)[: n // 32], alone[2])
+
+
+def test_encode_calls_replayed_from_a_cuda_graph(c3_inputs):
+    """The eight encode calls of a step, captured once into a CUDA graph and replayed: an encode kernel leaves
+    its workspace as it found it and takes nothing from the host but its arguments, so every replay writes the
+    containers of the gradients that are in the input buffers at that time."""
+    from gpu_util import require_cuda
+    torch, nuq = require_cuda()
+    src = [torch.from_numpy(g).cuda() for g in c3_inputs]
+    d = src[0].numel()
+    cases = [(8192, 0), (8192, O.make_flags(mode=O.MODE_FIXED)), (65536, 0)]
+    side = torch.cuda.Stream()
+    gs = [torch.zeros(d, dtype=torch.float32, device="cuda") for _ in range(3)]
+    outs = [torch.zeros(nuq.encode_bound(d, b, 4, f) // 4, dtype=torch.int32, device="cuda") for b, f in cases]
+    bits = [torch.zeros(1, dtype=torch.int64, device="cuda") for _ in cases]
+
+    def enqueue():
+        for i, (b, f) in enumerate(cases):
+            nuq.encode(gs[i], b, 4, f, seed=11 + i, offset=5, out=outs[i], out_bits=bits[i], stream=side)
+
+    with torch.cuda.stream(side):                            # first use of the stream: the workspace is allocated here
+        enqueue()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        enqueue()
+    for rnd in range(3):
+        for i in range(3):
+            gs[i].copy_(src[(i + rnd) % 3])
+            outs[i].zero_()
+            bits[i].zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert nuq.last_status(side) == 0
+        for i, (b, f) in enumerate(cases):
+            want = torch.zeros_like(outs[i])
+            _, wbits = nuq.encode(src[(i + rnd) % 3], b, 4, f, seed=11 + i, offset=5, out=want)
+            n = int(wbits.item())
+            assert int(bits[i].item()) == n
+            assert torch.equal(outs[i][: n // 32], want[: n // 32])
